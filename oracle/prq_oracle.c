@@ -1,0 +1,337 @@
+/*
+ * PRQuant oracle -- TEST INFRASTRUCTURE, NOT THE PRODUCT.
+ *
+ * A plain, slow, scalar CPU statement of what the compensated W4A4 MXFP4 linear
+ * layer computes.  It exists so that the CUDA library can be checked against
+ * something written directly from the paper; it shares no code, header, table
+ * or helper with the CUDA library and must never be called from it.  Only the
+ * tests, the smoke check and the benchmark's CPU-baseline leg may use it.
+ *
+ * Every function names the passage of the paper it follows.  Floating point is
+ * FP64 unless the step is defined on fp32 values (the quantiser input, the
+ * scaled weight), in which case the fp32 value is produced by rounding an exact
+ * FP64 result once.
+ *
+ * Readings taken where the paper is silent (the MXFP4 details come from the OCP
+ * microscaling format the paper cites in its Introduction):
+ *   - block = 32 consecutive input channels of one row; shared scale 2^e with
+ *     e = clamp(floor(log2(amax)) - 2, -127, 127), stored as the byte e + 127;
+ *     an all-zero block stores byte 0;
+ *   - elements are E2M1 (values 0, .5, 1, 1.5, 2, 3, 4, 6 and a sign bit),
+ *     rounded to nearest with ties to the even code, magnitudes above 6
+ *     saturate to 6, the sign bit of the input is kept even when the magnitude
+ *     rounds to zero;
+ *   - packed storage: byte i of a row = code[2i] | code[2i+1] << 4;
+ *   - "column-wise quantization error" of channel j = sum over output rows of
+ *     the squared difference between the scaled weight and its MXFP4 image,
+ *     accumulated in FP64 in ascending row order;
+ *   - top-k ties break toward the lower channel index; the permutation lists the
+ *     unselected channels in ascending order, then the selected ones ascending;
+ *   - s_j = max(amax_j, 1e-5)^alpha.
+ *
+ * Pins (see tests/test_oracle_*.py): hand-worked encodings, a brute-force
+ * nearest-value quantiser in exact rational arithmetic, the worked prep example,
+ * k = 0 reducing to plain MXFP4, Eq. (1) invariance, exact residual identity,
+ * brute-force top-k, Eq. (3) = main + correction.  The alpha selection is
+ * "parity unpinned": the paper fixes only "argmin of the normalised error".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORC_BLOCK 32
+
+/* E2M1 magnitudes by 3-bit index (OCP MX element format cited in the Introduction). */
+static const double orc_e2m1_value[8] = {0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0};
+
+static float orc_bf16_to_f32(uint16_t h) {
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+static int orc_signbit_f32(float v) {
+    uint32_t u;
+    memcpy(&u, &v, 4);
+    return (int)(u >> 31);
+}
+
+/* Shared block scale (E8M0 byte) of one block of 32 fp32 values.
+ * floor(log2(amax)) - 2 puts amax/2^e in [4, 8), i.e. just inside the E2M1
+ * range up to its saturation band. */
+static uint8_t orc_block_scale_byte(const float *v) {
+    double amax = 0.0;
+    for (int i = 0; i < ORC_BLOCK; ++i) {
+        double a = fabs((double)v[i]);
+        if (a > amax) amax = a;
+    }
+    if (amax == 0.0) return 0;
+    int ex;
+    (void)frexp(amax, &ex); /* amax = m * 2^ex with m in [0.5, 1)  =>  floor(log2) = ex - 1 */
+    int e = (ex - 1) - 2;
+    if (e < -127) e = -127;
+    if (e > 127) e = 127;
+    return (uint8_t)(e + 127);
+}
+
+/* One element: a = |v| / 2^e is exact in FP64; round to the nearest E2M1
+ * magnitude, ties to the even code, saturating at 6. */
+static uint8_t orc_e2m1_code(float v, int e) {
+    double a = ldexp(fabs((double)v), -e);
+    uint8_t mag;
+    if (a <= 0.25) mag = 0;
+    else if (a < 0.75) mag = 1;
+    else if (a <= 1.25) mag = 2;
+    else if (a < 1.75) mag = 3;
+    else if (a <= 2.5) mag = 4;
+    else if (a < 3.5) mag = 5;
+    else if (a <= 5.0) mag = 6;
+    else mag = 7;
+    return (uint8_t)(mag | (orc_signbit_f32(v) << 3));
+}
+
+/* The MXFP4 quantiser Q of Eq. (2), storage half: rows x cols fp32 -> packed
+ * codes (rows x cols/2 bytes) and scale bytes (rows x cols/32). */
+int orc_quantize_rows(const float *v, long rows, long cols, uint8_t *codes, uint8_t *scales) {
+    if (cols % ORC_BLOCK) return 1;
+    for (long r = 0; r < rows; ++r) {
+        for (long b = 0; b < cols / ORC_BLOCK; ++b) {
+            const float *blk = v + r * cols + b * ORC_BLOCK;
+            uint8_t byte = orc_block_scale_byte(blk);
+            scales[r * (cols / ORC_BLOCK) + b] = byte;
+            int e = (int)byte - 127;
+            for (int i = 0; i < ORC_BLOCK; i += 2) {
+                uint8_t lo = orc_e2m1_code(blk[i], e);
+                uint8_t hi = orc_e2m1_code(blk[i + 1], e);
+                codes[(r * cols + b * ORC_BLOCK + i) / 2] = (uint8_t)(lo | (hi << 4));
+            }
+        }
+    }
+    return 0;
+}
+
+static double orc_dequant_one(const uint8_t *codes, const uint8_t *scales, long cols, long r, long j) {
+    uint8_t byte = codes[(r * cols + j) / 2];
+    uint8_t c = (j & 1) ? (uint8_t)(byte >> 4) : (uint8_t)(byte & 0xF);
+    double mag = orc_e2m1_value[c & 7];
+    int e = (int)scales[r * (cols / ORC_BLOCK) + j / ORC_BLOCK] - 127;
+    double x = ldexp(mag, e);
+    return (c & 8) ? -x : x;
+}
+
+/* The dequantise half of Q: sign * value[code & 7] * 2^(byte - 127), in FP64 (exact). */
+int orc_dequantize_rows(const uint8_t *codes, const uint8_t *scales, long rows, long cols, double *out) {
+    if (cols % ORC_BLOCK) return 1;
+    for (long r = 0; r < rows; ++r)
+        for (long j = 0; j < cols; ++j) out[r * cols + j] = orc_dequant_one(codes, scales, cols, r, j);
+    return 0;
+}
+
+/* Algorithm 1 step 1: per-channel maxima of |Z_cal| (exact, any precision). */
+int orc_channel_amax(const uint16_t *z_bf16, long T, long K, float *amax) {
+    for (long j = 0; j < K; ++j) amax[j] = 0.0f;
+    for (long t = 0; t < T; ++t)
+        for (long j = 0; j < K; ++j) {
+            float a = fabsf(orc_bf16_to_f32(z_bf16[t * K + j]));
+            if (a > amax[j]) amax[j] = a;
+        }
+    return 0;
+}
+
+/* Method, "Offline scaling": s_j = (max_t |Z_tj|)^alpha, stored in fp32, and the
+ * reciprocal the activation side multiplies by.  The grid values 0, .25, .5, .75, 1
+ * use only correctly rounded operations so that any implementation agrees. */
+int orc_scales_from_amax(const float *amax, long K, double alpha, float *s, float *inv_s) {
+    for (long j = 0; j < K; ++j) {
+        double a = (double)amax[j];
+        if (a < 1e-5) a = 1e-5;
+        double p;
+        if (alpha == 0.0) p = 1.0;
+        else if (alpha == 1.0) p = a;
+        else if (alpha == 0.5) p = sqrt(a);
+        else if (alpha == 0.25) p = sqrt(sqrt(a));
+        else if (alpha == 0.75) p = sqrt(a) * sqrt(sqrt(a));
+        else p = pow(a, alpha);
+        s[j] = (float)p;
+        inv_s[j] = (float)(1.0 / (double)s[j]);
+    }
+    return 0;
+}
+
+typedef struct {
+    double err;
+    int32_t idx;
+} orc_rank_t;
+
+static int orc_rank_cmp(const void *pa, const void *pb) {
+    const orc_rank_t *a = (const orc_rank_t *)pa, *b = (const orc_rank_t *)pb;
+    if (a->err > b->err) return -1;
+    if (a->err < b->err) return 1;
+    return (a->idx > b->idx) - (a->idx < b->idx);
+}
+
+/* Algorithm 1 steps 3-7 and 11 for one alpha:
+ *   W0 = fl32(W * s)                                  (step 3, scaled weight W D)
+ *   err_j = sum_n (W0[n,j] - deq(Q(W0))[n,j])^2       (step 4, original channel order)
+ *   top-k by err, perm = [unselected asc | selected asc]   (steps 4-5)
+ *   Wt = W0[:, perm]                                  (step 6, Eq. (1) W D P)
+ *   Qw = Q(Wt);  R = Wt_tail - deq(Qw)_tail           (step 7, Eq. (2))
+ *   export [Qw | Q(R)]                                (step 11, right factor of Eq. (3))
+ * Outputs: s, inv_s (K), col_err (K), perm (K, new -> old), wcodes N x (K+k)/2,
+ * wscales N x (K+k)/32, R (N x k fp32, may be NULL). */
+int orc_prepare(const uint16_t *W_bf16, long N, long K, const float *amax, double alpha, long k,
+                float *s, float *inv_s, double *col_err, int32_t *perm,
+                uint8_t *wcodes, uint8_t *wscales, float *R_out) {
+    if (K % ORC_BLOCK || k % ORC_BLOCK || k < 0 || k > K) return 1;
+    long Ka = K + k;
+    orc_scales_from_amax(amax, K, alpha, s, inv_s);
+
+    float *W0 = (float *)malloc(sizeof(float) * N * K);
+    uint8_t *c0 = (uint8_t *)malloc((size_t)N * K / 2);
+    uint8_t *s0 = (uint8_t *)malloc((size_t)N * K / ORC_BLOCK);
+    for (long n = 0; n < N; ++n)
+        for (long j = 0; j < K; ++j)
+            W0[n * K + j] = (float)((double)orc_bf16_to_f32(W_bf16[n * K + j]) * (double)s[j]);
+
+    orc_quantize_rows(W0, N, K, c0, s0);
+    for (long j = 0; j < K; ++j) col_err[j] = 0.0;
+    for (long n = 0; n < N; ++n)
+        for (long j = 0; j < K; ++j) {
+            double d = (double)W0[n * K + j] - orc_dequant_one(c0, s0, K, n, j);
+            col_err[j] += d * d;
+        }
+
+    orc_rank_t *rank = (orc_rank_t *)malloc(sizeof(orc_rank_t) * K);
+    for (long j = 0; j < K; ++j) {
+        rank[j].err = col_err[j];
+        rank[j].idx = (int32_t)j;
+    }
+    qsort(rank, (size_t)K, sizeof(orc_rank_t), orc_rank_cmp);
+    uint8_t *selected = (uint8_t *)calloc((size_t)K, 1);
+    for (long i = 0; i < k; ++i) selected[rank[i].idx] = 1;
+    long head = 0, tail = K - k;
+    for (long j = 0; j < K; ++j) {
+        if (selected[j]) perm[tail++] = (int32_t)j;
+        else perm[head++] = (int32_t)j;
+    }
+
+    float *Wt = (float *)malloc(sizeof(float) * N * K);
+    for (long n = 0; n < N; ++n)
+        for (long j = 0; j < K; ++j) Wt[n * K + j] = W0[n * K + perm[j]];
+    uint8_t *c1 = (uint8_t *)malloc((size_t)N * K / 2);
+    uint8_t *s1 = (uint8_t *)malloc((size_t)N * K / ORC_BLOCK);
+    orc_quantize_rows(Wt, N, K, c1, s1);
+
+    float *R = (float *)malloc(sizeof(float) * (size_t)(N * (k ? k : 1)));
+    for (long n = 0; n < N; ++n)
+        for (long i = 0; i < k; ++i) {
+            long j = K - k + i;
+            /* the difference is exactly representable in fp32 (both terms are
+             * multiples of the weight's last bit and the result is no larger) */
+            R[n * k + i] = (float)((double)Wt[n * K + j] - orc_dequant_one(c1, s1, K, n, j));
+        }
+    uint8_t *cr = (uint8_t *)malloc((size_t)(N * (k ? k : ORC_BLOCK)) / 2);
+    uint8_t *sr = (uint8_t *)malloc((size_t)(N * (k ? k : ORC_BLOCK)) / ORC_BLOCK);
+    if (k) orc_quantize_rows(R, N, k, cr, sr);
+
+    for (long n = 0; n < N; ++n) {
+        memcpy(wcodes + n * (Ka / 2), c1 + n * (K / 2), (size_t)K / 2);
+        memcpy(wscales + n * (Ka / ORC_BLOCK), s1 + n * (K / ORC_BLOCK), (size_t)K / ORC_BLOCK);
+        if (k) {
+            memcpy(wcodes + n * (Ka / 2) + K / 2, cr + n * (k / 2), (size_t)k / 2);
+            memcpy(wscales + n * (Ka / ORC_BLOCK) + K / ORC_BLOCK, sr + n * (k / ORC_BLOCK), (size_t)k / ORC_BLOCK);
+        }
+    }
+    if (R_out && k) memcpy(R_out, R, sizeof(float) * N * k);
+
+    free(W0); free(c0); free(s0); free(rank); free(selected); free(Wt); free(c1); free(s1); free(R); free(cr); free(sr);
+    return 0;
+}
+
+/* Eq. (1), activation side: Zt = Z D^-1 P, i.e. xt[t,j'] = fl32(x[t,perm[j']] * inv_s[perm[j']]);
+ * identity when perm and inv_s are NULL (folded into the producer layers).  Then Q by rows
+ * ("quantizes the reordered activation once", Kernel design paragraph). */
+int orc_quantize_act(const uint16_t *x_bf16, long M, long K, const int32_t *perm, const float *inv_s,
+                     uint8_t *codes, uint8_t *scales) {
+    if (K % ORC_BLOCK) return 1;
+    float *row = (float *)malloc(sizeof(float) * K);
+    for (long t = 0; t < M; ++t) {
+        for (long j = 0; j < K; ++j) {
+            long src = perm ? perm[j] : j;
+            double v = (double)orc_bf16_to_f32(x_bf16[t * K + src]);
+            if (inv_s) v = v * (double)inv_s[src];
+            row[j] = (float)v;
+        }
+        orc_quantize_rows(row, 1, K, codes + t * (K / 2), scales + t * (K / ORC_BLOCK));
+    }
+    free(row);
+    return 0;
+}
+
+/* "Online copy": the augmented activation [Q(Zt) | Q(Zt)[:, K-k:K]] -- the copied
+ * blocks keep their own codes and scales (Kernel design paragraph). */
+int orc_augment_act(const uint8_t *codes, const uint8_t *scales, long M, long K, long k,
+                    uint8_t *codes_aug, uint8_t *scales_aug) {
+    if (K % ORC_BLOCK || k % ORC_BLOCK || k > K) return 1;
+    long Ka = K + k;
+    for (long t = 0; t < M; ++t) {
+        memcpy(codes_aug + t * (Ka / 2), codes + t * (K / 2), (size_t)K / 2);
+        memcpy(codes_aug + t * (Ka / 2) + K / 2, codes + t * (K / 2) + (K - k) / 2, (size_t)k / 2);
+        memcpy(scales_aug + t * (Ka / ORC_BLOCK), scales + t * (K / ORC_BLOCK), (size_t)K / ORC_BLOCK);
+        memcpy(scales_aug + t * (Ka / ORC_BLOCK) + K / ORC_BLOCK,
+               scales + t * (K / ORC_BLOCK) + (K - k) / ORC_BLOCK, (size_t)k / ORC_BLOCK);
+    }
+    return 0;
+}
+
+/* Eq. (3): y[t,n] = sum_{j < Ka} deq(A)[t,j] * deq(W)[n,j], FP64, ascending j.
+ * Rows of y are independent; they are split across threads and nothing else is
+ * reordered. */
+int orc_matmul(const uint8_t *acodes, const uint8_t *ascales, long M,
+               const uint8_t *wcodes, const uint8_t *wscales, long N, long Ka, double *y) {
+    if (Ka % ORC_BLOCK) return 1;
+    double *A = (double *)malloc(sizeof(double) * (size_t)(M * Ka));
+    double *W = (double *)malloc(sizeof(double) * (size_t)(N * Ka));
+    orc_dequantize_rows(acodes, ascales, M, Ka, A);
+    orc_dequantize_rows(wcodes, wscales, N, Ka, W);
+    long t;
+#pragma omp parallel for schedule(static)
+    for (t = 0; t < M; ++t)
+        for (long n = 0; n < N; ++n) {
+            double acc = 0.0;
+            const double *a = A + t * Ka, *w = W + n * Ka;
+            for (long j = 0; j < Ka; ++j) acc += a[j] * w[j];
+            y[t * N + n] = acc;
+        }
+    free(A);
+    free(W);
+    return 0;
+}
+
+/* Unquantised reference Y = Z W^T in FP64 from the bf16 inputs (the target of the
+ * normalised reconstruction error after Eq. (3)). */
+int orc_matmul_bf16(const uint16_t *x_bf16, long M, const uint16_t *W_bf16, long N, long K, double *y) {
+    long t;
+#pragma omp parallel for schedule(static)
+    for (t = 0; t < M; ++t)
+        for (long n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (long j = 0; j < K; ++j)
+                acc += (double)orc_bf16_to_f32(x_bf16[t * K + j]) * (double)orc_bf16_to_f32(W_bf16[n * K + j]);
+            y[t * N + n] = acc;
+        }
+    return 0;
+}
+
+int orc_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
