@@ -1,0 +1,186 @@
+/*
+ * prq.h -- C ABI of libprq: the PRQuant compensated W4A4 MXFP4 linear layer on
+ * NVIDIA B200 (sm_100a).
+ *
+ * The library implements the inference hot path of the paper's Method section:
+ * offline, a weight W (N x K) is scaled per input channel, its k hardest channels
+ * are permuted into a contiguous tail and the tail's quantisation residual is
+ * appended, giving one MXFP4 matrix over K + k columns (Algorithm 1, Eq. (2));
+ * online, the activation is quantised to MXFP4 once and a single block-scaled FP4
+ * GEMM over K + k, which re-reads the activation tail against the residual
+ * columns, produces y (Eq. (3), "Kernel design for efficient inference").
+ *
+ * Conventions
+ *   - Every function returns a prq_status; nothing throws across the boundary and
+ *     outputs are left untouched when an argument check fails.
+ *   - "host" / "device" is stated for every pointer.  Device buffers are owned by
+ *     the caller (for example torch tensors); online calls never allocate, never
+ *     synchronise the device and run on the given CUDA stream.
+ *   - bf16 values are raw 16-bit patterns.  MXFP4 storage: 32-element blocks along
+ *     the reduction axis, one E8M0 scale byte per block (value 2^(byte-127)),
+ *     E2M1 elements packed two per byte with the even column in the low nibble.
+ *   - K % 32 == 0, k_tail % 32 == 0 and 0 <= k_tail <= K are required ("the tail and
+ *     concatenation boundaries are aligned with the MXFP4 quantization blocks").
+ *   - A prq_weights handle is immutable after creation and may be used from several
+ *     streams at once.  It belongs to the device that was current when it was made.
+ *   - A kernel that gives up on a bounded wait records PRQ_ERR_TIMEOUT in a device
+ *     status word that prq_last_device_status() reads; it never traps or spins forever.
+ */
+#ifndef PRQ_H_
+#define PRQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PRQ_OK = 0,
+    PRQ_ERR_INVALID_ARG = 1,
+    PRQ_ERR_ALIGNMENT = 2,
+    PRQ_ERR_UNSUPPORTED_ARCH = 3,
+    PRQ_ERR_CUDA = 4,
+    PRQ_ERR_OOM = 5,
+    PRQ_ERR_TIMEOUT = 6,
+    PRQ_ERR_NONFINITE = 7,
+    PRQ_ERR_WORKSPACE = 8
+} prq_status;
+
+typedef struct prq_weights prq_weights; /* opaque: prepared weights of one layer (or of E stacked experts) */
+typedef void *prq_stream_t;             /* a cudaStream_t; NULL is the default stream */
+
+typedef enum { PRQ_F32 = 0, PRQ_BF16 = 1 } prq_dtype;
+
+/* Which activation transform prq_quantize_act applies before quantising. */
+typedef enum {
+    PRQ_ACT_IDENTITY = 0,  /* x is already Z D^-1 P (folded into the producer layers, Eq. (1)) */
+    PRQ_ACT_SCALE_PERM = 1 /* apply x[t, perm[j]] * inv_s[perm[j]] online */
+} prq_act_mode;
+
+/* Host-side views that prq_weights_get copies out (for parity checks and export). */
+typedef enum {
+    PRQ_FIELD_CODES = 0,   /* uint8  N x (K+k)/2   packed E2M1 codes of [Q(W D P) | Q(R)]            */
+    PRQ_FIELD_SCALES = 1,  /* uint8  N x (K+k)/32  E8M0 bytes, row-major                             */
+    PRQ_FIELD_PERM = 2,    /* int32  K             new position -> original channel                   */
+    PRQ_FIELD_TOPK = 3,    /* int32  k             selected channels, ascending (= perm[K-k..K))      */
+    PRQ_FIELD_S = 4,       /* float  K             s_j = max(amax_j, 1e-5)^alpha, original order      */
+    PRQ_FIELD_INV_S = 5,   /* float  K             fl32(1 / s_j)                                      */
+    PRQ_FIELD_COL_ERR = 6  /* double K             column-wise quantisation error used for the ranking */
+} prq_field;
+
+typedef enum {
+    PRQ_BUF_CODES = 0,      /* M x K/2 bytes                                                    */
+    PRQ_BUF_SCALES_ROW = 1, /* M x K/32 bytes, row-major (optional output, parity view)         */
+    PRQ_BUF_SCALES_SF = 2   /* scale bytes in the GEMM's tile order, tail scales duplicated     */
+} prq_buf;
+
+/* ---- offline (Algorithm 1) ------------------------------------------------------------- */
+
+/* Algorithm 1 steps 3-7 and 11 for one given alpha: scale W by s = amax^alpha, rank the input
+ * channels by the MXFP4 quantisation error of the scaled weight, move the k_tail worst to a
+ * contiguous tail, quantise, compute the tail residual R (Eq. (2)), quantise it and store
+ * [Q(W D P) | Q(R)] on the current device in the GEMM's layout.
+ *   W         host, n_experts x N x K bf16, row-major (ld = K)
+ *   act_amax  host, n_experts x K float: max_t |Z_cal[t, j]| per input channel (step 1)
+ *   out       receives the handle; release it with prq_weights_free
+ * Runs on the host (multi-threaded) and uploads once.  Errors: INVALID_ARG (NULL, sizes,
+ * alignment of K / k_tail), NONFINITE (W, amax), UNSUPPORTED_ARCH (no sm_100 device), CUDA, OOM. */
+prq_status prq_prepare_weights(const uint16_t *W, int n_experts, int N, int K, const float *act_amax,
+                               float alpha, int k_tail, prq_weights **out);
+
+/* The same per-alpha pipeline as prq_prepare_weights, host buffers in and out, no device involved
+ * (offline tooling, export, checks on machines without a GPU).  One layer.
+ *   codes   host out, N x (K+k)/2    scales  host out, N x (K+k)/32    perm  host out, K int32
+ *   s, inv_s (K floats) and col_err (K doubles) are optional (NULL to skip). */
+prq_status prq_prepare_weights_host(const uint16_t *W, int N, int K, const float *act_amax, float alpha,
+                                    int k_tail, uint8_t *codes, uint8_t *scales, int32_t *perm, float *s,
+                                    float *inv_s, double *col_err);
+
+/* Algorithm 1 steps 1-10: derive amax from the calibration rows, run the per-alpha pipeline for
+ * every candidate, evaluate Eq. (3) on the calibration rows with the GPU kernels and keep the
+ * alpha with the smallest normalised error ||Yhat - Z W^T||_F / ||Z W^T||_F (first minimum).
+ *   Zcal       host, T x K bf16 (one layer; n_experts must be 1)
+ *   alphas     host, n_alphas candidates
+ *   alpha_star receives the chosen alpha; nrmse (host, n_alphas doubles, nullable) every error */
+prq_status prq_prepare_weights_search(const uint16_t *W, int N, int K, const uint16_t *Zcal, int T,
+                                      const float *alphas, int n_alphas, int k_tail, prq_weights **out,
+                                      float *alpha_star, double *nrmse);
+
+void prq_weights_free(prq_weights *w);
+
+/* Shape of a handle.  Any output pointer may be NULL. */
+prq_status prq_weights_info(const prq_weights *w, int *n_experts, int *N, int *K, int *k_tail, float *alpha);
+
+/* Copy one canonical host-side view of expert `expert` into dst (host, dst_bytes must match). */
+prq_status prq_weights_get(const prq_weights *w, int expert, prq_field which, void *dst, size_t dst_bytes);
+
+/* ---- online ------------------------------------------------------------------------------ */
+
+/* Size in bytes of an activation-side buffer for M rows.  For grouped calls pass the total row
+ * count and n_groups = number of experts (each group's scale tiles are padded to 128 rows);
+ * dense calls pass n_groups = 1.  Returns 0 for invalid arguments. */
+size_t prq_act_bytes(int M, int K, int k_tail, int n_groups, prq_buf which);
+
+/* "The kernel quantizes the reordered activation to MXFP4 once" (Kernel design paragraph).
+ * One launch: optional scale + permute (Eq. (1), activation side), per-32 amax, E8M0 scale,
+ * E2M1 round-to-nearest-even codes.  The quantised tail is not copied: only its k_tail/32 scale
+ * bytes per row are duplicated into the tile-ordered scale buffer, the GEMM re-reads the codes.
+ *   w               handle (gives K, k_tail, perm, inv_s); required
+ *   mode            PRQ_ACT_IDENTITY or PRQ_ACT_SCALE_PERM
+ *   x               device, M x K bf16, row stride ldx elements (ldx >= K, ldx % 8 == 0, 16-byte aligned)
+ *   expert_offsets  device, n_experts + 1 int32 row boundaries when w stacks experts (rows sorted by
+ *                   expert; expert e uses its own perm / inv_s); NULL for a dense layer
+ *   codes           device out, PRQ_BUF_CODES bytes (16-byte aligned)
+ *   scales_row      device out or NULL, PRQ_BUF_SCALES_ROW bytes
+ *   scales_sf       device out, PRQ_BUF_SCALES_SF bytes (16-byte aligned)
+ * M == 0 is a no-op. */
+prq_status prq_quantize_act(const prq_weights *w, prq_act_mode mode, const void *x, int M, int ldx,
+                            const int32_t *expert_offsets, void *codes, void *scales_row, void *scales_sf,
+                            prq_stream_t stream);
+
+/* Scratch the GEMM needs for M rows (split-K partial sums and tile counters); may be 0. */
+size_t prq_linear_workspace_bytes(const prq_weights *w, int M);
+
+/* Eq. (3): y = [Q(x) | Q(x)_tail] [Q(W D P) | Q(R)]^T, one block-scaled FP4 GEMM over K + k with fp32
+ * accumulation.  Reads activation columns [0, K) and then [K - k, K) again; no M x (K + k) buffer exists.
+ *   codes, scales_sf  device, as written by prq_quantize_act for the same w and M
+ *   y                 device out, M x N, row stride ldy elements, dtype y_dtype (fp32 for parity)
+ *   workspace         device, at least prq_linear_workspace_bytes(w, M) bytes, 16-byte aligned; its first
+ *                     use must be zero-filled by the caller, the kernels leave it zeroed again
+ * M <= 128 takes the weight-streaming split-K path, larger M the persistent prefill path. */
+prq_status prq_linear(const prq_weights *w, const void *codes, const void *scales_sf, int M, void *y, int ldy,
+                      prq_dtype y_dtype, void *workspace, size_t workspace_bytes, prq_stream_t stream);
+
+/* The same product for stacked experts (MoE): rows [expert_offsets[e], expert_offsets[e+1]) of the
+ * activation use expert e's weights.  expert_offsets: device, n_experts + 1 int32, non-decreasing,
+ * last = M_total. */
+prq_status prq_linear_grouped(const prq_weights *w, const void *codes, const void *scales_sf,
+                              const int32_t *expert_offsets, int M_total, void *y, int ldy, prq_dtype y_dtype,
+                              prq_stream_t stream);
+
+/* Whole online path from HOST buffers: copies x (host, M x K bf16, pinned for speed) to the device,
+ * quantises, multiplies and copies y (M x N, y_dtype) back to y_host, all on `stream`, using
+ * caller-provided device scratch of at least prq_forward_host_scratch_bytes(w, M) bytes (zero-filled
+ * before its first use).  Returns after enqueueing; synchronise the stream before reading y_host. */
+size_t prq_forward_host_scratch_bytes(const prq_weights *w, int M);
+prq_status prq_forward_host(const prq_weights *w, prq_act_mode mode, const uint16_t *x_host, int M,
+                            void *y_host, prq_dtype y_dtype, void *dev_scratch, size_t scratch_bytes,
+                            prq_stream_t stream);
+
+/* ---- diagnostics ----------------------------------------------------------------------- */
+
+const char *prq_status_string(prq_status s);
+
+/* Synchronises `stream`, then reads and clears the device status word that a kernel sets when a
+ * bounded wait expired (PRQ_ERR_TIMEOUT).  PRQ_OK when nothing went wrong. */
+prq_status prq_last_device_status(prq_stream_t stream);
+
+/* Number of kernels this library has launched in this process (for benchmark bookkeeping). */
+unsigned long long prq_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRQ_H_ */

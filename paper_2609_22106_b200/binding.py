@@ -1,0 +1,258 @@
+"""Thin ctypes binding over libprq.so (the C ABI declared in include/prq.h).
+
+Argument marshalling only: every step of the hot path runs inside the library's CUDA
+kernels.  torch is used for device memory and streams.  There is no CPU fallback: if the
+library cannot be loaded or a call fails, a ``PrqError`` is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libprq.so")
+
+OK = 0
+F32, BF16 = 0, 1
+ACT_IDENTITY, ACT_SCALE_PERM = 0, 1
+FIELD_CODES, FIELD_SCALES, FIELD_PERM, FIELD_TOPK, FIELD_S, FIELD_INV_S, FIELD_COL_ERR = range(7)
+BUF_CODES, BUF_SCALES_ROW, BUF_SCALES_SF = range(3)
+
+EXPORTS = [
+    "prq_prepare_weights", "prq_prepare_weights_host", "prq_prepare_weights_search", "prq_weights_free",
+    "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
+    "prq_linear", "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
+    "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count",
+]
+
+
+class PrqError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+_lib = None
+
+
+def lib():
+    """Load libprq.so (built in-tree by paper_2609_22106_b200.build).  Fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise PrqError(-1, f"libprq.so not found at {LIB_PATH}; run paper_2609_22106_b200.build.build()")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci, cf, cs = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        L.prq_prepare_weights.argtypes = [vp, ci, ci, ci, vp, cf, ci, ctypes.POINTER(vp)]
+        L.prq_prepare_weights_host.argtypes = [vp, ci, ci, vp, cf, ci, vp, vp, vp, vp, vp, vp]
+        L.prq_prepare_weights_search.argtypes = [vp, ci, ci, vp, ci, vp, ci, ci, ctypes.POINTER(vp),
+                                                 ctypes.POINTER(cf), vp]
+        L.prq_weights_free.argtypes = [vp]
+        L.prq_weights_free.restype = None
+        L.prq_weights_info.argtypes = [vp] + [ctypes.POINTER(ci)] * 4 + [ctypes.POINTER(cf)]
+        L.prq_weights_get.argtypes = [vp, ci, ci, vp, cs]
+        L.prq_act_bytes.argtypes = [ci, ci, ci, ci, ci]
+        L.prq_act_bytes.restype = cs
+        L.prq_quantize_act.argtypes = [vp, ci, vp, ci, ci, vp, vp, vp, vp, vp]
+        L.prq_linear_workspace_bytes.argtypes = [vp, ci]
+        L.prq_linear_workspace_bytes.restype = cs
+        L.prq_linear.argtypes = [vp, vp, vp, ci, vp, ci, ci, vp, cs, vp]
+        L.prq_linear_grouped.argtypes = [vp, vp, vp, vp, ci, vp, ci, ci, vp]
+        L.prq_forward_host_scratch_bytes.argtypes = [vp, ci]
+        L.prq_forward_host_scratch_bytes.restype = cs
+        L.prq_forward_host.argtypes = [vp, ci, vp, ci, vp, ci, vp, cs, vp]
+        L.prq_status_string.argtypes = [ci]
+        L.prq_status_string.restype = ctypes.c_char_p
+        L.prq_last_device_status.argtypes = [vp]
+        L.prq_kernel_launch_count.restype = ctypes.c_ulonglong
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    if code < 0:
+        return "library not loaded"
+    return lib().prq_status_string(code).decode()
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise PrqError(code, where)
+
+
+def _np_ptr(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _stream_ptr(stream=None):
+    import torch
+
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _dptr(t):
+    return ctypes.c_void_p(t.data_ptr()) if t is not None else None
+
+
+class Weights:
+    """Owner of a prq_weights handle."""
+
+    def __init__(self, handle):
+        self._h = handle
+        ne, N, K, k = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+        a = ctypes.c_float()
+        _check(lib().prq_weights_info(handle, ne, N, K, k, a), "prq_weights_info")
+        self.n_experts, self.N, self.K, self.k_tail, self.alpha = ne.value, N.value, K.value, k.value, a.value
+
+    @property
+    def handle(self):
+        return self._h
+
+    def get(self, field: int, expert: int = 0) -> np.ndarray:
+        Ka = self.K + self.k_tail
+        shape, dt = {
+            FIELD_CODES: ((self.N, Ka // 2), np.uint8),
+            FIELD_SCALES: ((self.N, Ka // 32), np.uint8),
+            FIELD_PERM: ((self.K,), np.int32),
+            FIELD_TOPK: ((self.k_tail,), np.int32),
+            FIELD_S: ((self.K,), np.float32),
+            FIELD_INV_S: ((self.K,), np.float32),
+            FIELD_COL_ERR: ((self.K,), np.float64),
+        }[field]
+        out = np.empty(shape, dt)
+        _check(lib().prq_weights_get(self._h, expert, field, _np_ptr(out), out.nbytes), "prq_weights_get")
+        return out
+
+    def free(self):
+        if self._h:
+            lib().prq_weights_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_tail: int) -> Weights:
+    """W_bf16: uint16 (N, K) or (E, N, K); act_amax: float32 (K,) or (E, K)."""
+    W = np.ascontiguousarray(W_bf16, np.uint16)
+    amax = np.ascontiguousarray(act_amax, np.float32)
+    if W.ndim == 2:
+        W = W[None]
+        amax = amax[None]
+    E, N, K = W.shape
+    h = ctypes.c_void_p()
+    _check(lib().prq_prepare_weights(_np_ptr(W), E, N, K, _np_ptr(amax), alpha, k_tail, ctypes.byref(h)),
+           "prq_prepare_weights")
+    return Weights(h)
+
+
+def prepare_weights_host(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_tail: int) -> dict:
+    W = np.ascontiguousarray(W_bf16, np.uint16)
+    amax = np.ascontiguousarray(act_amax, np.float32)
+    N, K = W.shape
+    Ka = K + k_tail
+    out = dict(codes=np.empty((N, Ka // 2), np.uint8), scales=np.empty((N, Ka // 32), np.uint8),
+               perm=np.empty(K, np.int32), s=np.empty(K, np.float32), inv_s=np.empty(K, np.float32),
+               col_err=np.empty(K, np.float64))
+    _check(lib().prq_prepare_weights_host(_np_ptr(W), N, K, _np_ptr(amax), alpha, k_tail, _np_ptr(out["codes"]),
+                                          _np_ptr(out["scales"]), _np_ptr(out["perm"]), _np_ptr(out["s"]),
+                                          _np_ptr(out["inv_s"]), _np_ptr(out["col_err"])), "prq_prepare_weights_host")
+    return out
+
+
+def prepare_weights_search(W_bf16, zcal_bf16, alphas, k_tail: int):
+    W = np.ascontiguousarray(W_bf16, np.uint16)
+    Z = np.ascontiguousarray(zcal_bf16, np.uint16)
+    al = np.ascontiguousarray(alphas, np.float32)
+    N, K = W.shape
+    T = Z.shape[0]
+    h = ctypes.c_void_p()
+    star = ctypes.c_float()
+    errs = np.empty(len(al), np.float64)
+    _check(lib().prq_prepare_weights_search(_np_ptr(W), N, K, _np_ptr(Z), T, _np_ptr(al), len(al), k_tail,
+                                            ctypes.byref(h), ctypes.byref(star), _np_ptr(errs)),
+           "prq_prepare_weights_search")
+    return Weights(h), star.value, errs
+
+
+def act_bytes(M: int, K: int, k_tail: int, n_groups: int, which: int) -> int:
+    return int(lib().prq_act_bytes(M, K, k_tail, n_groups, which))
+
+
+def quantize_act(w: Weights, x, mode: int = ACT_IDENTITY, expert_offsets=None, row_scales: bool = False,
+                 out=None, stream=None):
+    """x: torch bf16 CUDA tensor (M, K).  Returns (codes, scales_row or None, scales_sf) uint8 tensors."""
+    import torch
+
+    M = x.shape[0]
+    ng = w.n_experts
+    if out is None:
+        codes = torch.empty(max(act_bytes(M, w.K, w.k_tail, ng, BUF_CODES), 16), dtype=torch.uint8, device=x.device)
+        sf = torch.empty(max(act_bytes(M, w.K, w.k_tail, ng, BUF_SCALES_SF), 16), dtype=torch.uint8, device=x.device)
+        srow = torch.empty(max(act_bytes(M, w.K, w.k_tail, ng, BUF_SCALES_ROW), 16), dtype=torch.uint8,
+                           device=x.device) if row_scales else None
+    else:
+        codes, srow, sf = out
+    _check(lib().prq_quantize_act(w.handle, mode, _dptr(x), M, x.stride(0) if M else w.K, _dptr(expert_offsets),
+                                  _dptr(codes), _dptr(srow), _dptr(sf), _stream_ptr(stream)), "prq_quantize_act")
+    return codes, srow, sf
+
+
+def linear_workspace_bytes(w: Weights, M: int) -> int:
+    return int(lib().prq_linear_workspace_bytes(w.handle, M))
+
+
+def new_workspace(w: Weights, M: int, device="cuda"):
+    import torch
+
+    return torch.zeros(max(linear_workspace_bytes(w, M), 16), dtype=torch.uint8, device=device)
+
+
+def linear(w: Weights, codes, scales_sf, M: int, y_dtype: int = F32, workspace=None, out=None, stream=None):
+    import torch
+
+    if out is None:
+        out = torch.empty((M, w.N), dtype=torch.float32 if y_dtype == F32 else torch.bfloat16, device=codes.device)
+    if workspace is None:
+        workspace = new_workspace(w, M, codes.device)
+    _check(lib().prq_linear(w.handle, _dptr(codes), _dptr(scales_sf), M, _dptr(out), out.stride(0) if M else w.N,
+                            y_dtype, _dptr(workspace), workspace.numel(), _stream_ptr(stream)), "prq_linear")
+    return out
+
+
+def linear_grouped(w: Weights, codes, scales_sf, expert_offsets, M_total: int, y_dtype: int = F32, out=None,
+                   stream=None):
+    import torch
+
+    if out is None:
+        out = torch.empty((M_total, w.N), dtype=torch.float32 if y_dtype == F32 else torch.bfloat16,
+                          device=codes.device)
+    _check(lib().prq_linear_grouped(w.handle, _dptr(codes), _dptr(scales_sf), _dptr(expert_offsets), M_total,
+                                    _dptr(out), out.stride(0) if M_total else w.N, y_dtype, _stream_ptr(stream)),
+           "prq_linear_grouped")
+    return out
+
+
+def forward_host_scratch_bytes(w: Weights, M: int) -> int:
+    return int(lib().prq_forward_host_scratch_bytes(w.handle, M))
+
+
+def forward_host(w: Weights, x_host, y_host, mode: int, scratch, y_dtype: int = F32, stream=None):
+    """x_host / y_host: pinned torch CPU tensors (bf16 M x K, fp32 or bf16 M x N); scratch: CUDA uint8 tensor."""
+    M = x_host.shape[0]
+    _check(lib().prq_forward_host(w.handle, mode, _dptr(x_host), M, _dptr(y_host), y_dtype, _dptr(scratch),
+                                  scratch.numel(), _stream_ptr(stream)), "prq_forward_host")
+
+
+def last_device_status(stream=None) -> int:
+    return int(lib().prq_last_device_status(_stream_ptr(stream)))
+
+
+def kernel_launch_count() -> int:
+    return int(lib().prq_kernel_launch_count())

@@ -1,0 +1,582 @@
+// C-ABI entry points of libprq: argument checks, the weight handle, tensor-map construction,
+// kernel selection.  See include/prq.h for the contract of every call.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <thread>
+#include <vector>
+
+#include "prq_internal.h"
+#include "prq_kernels.h"
+
+namespace prq {
+namespace {
+
+__device__ int g_device_status = 0;
+
+std::atomic<unsigned long long> g_launches{0};
+
+struct DeviceInfo {
+    bool ok = false;
+    int num_sms = 0;
+    int* status_ptr = nullptr;
+};
+std::mutex g_dev_mutex;
+DeviceInfo g_dev[64];
+
+// Per-device facts, looked up once: sm_100 check, SM count, address of the status word.
+prq_status device_info(int dev, DeviceInfo** out) {
+    if (dev < 0 || dev >= 64) return PRQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    DeviceInfo& d = g_dev[dev];
+    if (!d.ok) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return PRQ_ERR_CUDA;
+        if (prop.major != 10) return PRQ_ERR_UNSUPPORTED_ARCH;
+        d.num_sms = prop.multiProcessorCount;
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return PRQ_ERR_CUDA;
+        d.status_ptr = static_cast<int*>(p);
+        d.ok = true;
+    }
+    *out = &d;
+    return PRQ_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// Packed E2M1 codes are plain bytes: a row-major (rows x row_bytes) byte matrix, boxes of 128 bytes
+// (256 codes, one swizzle row) x box_rows rows, 128-byte swizzle, zero fill outside the matrix.
+prq_status make_code_map(CUtensorMap* map, const void* base, uint64_t row_bytes, uint64_t rows, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return PRQ_ERR_CUDA;
+    cuuint64_t dims[2] = {row_bytes, rows};
+    cuuint64_t strides[1] = {row_bytes};
+    cuuint32_t box[2] = {128, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
+int env_int(const char* name, int dflt) {
+    const char* v = std::getenv(name);
+    return v && *v ? std::atoi(v) : dflt;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int dense_groups(int M) { return (M + kGroupRows - 1) / kGroupRows; }
+int grouped_groups(int M, int n_groups) { return (M + kGroupRows - 1) / kGroupRows + n_groups; }
+
+int decode_bn(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
+
+int decode_splits(const prq_weights* w, int M, int num_sms) {
+    const int n_tiles = (w->N + 127) / 128;
+    const int ctas_per_sm = decode_bn(M) <= 32 ? 2 : 1;
+    int splits = env_int("PRQ_DECODE_SPLITS", 0);
+    if (splits <= 0) splits = std::max(1, (num_sms * ctas_per_sm) / n_tiles);
+    splits = std::min(splits, std::min(w->plan.S, 64));
+    return std::max(1, splits);
+}
+
+int prefill_bn(const prq_weights* w, int M, int num_sms) {
+    int forced = env_int("PRQ_PREFILL_BN", 0);
+    if (forced) return forced;
+    const int cand[4] = {256, 192, 160, 128};
+    const long m_tiles = (M + 127) / 128;
+    long best_cost = -1;
+    int best = 256;
+    for (int bn : cand) {
+        const long units = m_tiles * ((w->N + bn - 1) / bn);
+        const long waves = (units + num_sms - 1) / num_sms;
+        const long cost = waves * bn;  // MMA time per tile is proportional to bn
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
+    }
+    return best;
+}
+
+constexpr size_t kCounterBytes = 4096;  // 1024 tile counters
+
+}  // namespace
+}  // namespace prq
+
+using namespace prq;
+
+extern "C" {
+
+const char* prq_status_string(prq_status s) {
+    switch (s) {
+        case PRQ_OK: return "ok";
+        case PRQ_ERR_INVALID_ARG: return "invalid argument";
+        case PRQ_ERR_ALIGNMENT: return "misaligned pointer or stride";
+        case PRQ_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+        case PRQ_ERR_CUDA: return "CUDA runtime error";
+        case PRQ_ERR_OOM: return "out of memory";
+        case PRQ_ERR_TIMEOUT: return "a device-side wait expired";
+        case PRQ_ERR_NONFINITE: return "non-finite input";
+        case PRQ_ERR_WORKSPACE: return "workspace too small";
+    }
+    return "unknown status";
+}
+
+unsigned long long prq_kernel_launch_count(void) { return g_launches.load(); }
+
+prq_status prq_last_device_status(prq_stream_t stream) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PRQ_ERR_CUDA;
+    DeviceInfo* di;
+    prq_status st = device_info(dev, &di);
+    if (st != PRQ_OK) return st;
+    if (cudaStreamSynchronize(static_cast<cudaStream_t>(stream)) != cudaSuccess) return PRQ_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, di->status_ptr, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return PRQ_ERR_CUDA;
+    if (v != 0) {
+        int zero = 0;
+        cudaMemcpy(di->status_ptr, &zero, sizeof(int), cudaMemcpyHostToDevice);
+    }
+    return static_cast<prq_status>(v);
+}
+
+void prq_weights_free(prq_weights* w) {
+    if (!w) return;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (w->device >= 0 && w->device != cur) cudaSetDevice(w->device);
+    cudaFree(w->d_codes);
+    cudaFree(w->d_sf);
+    cudaFree(w->d_perm);
+    cudaFree(w->d_inv_s_perm);
+    if (w->device >= 0 && w->device != cur) cudaSetDevice(cur);
+    delete w;
+}
+
+prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, const float* act_amax, float alpha,
+                               int k_tail, prq_weights** out) {
+    if (!W || !act_amax || !out) return PRQ_ERR_INVALID_ARG;
+    if (n_experts < 1 || n_experts > kMaxExperts || N < 1 || K < kBlock) return PRQ_ERR_INVALID_ARG;
+    if (K % kBlock || k_tail % kBlock || k_tail < 0 || k_tail > K) return PRQ_ERR_INVALID_ARG;
+    if (!std::isfinite(alpha)) return PRQ_ERR_INVALID_ARG;
+    if (static_cast<long long>(n_experts) * N > 0x7fffffffll) return PRQ_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PRQ_ERR_CUDA;
+    DeviceInfo* di;
+    prq_status st = device_info(dev, &di);
+    if (st != PRQ_OK) return st;
+
+    prq_weights* w = new (std::nothrow) prq_weights;
+    if (!w) return PRQ_ERR_OOM;
+    w->n_experts = n_experts; w->N = N; w->K = K; w->k_tail = k_tail; w->alpha = alpha;
+    w->plan = StagePlan(K, k_tail);
+    w->w_groups = (N + kGroupRows - 1) / kGroupRows;
+    w->device = dev;
+    const size_t Ka = static_cast<size_t>(K) + k_tail;
+    const size_t E = n_experts;
+    try {
+        w->h_codes.resize(E * N * Ka / 2);
+        w->h_scales.resize(E * N * Ka / kBlock);
+        w->h_perm.resize(E * K);
+        w->h_s.resize(E * K);
+        w->h_inv_s.resize(E * K);
+        w->h_col_err.resize(E * K);
+        const int S = w->plan.S, S1 = w->plan.S1, nb = kStageK / kBlock;
+        // scale bytes in stage order, padded by a few groups so that a tile's bulk copy never runs off the end
+        w->d_sf_bytes = (E * S * w->w_groups + 4) * kSfGroupBytes;
+        std::vector<uint8_t> sf(w->d_sf_bytes, 0);
+        std::vector<float> inv_s_perm(E * K);
+        PrepResult r;
+        for (size_t e = 0; e < E; ++e) {
+            st = prepare_layer(W + e * N * K, N, K, act_amax + e * K, alpha, k_tail, r);
+            if (st != PRQ_OK) { delete w; return st; }
+            std::memcpy(&w->h_codes[e * N * Ka / 2], r.codes.data(), r.codes.size());
+            std::memcpy(&w->h_scales[e * N * Ka / kBlock], r.scales.data(), r.scales.size());
+            std::memcpy(&w->h_perm[e * K], r.perm.data(), sizeof(int32_t) * K);
+            std::memcpy(&w->h_s[e * K], r.s.data(), sizeof(float) * K);
+            std::memcpy(&w->h_inv_s[e * K], r.inv_s.data(), sizeof(float) * K);
+            std::memcpy(&w->h_col_err[e * K], r.col_err.data(), sizeof(double) * K);
+            for (int j = 0; j < K; ++j) inv_s_perm[e * K + j] = r.inv_s[r.perm[j]];
+            const int nblk_main = K / kBlock, nblk = static_cast<int>(Ka / kBlock);
+            for (int n = 0; n < N; ++n) {
+                const uint8_t* srow = &r.scales[static_cast<size_t>(n) * nblk];
+                const int g = n / kGroupRows, rr = n % kGroupRows;
+                for (int b = 0; b < nblk; ++b) {
+                    const int stage = b < nblk_main ? b / nb : S1 + (b - nblk_main) / nb;
+                    const int bis = b < nblk_main ? b % nb : (b - nblk_main) % nb;
+                    sf[((e * S + stage) * w->w_groups + g) * kSfGroupBytes + sf_offset_in_group(rr, bis)] = srow[b];
+                }
+            }
+        }
+        w->d_codes_bytes = w->h_codes.size() + 256;
+        if (cudaMalloc(&w->d_codes, w->d_codes_bytes) != cudaSuccess || cudaMalloc(&w->d_sf, w->d_sf_bytes) != cudaSuccess ||
+            cudaMalloc(&w->d_perm, sizeof(int32_t) * E * K) != cudaSuccess ||
+            cudaMalloc(&w->d_inv_s_perm, sizeof(float) * E * K) != cudaSuccess) {
+            cudaGetLastError();
+            prq_weights_free(w);
+            return PRQ_ERR_OOM;
+        }
+        bool ok = cudaMemcpy(w->d_codes, w->h_codes.data(), w->h_codes.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(w->d_sf, sf.data(), sf.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(w->d_perm, w->h_perm.data(), sizeof(int32_t) * E * K, cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(w->d_inv_s_perm, inv_s_perm.data(), sizeof(float) * E * K, cudaMemcpyHostToDevice) == cudaSuccess;
+        if (!ok) { prq_weights_free(w); return PRQ_ERR_CUDA; }
+    } catch (const std::bad_alloc&) {
+        prq_weights_free(w);
+        return PRQ_ERR_OOM;
+    }
+    *out = w;
+    return PRQ_OK;
+}
+
+prq_status prq_prepare_weights_search(const uint16_t* W, int N, int K, const uint16_t* Zcal, int T, const float* alphas,
+                                      int n_alphas, int k_tail, prq_weights** out, float* alpha_star, double* nrmse) {
+    if (!W || !Zcal || !alphas || !out || !alpha_star || T < 1 || n_alphas < 1) return PRQ_ERR_INVALID_ARG;
+    if (N < 1 || K < kBlock || K % kBlock || k_tail % kBlock || k_tail < 0 || k_tail > K) return PRQ_ERR_INVALID_ARG;
+    auto bf = [](uint16_t h) { uint32_t u = static_cast<uint32_t>(h) << 16; float f; std::memcpy(&f, &u, 4); return f; };
+    // step 1: per-channel maxima of the calibration activations
+    std::vector<float> amax(K, 0.f);
+    for (int t = 0; t < T; ++t)
+        for (int j = 0; j < K; ++j) amax[j] = std::max(amax[j], std::fabs(bf(Zcal[static_cast<size_t>(t) * K + j])));
+    // the target Z W^T in double, rows split over host threads
+    std::vector<double> yref(static_cast<size_t>(T) * N);
+    {
+        std::vector<double> Wd(static_cast<size_t>(N) * K);
+        for (size_t i = 0; i < Wd.size(); ++i) Wd[i] = bf(W[i]);
+        unsigned nt = std::max(1u, std::min(std::thread::hardware_concurrency(), 64u));
+        std::vector<std::thread> th;
+        for (unsigned ti = 0; ti < nt; ++ti)
+            th.emplace_back([&, ti] {
+                std::vector<double> z(K);
+                for (int t = ti; t < T; t += nt) {
+                    for (int j = 0; j < K; ++j) z[j] = bf(Zcal[static_cast<size_t>(t) * K + j]);
+                    for (int n = 0; n < N; ++n) {
+                        const double* wr = &Wd[static_cast<size_t>(n) * K];
+                        double acc = 0.0;
+                        for (int j = 0; j < K; ++j) acc += z[j] * wr[j];
+                        yref[static_cast<size_t>(t) * N + n] = acc;
+                    }
+                }
+            });
+        for (auto& x : th) x.join();
+    }
+    double ref_norm2 = 0.0;
+    for (double v : yref) ref_norm2 += v * v;
+
+    const size_t x_bytes = static_cast<size_t>(T) * K * 2;
+    const size_t c_bytes = prq_act_bytes(T, K, k_tail, 1, PRQ_BUF_CODES);
+    const size_t sf_bytes = prq_act_bytes(T, K, k_tail, 1, PRQ_BUF_SCALES_SF);
+    const size_t y_bytes = static_cast<size_t>(T) * N * 4;
+    void *dx = nullptr, *dc = nullptr, *dsf = nullptr, *dy = nullptr, *dws = nullptr;
+    size_t ws_bytes = 0;
+    std::vector<float> y(static_cast<size_t>(T) * N);
+    prq_weights* best = nullptr;
+    double best_err = 0.0;
+    prq_status st = PRQ_OK;
+    for (int a = 0; a < n_alphas && st == PRQ_OK; ++a) {
+        prq_weights* w = nullptr;
+        st = prq_prepare_weights(W, 1, N, K, amax.data(), alphas[a], k_tail, &w);
+        if (st != PRQ_OK) break;
+        if (!dx) {
+            ws_bytes = prq_linear_workspace_bytes(w, T);
+            bool ok = cudaMalloc(&dx, x_bytes) == cudaSuccess && cudaMalloc(&dc, c_bytes) == cudaSuccess &&
+                      cudaMalloc(&dsf, sf_bytes) == cudaSuccess && cudaMalloc(&dy, y_bytes) == cudaSuccess &&
+                      cudaMalloc(&dws, ws_bytes) == cudaSuccess;
+            ok = ok && cudaMemset(dws, 0, ws_bytes) == cudaSuccess;
+            ok = ok && cudaMemcpy(dx, Zcal, x_bytes, cudaMemcpyHostToDevice) == cudaSuccess;
+            if (!ok) { cudaGetLastError(); prq_weights_free(w); st = PRQ_ERR_OOM; break; }
+        }
+        st = prq_quantize_act(w, PRQ_ACT_SCALE_PERM, dx, T, K, nullptr, dc, nullptr, dsf, nullptr);
+        if (st == PRQ_OK) st = prq_linear(w, dc, dsf, T, dy, N, PRQ_F32, dws, ws_bytes, nullptr);
+        if (st == PRQ_OK) st = prq_last_device_status(nullptr);
+        if (st == PRQ_OK && cudaMemcpy(y.data(), dy, y_bytes, cudaMemcpyDeviceToHost) != cudaSuccess) st = PRQ_ERR_CUDA;
+        if (st != PRQ_OK) { prq_weights_free(w); break; }
+        double d2 = 0.0;
+        for (size_t i = 0; i < y.size(); ++i) { const double d = static_cast<double>(y[i]) - yref[i]; d2 += d * d; }
+        const double err = std::sqrt(d2 / ref_norm2);
+        if (nrmse) nrmse[a] = err;
+        if (!best || err < best_err) {
+            prq_weights_free(best);
+            best = w; best_err = err; *alpha_star = alphas[a];
+        } else {
+            prq_weights_free(w);
+        }
+    }
+    cudaFree(dx); cudaFree(dc); cudaFree(dsf); cudaFree(dy); cudaFree(dws);
+    if (st != PRQ_OK) { prq_weights_free(best); return st; }
+    *out = best;
+    return PRQ_OK;
+}
+
+prq_status prq_prepare_weights_host(const uint16_t* W, int N, int K, const float* act_amax, float alpha, int k_tail,
+                                    uint8_t* codes, uint8_t* scales, int32_t* perm, float* s_out, float* inv_s_out,
+                                    double* col_err) {
+    if (!W || !act_amax || !codes || !scales || !perm) return PRQ_ERR_INVALID_ARG;
+    if (N < 1 || K < kBlock || K % kBlock || k_tail % kBlock || k_tail < 0 || k_tail > K) return PRQ_ERR_INVALID_ARG;
+    if (!std::isfinite(alpha)) return PRQ_ERR_INVALID_ARG;
+    PrepResult r;
+    try {
+        prq_status st = prepare_layer(W, N, K, act_amax, alpha, k_tail, r);
+        if (st != PRQ_OK) return st;
+    } catch (const std::bad_alloc&) {
+        return PRQ_ERR_OOM;
+    }
+    std::memcpy(codes, r.codes.data(), r.codes.size());
+    std::memcpy(scales, r.scales.data(), r.scales.size());
+    std::memcpy(perm, r.perm.data(), sizeof(int32_t) * K);
+    if (s_out) std::memcpy(s_out, r.s.data(), sizeof(float) * K);
+    if (inv_s_out) std::memcpy(inv_s_out, r.inv_s.data(), sizeof(float) * K);
+    if (col_err) std::memcpy(col_err, r.col_err.data(), sizeof(double) * K);
+    return PRQ_OK;
+}
+
+prq_status prq_weights_info(const prq_weights* w, int* n_experts, int* N, int* K, int* k_tail, float* alpha) {
+    if (!w) return PRQ_ERR_INVALID_ARG;
+    if (n_experts) *n_experts = w->n_experts;
+    if (N) *N = w->N;
+    if (K) *K = w->K;
+    if (k_tail) *k_tail = w->k_tail;
+    if (alpha) *alpha = w->alpha;
+    return PRQ_OK;
+}
+
+prq_status prq_weights_get(const prq_weights* w, int expert, prq_field which, void* dst, size_t dst_bytes) {
+    if (!w || !dst || expert < 0 || expert >= w->n_experts) return PRQ_ERR_INVALID_ARG;
+    const size_t Ka = static_cast<size_t>(w->K) + w->k_tail, N = w->N, K = w->K, e = expert;
+    const void* src = nullptr;
+    size_t bytes = 0;
+    switch (which) {
+        case PRQ_FIELD_CODES: bytes = N * Ka / 2; src = &w->h_codes[e * bytes]; break;
+        case PRQ_FIELD_SCALES: bytes = N * Ka / kBlock; src = &w->h_scales[e * bytes]; break;
+        case PRQ_FIELD_PERM: bytes = K * sizeof(int32_t); src = &w->h_perm[e * K]; break;
+        case PRQ_FIELD_TOPK: bytes = w->k_tail * sizeof(int32_t); src = w->h_perm.data() + e * K + (K - w->k_tail); break;
+        case PRQ_FIELD_S: bytes = K * sizeof(float); src = &w->h_s[e * K]; break;
+        case PRQ_FIELD_INV_S: bytes = K * sizeof(float); src = &w->h_inv_s[e * K]; break;
+        case PRQ_FIELD_COL_ERR: bytes = K * sizeof(double); src = &w->h_col_err[e * K]; break;
+        default: return PRQ_ERR_INVALID_ARG;
+    }
+    if (dst_bytes != bytes) return PRQ_ERR_INVALID_ARG;
+    if (bytes) std::memcpy(dst, src, bytes);
+    return PRQ_OK;
+}
+
+size_t prq_act_bytes(int M, int K, int k_tail, int n_groups, prq_buf which) {
+    if (M < 0 || K < kBlock || K % kBlock || k_tail % kBlock || k_tail < 0 || k_tail > K || n_groups < 1) return 0;
+    const StagePlan plan(K, k_tail);
+    switch (which) {
+        case PRQ_BUF_CODES: return static_cast<size_t>(M) * K / 2;
+        case PRQ_BUF_SCALES_ROW: return static_cast<size_t>(M) * K / kBlock;
+        case PRQ_BUF_SCALES_SF: {
+            const int groups = n_groups == 1 ? dense_groups(M) : grouped_groups(M, n_groups);
+            return static_cast<size_t>(plan.S) * std::max(groups, 1) * kSfGroupBytes;
+        }
+    }
+    return 0;
+}
+
+prq_status prq_quantize_act(const prq_weights* w, prq_act_mode mode, const void* x, int M, int ldx,
+                            const int32_t* expert_offsets, void* codes, void* scales_row, void* scales_sf,
+                            prq_stream_t stream) {
+    if (!w || M < 0) return PRQ_ERR_INVALID_ARG;
+    if (mode != PRQ_ACT_IDENTITY && mode != PRQ_ACT_SCALE_PERM) return PRQ_ERR_INVALID_ARG;
+    if (M == 0) return PRQ_OK;
+    if (!x || !codes || !scales_sf || ldx < w->K) return PRQ_ERR_INVALID_ARG;
+    if ((w->n_experts > 1) != (expert_offsets != nullptr)) return PRQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(codes) || !aligned16(scales_sf) || ldx % 8) return PRQ_ERR_ALIGNMENT;
+    QuantParams p;
+    p.x = static_cast<const uint16_t*>(x);
+    p.M = M; p.ldx = ldx; p.K = w->K; p.k_tail = w->k_tail;
+    p.n_experts = w->n_experts;
+    p.expert_offsets = expert_offsets;
+    p.act_groups = expert_offsets ? grouped_groups(M, w->n_experts) : dense_groups(M);
+    p.perm = w->d_perm;
+    p.inv_s_perm = w->d_inv_s_perm;
+    p.codes = static_cast<uint8_t*>(codes);
+    p.scales_row = static_cast<uint8_t*>(scales_row);
+    p.scales_sf = static_cast<uint8_t*>(scales_sf);
+    cudaError_t e = launch_quant_act(p, mode == PRQ_ACT_SCALE_PERM, p.act_groups, static_cast<cudaStream_t>(stream));
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
+size_t prq_linear_workspace_bytes(const prq_weights* w, int M) {
+    if (!w || M < 0) return 0;
+    if (M > 128) return kCounterBytes;
+    // decode: counters + the largest split count this layer can use x token tile x padded N
+    const size_t n_pad = static_cast<size_t>((w->N + 127) / 128) * 128;
+    const size_t splits = std::min(w->plan.S, 64);
+    return kCounterBytes + splits * decode_bn(M) * n_pad * sizeof(float);
+}
+
+static prq_status check_linear_common(const prq_weights* w, const void* codes, const void* scales_sf, void* y, int ldy,
+                                      prq_dtype y_dtype) {
+    if (!w || !codes || !scales_sf || !y) return PRQ_ERR_INVALID_ARG;
+    if (y_dtype != PRQ_F32 && y_dtype != PRQ_BF16) return PRQ_ERR_INVALID_ARG;
+    if (ldy < w->N) return PRQ_ERR_INVALID_ARG;
+    if (!aligned16(codes) || !aligned16(scales_sf) || !aligned16(y)) return PRQ_ERR_ALIGNMENT;
+    if (ldy % (y_dtype == PRQ_F32 ? 4 : 8)) return PRQ_ERR_ALIGNMENT;
+    return PRQ_OK;
+}
+
+prq_status prq_linear(const prq_weights* w, const void* codes, const void* scales_sf, int M, void* y, int ldy,
+                      prq_dtype y_dtype, void* workspace, size_t workspace_bytes, prq_stream_t stream) {
+    if (w && M == 0) return PRQ_OK;
+    prq_status st = check_linear_common(w, codes, scales_sf, y, ldy, y_dtype);
+    if (st != PRQ_OK) return st;
+    if (M < 0 || w->n_experts != 1) return PRQ_ERR_INVALID_ARG;
+    DeviceInfo* di;
+    st = device_info(w->device, &di);
+    if (st != PRQ_OK) return st;
+    const size_t Ka = static_cast<size_t>(w->K) + w->k_tail;
+
+    GemmParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = M; p.N = w->N; p.K = w->K; p.k_tail = w->k_tail;
+    p.n_experts = 1;
+    p.act_groups = dense_groups(M);
+    p.w_groups = w->w_groups;
+    p.act_sf = static_cast<const uint8_t*>(scales_sf);
+    p.w_sf = w->d_sf;
+    p.y = y; p.ldy = ldy; p.y_bf16 = y_dtype == PRQ_BF16;
+    p.status = di->status_ptr;
+    p.splits = 1;
+
+    CUtensorMap tm_act, tm_w;
+    GemmKind kind;
+    int bn, grid;
+    if (M <= 128) {
+        kind = GemmKind::kDecode;
+        bn = decode_bn(M);
+        p.splits = decode_splits(w, M, di->num_sms);
+        const size_t n_pad = static_cast<size_t>((w->N + 127) / 128) * 128;
+        if (p.splits > 1) {
+            const size_t need = kCounterBytes + static_cast<size_t>(p.splits) * bn * n_pad * sizeof(float);
+            if (!workspace || workspace_bytes < need) return PRQ_ERR_WORKSPACE;
+            if (!aligned16(workspace)) return PRQ_ERR_ALIGNMENT;
+            if ((w->N + 127) / 128 > static_cast<int>(kCounterBytes / sizeof(int))) return PRQ_ERR_INVALID_ARG;
+            p.counters = static_cast<int*>(workspace);
+            p.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kCounterBytes);
+        }
+        grid = ((w->N + 127) / 128) * p.splits;
+        st = make_code_map(&tm_act, codes, w->K / 2, M, bn);
+        if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, 128);
+    } else {
+        kind = GemmKind::kPrefill;
+        bn = prefill_bn(w, M, di->num_sms);
+        const long units = static_cast<long>((M + 127) / 128) * ((w->N + bn - 1) / bn);
+        grid = static_cast<int>(std::min<long>(units, di->num_sms));
+        st = make_code_map(&tm_act, codes, w->K / 2, M, 128);
+        if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, bn);
+    }
+    if (st != PRQ_OK) return st;
+    bool unsupported = false;
+    cudaError_t e = launch_gemm(kind, bn, tm_act, tm_w, p, grid, static_cast<cudaStream_t>(stream), &unsupported);
+    if (unsupported) return PRQ_ERR_INVALID_ARG;
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
+prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const void* scales_sf,
+                              const int32_t* expert_offsets, int M_total, void* y, int ldy, prq_dtype y_dtype,
+                              prq_stream_t stream) {
+    if (w && M_total == 0) return PRQ_OK;
+    prq_status st = check_linear_common(w, codes, scales_sf, y, ldy, y_dtype);
+    if (st != PRQ_OK) return st;
+    if (M_total < 0 || !expert_offsets) return PRQ_ERR_INVALID_ARG;
+    DeviceInfo* di;
+    st = device_info(w->device, &di);
+    if (st != PRQ_OK) return st;
+    const size_t Ka = static_cast<size_t>(w->K) + w->k_tail;
+
+    GemmParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.M = M_total; p.N = w->N; p.K = w->K; p.k_tail = w->k_tail;
+    p.n_experts = w->n_experts;
+    p.act_groups = grouped_groups(M_total, w->n_experts);
+    p.w_groups = w->w_groups;
+    p.act_sf = static_cast<const uint8_t*>(scales_sf);
+    p.w_sf = w->d_sf;
+    p.expert_offsets = expert_offsets;
+    p.y = y; p.ldy = ldy; p.y_bf16 = y_dtype == PRQ_BF16;
+    p.status = di->status_ptr;
+    p.splits = 1;
+    int bn = env_int("PRQ_GROUPED_BN", 0);
+    if (!bn) bn = (M_total >= 8192 && w->N % 256 == 0) ? 256 : 128;
+    CUtensorMap tm_act, tm_w;
+    st = make_code_map(&tm_act, codes, w->K / 2, M_total, 128);
+    if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, static_cast<uint64_t>(w->n_experts) * w->N, bn);
+    if (st != PRQ_OK) return st;
+    bool unsupported = false;
+    cudaError_t e = launch_gemm(GemmKind::kGrouped, bn, tm_act, tm_w, p, di->num_sms, static_cast<cudaStream_t>(stream),
+                                &unsupported);
+    if (unsupported) return PRQ_ERR_INVALID_ARG;
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
+// Device scratch layout of prq_forward_host: [workspace | x | codes | scales_sf | y], each 256-byte aligned.
+namespace {
+size_t align256(size_t v) { return (v + 255) & ~static_cast<size_t>(255); }
+struct HostFwdLayout {
+    size_t ws, x, codes, sf, y, total;
+};
+HostFwdLayout host_fwd_layout(const prq_weights* w, int M) {
+    HostFwdLayout l;
+    l.ws = 0;
+    l.x = align256(prq_linear_workspace_bytes(w, M));
+    l.codes = l.x + align256(static_cast<size_t>(M) * w->K * 2);
+    l.sf = l.codes + align256(prq_act_bytes(M, w->K, w->k_tail, 1, PRQ_BUF_CODES));
+    l.y = l.sf + align256(prq_act_bytes(M, w->K, w->k_tail, 1, PRQ_BUF_SCALES_SF));
+    l.total = l.y + align256(static_cast<size_t>(M) * w->N * 4);
+    return l;
+}
+}  // namespace
+
+size_t prq_forward_host_scratch_bytes(const prq_weights* w, int M) {
+    if (!w || M < 0 || w->n_experts != 1) return 0;
+    return host_fwd_layout(w, M).total;
+}
+
+prq_status prq_forward_host(const prq_weights* w, prq_act_mode mode, const uint16_t* x_host, int M, void* y_host,
+                            prq_dtype y_dtype, void* dev_scratch, size_t scratch_bytes, prq_stream_t stream) {
+    if (!w || w->n_experts != 1 || M < 0) return PRQ_ERR_INVALID_ARG;
+    if (M == 0) return PRQ_OK;
+    if (!x_host || !y_host || !dev_scratch) return PRQ_ERR_INVALID_ARG;
+    if (y_dtype != PRQ_F32 && y_dtype != PRQ_BF16) return PRQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(dev_scratch) & 255) return PRQ_ERR_ALIGNMENT;
+    const HostFwdLayout l = host_fwd_layout(w, M);
+    if (scratch_bytes < l.total) return PRQ_ERR_WORKSPACE;
+    uint8_t* base = static_cast<uint8_t*>(dev_scratch);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t x_bytes = static_cast<size_t>(M) * w->K * 2;
+    if (cudaMemcpyAsync(base + l.x, x_host, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return PRQ_ERR_CUDA;
+    prq_status st = prq_quantize_act(w, mode, base + l.x, M, w->K, nullptr, base + l.codes, nullptr, base + l.sf, stream);
+    if (st != PRQ_OK) return st;
+    st = prq_linear(w, base + l.codes, base + l.sf, M, base + l.y, w->N, y_dtype, base + l.ws, l.x, stream);
+    if (st != PRQ_OK) return st;
+    const size_t y_bytes = static_cast<size_t>(M) * w->N * (y_dtype == PRQ_F32 ? 4 : 2);
+    if (cudaMemcpyAsync(y_host, base + l.y, y_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return PRQ_ERR_CUDA;
+    return PRQ_OK;
+}
+
+}  // extern "C"

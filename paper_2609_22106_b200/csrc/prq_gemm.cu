@@ -1,0 +1,458 @@
+// Block-scaled FP4 GEMM over the augmented reduction K + k (Eq. (3)):
+//     y[t, n] = sum_b 2^(ea[t,b] + ew[n,b] - 254) * sum_{i<32} a[t, 32 b + i] * w[n, 32 b + i]
+// with a = E2M1 codes of [Q(x) | Q(x)_tail] and w = E2M1 codes of [Q(W D P) | Q(R)].
+//
+// sm_100a design.  One CTA per SM, 6 warps:
+//   warp 0  producer: per 256-element reduction stage, one TMA tile load per operand (128-byte rows,
+//           128B swizzle) and one flat bulk copy per operand for the stage's scale bytes, all landing
+//           on the stage's "full" mbarrier;
+//   warp 1  MMA issuer: copies the stage's scale atoms shared -> tensor memory (tcgen05.cp), then issues
+//           up to four K = 64 tcgen05.mma.kind::mxf4.block_scale steps into a tensor-memory accumulator
+//           and commits to the stage's "empty" mbarrier; after the last stage commits "accumulator full";
+//   warps 2-5 epilogue: tcgen05.ld of their 32-lane quarter, store to y, release the accumulator.
+// The augmented activation is never materialised: in the residual stages the activation tile is loaded
+// again from column K - k while the weight tile continues at column K ("reuses the quantized
+// representation of the tail", Kernel design paragraph); only the tail's scale bytes were duplicated.
+//
+// Operand roles.  "P" is the operand on the MMA M axis (always 128 rows), "Q" the operand on the MMA N
+// axis (BN rows).  Prefill / grouped: P = activation tokens, Q = weight rows.  Decode (M <= 128): P =
+// weight rows, Q = tokens, and the reduction is split over CTAs so that all SMs stream weights; the
+// partial sums meet in a workspace and the last CTA of a tile adds them in a fixed order.
+//
+// Every wait is bounded; on expiry the CTA raises an abort flag, all roles unwind, tensor memory is
+// freed and PRQ_ERR_TIMEOUT is recorded in the device status word.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "prq_kernels.h"
+#include "prq_ptx.cuh"
+
+namespace prq {
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kPTileBytes = 128 * 128;
+constexpr int kKindPrefill = 0, kKindDecode = 1, kKindGrouped = 2;
+
+constexpr int cgcd(int a, int b) { return b == 0 ? a : cgcd(b, a % b); }
+constexpr int cmin(int a, int b) { return a < b ? a : b; }
+constexpr int cmax(int a, int b) { return a > b ? a : b; }
+constexpr int pow2_at_least(int x) { int p = 32; while (p < x) p *= 2; return p; }
+
+template <int BN, int KIND>
+struct Cfg {
+    static constexpr bool kSwap = KIND == kKindDecode;
+    // 128-row scale groups a Q tile can touch (its first row is a multiple of gcd(BN, 128))
+    static constexpr int kNgq = kSwap ? 1 : (128 - cgcd(BN, 128) + BN + 127) / 128;
+    static constexpr int kQTileBytes = BN * 128;
+    static constexpr int kSfpBytes = kSfGroupBytes;
+    static constexpr int kSfqBytes = kNgq * kSfGroupBytes;
+    static constexpr int kStageBytes = kPTileBytes + kQTileBytes + kSfpBytes + kSfqBytes;
+    static constexpr int kStages = cmin(8, (232448 - 1024 - 8192) / kStageBytes);
+    // tensor memory columns: accumulators first, then scale words
+    static constexpr int kAccStride = cmax(BN, 32);
+    static constexpr int kSfpCols = 8;              // 2 atoms x 4 columns
+    static constexpr int kSfqCols = 8 * kNgq;       // 2 atoms x 4 columns x groups
+    static constexpr int kSfCols = kSfpCols + 4 + kSfqCols;  // 4 spare columns absorb the group shift
+    static constexpr int kAcc = (!kSwap && 2 * kAccStride + kSfCols <= 512) ? 2 : 1;
+    static constexpr int kTmemCols = pow2_at_least(kAcc * kAccStride + kSfCols);
+    static constexpr int kSfpCol = kAcc * kAccStride;
+    static constexpr int kSfqCol = kSfpCol + kSfpCols + 4;
+    static constexpr uint32_t kTxBytes = kStageBytes;
+    static_assert(kStages >= 2, "tile too large for shared memory");
+    static_assert(kTmemCols <= 512, "tile too large for tensor memory");
+    static_assert(BN % 16 == 0 && BN >= 16 && BN <= 256, "MMA N must be a multiple of 16 in [16, 256]");
+};
+
+struct Unit {
+    int p_row, q_row;            // first row of each operand tile in its code tensor
+    const uint8_t* sfp;          // stage-0 scale tile of P; advance by sfp_stride per stage
+    const uint8_t* sfq;
+    size_t sfp_stride, sfq_stride;
+    int sfq_shift;               // 32-row chunks to drop in front of the first Q scale group
+    int s_begin, s_end;          // reduction stages of this unit
+    int row0, row_end;           // token rows covered / first row past the valid ones
+    int n0;                      // first output feature
+    int tile, split;             // decode bookkeeping
+};
+
+template <int BN, int KIND>
+__device__ __forceinline__ int unit_count(const GemmParams& p, const int* tile_start) {
+    if (KIND == kKindPrefill) return ((p.M + 127) / 128) * ((p.N + BN - 1) / BN);
+    if (KIND == kKindDecode) return ((p.N + 127) / 128) * p.splits;
+    return tile_start[p.n_experts] * ((p.N + BN - 1) / BN);
+}
+
+template <int BN, int KIND>
+__device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_start, int u, int S) {
+    Unit t;
+    if (KIND == kKindPrefill) {
+        const int m_tiles = (p.M + 127) / 128;
+        const int mi = u % m_tiles, ni = u / m_tiles;
+        t.p_row = mi * 128;
+        t.q_row = ni * BN;
+        t.sfp = p.act_sf + static_cast<size_t>(mi) * kSfGroupBytes;
+        t.sfp_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
+        t.sfq = p.w_sf + static_cast<size_t>((ni * BN) / 128) * kSfGroupBytes;
+        t.sfq_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
+        t.sfq_shift = ((ni * BN) / 32) & 3;
+        t.s_begin = 0; t.s_end = S;
+        t.row0 = mi * 128; t.row_end = min(p.M, t.row0 + 128);
+        t.n0 = ni * BN;
+        t.tile = u; t.split = 0;
+    } else if (KIND == kKindDecode) {
+        const int ni = u / p.splits, sp = u % p.splits;
+        t.p_row = ni * 128;
+        t.q_row = 0;
+        t.sfp = p.w_sf + static_cast<size_t>(ni) * kSfGroupBytes;
+        t.sfp_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
+        t.sfq = p.act_sf;
+        t.sfq_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
+        t.sfq_shift = 0;
+        t.s_begin = static_cast<int>(static_cast<long long>(S) * sp / p.splits);
+        t.s_end = static_cast<int>(static_cast<long long>(S) * (sp + 1) / p.splits);
+        t.row0 = 0; t.row_end = p.M;
+        t.n0 = ni * 128;
+        t.tile = ni; t.split = sp;
+    } else {
+        const int total_mt = tile_start[p.n_experts];
+        const int mt = u % total_mt, ni = u / total_mt;
+        int lo = 0, hi = p.n_experts - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (tile_start[mid] <= mt) lo = mid; else hi = mid - 1;
+        }
+        const int e = lo;
+        t.p_row = p.expert_offsets[e] + (mt - tile_start[e]) * 128;
+        t.q_row = e * p.N + ni * BN;
+        t.sfp = p.act_sf + static_cast<size_t>(mt) * kSfGroupBytes;
+        t.sfp_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
+        t.sfq = p.w_sf + (static_cast<size_t>(e) * S * p.w_groups + (ni * BN) / 128) * kSfGroupBytes;
+        t.sfq_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
+        t.sfq_shift = ((ni * BN) / 32) & 3;
+        t.s_begin = 0; t.s_end = S;
+        t.row0 = t.p_row; t.row_end = min(p.expert_offsets[e + 1], t.p_row + 128);
+        t.n0 = ni * BN;
+        t.tile = u; t.split = 0;
+    }
+    return t;
+}
+
+__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+template <int BN, int KIND>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
+            const GemmParams p) {
+    using C = Cfg<BN, KIND>;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[C::kStages], bar_empty[C::kStages], bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag_s;
+    __shared__ int is_last_s;
+    __shared__ int tile_start[KIND == kKindGrouped ? kMaxExperts + 1 : 1];
+    volatile int* abort_flag = &abort_flag_s;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const StagePlan plan(p.K, p.k_tail);
+    const int S = plan.S, S1 = plan.S1;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < C::kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_empty[i]), 4); }
+        abort_flag_s = 0;
+        is_last_s = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tm_act);
+        tma_prefetch_desc(&tm_w);
+    }
+    if (KIND == kKindGrouped && threadIdx.x == 64) {
+        int acc = 0;
+        for (int e = 0; e < p.n_experts; ++e) {
+            tile_start[e] = acc;
+            acc += (p.expert_offsets[e + 1] - p.expert_offsets[e] + 127) / 128;
+        }
+        tile_start[p.n_experts] = acc;
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tmem_slot), C::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+    const int n_units = unit_count<BN, KIND>(p, tile_start);
+
+    const CUtensorMap* tm_p = C::kSwap ? &tm_w : &tm_act;
+    const CUtensorMap* tm_q = C::kSwap ? &tm_act : &tm_w;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+                const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
+                for (int s = t.s_begin; s < t.s_end; ++s, ++it) {
+                    const int st = it % C::kStages;
+                    const uint32_t ph = (it / C::kStages) & 1;
+                    if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t full = smem_u32(&bar_full[st]);
+                    mbar_arrive_expect_tx(full, C::kTxBytes);
+                    // byte column of each operand in this stage
+                    const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
+                    const int xa = s < S1 ? s * 128 : (p.K - p.k_tail) / 2 + (s - S1) * 128;
+                    const uint32_t sb = smem_base + st * C::kStageBytes;
+                    tma_load_2d(sb, tm_p, C::kSwap ? xw : xa, t.p_row, full);
+                    tma_load_2d(sb + kPTileBytes, tm_q, C::kSwap ? xa : xw, t.q_row, full);
+                    bulk_load(sb + kPTileBytes + C::kQTileBytes, t.sfp + s * t.sfp_stride, C::kSfpBytes, full);
+                    bulk_load(sb + kPTileBytes + C::kQTileBytes + C::kSfpBytes, t.sfq + s * t.sfq_stride,
+                              C::kSfqBytes, full);
+                }
+            }
+            if (!ok) {
+                // let this CTA's copies in flight land before shared memory is given up (bounded)
+                for (int j = max(0, it - C::kStages); j < it; ++j) {
+                    const uint32_t bar = smem_u32(&bar_full[j % C::kStages]);
+                    const uint32_t ph = (j / C::kStages) & 1;
+                    for (int tries = 0; tries < (1 << 16) && !mbar_try_wait(bar, ph); ++tries) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int it = 0, acc_it = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
+                const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
+                const int buf = acc_it % C::kAcc;
+                const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
+                if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + buf * C::kAccStride;
+                const uint32_t sfp_t = tmem_base + C::kSfpCol;
+                const uint32_t sfq_t = tmem_base + C::kSfqCol;
+                uint32_t accumulate = 0;
+                for (int s = t.s_begin; s < t.s_end; ++s, ++it) {
+                    const int st = it % C::kStages;
+                    const uint32_t ph = (it / C::kStages) & 1;
+                    if (!mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t sb = smem_base + st * C::kStageBytes;
+                    const uint32_t sfp_s = sb + kPTileBytes + C::kQTileBytes;
+                    const uint32_t sfq_s = sfp_s + C::kSfpBytes;
+                    const int rem = s < S1 ? p.K - s * kStageK : p.k_tail - (s - S1) * kStageK;
+                    const int ksteps = min(4, (rem + 63) / 64);
+#pragma unroll
+                    for (int ka = 0; ka < 2; ++ka) {
+                        if (ka * 2 < ksteps) {
+                            tc_copy_sf_atom(sfp_t + ka * 4, make_smem_desc(sfp_s + ka * 512, 16, 128, kSwizzleNone));
+#pragma unroll
+                            for (int g = 0; g < C::kNgq; ++g)
+                                tc_copy_sf_atom(sfq_t + ka * 4 * C::kNgq + g * 4 - t.sfq_shift,
+                                                make_smem_desc(sfq_s + g * kSfGroupBytes + ka * 512, 16, 128, kSwizzleNone));
+                        }
+                    }
+                    const uint64_t pd = make_smem_desc(sb, 16, 1024, kSwizzle128B);
+                    const uint64_t qd = make_smem_desc(sb + kPTileBytes, 16, 1024, kSwizzle128B);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (j < ksteps) {
+                            const uint32_t sf_id = (j & 1) * 2;
+                            tc_mma_mxf4(d_tmem, pd + 2 * j, qd + 2 * j, make_idesc_mxf4(BN, sf_id, sf_id),
+                                        sfp_t + (j >> 1) * 4, sfq_t + (j >> 1) * 4 * C::kNgq, accumulate);
+                            accumulate = 1;
+                        }
+                    }
+                    tc_commit(smem_u32(&bar_empty[st]));
+                }
+                if (!ok) break;
+                tc_commit(smem_u32(&bar_acc_full[buf]));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;                 // tensor-memory lane quarter this warp may read
+        const int et = q * 32 + lane;           // 0..127: accumulator row
+        int acc_it = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
+            const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
+            const int buf = acc_it % C::kAcc;
+            const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
+            if (!mbar_wait(smem_u32(&bar_acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t acc_t = tmem_base + buf * C::kAccStride + (static_cast<uint32_t>(q * 32) << 16);
+            if (!C::kSwap) {
+                const int row = t.row0 + et;
+                const bool row_ok = row < t.row_end;
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(acc_t + c * 32, r);
+                    tmem_ld_wait();
+                    const int col = t.n0 + c * 32;
+                    if (row_ok && col < p.N) {
+                        if (p.y_bf16) {
+                            __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<size_t>(row) * p.ldy + col;
+                            if (col + 32 <= p.N) {
+#pragma unroll
+                                for (int i = 0; i < 32; i += 8) {
+                                    uint4 v;
+                                    __nv_bfloat162 h0 = __floats2bfloat162_rn(__uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+                                    __nv_bfloat162 h1 = __floats2bfloat162_rn(__uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+                                    __nv_bfloat162 h2 = __floats2bfloat162_rn(__uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+                                    __nv_bfloat162 h3 = __floats2bfloat162_rn(__uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+                                    v.x = *reinterpret_cast<uint32_t*>(&h0); v.y = *reinterpret_cast<uint32_t*>(&h1);
+                                    v.z = *reinterpret_cast<uint32_t*>(&h2); v.w = *reinterpret_cast<uint32_t*>(&h3);
+                                    *reinterpret_cast<uint4*>(yp + i) = v;
+                                }
+                            } else {
+                                for (int i = 0; i < 32 && col + i < p.N; ++i) yp[i] = __float2bfloat16_rn(__uint_as_float(r[i]));
+                            }
+                        } else {
+                            float* yp = reinterpret_cast<float*>(p.y) + static_cast<size_t>(row) * p.ldy + col;
+                            if (col + 32 <= p.N) {
+#pragma unroll
+                                for (int i = 0; i < 32; i += 4)
+                                    *reinterpret_cast<uint4*>(yp + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+                            } else {
+                                for (int i = 0; i < 32 && col + i < p.N; ++i) yp[i] = __uint_as_float(r[i]);
+                            }
+                        }
+                    }
+                }
+            } else {
+                // decode: accumulator row = weight row n, column = token
+                const int n = t.n0 + et;
+                const int n_pad = ((p.N + 127) / 128) * 128;
+                const bool direct = p.splits == 1;
+#pragma unroll 1
+                for (int c = 0; c < BN / 16; ++c) {
+                    uint32_t r[16];
+                    tmem_ld_32x16(acc_t + c * 16, r);
+                    tmem_ld_wait();
+                    if (c * 16 < p.M) {
+                        if (direct) {
+                            if (n < p.N) {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) {
+                                    const int tok = c * 16 + i;
+                                    if (tok < p.M) {
+                                        if (p.y_bf16)
+                                            reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] =
+                                                __float2bfloat16_rn(__uint_as_float(r[i]));
+                                        else
+                                            reinterpret_cast<float*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = __uint_as_float(r[i]);
+                                    }
+                                }
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const int tok = c * 16 + i;
+                                if (tok < p.M)
+                                    __stcg(&p.partial[(static_cast<size_t>(t.split) * BN + tok) * n_pad + n], __uint_as_float(r[i]));
+                            }
+                        }
+                    }
+                }
+                if (!direct) {
+                    // all partial sums of this CTA are visible before its arrival is counted
+                    __threadfence();
+                    epi_barrier();
+                    if (et == 0) {
+                        const int old = atomicAdd(&p.counters[t.tile], 1);
+                        const int last = old == p.splits - 1;
+                        if (last) p.counters[t.tile] = 0;  // leave the workspace clean for the next launch
+                        is_last_s = last;
+                    }
+                    epi_barrier();
+                    if (is_last_s) {
+                        __threadfence();
+                        if (n < p.N) {
+                            for (int tok = 0; tok < p.M; ++tok) {
+                                float sum = 0.f;
+                                for (int sp = 0; sp < p.splits; ++sp)
+                                    sum += __ldcg(&p.partial[(static_cast<size_t>(sp) * BN + tok) * n_pad + n]);
+                                if (p.y_bf16)
+                                    reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = __float2bfloat16_rn(sum);
+                                else
+                                    reinterpret_cast<float*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = sum;
+                            }
+                        }
+                    }
+                    epi_barrier();
+                }
+            }
+            // hand the accumulator back to the MMA issuer
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
+        }
+    }
+
+    // ------------------------------------------------------------ teardown (normal and aborted)
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+    if (threadIdx.x == 0 && abort_flag_s) atomicExch(p.status, static_cast<int>(PRQ_ERR_TIMEOUT));
+}
+
+template <int BN, int KIND>
+cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
+                       cudaStream_t stream) {
+    using C = Cfg<BN, KIND>;
+    constexpr int smem = C::kStages * C::kStageBytes + 1024;
+    static bool configured = false;  // per template instance; the attribute is per function, setting it twice is harmless
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BN, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    gemm_kernel<BN, KIND><<<grid, kThreads, smem, stream>>>(tm_act, tm_w, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_gemm(GemmKind kind, int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w,
+                        const GemmParams& p, int grid, cudaStream_t stream, bool* unsupported) {
+    *unsupported = false;
+#define PRQ_CASE(KINDV, BNV) \
+    if (bn == BNV) return launch_one<BNV, KINDV>(tm_act, tm_w, p, grid, stream);
+    if (kind == GemmKind::kPrefill) {
+        PRQ_CASE(kKindPrefill, 128)
+        PRQ_CASE(kKindPrefill, 160)
+        PRQ_CASE(kKindPrefill, 192)
+        PRQ_CASE(kKindPrefill, 256)
+    } else if (kind == GemmKind::kDecode) {
+        PRQ_CASE(kKindDecode, 16)
+        PRQ_CASE(kKindDecode, 32)
+        PRQ_CASE(kKindDecode, 64)
+        PRQ_CASE(kKindDecode, 128)
+    } else {
+        PRQ_CASE(kKindGrouped, 128)
+        PRQ_CASE(kKindGrouped, 256)
+    }
+#undef PRQ_CASE
+    *unsupported = true;
+    return cudaSuccess;
+}
+
+int gemm_smem_bytes(GemmKind kind, int bn) {
+    const int stage = kPTileBytes + bn * 128 + kSfGroupBytes + 2 * kSfGroupBytes;
+    (void)kind;
+    return stage;
+}
+
+}  // namespace prq

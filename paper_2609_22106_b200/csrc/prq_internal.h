@@ -1,0 +1,66 @@
+// Internal declarations shared by the translation units of libprq.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "prq.h"
+
+namespace prq {
+
+constexpr int kBlock = 32;        // MXFP4 block length
+constexpr int kStageK = 256;      // reduction elements per pipeline stage (one 128-byte swizzled row)
+constexpr int kGroupRows = 128;   // rows per scale-factor group
+constexpr int kSfGroupBytes = 1024;  // one (stage, 128-row group) of scale bytes: 2 atoms of 512 bytes
+constexpr int kMaxExperts = 1024;
+
+// Reduction stages of a layer: S1 cover the K main columns, S - S1 the k_tail residual columns.
+struct StagePlan {
+    int K, k_tail, S1, S;
+    __host__ __device__ StagePlan() : K(0), k_tail(0), S1(0), S(0) {}
+    __host__ __device__ StagePlan(int K_, int k_) : K(K_), k_tail(k_) {
+        S1 = (K_ + kStageK - 1) / kStageK;
+        S = S1 + (k_ + kStageK - 1) / kStageK;
+    }
+};
+
+// Byte offset of the scale of (row r of a 128-row group, block b of a stage) inside the group's
+// 1024-byte tile: two 512-byte atoms (4 blocks each); inside an atom 16 bytes per (r % 32) holding
+// 4 bytes per (r / 32), one per block.  This is the order the tensor-memory scale copy consumes.
+__host__ __device__ inline int sf_offset_in_group(int r, int blk_in_stage) {
+    return (blk_in_stage >> 2) * 512 + (r & 31) * 16 + (r >> 5) * 4 + (blk_in_stage & 3);
+}
+
+struct PrepResult {
+    std::vector<float> s, inv_s;
+    std::vector<double> col_err;
+    std::vector<int32_t> perm;
+    std::vector<uint8_t> codes;   // N x (K + k)/2
+    std::vector<uint8_t> scales;  // N x (K + k)/32
+};
+
+// Algorithm 1 steps 3-7 and 11 for one layer and one alpha, on the host.
+// Returns PRQ_ERR_NONFINITE if W or amax hold a NaN or an infinity.
+prq_status prepare_layer(const uint16_t* W, int N, int K, const float* amax, float alpha, int k_tail,
+                         PrepResult& out);
+
+}  // namespace prq
+
+struct prq_weights {
+    int n_experts = 0, N = 0, K = 0, k_tail = 0;
+    float alpha = 0.f;
+    prq::StagePlan plan;
+    int w_groups = 0;  // ceil(N / 128) scale groups per expert
+    int device = -1;
+    // canonical host copies (all experts concatenated)
+    std::vector<uint8_t> h_codes, h_scales;
+    std::vector<int32_t> h_perm;
+    std::vector<float> h_s, h_inv_s;
+    std::vector<double> h_col_err;
+    // device copies
+    uint8_t* d_codes = nullptr;      // E x N x (K + k)/2
+    uint8_t* d_sf = nullptr;         // E x S x w_groups x 1024 (+ padding)
+    int32_t* d_perm = nullptr;       // E x K
+    float* d_inv_s_perm = nullptr;   // E x K : inv_s[perm[j]] in the new channel order
+    size_t d_codes_bytes = 0, d_sf_bytes = 0;
+};

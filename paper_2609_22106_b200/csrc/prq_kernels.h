@@ -1,0 +1,58 @@
+// Launch interfaces of the device kernels (used by the C-ABI entry points).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "prq_internal.h"
+
+namespace prq {
+
+struct QuantParams {
+    const uint16_t* x;       // M x K bf16, row stride ldx
+    int M, ldx, K, k_tail;
+    int n_experts;
+    int act_groups;          // 128-row scale groups per stage in scales_sf
+    const int32_t* expert_offsets;  // nullptr when dense
+    const int32_t* perm;     // E x K (scale+perm mode)
+    const float* inv_s_perm; // E x K
+    uint8_t* codes;          // M x K/2
+    uint8_t* scales_row;     // M x K/32 or nullptr
+    uint8_t* scales_sf;      // S x act_groups x 1024
+};
+
+cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_groups, cudaStream_t stream);
+
+// Which GEMM variant to run.
+enum class GemmKind {
+    kPrefill,  // tokens on the MMA M axis (128-row tiles), weights on the N axis, persistent CTAs
+    kDecode,   // weights on the MMA M axis, tokens on the N axis, split-K with a workspace reduction
+    kGrouped   // prefill layout with per-expert row ranges
+};
+
+struct GemmParams {
+    int M;                   // activation rows (all experts)
+    int N, K, k_tail;
+    int n_experts;
+    int act_groups;          // 128-row groups per stage in act_sf
+    int w_groups;            // 128-row groups per stage per expert in w_sf
+    const uint8_t* act_sf;
+    const uint8_t* w_sf;
+    const int32_t* expert_offsets;  // grouped only
+    void* y;
+    int ldy;
+    int y_bf16;
+    float* partial;          // decode: splits x bn x N_pad fp32 partial sums
+    int* counters;           // decode: one arrival counter per 128-row weight tile
+    int splits;
+    int* status;             // device status word
+};
+
+// Creates the tensor maps and launches.  `bn` is the N-axis tile (weights rows for prefill / grouped,
+// tokens for decode).  Returns cudaSuccess or the launch error; sets *unsupported when `bn` has no
+// compiled instance.
+cudaError_t launch_gemm(GemmKind kind, int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w,
+                        const GemmParams& p, int grid, cudaStream_t stream, bool* unsupported);
+
+int gemm_smem_bytes(GemmKind kind, int bn);
+
+}  // namespace prq

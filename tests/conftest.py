@@ -19,3 +19,13 @@ def oracle():
 
     prq_oracle.build()
     return prq_oracle
+
+
+@pytest.fixture(scope="session")
+def prq():
+    """The ctypes binding over libprq.so, built in-tree if needed."""
+    from paper_2609_22106_b200 import binding, build
+
+    build.build()
+    binding.lib()
+    return binding
