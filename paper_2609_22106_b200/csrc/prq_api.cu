@@ -119,6 +119,7 @@ int prefill_bn(const prq_weights* w, int M, int num_sms) {
 }
 
 constexpr size_t kCounterBytes = 4096;  // 1024 tile counters
+constexpr int kAltTileRows[2] = {160, 192};  // weight tile widths with their own scale layout
 
 }  // namespace
 }  // namespace prq
@@ -169,6 +170,8 @@ void prq_weights_free(prq_weights* w) {
     cudaFree(w->d_sf);
     cudaFree(w->d_perm);
     cudaFree(w->d_inv_s_perm);
+    cudaFree(w->d_sf_alt[0]);
+    cudaFree(w->d_sf_alt[1]);
     if (w->device >= 0 && w->device != cur) cudaSetDevice(cur);
     delete w;
 }
@@ -206,6 +209,11 @@ prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, c
         w->d_sf_bytes = (E * S * w->w_groups + 4) * kSfGroupBytes;
         std::vector<uint8_t> sf(w->d_sf_bytes, 0);
         std::vector<float> inv_s_perm(E * K);
+        std::vector<uint8_t> sf_alt[2];
+        for (int a = 0; a < 2 && E == 1; ++a) {
+            w->w_groups_alt[a] = ((N + kAltTileRows[a] - 1) / kAltTileRows[a]) * 2;
+            sf_alt[a].assign((static_cast<size_t>(S) * w->w_groups_alt[a] + 4) * kSfGroupBytes, 0);
+        }
         PrepResult r;
         for (size_t e = 0; e < E; ++e) {
             st = prepare_layer(W + e * N * K, N, K, act_amax + e * K, alpha, k_tail, r);
@@ -225,6 +233,12 @@ prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, c
                     const int stage = b < nblk_main ? b / nb : S1 + (b - nblk_main) / nb;
                     const int bis = b < nblk_main ? b % nb : (b - nblk_main) % nb;
                     sf[((e * S + stage) * w->w_groups + g) * kSfGroupBytes + sf_offset_in_group(rr, bis)] = srow[b];
+                    for (int a = 0; a < 2 && E == 1; ++a) {
+                        const int tile_rows = kAltTileRows[a];
+                        const int ga = (n / tile_rows) * 2 + (n % tile_rows) / kGroupRows;
+                        sf_alt[a][(static_cast<size_t>(stage) * w->w_groups_alt[a] + ga) * kSfGroupBytes +
+                                  sf_offset_in_group((n % tile_rows) % kGroupRows, bis)] = srow[b];
+                    }
                 }
             }
         }
@@ -240,6 +254,14 @@ prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, c
         ok = ok && cudaMemcpy(w->d_sf, sf.data(), sf.size(), cudaMemcpyHostToDevice) == cudaSuccess;
         ok = ok && cudaMemcpy(w->d_perm, w->h_perm.data(), sizeof(int32_t) * E * K, cudaMemcpyHostToDevice) == cudaSuccess;
         ok = ok && cudaMemcpy(w->d_inv_s_perm, inv_s_perm.data(), sizeof(float) * E * K, cudaMemcpyHostToDevice) == cudaSuccess;
+        for (int a = 0; a < 2 && E == 1 && ok; ++a) {
+            if (cudaMalloc(&w->d_sf_alt[a], sf_alt[a].size()) != cudaSuccess) {
+                cudaGetLastError();
+                prq_weights_free(w);
+                return PRQ_ERR_OOM;
+            }
+            ok = cudaMemcpy(w->d_sf_alt[a], sf_alt[a].data(), sf_alt[a].size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        }
         if (!ok) { prq_weights_free(w); return PRQ_ERR_CUDA; }
     } catch (const std::bad_alloc&) {
         prq_weights_free(w);
@@ -485,6 +507,8 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         bn = prefill_bn(w, M, di->num_sms);
         const long units = static_cast<long>((M + 127) / 128) * ((w->N + bn - 1) / bn);
         grid = static_cast<int>(std::min<long>(units, di->num_sms));
+        for (int a = 0; a < 2; ++a)
+            if (bn == kAltTileRows[a]) { p.w_sf = w->d_sf_alt[a]; p.w_groups = w->w_groups_alt[a]; }
         st = make_code_map(&tm_act, codes, w->K / 2, M, 128);
         if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, bn);
     }

@@ -43,8 +43,9 @@ constexpr int pow2_at_least(int x) { int p = 32; while (p < x) p *= 2; return p;
 template <int BN, int KIND>
 struct Cfg {
     static constexpr bool kSwap = KIND == kKindDecode;
-    // 128-row scale groups a Q tile can touch (its first row is a multiple of gcd(BN, 128))
-    static constexpr int kNgq = kSwap ? 1 : (128 - cgcd(BN, 128) + BN + 127) / 128;
+    // 128-row scale groups of a Q tile; the weight scale buffer is laid out per BN-row tile, so a
+    // tile's groups are contiguous and start at the tile's first row
+    static constexpr int kNgq = (BN + 127) / 128;
     static constexpr int kQTileBytes = BN * 128;
     static constexpr int kSfpBytes = kSfGroupBytes;
     static constexpr int kSfqBytes = kNgq * kSfGroupBytes;
@@ -54,11 +55,11 @@ struct Cfg {
     static constexpr int kAccStride = cmax(BN, 32);
     static constexpr int kSfpCols = 8;              // 2 atoms x 4 columns
     static constexpr int kSfqCols = 8 * kNgq;       // 2 atoms x 4 columns x groups
-    static constexpr int kSfCols = kSfpCols + 4 + kSfqCols;  // 4 spare columns absorb the group shift
+    static constexpr int kSfCols = kSfpCols + kSfqCols;
     static constexpr int kAcc = (!kSwap && 2 * kAccStride + kSfCols <= 512) ? 2 : 1;
     static constexpr int kTmemCols = pow2_at_least(kAcc * kAccStride + kSfCols);
     static constexpr int kSfpCol = kAcc * kAccStride;
-    static constexpr int kSfqCol = kSfpCol + kSfpCols + 4;
+    static constexpr int kSfqCol = kSfpCol + kSfpCols;
     static constexpr uint32_t kTxBytes = kStageBytes;
     static_assert(kStages >= 2, "tile too large for shared memory");
     static_assert(kTmemCols <= 512, "tile too large for tensor memory");
@@ -70,7 +71,6 @@ struct Unit {
     const uint8_t* sfp;          // stage-0 scale tile of P; advance by sfp_stride per stage
     const uint8_t* sfq;
     size_t sfp_stride, sfq_stride;
-    int sfq_shift;               // 32-row chunks to drop in front of the first Q scale group
     int s_begin, s_end;          // reduction stages of this unit
     int row0, row_end;           // token rows covered / first row past the valid ones
     int n0;                      // first output feature
@@ -94,9 +94,8 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
         t.q_row = ni * BN;
         t.sfp = p.act_sf + static_cast<size_t>(mi) * kSfGroupBytes;
         t.sfp_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
-        t.sfq = p.w_sf + static_cast<size_t>((ni * BN) / 128) * kSfGroupBytes;
+        t.sfq = p.w_sf + static_cast<size_t>(ni) * Cfg<BN, KIND>::kNgq * kSfGroupBytes;
         t.sfq_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
-        t.sfq_shift = ((ni * BN) / 32) & 3;
         t.s_begin = 0; t.s_end = S;
         t.row0 = mi * 128; t.row_end = min(p.M, t.row0 + 128);
         t.n0 = ni * BN;
@@ -109,7 +108,6 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
         t.sfp_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
         t.sfq = p.act_sf;
         t.sfq_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
-        t.sfq_shift = 0;
         t.s_begin = static_cast<int>(static_cast<long long>(S) * sp / p.splits);
         t.s_end = static_cast<int>(static_cast<long long>(S) * (sp + 1) / p.splits);
         t.row0 = 0; t.row_end = p.M;
@@ -128,9 +126,8 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
         t.q_row = e * p.N + ni * BN;
         t.sfp = p.act_sf + static_cast<size_t>(mt) * kSfGroupBytes;
         t.sfp_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
-        t.sfq = p.w_sf + (static_cast<size_t>(e) * S * p.w_groups + (ni * BN) / 128) * kSfGroupBytes;
+        t.sfq = p.w_sf + (static_cast<size_t>(e) * S * p.w_groups + static_cast<size_t>(ni) * Cfg<BN, KIND>::kNgq) * kSfGroupBytes;
         t.sfq_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
-        t.sfq_shift = ((ni * BN) / 32) & 3;
         t.s_begin = 0; t.s_end = S;
         t.row0 = t.p_row; t.row_end = min(p.expert_offsets[e + 1], t.p_row + 128);
         t.n0 = ni * BN;
@@ -254,7 +251,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                             tc_copy_sf_atom(sfp_t + ka * 4, make_smem_desc(sfp_s + ka * 512, 16, 128, kSwizzleNone));
 #pragma unroll
                             for (int g = 0; g < C::kNgq; ++g)
-                                tc_copy_sf_atom(sfq_t + ka * 4 * C::kNgq + g * 4 - t.sfq_shift,
+                                tc_copy_sf_atom(sfq_t + ka * 4 * C::kNgq + g * 4,
                                                 make_smem_desc(sfq_s + g * kSfGroupBytes + ka * 512, 16, 128, kSwizzleNone));
                         }
                     }

