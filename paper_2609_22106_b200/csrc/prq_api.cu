@@ -86,6 +86,13 @@ int env_int(const char* name, int dflt) {
     return v && *v ? std::atoi(v) : dflt;
 }
 
+// Developer aid: PRQ_TRACE_PTR holds the address of a device buffer (4 x 512 int64) that the GEMM
+// fills with clock stamps.  Unset in normal use.
+long long* trace_ptr() {
+    const char* v = std::getenv("PRQ_TRACE_PTR");
+    return v && *v ? reinterpret_cast<long long*>(std::strtoull(v, nullptr, 0)) : nullptr;
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 int dense_groups(int M) { return (M + kGroupRows - 1) / kGroupRows; }
@@ -94,11 +101,14 @@ int grouped_groups(int M, int n_groups) { return (M + kGroupRows - 1) / kGroupRo
 int decode_bn(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
 
 int decode_splits(const prq_weights* w, int M, int num_sms) {
+    // The split CTAs of a tile wait for one another, so the whole grid must be resident at once:
+    // at most one CTA per SM.
     const int n_tiles = (w->N + 127) / 128;
-    const int ctas_per_sm = decode_bn(M) <= 32 ? 2 : 1;
+    (void)M;
+    const int max_splits = std::max(1, num_sms / n_tiles);
     int splits = env_int("PRQ_DECODE_SPLITS", 0);
-    if (splits <= 0) splits = std::max(1, (num_sms * ctas_per_sm) / n_tiles);
-    splits = std::min(splits, std::min(w->plan.S, 64));
+    if (splits <= 0) splits = max_splits;
+    splits = std::min(splits, std::min(max_splits, std::min(w->plan.S, 64)));
     return std::max(1, splits);
 }
 
@@ -482,6 +492,8 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
     p.y = y; p.ldy = ldy; p.y_bf16 = y_dtype == PRQ_BF16;
     p.status = di->status_ptr;
     p.splits = 1;
+    p.trace = trace_ptr();
+    p.dbg = env_int("PRQ_DBG", 0);
 
     CUtensorMap tm_act, tm_w;
     GemmKind kind;

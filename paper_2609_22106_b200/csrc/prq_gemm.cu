@@ -182,6 +182,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
+    // optional developer trace: SM clock stamps of the first iterations of each role (CTA 0..3 only)
+    long long* trace = (p.trace && blockIdx.x < 4) ? p.trace + blockIdx.x * 512 : nullptr;
+    if (trace && threadIdx.x == 0) trace[500] = clock64();
     const int n_units = unit_count<BN, KIND>(p, tile_start);
 
     const CUtensorMap* tm_p = C::kSwap ? &tm_w : &tm_act;
@@ -189,15 +192,17 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        if (lane == 0) {
-            int it = 0;
-            bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-                const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
-                for (int s = t.s_begin; s < t.s_end; ++s, ++it) {
-                    const int st = it % C::kStages;
-                    const uint32_t ph = (it / C::kStages) & 1;
-                    if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
+        // The whole warp walks the loop (a lone diverged lane runs this code several times slower);
+        // one elected lane arms the barrier and issues the copies.
+        int it = 0, st = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+            const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
+            for (int s = t.s_begin; s < t.s_end; ++s, ++it) {
+                if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
+                if (trace && lane == 0 && it < 64) trace[it] = clock64();
+                if (elect_one()) {
                     const uint32_t full = smem_u32(&bar_full[st]);
                     mbar_arrive_expect_tx(full, C::kTxBytes);
                     // byte column of each operand in this stage
@@ -210,44 +215,46 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                     bulk_load(sb + kPTileBytes + C::kQTileBytes + C::kSfpBytes, t.sfq + s * t.sfq_stride,
                               C::kSfqBytes, full);
                 }
+                if (++st == C::kStages) { st = 0; ph ^= 1; }
             }
-            if (!ok) {
-                // let this CTA's copies in flight land before shared memory is given up (bounded)
-                for (int j = max(0, it - C::kStages); j < it; ++j) {
-                    const uint32_t bar = smem_u32(&bar_full[j % C::kStages]);
-                    const uint32_t ph = (j / C::kStages) & 1;
-                    for (int tries = 0; tries < (1 << 16) && !mbar_try_wait(bar, ph); ++tries) {}
-                }
+        }
+        if (!ok && lane == 0) {
+            // let this CTA's copies in flight land before shared memory is given up (bounded)
+            for (int j = max(0, it - C::kStages); j < it; ++j) {
+                const uint32_t bar = smem_u32(&bar_full[j % C::kStages]);
+                const uint32_t ph = (j / C::kStages) & 1;
+                for (int tries = 0; tries < (1 << 16) && !mbar_try_wait(bar, ph); ++tries) {}
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            int it = 0, acc_it = 0;
-            bool ok = true;
-            for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
-                const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
-                const int buf = acc_it % C::kAcc;
-                const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
-                if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1, abort_flag)) { ok = false; break; }
-                tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + buf * C::kAccStride;
-                const uint32_t sfp_t = tmem_base + C::kSfpCol;
-                const uint32_t sfq_t = tmem_base + C::kSfqCol;
-                uint32_t accumulate = 0;
-                for (int s = t.s_begin; s < t.s_end; ++s, ++it) {
-                    const int st = it % C::kStages;
-                    const uint32_t ph = (it / C::kStages) & 1;
-                    if (!mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
-                    tc_fence_after_sync();
+        // The whole warp walks the loop and waits on the barriers; one elected lane issues the
+        // tensor-core instructions (and therefore also the commits that track them).
+        int it = 0, acc_it = 0, st = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        const uint32_t sfp_t = tmem_base + C::kSfpCol;
+        const uint32_t sfq_t = tmem_base + C::kSfqCol;
+        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
+            const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
+            const int buf = acc_it % C::kAcc;
+            const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
+            if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t d_tmem = tmem_base + buf * C::kAccStride;
+            uint32_t accumulate = 0;
+            for (int s = t.s_begin; s < t.s_end; ++s, ++it) {
+                if (!mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
+                if (trace && lane == 0 && it < 64) trace[64 + it] = clock64();
+                const int rem = s < S1 ? p.K - s * kStageK : p.k_tail - (s - S1) * kStageK;
+                const int ksteps = min(4, (rem + 63) / 64);
+                if (elect_one()) {
                     const uint32_t sb = smem_base + st * C::kStageBytes;
                     const uint32_t sfp_s = sb + kPTileBytes + C::kQTileBytes;
                     const uint32_t sfq_s = sfp_s + C::kSfpBytes;
-                    const int rem = s < S1 ? p.K - s * kStageK : p.k_tail - (s - S1) * kStageK;
-                    const int ksteps = min(4, (rem + 63) / 64);
 #pragma unroll
                     for (int ka = 0; ka < 2; ++ka) {
-                        if (ka * 2 < ksteps) {
+                        if (ka * 2 < ksteps && !(p.dbg & 1)) {
                             tc_copy_sf_atom(sfp_t + ka * 4, make_smem_desc(sfp_s + ka * 512, 16, 128, kSwizzleNone));
 #pragma unroll
                             for (int g = 0; g < C::kNgq; ++g)
@@ -259,7 +266,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                     const uint64_t qd = make_smem_desc(sb + kPTileBytes, 16, 1024, kSwizzle128B);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        if (j < ksteps) {
+                        if (j < ksteps && !(p.dbg & 2)) {
                             const uint32_t sf_id = (j & 1) * 2;
                             tc_mma_mxf4(d_tmem, pd + 2 * j, qd + 2 * j, make_idesc_mxf4(BN, sf_id, sf_id),
                                         sfp_t + (j >> 1) * 4, sfq_t + (j >> 1) * 4 * C::kNgq, accumulate);
@@ -268,9 +275,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                     }
                     tc_commit(smem_u32(&bar_empty[st]));
                 }
-                if (!ok) break;
-                tc_commit(smem_u32(&bar_acc_full[buf]));
+                accumulate = 1;
+                if (trace && lane == 0 && it < 64) trace[128 + it] = clock64();
+                if (++st == C::kStages) { st = 0; ph ^= 1; }
             }
+            if (!ok) break;
+            if (elect_one()) tc_commit(smem_u32(&bar_acc_full[buf]));
+            __syncwarp();
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5)
@@ -283,6 +294,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
             const int buf = acc_it % C::kAcc;
             const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
             if (!mbar_wait(smem_u32(&bar_acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
+            if (trace && et == 0 && acc_it < 8) trace[192 + 2 * acc_it] = clock64();
             tc_fence_after_sync();
             const uint32_t acc_t = tmem_base + buf * C::kAccStride + (static_cast<uint32_t>(q * 32) << 16);
             if (!C::kSwap) {
@@ -360,43 +372,63 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                     }
                 }
                 if (!direct) {
-                    // all partial sums of this CTA are visible before its arrival is counted
+                    // Split-K meeting point.  Every CTA of a tile publishes its partial sums, waits
+                    // (bounded) until all `splits` partials of the tile are there, then adds up its own
+                    // share of the tokens in a fixed order.  All CTAs of the launch are co-resident
+                    // (the host keeps the grid within one wave), so the wait cannot starve.
                     __threadfence();
                     epi_barrier();
                     if (et == 0) {
-                        const int old = atomicAdd(&p.counters[t.tile], 1);
-                        const int last = old == p.splits - 1;
-                        if (last) p.counters[t.tile] = 0;  // leave the workspace clean for the next launch
-                        is_last_s = last;
-                    }
-                    epi_barrier();
-                    if (is_last_s) {
-                        __threadfence();
-                        if (n < p.N) {
-                            for (int tok = 0; tok < p.M; ++tok) {
-                                float sum = 0.f;
-                                for (int sp = 0; sp < p.splits; ++sp)
-                                    sum += __ldcg(&p.partial[(static_cast<size_t>(sp) * BN + tok) * n_pad + n]);
-                                if (p.y_bf16)
-                                    reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = __float2bfloat16_rn(sum);
-                                else
-                                    reinterpret_cast<float*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = sum;
-                            }
+                        atomicAdd(&p.counters[t.tile], 1);
+                        const long long t0 = clock64();
+                        volatile int* cnt = p.counters + t.tile;
+                        while (*cnt < p.splits) {
+                            if (*abort_flag) break;
+                            if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
                         }
                     }
                     epi_barrier();
+                    if (*abort_flag) { ok = false; break; }
+                    __threadfence();
+                    if (n < p.N) {
+                        for (int tok = t.split; tok < p.M; tok += p.splits) {
+                            const float* src = p.partial + static_cast<size_t>(tok) * n_pad + n;
+                            const size_t sp_stride = static_cast<size_t>(BN) * n_pad;
+                            float sum = 0.f;
+                            for (int sp0 = 0; sp0 < p.splits; sp0 += 8) {
+                                float v[8];
+#pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    v[i] = sp0 + i < p.splits ? __ldcg(src + (sp0 + i) * sp_stride) : 0.f;
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) sum += v[i];
+                            }
+                            if (p.y_bf16)
+                                reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = __float2bfloat16_rn(sum);
+                            else
+                                reinterpret_cast<float*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = sum;
+                        }
+                    }
+                    epi_barrier();
+                    // the last CTA to finish reading leaves the counter at zero for the next launch
+                    if (et == 0) {
+                        const int old = atomicAdd(&p.counters[t.tile], 1);
+                        if (old == 2 * p.splits - 1) p.counters[t.tile] = 0;
+                    }
                 }
             }
             // hand the accumulator back to the MMA issuer
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
+            if (trace && et == 0 && acc_it < 8) trace[193 + 2 * acc_it] = clock64();
         }
     }
 
     // ------------------------------------------------------------ teardown (normal and aborted)
     tc_fence_before_sync();
     __syncthreads();
+    if (trace && threadIdx.x == 0) trace[501] = clock64();
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();

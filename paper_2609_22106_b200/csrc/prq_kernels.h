@@ -45,6 +45,8 @@ struct GemmParams {
     int* counters;           // decode: one arrival counter per 128-row weight tile
     int splits;
     int* status;             // device status word
+    long long* trace;        // developer trace buffer (nullptr in normal use)
+    int dbg;                 // developer switches for timing experiments (0 in normal use)
 };
 
 // Creates the tensor maps and launches.  `bn` is the N-axis tile (weights rows for prefill / grouped,
