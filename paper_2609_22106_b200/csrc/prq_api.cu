@@ -81,6 +81,23 @@ prq_status make_code_map(CUtensorMap* map, const void* base, uint64_t row_bytes,
     return r == CUDA_SUCCESS ? PRQ_OK : PRQ_ERR_CUDA;
 }
 
+// Output matrix for the epilogue's TMA stores: boxes of 32 columns x 32 rows (128-byte rows with the
+// 128-byte swizzle for fp32, 64-byte rows with the 64-byte swizzle for bf16).
+prq_status make_out_map(CUtensorMap* map, void* y, int M, int N, int ldy, bool bf16) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return PRQ_ERR_CUDA;
+    const uint64_t es = bf16 ? 2 : 4;
+    cuuint64_t dims[2] = {static_cast<cuuint64_t>(N), static_cast<cuuint64_t>(M)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(ldy) * es};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides,
+                    box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
 int env_int(const char* name, int dflt) {
     const char* v = std::getenv(name);
     return v && *v ? std::atoi(v) : dflt;
@@ -129,7 +146,14 @@ int prefill_bn(const prq_weights* w, int M, int num_sms) {
 }
 
 constexpr size_t kCounterBytes = 4096;  // 1024 tile counters
-constexpr int kAltTileRows[2] = {160, 192};  // weight tile widths with their own scale layout
+constexpr int kNumAlt = 3;
+constexpr int kAltTileRows[kNumAlt] = {160, 192, 224};  // weight tile widths with their own scale layout
+constexpr size_t kPrefillSlotBytes = 128 * kPrefillTileN * sizeof(float);
+
+size_t prefill_flag_bytes(const prq_weights* w, int M) {
+    const size_t tiles = static_cast<size_t>((M + 127) / 128) * ((w->N + kPrefillTileN - 1) / kPrefillTileN);
+    return (tiles * sizeof(int) + 255) & ~static_cast<size_t>(255);
+}
 
 }  // namespace
 }  // namespace prq
@@ -180,8 +204,7 @@ void prq_weights_free(prq_weights* w) {
     cudaFree(w->d_sf);
     cudaFree(w->d_perm);
     cudaFree(w->d_inv_s_perm);
-    cudaFree(w->d_sf_alt[0]);
-    cudaFree(w->d_sf_alt[1]);
+    for (int a = 0; a < 3; ++a) cudaFree(w->d_sf_alt[a]);
     if (w->device >= 0 && w->device != cur) cudaSetDevice(cur);
     delete w;
 }
@@ -219,8 +242,8 @@ prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, c
         w->d_sf_bytes = (E * S * w->w_groups + 4) * kSfGroupBytes;
         std::vector<uint8_t> sf(w->d_sf_bytes, 0);
         std::vector<float> inv_s_perm(E * K);
-        std::vector<uint8_t> sf_alt[2];
-        for (int a = 0; a < 2 && E == 1; ++a) {
+        std::vector<uint8_t> sf_alt[kNumAlt];
+        for (int a = 0; a < kNumAlt && E == 1; ++a) {
             w->w_groups_alt[a] = ((N + kAltTileRows[a] - 1) / kAltTileRows[a]) * 2;
             sf_alt[a].assign((static_cast<size_t>(S) * w->w_groups_alt[a] + 4) * kSfGroupBytes, 0);
         }
@@ -243,7 +266,7 @@ prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, c
                     const int stage = b < nblk_main ? b / nb : S1 + (b - nblk_main) / nb;
                     const int bis = b < nblk_main ? b % nb : (b - nblk_main) % nb;
                     sf[((e * S + stage) * w->w_groups + g) * kSfGroupBytes + sf_offset_in_group(rr, bis)] = srow[b];
-                    for (int a = 0; a < 2 && E == 1; ++a) {
+                    for (int a = 0; a < kNumAlt && E == 1; ++a) {
                         const int tile_rows = kAltTileRows[a];
                         const int ga = (n / tile_rows) * 2 + (n % tile_rows) / kGroupRows;
                         sf_alt[a][(static_cast<size_t>(stage) * w->w_groups_alt[a] + ga) * kSfGroupBytes +
@@ -264,7 +287,7 @@ prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, c
         ok = ok && cudaMemcpy(w->d_sf, sf.data(), sf.size(), cudaMemcpyHostToDevice) == cudaSuccess;
         ok = ok && cudaMemcpy(w->d_perm, w->h_perm.data(), sizeof(int32_t) * E * K, cudaMemcpyHostToDevice) == cudaSuccess;
         ok = ok && cudaMemcpy(w->d_inv_s_perm, inv_s_perm.data(), sizeof(float) * E * K, cudaMemcpyHostToDevice) == cudaSuccess;
-        for (int a = 0; a < 2 && E == 1 && ok; ++a) {
+        for (int a = 0; a < kNumAlt && E == 1 && ok; ++a) {
             if (cudaMalloc(&w->d_sf_alt[a], sf_alt[a].size()) != cudaSuccess) {
                 cudaGetLastError();
                 prq_weights_free(w);
@@ -453,7 +476,12 @@ prq_status prq_quantize_act(const prq_weights* w, prq_act_mode mode, const void*
 
 size_t prq_linear_workspace_bytes(const prq_weights* w, int M) {
     if (!w || M < 0) return 0;
-    if (M > 128) return kCounterBytes;
+    if (M > 128) {
+        // stream-K prefill: one flag per 128 x 256 tile, one fp32 partial tile per CTA (at most one CTA per SM)
+        DeviceInfo* di;
+        if (device_info(w->device, &di) != PRQ_OK) return 0;
+        return prefill_flag_bytes(w, M) + static_cast<size_t>(di->num_sms) * kPrefillSlotBytes;
+    }
     // decode: counters + the largest split count this layer can use x token tile x padded N
     const size_t n_pad = static_cast<size_t>((w->N + 127) / 128) * 128;
     const size_t splits = std::min(w->plan.S, 64);
@@ -514,12 +542,36 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         grid = ((w->N + 127) / 128) * p.splits;
         st = make_code_map(&tm_act, codes, w->K / 2, M, bn);
         if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, 128);
+    } else if (env_int("PRQ_PREFILL_BN", 0) == 0) {
+        // stream-K kernel with 128 x 224 tiles (scale bytes grouped per 224-row weight tile)
+        PrefillParams q;
+        std::memset(&q, 0, sizeof(q));
+        q.M = M; q.N = w->N; q.K = w->K; q.k_tail = w->k_tail;
+        q.m_tiles = (M + 127) / 128; q.n_tiles = (w->N + kPrefillTileN - 1) / kPrefillTileN;
+        q.act_groups = p.act_groups; q.w_groups = w->w_groups_alt[2];
+        q.act_sf = p.act_sf; q.w_sf = w->d_sf_alt[2];
+        q.y_bf16 = p.y_bf16; q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
+        const size_t flag_bytes = prefill_flag_bytes(w, M);
+        const long long units = static_cast<long long>(q.m_tiles) * q.n_tiles * w->plan.S;
+        const int g = static_cast<int>(std::min<long long>(units, di->num_sms));
+        if (!workspace || workspace_bytes < flag_bytes + static_cast<size_t>(g) * kPrefillSlotBytes) return PRQ_ERR_WORKSPACE;
+        if (!aligned16(workspace)) return PRQ_ERR_ALIGNMENT;
+        q.flags = static_cast<int*>(workspace);
+        q.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + flag_bytes);
+        CUtensorMap tm_y;
+        st = make_code_map(&tm_act, codes, w->K / 2, M, 128);
+        if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, kPrefillTileN);
+        if (st == PRQ_OK) st = make_out_map(&tm_y, y, M, w->N, ldy, y_dtype == PRQ_BF16);
+        if (st != PRQ_OK) return st;
+        cudaError_t e = launch_prefill(tm_act, tm_w, tm_y, q, g, static_cast<cudaStream_t>(stream));
+        g_launches.fetch_add(1);
+        return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     } else {
         kind = GemmKind::kPrefill;
         bn = prefill_bn(w, M, di->num_sms);
         const long units = static_cast<long>((M + 127) / 128) * ((w->N + bn - 1) / bn);
         grid = static_cast<int>(std::min<long>(units, di->num_sms));
-        for (int a = 0; a < 2; ++a)
+        for (int a = 0; a < kNumAlt; ++a)
             if (bn == kAltTileRows[a]) { p.w_sf = w->d_sf_alt[a]; p.w_groups = w->w_groups_alt[a]; }
         st = make_code_map(&tm_act, codes, w->K / 2, M, 128);
         if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, bn);

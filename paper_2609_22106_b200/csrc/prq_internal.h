@@ -60,10 +60,10 @@ struct prq_weights {
     // device copies
     uint8_t* d_codes = nullptr;      // E x N x (K + k)/2
     uint8_t* d_sf = nullptr;         // E x S x w_groups x 1024 (+ padding)
-    // Dense layers also keep the scale bytes grouped per 160- and 192-row weight tile (two 128-row
-    // groups per tile, the second partly empty) so that those tile widths need no re-alignment.
-    uint8_t* d_sf_alt[2] = {nullptr, nullptr};
-    int w_groups_alt[2] = {0, 0};
+    // Dense layers also keep the scale bytes grouped per 160-, 192- and 224-row weight tile (two
+    // 128-row groups per tile, the second partly empty) so that those tile widths need no re-alignment.
+    uint8_t* d_sf_alt[3] = {nullptr, nullptr, nullptr};
+    int w_groups_alt[3] = {0, 0, 0};
     int32_t* d_perm = nullptr;       // E x K
     float* d_inv_s_perm = nullptr;   // E x K : inv_s[perm[j]] in the new channel order
     size_t d_codes_bytes = 0, d_sf_bytes = 0;

@@ -57,4 +57,22 @@ cudaError_t launch_gemm(GemmKind kind, int bn, const CUtensorMap& tm_act, const 
 
 int gemm_smem_bytes(GemmKind kind, int bn);
 
+// Stream-K prefill kernel (128 x 224 tiles).
+constexpr int kPrefillTileN = 224;
+struct PrefillParams {
+    int M, N, K, k_tail;
+    int m_tiles, n_tiles;
+    int act_groups, w_groups;   // 128-row scale groups per stage in act_sf / w_sf
+    const uint8_t* act_sf;
+    const uint8_t* w_sf;
+    float* partial;             // one 128 x 224 fp32 slot per CTA (column-major inside a slot)
+    int* flags;                 // one arrival counter per tile, zero between launches
+    int y_bf16;
+    int* status;
+    long long* trace;
+    int dbg;
+};
+cudaError_t launch_prefill(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_y,
+                           const PrefillParams& p, int grid, cudaStream_t stream);
+
 }  // namespace prq

@@ -114,7 +114,7 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
 // Shared -> tensor memory copy of one 512-byte scale atom: 32 rows of 16 bytes, broadcast to the
 // four 32-lane quarters of tensor memory.
 __device__ __forceinline__ void tc_copy_sf_atom(uint32_t taddr, uint64_t smem_desc) {
-    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(smem_desc) : "memory");
+    asm volatile("tcgen05.cp.cta_group::1.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(smem_desc));
 }
 // D[tmem] (+)= A[smem] * B[smem] with per-32 block scales from tensor memory, E2M1 x E2M1, K = 64.
 __device__ __forceinline__ void tc_mma_mxf4(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
@@ -123,8 +123,7 @@ __device__ __forceinline__ void tc_mma_mxf4(uint32_t d_tmem, uint64_t a_desc, ui
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::mxf4.block_scale.block32 [%0], %1, %2, %3, [%5], [%6], p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
-        : "memory");
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem));
 }
 // 32 lanes x 32 consecutive 32-bit columns -> 32 registers per thread (thread i = lane base + i).
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {

@@ -173,14 +173,23 @@ def test_decode_split_counts(prq, oracle, splits, monkeypatch):
     layer_case(prq, oracle, N=300, K=2560, M=8, k=128, alpha=0.5, mode=prq.ACT_IDENTITY)
 
 
-@pytest.mark.parametrize("bn", [128, 160, 192, 256])
+@pytest.mark.parametrize("bn", [0, 128, 160, 192, 256])
 @pytest.mark.parametrize("shape", [(300, 608, 2336, 96), (1000, 2560, 1024, 0), (260, 328, 512, 512)])
 def test_prefill_tiles(prq, oracle, bn, shape, monkeypatch):
-    """M > 128: persistent prefill kernel with every weight-tile width; ragged M and N, a reduction that
-    is not a multiple of the stage, k = 0 and k = K."""
-    monkeypatch.setenv("PRQ_PREFILL_BN", str(bn))
+    """M > 128: the stream-K prefill kernel (bn = 0, the default) and the tile-per-CTA kernel with every
+    weight-tile width; ragged M and N, a reduction that is not a multiple of the stage, k = 0 and k = K."""
+    if bn:
+        monkeypatch.setenv("PRQ_PREFILL_BN", str(bn))
     M, N, K, k = shape
     layer_case(prq, oracle, N=N, K=K, M=M, k=k, alpha=0.5, mode=prq.ACT_SCALE_PERM, seed=bn)
+
+
+@pytest.mark.parametrize("shape", [(200, 256, 9728, 256), (129, 520, 4096, 128), (1500, 1024, 2560, 128), (4100, 768, 512, 64)])
+def test_prefill_stream_k_splits(prq, oracle, shape):
+    """Stream-K corner cases: a tile shared by dozens of CTAs (few tiles, long reduction), ranges that
+    start and end inside tiles, more tiles than CTAs."""
+    M, N, K, k = shape
+    layer_case(prq, oracle, N=N, K=K, M=M, k=k, alpha=0.5, mode=prq.ACT_IDENTITY, seed=M)
 
 
 def test_k0_runs_the_same_kernels_as_plain_mxfp4(prq, oracle):
@@ -220,6 +229,14 @@ def test_deterministic(prq, oracle):
     y2 = prq.linear(w, codes, sf, 16, workspace=ws).clone()
     assert torch.equal(y1, y2)
     assert int(ws.view(torch.int32)[:1024].abs().sum()) == 0  # counters are left clean
+    # prefill: the stream-K flags are left clean too and the fixed summation order reproduces bits
+    x2 = to_dev_bf16(synth.layer(95, 512, 2560, 700, T_cal=32)["x"])
+    codes, _, sf = prq.quantize_act(w, x2, prq.ACT_SCALE_PERM)
+    ws = prq.new_workspace(w, 700)
+    y1 = prq.linear(w, codes, sf, 700, workspace=ws).clone()
+    y2 = prq.linear(w, codes, sf, 700, workspace=ws).clone()
+    assert torch.equal(y1, y2)
+    assert int(ws.view(torch.int32)[:64].abs().sum()) == 0
     w.free()
 
 
