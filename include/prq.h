@@ -110,6 +110,11 @@ prq_status prq_prepare_weights_search(const uint16_t *W, int N, int K, const uin
 
 void prq_weights_free(prq_weights *w);
 
+/* A second, independent device copy of a handle's prepared weights (same device): serving several
+ * streams from separate memory, or benchmarks that rotate over more weight bytes than the L2 holds.
+ * Not part of the paper's method.  Free it with prq_weights_free. */
+prq_status prq_weights_clone(const prq_weights *w, prq_weights **out);
+
 /* Shape of a handle.  Any output pointer may be NULL. */
 prq_status prq_weights_info(const prq_weights *w, int *n_experts, int *N, int *K, int *k_tail, float *alpha);
 

@@ -22,7 +22,7 @@ BUF_CODES, BUF_SCALES_ROW, BUF_SCALES_SF = range(3)
 
 EXPORTS = [
     "prq_prepare_weights", "prq_prepare_weights_host", "prq_prepare_weights_search", "prq_weights_free",
-    "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
+    "prq_weights_clone", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
     "prq_linear", "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count",
 ]
@@ -49,6 +49,7 @@ def lib():
         L.prq_prepare_weights_host.argtypes = [vp, ci, ci, vp, cf, ci, vp, vp, vp, vp, vp, vp]
         L.prq_prepare_weights_search.argtypes = [vp, ci, ci, vp, ci, vp, ci, ci, ctypes.POINTER(vp),
                                                  ctypes.POINTER(cf), vp]
+        L.prq_weights_clone.argtypes = [vp, ctypes.POINTER(vp)]
         L.prq_weights_free.argtypes = [vp]
         L.prq_weights_free.restype = None
         L.prq_weights_info.argtypes = [vp] + [ctypes.POINTER(ci)] * 4 + [ctypes.POINTER(cf)]
@@ -125,6 +126,11 @@ class Weights:
         out = np.empty(shape, dt)
         _check(lib().prq_weights_get(self._h, expert, field, _np_ptr(out), out.nbytes), "prq_weights_get")
         return out
+
+    def clone(self) -> "Weights":
+        h = ctypes.c_void_p()
+        _check(lib().prq_weights_clone(self._h, ctypes.byref(h)), "prq_weights_clone")
+        return Weights(h)
 
     def free(self):
         if self._h:

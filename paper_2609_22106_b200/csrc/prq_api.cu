@@ -27,6 +27,7 @@ struct DeviceInfo {
     bool ok = false;
     int num_sms = 0;
     int* status_ptr = nullptr;
+    int max_clusters[4][9] = {};  // decode kernel: [token-tile index][cluster size], 0 = not queried yet
 };
 std::mutex g_dev_mutex;
 DeviceInfo g_dev[64];
@@ -117,16 +118,30 @@ int grouped_groups(int M, int n_groups) { return (M + kGroupRows - 1) / kGroupRo
 
 int decode_bn(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
 
-int decode_splits(const prq_weights* w, int M, int num_sms) {
-    // The split CTAs of a tile wait for one another, so the whole grid must be resident at once:
-    // at most one CTA per SM.
+// Cluster size (= number of K-splits) of the decode kernel: the one that puts the most SMs to work in
+// the first wave, given how many clusters of each size the device can hold at once.
+int decode_splits(const prq_weights* w, int M, DeviceInfo* di) {
     const int n_tiles = (w->N + 127) / 128;
-    (void)M;
-    const int max_splits = std::max(1, num_sms / n_tiles);
-    int splits = env_int("PRQ_DECODE_SPLITS", 0);
-    if (splits <= 0) splits = max_splits;
-    splits = std::min(splits, std::min(max_splits, std::min(w->plan.S, 64)));
-    return std::max(1, splits);
+    const int bn = decode_bn(M);
+    const int bi = bn == 16 ? 0 : bn == 32 ? 1 : bn == 64 ? 2 : 3;
+    const int forced = env_int("PRQ_DECODE_SPLITS", 0);
+    const int limit = std::min(8, w->plan.S);
+    if (forced > 0) return std::min(forced, limit);
+    int best = 1, best_ctas = 0;
+    for (int s = 1; s <= limit; ++s) {
+        int mc;
+        {
+            std::lock_guard<std::mutex> lock(g_dev_mutex);
+            if (di->max_clusters[bi][s] == 0) di->max_clusters[bi][s] = std::max(1, decode_max_active_clusters(bn, s));
+            mc = di->max_clusters[bi][s];
+        }
+        const int ctas = std::min(n_tiles, mc) * s;
+        const bool one_wave = mc >= n_tiles;
+        // prefer configurations that fit in one wave; among them the most CTAs
+        const int score = ctas + (one_wave ? 100000 : 0);
+        if (score > best_ctas) { best_ctas = score; best = s; }
+    }
+    return best;
 }
 
 int prefill_bn(const prq_weights* w, int M, int num_sms) {
@@ -145,7 +160,6 @@ int prefill_bn(const prq_weights* w, int M, int num_sms) {
     return best;
 }
 
-constexpr size_t kCounterBytes = 4096;  // 1024 tile counters
 constexpr int kNumAlt = 3;
 constexpr int kAltTileRows[kNumAlt] = {160, 192, 224};  // weight tile widths with their own scale layout
 constexpr size_t kPrefillSlotBytes = 128 * kPrefillTileN * sizeof(float);
@@ -405,6 +419,45 @@ prq_status prq_prepare_weights_host(const uint16_t* W, int N, int K, const float
     return PRQ_OK;
 }
 
+prq_status prq_weights_clone(const prq_weights* w, prq_weights** out) {
+    if (!w || !out) return PRQ_ERR_INVALID_ARG;
+    prq_weights* c = new (std::nothrow) prq_weights;
+    if (!c) return PRQ_ERR_OOM;
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (cur != w->device) cudaSetDevice(w->device);
+    prq_status st = PRQ_OK;
+    try {
+        c->n_experts = w->n_experts; c->N = w->N; c->K = w->K; c->k_tail = w->k_tail; c->alpha = w->alpha;
+        c->plan = w->plan; c->w_groups = w->w_groups; c->device = w->device;
+        c->h_codes = w->h_codes; c->h_scales = w->h_scales; c->h_perm = w->h_perm;
+        c->h_s = w->h_s; c->h_inv_s = w->h_inv_s; c->h_col_err = w->h_col_err;
+        c->d_codes_bytes = w->d_codes_bytes; c->d_sf_bytes = w->d_sf_bytes;
+        const size_t EK = static_cast<size_t>(w->n_experts) * w->K;
+        auto dup = [&](void* dst_pp, const void* src, size_t bytes) {
+            void** pp = static_cast<void**>(dst_pp);
+            if (st != PRQ_OK || !src) return;
+            if (cudaMalloc(pp, bytes) != cudaSuccess) { cudaGetLastError(); st = PRQ_ERR_OOM; return; }
+            if (cudaMemcpy(*pp, src, bytes, cudaMemcpyDeviceToDevice) != cudaSuccess) st = PRQ_ERR_CUDA;
+        };
+        dup(&c->d_codes, w->d_codes, w->d_codes_bytes);
+        dup(&c->d_sf, w->d_sf, w->d_sf_bytes);
+        dup(&c->d_perm, w->d_perm, sizeof(int32_t) * EK);
+        dup(&c->d_inv_s_perm, w->d_inv_s_perm, sizeof(float) * EK);
+        for (int a = 0; a < kNumAlt; ++a) {
+            c->w_groups_alt[a] = w->w_groups_alt[a];
+            if (w->d_sf_alt[a])
+                dup(&c->d_sf_alt[a], w->d_sf_alt[a], (static_cast<size_t>(w->plan.S) * w->w_groups_alt[a] + 4) * kSfGroupBytes);
+        }
+    } catch (const std::bad_alloc&) {
+        st = PRQ_ERR_OOM;
+    }
+    if (cur != w->device) cudaSetDevice(cur);
+    if (st != PRQ_OK) { prq_weights_free(c); return st; }
+    *out = c;
+    return PRQ_OK;
+}
+
 prq_status prq_weights_info(const prq_weights* w, int* n_experts, int* N, int* K, int* k_tail, float* alpha) {
     if (!w) return PRQ_ERR_INVALID_ARG;
     if (n_experts) *n_experts = w->n_experts;
@@ -482,10 +535,7 @@ size_t prq_linear_workspace_bytes(const prq_weights* w, int M) {
         if (device_info(w->device, &di) != PRQ_OK) return 0;
         return prefill_flag_bytes(w, M) + static_cast<size_t>(di->num_sms) * kPrefillSlotBytes;
     }
-    // decode: counters + the largest split count this layer can use x token tile x padded N
-    const size_t n_pad = static_cast<size_t>((w->N + 127) / 128) * 128;
-    const size_t splits = std::min(w->plan.S, 64);
-    return kCounterBytes + splits * decode_bn(M) * n_pad * sizeof(float);
+    return 0;  // decode: the split-K partial sums meet in distributed shared memory
 }
 
 static prq_status check_linear_common(const prq_weights* w, const void* codes, const void* scales_sf, void* y, int ldy,
@@ -527,21 +577,22 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
     GemmKind kind;
     int bn, grid;
     if (M <= 128) {
-        kind = GemmKind::kDecode;
+        // weight-streaming kernel: weights on the MMA M axis, K split over a thread-block cluster
+        DecodeParams q;
+        std::memset(&q, 0, sizeof(q));
+        q.M = M; q.N = w->N; q.K = w->K; q.k_tail = w->k_tail;
+        q.w_groups = w->w_groups;
+        q.act_sf = p.act_sf; q.w_sf = w->d_sf;
+        q.y = y; q.ldy = ldy; q.y_bf16 = p.y_bf16;
+        q.status = p.status; q.trace = p.trace;
+        q.splits = decode_splits(w, M, di);
         bn = decode_bn(M);
-        p.splits = decode_splits(w, M, di->num_sms);
-        const size_t n_pad = static_cast<size_t>((w->N + 127) / 128) * 128;
-        if (p.splits > 1) {
-            const size_t need = kCounterBytes + static_cast<size_t>(p.splits) * bn * n_pad * sizeof(float);
-            if (!workspace || workspace_bytes < need) return PRQ_ERR_WORKSPACE;
-            if (!aligned16(workspace)) return PRQ_ERR_ALIGNMENT;
-            if ((w->N + 127) / 128 > static_cast<int>(kCounterBytes / sizeof(int))) return PRQ_ERR_INVALID_ARG;
-            p.counters = static_cast<int*>(workspace);
-            p.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kCounterBytes);
-        }
-        grid = ((w->N + 127) / 128) * p.splits;
         st = make_code_map(&tm_act, codes, w->K / 2, M, bn);
         if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, 128);
+        if (st != PRQ_OK) return st;
+        cudaError_t e = launch_decode(bn, tm_act, tm_w, q, (w->N + 127) / 128, static_cast<cudaStream_t>(stream));
+        g_launches.fetch_add(1);
+        return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     } else if (env_int("PRQ_PREFILL_BN", 0) == 0) {
         // stream-K kernel with 128 x 224 tiles (scale bytes grouped per 224-row weight tile)
         PrefillParams q;
@@ -554,6 +605,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         const size_t flag_bytes = prefill_flag_bytes(w, M);
         const long long units = static_cast<long long>(q.m_tiles) * q.n_tiles * w->plan.S;
         const int g = static_cast<int>(std::min<long long>(units, di->num_sms));
+        if (units * g >= (1ll << 32)) return PRQ_ERR_INVALID_ARG;  // the kernel's range arithmetic is 32-bit
         if (!workspace || workspace_bytes < flag_bytes + static_cast<size_t>(g) * kPrefillSlotBytes) return PRQ_ERR_WORKSPACE;
         if (!aligned16(workspace)) return PRQ_ERR_ALIGNMENT;
         q.flags = static_cast<int*>(workspace);

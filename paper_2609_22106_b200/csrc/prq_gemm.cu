@@ -464,12 +464,7 @@ cudaError_t launch_gemm(GemmKind kind, int bn, const CUtensorMap& tm_act, const 
         PRQ_CASE(kKindPrefill, 160)
         PRQ_CASE(kKindPrefill, 192)
         PRQ_CASE(kKindPrefill, 256)
-    } else if (kind == GemmKind::kDecode) {
-        PRQ_CASE(kKindDecode, 16)
-        PRQ_CASE(kKindDecode, 32)
-        PRQ_CASE(kKindDecode, 64)
-        PRQ_CASE(kKindDecode, 128)
-    } else {
+    } else if (kind == GemmKind::kGrouped) {
         PRQ_CASE(kKindGrouped, 128)
         PRQ_CASE(kKindGrouped, 256)
     }

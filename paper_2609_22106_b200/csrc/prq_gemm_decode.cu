@@ -1,0 +1,358 @@
+// Decode GEMM (M <= 128 tokens): the block-scaled FP4 product of Eq. (3) as a weight-streaming kernel.
+//
+// With few tokens the layer is bound by reading its 4-bit weights once.  The weight rows sit on the MMA
+// M axis (128-row tiles), the tokens on the N axis (16, 32, 64 or 128 columns), and the reduction axis
+// K + k is split over the CTAs of a thread-block cluster so that every SM streams a share of the
+// weights.  Each CTA of a cluster accumulates its K-range in tensor memory, parks the fp32 partial tile
+// in its own shared memory, and after one cluster barrier every CTA sums, over its peers' shared memory
+// (distributed shared memory), the tokens assigned to it and writes them to y.  No global scratch, no
+// atomics, and the summation order is fixed (peer 0, 1, ...), so the result is reproducible.
+//
+// Roles per CTA (6 warps): warp 0 TMA producer, warp 1 tcgen05 issuer (scale copies + MMAs), warps 2-5
+// epilogue and reduction.  The activation tail is re-read: stages past the K main columns load the
+// token tile from column K - k and the weight tile from column K onwards (Kernel design paragraph).
+// Every wait is bounded; the cluster barriers sit on the common path so that a CTA that gave up still
+// arrives and its peers are released.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "prq_kernels.h"
+#include "prq_ptx.cuh"
+
+namespace prq {
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kPTile = 128 * 128;   // weight tile bytes: 128 rows x 256 codes
+constexpr int kSf = kSfGroupBytes;  // one 128-row scale group per operand and stage
+constexpr int kStages = 6;
+
+constexpr uint32_t kHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+constexpr uint32_t kHiPlain = (128u >> 4) | (1u << 14);
+__device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo) { return (static_cast<uint64_t>(hi) << 32) | lo; }
+constexpr int pow2_cols(int x) { int p = 32; while (p < x) p *= 2; return p; }
+
+template <int BN>
+struct DCfg {
+    static constexpr int kQTile = BN * 128;
+    static constexpr int kStageBytes = kPTile + kQTile + 2 * kSf;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024;
+    static constexpr int kAccCols = BN < 32 ? 32 : BN;
+    static constexpr int kSfCol = kAccCols;          // 8 weight-scale + 8 token-scale columns behind the accumulator
+    static constexpr int kTmemCols = pow2_cols(kAccCols + 16);
+    static_assert(kStageBytes % 1024 == 0, "stage slots must keep 1024-byte alignment");
+    static_assert(BN * 128 * 4 <= kStages * kStageBytes, "the partial tile is parked in the pipeline buffers");
+};
+
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Address of `local_addr` in the shared memory of CTA `peer` of this cluster.
+__device__ __forceinline__ uint32_t peer_addr(uint32_t local_addr, uint32_t peer) {
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(peer));
+    return ra;
+}
+__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+
+// One reduction stage issued by the elected thread, ring slot Q known at compile time.
+template <int BN, int Q>
+__device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, uint32_t sf_t, int rem,
+                                            uint32_t accumulate, uint32_t empty_bar0) {
+    using C = DCfg<BN>;
+    constexpr uint32_t so = (Q * C::kStageBytes) >> 4;
+    constexpr uint32_t sfo = so + ((kPTile + C::kQTile) >> 4);
+    constexpr uint32_t idesc0 = (1u << 7) | (1u << 10) | ((BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+    constexpr uint32_t idesc2 = idesc0 | (2u << 4) | (2u << 29);
+    const uint32_t plo = lo_base + so, qlo = lo_base + so + (kPTile >> 4), slo = lo_base + sfo;
+    const uint32_t sfp_t = sf_t, sfq_t = sf_t + 8;
+    tc_copy_sf_atom(sfp_t, desc64(kHiPlain, slo));
+    tc_copy_sf_atom(sfq_t, desc64(kHiPlain, slo + (kSf >> 4)));
+    if (rem > 128) {
+        tc_copy_sf_atom(sfp_t + 4, desc64(kHiPlain, slo + (512 >> 4)));
+        tc_copy_sf_atom(sfq_t + 4, desc64(kHiPlain, slo + ((kSf + 512) >> 4)));
+    }
+    tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo), desc64(kHiSw128, qlo), idesc0, sfp_t, sfq_t, accumulate);
+    if (rem > 64) tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 2), desc64(kHiSw128, qlo + 2), idesc2, sfp_t, sfq_t, 1);
+    if (rem > 128) tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 4), desc64(kHiSw128, qlo + 4), idesc0, sfp_t + 4, sfq_t + 4, 1);
+    if (rem > 192) tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 6), desc64(kHiSw128, qlo + 6), idesc2, sfp_t + 4, sfq_t + 4, 1);
+    tc_commit(empty_bar0 + Q * 8);
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
+              const DecodeParams p) {
+    using C = DCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bar_full[kStages], bar_empty[kStages], bar_acc_full;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag_s;
+    volatile int* abort_flag = &abort_flag_s;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t smem_base = smem_u32(smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const StagePlan plan(p.K, p.k_tail);
+    const int S = plan.S, S1 = plan.S1;
+    const int splits = p.splits;
+    const int tile = blockIdx.x / splits;
+    const int split = blockIdx.x - tile * splits;   // = rank in the cluster
+    const int s_begin = static_cast<int>(static_cast<long long>(S) * split / splits);
+    const int s_end = static_cast<int>(static_cast<long long>(S) * (split + 1) / splits);
+    const int n0 = tile * 128;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
+        mbar_init(smem_u32(&bar_acc_full), 1);
+        abort_flag_s = 0;
+        fence_mbar_init();
+        tma_prefetch_desc(&tm_act);
+        tma_prefetch_desc(&tm_w);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&tmem_slot), C::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_slot;
+    long long* trace = (p.trace && blockIdx.x < 4) ? p.trace + blockIdx.x * 512 : nullptr;
+    if (trace && threadIdx.x == 0) trace[500] = clock64();
+    const uint32_t lo_base = ((smem_base & 0x3FFFF) >> 4) | (1u << 16);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        const uint8_t* sfp = p.w_sf + static_cast<size_t>(tile) * kSfGroupBytes;
+        const size_t sfp_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
+        const size_t sfq_stride = kSfGroupBytes;  // one token group per stage
+        int st = 0, it = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        for (int s = s_begin; s < s_end; ++s, ++it) {
+            if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
+            if (trace && lane == 0 && it < 64) trace[it] = clock64();
+            if (elect_one()) {
+                const uint32_t full = smem_u32(&bar_full[st]);
+                mbar_arrive_expect_tx(full, C::kStageBytes);
+                const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
+                const int xa = s < S1 ? s * 128 : (p.K - p.k_tail) / 2 + (s - S1) * 128;
+                const uint32_t sb = smem_base + st * C::kStageBytes;
+                tma_load_2d(sb, &tm_w, xw, n0, full);
+                tma_load_2d(sb + kPTile, &tm_act, xa, 0, full);
+                bulk_load(sb + kPTile + C::kQTile, sfp + s * sfp_stride, kSf, full);
+                bulk_load(sb + kPTile + C::kQTile + kSf, p.act_sf + s * sfq_stride, kSf, full);
+            }
+            if (++st == kStages) { st = 0; ph ^= 1; }
+        }
+        if (!ok && lane == 0) {
+            for (int j = max(0, it - kStages); j < it; ++j) {
+                const uint32_t bar = smem_u32(&bar_full[j % kStages]);
+                const uint32_t php = (j / kStages) & 1;
+                for (int tries = 0; tries < (1 << 16) && !mbar_try_wait(bar, php); ++tries) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ tcgen05 issuer
+        const bool leader = elect_one();
+        const uint32_t d_tmem = tmem_base;
+        const uint32_t sf_t = tmem_base + C::kSfCol;
+        const uint32_t eb = smem_u32(&bar_empty[0]);
+        int st = 0, it = 0;
+        uint32_t ph = 0, accumulate = 0;
+        bool ok = true;
+        for (int s = s_begin; s < s_end; ++s, ++it) {
+            if (!mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
+            if (trace && lane == 0 && it < 64) trace[64 + it] = clock64();
+            const int rem = s < S1 ? p.K - s * kStageK : p.k_tail - (s - S1) * kStageK;
+            if (leader) {
+                switch (st) {
+                    case 0: issue_stage<BN, 0>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                    case 1: issue_stage<BN, 1>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                    case 2: issue_stage<BN, 2>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                    case 3: issue_stage<BN, 3>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                    case 4: issue_stage<BN, 4>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                    default: issue_stage<BN, 5>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                }
+            }
+            accumulate = 1;
+            if (trace && lane == 0 && it < 64) trace[128 + it] = clock64();
+            if (++st == kStages) { st = 0; ph ^= 1; }
+        }
+        if (ok && leader) tc_commit(smem_u32(&bar_acc_full));
+    } else {
+        // ------------------------------------------------------------ epilogue, part 1: accumulator -> registers
+        // -> (splits == 1) y, or this CTA's partial tile in shared memory, token-major: partial[t][row]
+        const int q4 = warp & 3;
+        const int row = q4 * 32 + lane;              // weight row inside the tile
+        const int n = n0 + row;
+        const uint32_t acc_t = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
+        if (mbar_wait(smem_u32(&bar_acc_full), 0, abort_flag)) {
+            if (trace && row == 0) trace[192] = clock64();
+            tc_fence_after_sync();
+            float* partial = reinterpret_cast<float*>(smem);
+#pragma unroll 1
+            for (int c = 0; c < (BN + 15) / 16; ++c) {
+                uint32_t v[16];
+                tmem_ld_32x16(acc_t + c * 16, v);
+                tmem_ld_wait();
+                if (c * 16 < p.M) {
+                    if (splits == 1) {
+                        if (n < p.N) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const int tok = c * 16 + i;
+                                if (tok < p.M) {
+                                    if (p.y_bf16)
+                                        reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] =
+                                            __float2bfloat16_rn(__uint_as_float(v[i]));
+                                    else
+                                        reinterpret_cast<float*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = __uint_as_float(v[i]);
+                                }
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) partial[(c * 16 + i) * 128 + row] = __uint_as_float(v[i]);
+                    }
+                }
+            }
+            if (trace && row == 0) trace[193] = clock64();
+        }
+        tc_fence_before_sync();
+    }
+
+    if (splits > 1) {
+        // ------------------------------------------------------------ meeting point of the cluster
+        // (all threads of all CTAs; orders the partial tiles before the peers' reads)
+        __syncthreads();
+        cluster_sync_all();
+        if (warp >= 2 && !abort_flag_s) {
+            // epilogue, part 2: this CTA adds up tokens split, split + splits, ... over all peers.  A thread
+            // owns 4 consecutive weight rows (one 16-byte piece of the token-major partial tiles) and every
+            // fourth of the CTA's tokens; the loads from all peers are issued together, the sum runs
+            // in peer order.
+            const int et = threadIdx.x - 64;                 // 0..127
+            const int j = et & 31, tq = et >> 5;
+            const int n = n0 + 4 * j;
+            uint32_t base[8];
+#pragma unroll
+            for (int peer = 0; peer < 8; ++peer) base[peer] = peer_addr(smem_base + j * 16, peer < splits ? peer : 0);
+            for (int tok = split + splits * tq; tok < p.M; tok += splits * 4) {
+                float4 v[8];
+#pragma unroll
+                for (int peer = 0; peer < 8; ++peer)
+                    if (peer < splits) v[peer] = ld_cluster_f32x4(base[peer] + tok * 512);
+                float4 sum = v[0];
+#pragma unroll
+                for (int peer = 1; peer < 8; ++peer)
+                    if (peer < splits) { sum.x += v[peer].x; sum.y += v[peer].y; sum.z += v[peer].z; sum.w += v[peer].w; }
+                if (n + 3 < p.N) {
+                    if (p.y_bf16) {
+                        __nv_bfloat162 lo = __floats2bfloat162_rn(sum.x, sum.y), hi = __floats2bfloat162_rn(sum.z, sum.w);
+                        uint2 pk = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<size_t>(tok) * p.ldy + n) = pk;
+                    } else {
+                        *reinterpret_cast<float4*>(reinterpret_cast<float*>(p.y) + static_cast<size_t>(tok) * p.ldy + n) = sum;
+                    }
+                } else {
+                    const float e[4] = {sum.x, sum.y, sum.z, sum.w};
+                    for (int i = 0; i < 4 && n + i < p.N; ++i) {
+                        if (p.y_bf16)
+                            reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<size_t>(tok) * p.ldy + n + i] = __float2bfloat16_rn(e[i]);
+                        else
+                            reinterpret_cast<float*>(p.y)[static_cast<size_t>(tok) * p.ldy + n + i] = e[i];
+                    }
+                }
+            }
+            if (trace && et == 0) trace[194] = clock64();
+        }
+        // nobody leaves while a peer may still be reading its shared memory
+        cluster_sync_all();
+    }
+
+    // ------------------------------------------------------------ teardown (normal and aborted)
+    tc_fence_before_sync();
+    __syncthreads();
+    if (trace && threadIdx.x == 0) trace[501] = clock64();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::kTmemCols);
+    }
+    if (threadIdx.x == 0 && abort_flag_s) atomicExch(p.status, static_cast<int>(PRQ_ERR_TIMEOUT));
+}
+
+template <int BN>
+cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const DecodeParams& p, int n_tiles,
+                       cudaStream_t stream) {
+    using C = DCfg<BN>;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_tiles * p.splits);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = p.splits;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_kernel<BN>, tm_act, tm_w, p);
+}
+
+template <int BN>
+int max_clusters(int splits) {
+    using C = DCfg<BN>;
+    cudaFuncSetAttribute(decode_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(splits);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = C::kSmemBytes;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = splits;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<BN>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return n;
+}
+
+}  // namespace
+
+cudaError_t launch_decode(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const DecodeParams& p,
+                          int n_tiles, cudaStream_t stream) {
+    switch (bn) {
+        case 16: return launch_one<16>(tm_act, tm_w, p, n_tiles, stream);
+        case 32: return launch_one<32>(tm_act, tm_w, p, n_tiles, stream);
+        case 64: return launch_one<64>(tm_act, tm_w, p, n_tiles, stream);
+        default: return launch_one<128>(tm_act, tm_w, p, n_tiles, stream);
+    }
+}
+
+int decode_max_active_clusters(int bn, int splits) {
+    switch (bn) {
+        case 16: return max_clusters<16>(splits);
+        case 32: return max_clusters<32>(splits);
+        case 64: return max_clusters<64>(splits);
+        default: return max_clusters<128>(splits);
+    }
+}
+
+}  // namespace prq

@@ -79,21 +79,25 @@ struct Segment {
 };
 
 // The contiguous range of (tile, stage) units of one CTA, walked segment by segment.
+// All of this is 32-bit arithmetic (the host checks that W * G fits): 64-bit divisions cost hundreds of
+// cycles each and sit on the critical path of every role's first instruction.
 struct Range {
-    long long cur, end;
+    uint32_t cur, end;
     int S;
     __device__ __forceinline__ bool next(Segment& g) {
         if (cur >= end) return false;
-        g.tile = static_cast<int>(cur / S);
-        g.s0 = static_cast<int>(cur - static_cast<long long>(g.tile) * S);
-        const long long left = end - cur;
-        g.s1 = static_cast<int>(left < S - g.s0 ? g.s0 + left : S);
+        g.tile = static_cast<int>(cur / static_cast<uint32_t>(S));
+        g.s0 = static_cast<int>(cur - static_cast<uint32_t>(g.tile) * S);
+        const uint32_t left = end - cur;
+        g.s1 = left < static_cast<uint32_t>(S - g.s0) ? g.s0 + static_cast<int>(left) : S;
         cur += g.s1 - g.s0;
         return true;
     }
 };
 
-__device__ __forceinline__ long long range_begin(long long W, int g, int G) { return W * g / G; }
+__device__ __forceinline__ uint32_t range_begin(uint32_t W, int g, int G) {
+    return W * static_cast<uint32_t>(g) / static_cast<uint32_t>(G);
+}
 
 constexpr uint32_t kHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO 1024, version 1, 128B swizzle
 constexpr uint32_t kHiPlain = (128u >> 4) | (1u << 14);                // SBO 128, version 1, no swizzle
@@ -145,7 +149,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant
     const StagePlan plan(p.K, p.k_tail);
     const int S = plan.S, S1 = plan.S1;
     const int G = gridDim.x, g = blockIdx.x;
-    const long long W = static_cast<long long>(p.m_tiles) * p.n_tiles * S;
+    const uint32_t W = static_cast<uint32_t>(p.m_tiles) * p.n_tiles * S;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
@@ -263,7 +267,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant
             int n_contrib = 0;
             if (!contributor && sg.s1 < S) {
                 // owner of a tile that other CTAs finish: they are the next CTAs in order
-                const long long last_unit = static_cast<long long>(sg.tile + 1) * S - 1;
+                const uint32_t last_unit = static_cast<uint32_t>(sg.tile + 1) * S - 1;
                 int gl = g + 1;
                 while (gl + 1 < G && range_begin(W, gl + 1, G) <= last_unit) ++gl;
                 n_contrib = gl - g;

@@ -57,6 +57,24 @@ cudaError_t launch_gemm(GemmKind kind, int bn, const CUtensorMap& tm_act, const 
 
 int gemm_smem_bytes(GemmKind kind, int bn);
 
+// Decode kernel (M <= 128): cluster split-K with a distributed-shared-memory reduction.
+struct DecodeParams {
+    int M, N, K, k_tail;
+    int w_groups;               // 128-row scale groups per stage in w_sf
+    const uint8_t* act_sf;      // one group per stage
+    const uint8_t* w_sf;
+    void* y;
+    int ldy, y_bf16;
+    int splits;                 // = cluster size, 1..8
+    int* status;
+    long long* trace;
+};
+// `bn` in {16, 32, 64, 128} is the token tile; the grid is n_tiles * splits CTAs in clusters of `splits`.
+cudaError_t launch_decode(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const DecodeParams& p,
+                          int n_tiles, cudaStream_t stream);
+// How many clusters of `splits` CTAs of the decode kernel can be resident at once on the current device.
+int decode_max_active_clusters(int bn, int splits);
+
 // Stream-K prefill kernel (128 x 224 tiles).
 constexpr int kPrefillTileN = 224;
 struct PrefillParams {

@@ -1,15 +1,16 @@
 // Activation quantisation kernel ("the kernel quantizes the reordered activation to MXFP4 once",
 // Kernel design paragraph; Eq. (1) activation side when the scale and permutation are applied online).
 //
-// One CTA owns a tile of 128 rows x 256 columns (one reduction stage of the GEMM): 8 warps x 16 rows,
-// a warp covers the 256 columns of a row with one 16-byte load per lane (8 bf16).  A 32-element block
-// is 4 adjacent lanes: amax by two shuffles, E8M0 byte from the exponent field, eight
-// round-to-nearest-even E2M1 conversions per lane, one 4-byte packed store per lane (128 contiguous
-// bytes per warp).  The scale bytes of the tile are collected in shared memory in the GEMM's
-// 1024-byte (stage, 128-row group) order and written out coalesced; the bytes of tail blocks are
-// also duplicated into the residual stages, which is all the "tail copy" this design needs.
-//
-// HBM-bound: 2 bytes read + 0.5 + 1/32 written per element.
+// One CTA owns 128 rows x 128 columns: exactly one 512-byte scale atom of the GEMM's layout.  A warp
+// processes two rows per step (16 lanes x 8 bf16 = 128 columns each); the eight steps of a warp are
+// unrolled with all eight 16-byte loads issued first, so that about 100 KB per SM are in flight -- the
+// kernel is HBM-bound (2 bytes read + 0.5 + 1/32 written per element) and latency is hidden by loads
+// in flight, not by occupancy.  A 32-element block is 4 adjacent lanes: amax by packed 16-bit maxima and
+// two shuffles, E8M0 byte from the exponent field, eight round-to-nearest-even E2M1 conversions per
+// lane, one 4-byte packed store per lane.  The atom's scale bytes are collected in shared memory and
+// written out as one coalesced 512-byte piece; the bytes of tail blocks are also duplicated into the
+// residual stages, which is all the "tail copy" this design needs (the GEMM re-reads the tail codes).
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include "prq_internal.h"
@@ -19,30 +20,50 @@ namespace prq {
 namespace {
 
 constexpr int kQuantThreads = 256;
-constexpr int kRowsPerWarp = kGroupRows / (kQuantThreads / 32);  // 16
+constexpr int kAtomK = 128;    // columns per CTA (4 blocks = one scale atom)
+constexpr int kSteps = kGroupRows / (2 * (kQuantThreads / 32));  // 8 steps of 16 rows
 
-// Two floats -> one byte of E2M1 codes (lo in the low nibble), round to nearest even, saturating.
-__device__ __forceinline__ uint32_t cvt_e2m1x2(float lo, float hi) {
-    uint16_t out;
-    asm("{\n\t.reg .b8 t;\n\t"
-        "cvt.rn.satfinite.e2m1x2.f32 t, %2, %1;\n\t"
-        "cvt.u16.u8 %0, t;\n\t}"
-        : "=h"(out)
-        : "f"(lo), "f"(hi));
+// E2M1 conversion: round to nearest even, saturating; the sign of values that round to zero (and of
+// negative zero) is kept.
+// Eight floats -> four bytes of E2M1 codes (element 0 in the lowest nibble).
+__device__ __forceinline__ uint32_t cvt_e2m1x8(float f0, float f1, float f2, float f3, float f4, float f5, float f6,
+                                               float f7) {
+    uint32_t out;
+    asm("{\n\t.reg .b8 t0, t1, t2, t3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t2, %6, %5;\n\t"
+        "cvt.rn.satfinite.e2m1x2.f32 t3, %8, %7;\n\t"
+        "mov.b32 %0, {t0, t1, t2, t3};\n\t}"
+        : "=r"(out)
+        : "f"(f0), "f"(f1), "f"(f2), "f"(f3), "f"(f4), "f"(f5), "f"(f6), "f"(f7));
     return out;
 }
 
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t w) { return *reinterpret_cast<__nv_bfloat162*>(&w); }
+__device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t*>(&h); }
+
+// Scale byte from the block's largest magnitude given as fp32 bits: biased exponent - 2, floored at 0.
+__device__ __forceinline__ uint32_t scale_byte(uint32_t amax_f32_bits) {
+    const int eb = static_cast<int>(amax_f32_bits >> 23) - 2;
+    return eb < 0 ? 0u : static_cast<uint32_t>(eb);
+}
+
+// Eight values (as fp32) -> 4 bytes of codes under the block scale 2^(byte - 127).
+__device__ __forceinline__ uint32_t encode8(const float (&v)[8], uint32_t byte) {
+    const float inv = __uint_as_float((254u - byte) << 23);  // 2^(127 - byte), exact multiply
+    return cvt_e2m1x8(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv, v[4] * inv, v[5] * inv, v[6] * inv, v[7] * inv);
+}
 
 template <bool kScalePerm>
 __global__ void __launch_bounds__(kQuantThreads)
 quant_act_kernel(QuantParams p) {
-    __shared__ __align__(16) uint8_t sf_tile[kSfGroupBytes];
+    __shared__ __align__(16) uint8_t sf_atom[512];
     __shared__ int s_tile_start[kMaxExperts + 1];
 
-    const int stage = blockIdx.x;
+    const int atom = blockIdx.x;                  // 128-column slice of the reduction axis
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int half = lane >> 4, hl = lane & 15;   // which of the warp's two rows, lane inside the row
 
     // Which rows does this CTA own?  Dense: group g covers rows [128 g, 128 g + 128).  Grouped: the
     // scale groups are padded per expert, so walk the expert offsets to find ours.
@@ -63,7 +84,7 @@ quant_act_kernel(QuantParams p) {
         __syncthreads();
         if (group >= s_tile_start[p.n_experts]) return;  // padding CTA of the launch grid
         int lo = 0, hi = p.n_experts - 1;
-        while (lo < hi) {  // last expert whose first tile is <= group and that owns tiles
+        while (lo < hi) {  // last expert whose first tile is <= group
             int mid = (lo + hi + 1) >> 1;
             if (s_tile_start[mid] <= group) lo = mid; else hi = mid - 1;
         }
@@ -72,19 +93,21 @@ quant_act_kernel(QuantParams p) {
         row_end = min(p.expert_offsets[expert + 1], row0 + kGroupRows);
     }
 
-    for (int i = threadIdx.x; i < kSfGroupBytes / 4; i += kQuantThreads) reinterpret_cast<uint32_t*>(sf_tile)[i] = 0;
+    if (threadIdx.x < 128) reinterpret_cast<uint32_t*>(sf_atom)[threadIdx.x] = 0;
     __syncthreads();
 
     const int K = p.K, k_tail = p.k_tail;
-    const int col0 = stage * kStageK + lane * 8;  // first of this lane's 8 columns
+    const int col0 = atom * kAtomK + hl * 8;      // first of this lane's 8 columns
     const bool col_ok = col0 < K;                 // K % 32 == 0, so a lane is all in or all out
-    const int blk_in_stage = lane >> 2;
+    const int blk_in_atom = hl >> 2;
+    const int gblk = atom * (kAtomK / kBlock) + blk_in_atom;
     const int tail_blk0 = (K - k_tail) / kBlock;  // first tail block (global block index)
-    const int gblk = stage * (kStageK / kBlock) + blk_in_stage;
     const StagePlan plan(K, k_tail);
+    const int stage = atom >> 1;
     uint8_t* sf_base = p.scales_sf;
-    const size_t sf_group_stride = kSfGroupBytes;
     const size_t sf_stage_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
+    uint8_t* sf_group = sf_base + static_cast<size_t>(group) * kSfGroupBytes;
+    const int n_rows = row_end - row0;            // 1..128
 
     float inv_s[8];
     int src[8];
@@ -99,76 +122,117 @@ quant_act_kernel(QuantParams p) {
         inv_s[4] = s1.x; inv_s[5] = s1.y; inv_s[6] = s1.z; inv_s[7] = s1.w;
     }
 
-#pragma unroll 4
-    for (int i = 0; i < kRowsPerWarp; ++i) {
-        const int r = warp + i * (kQuantThreads / 32);  // row inside the group
-        const int row = row0 + r;
-        if (row >= row_end) break;  // warp-uniform
-        float v[8];
-        if (col_ok) {
-            const uint16_t* xrow = p.x + static_cast<size_t>(row) * p.ldx;
-            if (kScalePerm) {
+    // row of step i: 16 rows per step, 2 per warp
+    auto row_of = [&](int i) { return i * 16 + warp * 2 + half; };
+
+    if (!kScalePerm) {
+        // ---- identity: all eight 16-byte loads first, then the arithmetic on packed bf16 pairs ----
+        // Pointers advance by a constant per step (16 rows); nothing inside the loops multiplies.
+        const int c = warp * 2 + half;                       // row inside a 16-row step
+        const uint16_t* xp = p.x + static_cast<size_t>(row0 + c) * p.ldx + col0;
+        const size_t x_step = static_cast<size_t>(16) * p.ldx;
+        uint4 q[kSteps];
 #pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    v[e] = __uint_as_float(static_cast<uint32_t>(__ldg(xrow + src[e])) << 16) * inv_s[e];
-            } else {
-                const uint4 q = __ldg(reinterpret_cast<const uint4*>(xrow + col0));
-                v[0] = bf16_lo(q.x); v[1] = bf16_hi(q.x); v[2] = bf16_lo(q.y); v[3] = bf16_hi(q.y);
-                v[4] = bf16_lo(q.z); v[5] = bf16_hi(q.z); v[6] = bf16_lo(q.w); v[7] = bf16_hi(q.w);
+        for (int i = 0; i < kSteps; ++i) {
+            q[i] = make_uint4(0, 0, 0, 0);
+            if (col_ok && i * 16 + c < n_rows) q[i] = __ldg(reinterpret_cast<const uint4*>(xp + i * x_step));
+        }
+        uint8_t* cp = p.codes + static_cast<size_t>(row0 + c) * (K / 2) + col0 / 2;
+        const size_t c_step = static_cast<size_t>(16) * (K / 2);
+        uint8_t* rp = p.scales_row ? p.scales_row + static_cast<size_t>(row0 + c) * (K / kBlock) + gblk : nullptr;
+        const size_t r_step = static_cast<size_t>(16) * (K / kBlock);
+        const bool sf_lane = col_ok && (hl & 3) == 0;
+        const bool tail_lane = sf_lane && gblk >= tail_blk0;
+        uint8_t* tp = nullptr;                                // this lane's duplicate slot in the residual stages
+        if (tail_lane) {
+            const int t = gblk - tail_blk0;
+            tp = sf_group + (plan.S1 + t / 8) * sf_stage_stride + ((t % 8) >> 2) * 512 + ((t % 8) & 3);
+        }
+        uint8_t* ap = sf_atom + c * 16 + blk_in_atom;
+#pragma unroll
+        for (int i = 0; i < kSteps; ++i) {
+            // block amax: packed bf16 |.| and max, the two halves, then the block's 4 lanes
+            const __nv_bfloat162 a0 = __hmax2(__habs2(as_bf162(q[i].x)), __habs2(as_bf162(q[i].y)));
+            const __nv_bfloat162 a1 = __hmax2(__habs2(as_bf162(q[i].z)), __habs2(as_bf162(q[i].w)));
+            const uint32_t mm = as_u32(__hmax2(a0, a1));
+            uint32_t m = max(mm & 0xffffu, mm >> 16);
+            m = max(m, __shfl_xor_sync(0xffffffffu, m, 1));
+            m = max(m, __shfl_xor_sync(0xffffffffu, m, 2));
+            // E8M0 byte = biased exponent - 2 (floored at 0); 2^(127 - byte) as a packed bf16 pair.
+            // Multiplying bf16 by a power of two is exact (results too small for bf16 round to code 0
+            // in any case), so the scaling is done on pairs before widening to fp32.
+            const int eb = static_cast<int>(m >> 7) - 2;
+            const uint32_t byte = eb < 0 ? 0u : static_cast<uint32_t>(eb);
+            const uint32_t inv1 = (254u - byte) << 7;
+            const __nv_bfloat162 inv2 = as_bf162(inv1 | (inv1 << 16));
+            const uint32_t s0 = as_u32(__hmul2(as_bf162(q[i].x), inv2)), s1 = as_u32(__hmul2(as_bf162(q[i].y), inv2));
+            const uint32_t s2 = as_u32(__hmul2(as_bf162(q[i].z), inv2)), s3 = as_u32(__hmul2(as_bf162(q[i].w), inv2));
+            const uint32_t packed = cvt_e2m1x8(__uint_as_float(s0 << 16), __uint_as_float(s0 & 0xffff0000u),
+                                               __uint_as_float(s1 << 16), __uint_as_float(s1 & 0xffff0000u),
+                                               __uint_as_float(s2 << 16), __uint_as_float(s2 & 0xffff0000u),
+                                               __uint_as_float(s3 << 16), __uint_as_float(s3 & 0xffff0000u));
+            const bool row_ok = i * 16 + c < n_rows;
+            if (col_ok && row_ok) *reinterpret_cast<uint32_t*>(cp + i * c_step) = packed;
+            if (sf_lane && row_ok) {
+                // row r = 16 i + c of the group: atom offset (r % 32) * 16 + (r / 32) * 4 + block
+                ap[(i & 1) * 256 + (i >> 1) * 4] = static_cast<uint8_t>(byte);
+                if (rp) rp[i * r_step] = static_cast<uint8_t>(byte);
+                if (tail_lane) tp[((i & 1) * 16 + c) * 16 + (i >> 1) * 4] = static_cast<uint8_t>(byte);
             }
-        } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) v[e] = 0.f;
         }
-        // block amax over the 4 lanes of a 32-element block (bit patterns of |v| order like the values)
-        uint32_t am = 0;
+    } else {
+        // ---- scale + permute: gathered 2-byte loads (the head of the permutation is nearly the identity,
+        // so they coalesce), multiply by the stored reciprocal scale in fp32 ----
+#pragma unroll 2
+        for (int i = 0; i < kSteps; ++i) {
+            const int r = row_of(i);
+            const int rc = min(r, n_rows - 1);
+            float v[8];
+            const uint16_t* xrow = p.x + static_cast<size_t>(row0 + rc) * p.ldx;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) am = max(am, __float_as_uint(v[e]) & 0x7fffffffu);
-        am = max(am, __shfl_xor_sync(0xffffffffu, am, 1));
-        am = max(am, __shfl_xor_sync(0xffffffffu, am, 2));
-        // E8M0 byte = biased exponent - 2, floored at 0; multiply by 2^(127 - byte) (exact)
-        const int eb = static_cast<int>(am >> 23) - 2;
-        const uint32_t byte = eb < 0 ? 0u : static_cast<uint32_t>(eb);
-        const float inv = __uint_as_float((254u - byte) << 23);
-        uint32_t packed = 0;
+            for (int e = 0; e < 8; ++e)
+                v[e] = col_ok ? __uint_as_float(static_cast<uint32_t>(__ldg(xrow + src[e])) << 16) * inv_s[e] : 0.f;
+            uint32_t am = 0;
 #pragma unroll
-        for (int e = 0; e < 8; e += 2) {
-            uint32_t b = cvt_e2m1x2(v[e] * inv, v[e + 1] * inv);
-            // keep the sign bit of inputs whose magnitude rounded to zero
-            b |= ((__float_as_uint(v[e]) >> 28) & 0x8u) | ((__float_as_uint(v[e + 1]) >> 24) & 0x80u);
-            packed |= b << (4 * e);
-        }
-        if (col_ok) {
-            *reinterpret_cast<uint32_t*>(p.codes + static_cast<size_t>(row) * (K / 2) + col0 / 2) = packed;
-            if ((lane & 3) == 0) {
-                sf_tile[sf_offset_in_group(r, blk_in_stage)] = static_cast<uint8_t>(byte);
-                if (p.scales_row) p.scales_row[static_cast<size_t>(row) * (K / kBlock) + gblk] = static_cast<uint8_t>(byte);
-                if (gblk >= tail_blk0) {  // duplicate the tail block's scale into its residual stage
-                    const int t = gblk - tail_blk0;
-                    const int ts = plan.S1 + t / (kStageK / kBlock);
-                    sf_base[ts * sf_stage_stride + group * sf_group_stride +
-                            sf_offset_in_group(r, t % (kStageK / kBlock))] = static_cast<uint8_t>(byte);
+            for (int e = 0; e < 8; ++e) am = max(am, __float_as_uint(v[e]) & 0x7fffffffu);
+            am = max(am, __shfl_xor_sync(0xffffffffu, am, 1));
+            am = max(am, __shfl_xor_sync(0xffffffffu, am, 2));
+            const uint32_t byte = scale_byte(am);
+            const uint32_t packed = encode8(v, byte);
+            if (col_ok && r < n_rows) {
+                const int row = row0 + r;
+                *reinterpret_cast<uint32_t*>(p.codes + static_cast<size_t>(row) * (K / 2) + col0 / 2) = packed;
+                if ((hl & 3) == 0) {
+                    sf_atom[(r & 31) * 16 + (r >> 5) * 4 + blk_in_atom] = static_cast<uint8_t>(byte);
+                    if (p.scales_row) p.scales_row[static_cast<size_t>(row) * (K / kBlock) + gblk] = static_cast<uint8_t>(byte);
+                    if (gblk >= tail_blk0) {
+                        const int t = gblk - tail_blk0;
+                        sf_group[(plan.S1 + t / 8) * sf_stage_stride + sf_offset_in_group(r, t % 8)] = static_cast<uint8_t>(byte);
+                    }
                 }
             }
         }
     }
     __syncthreads();
-    // the tile's scale bytes, coalesced (rows past the end and blocks past K stay zero = 2^-127)
-    if (threadIdx.x < kSfGroupBytes / 16) {
-        reinterpret_cast<uint4*>(sf_base + stage * sf_stage_stride + group * sf_group_stride)[threadIdx.x] =
-            reinterpret_cast<const uint4*>(sf_tile)[threadIdx.x];
+    // the atom's scale bytes, coalesced (rows past the end and blocks past K stay zero = 2^-127)
+    if (threadIdx.x < 32) {
+        reinterpret_cast<uint4*>(sf_group + stage * sf_stage_stride + (atom & 1) * 512)[threadIdx.x] =
+            reinterpret_cast<const uint4*>(sf_atom)[threadIdx.x];
     }
-    // The CTA of the last main stage also zero-fills what nobody else writes in the residual stages:
+    const int n_atoms = gridDim.x;
+    // An odd atom count leaves the second half of the last main stage without an owner: zero it.
+    if (atom == n_atoms - 1 && (n_atoms & 1) && threadIdx.x >= 32 && threadIdx.x < 64)
+        reinterpret_cast<uint4*>(sf_group + stage * sf_stage_stride + 512)[threadIdx.x - 32] = make_uint4(0, 0, 0, 0);
+    // The CTA of the last atom also zero-fills what nobody else writes in the residual stages:
     // blocks past k_tail, and every byte of rows past the end of the group.
-    if (stage == plan.S1 - 1 && plan.S > plan.S1) {
+    if (atom == n_atoms - 1 && plan.S > plan.S1) {
         const int nb = kStageK / kBlock;
         for (int idx = threadIdx.x; idx < (plan.S - plan.S1) * kGroupRows * nb; idx += kQuantThreads) {
             const int ts = idx / (kGroupRows * nb);
             const int r = (idx / nb) % kGroupRows;
             const int b = idx % nb;
-            const bool live = (row0 + r < row_end) && (ts * nb + b) < k_tail / kBlock;
-            if (!live)
-                sf_base[(plan.S1 + ts) * sf_stage_stride + group * sf_group_stride + sf_offset_in_group(r, b)] = 0;
+            const bool live = (r < n_rows) && (ts * nb + b) < k_tail / kBlock;
+            if (!live) sf_group[(plan.S1 + ts) * sf_stage_stride + sf_offset_in_group(r, b)] = 0;
         }
     }
 }
@@ -176,8 +240,7 @@ quant_act_kernel(QuantParams p) {
 }  // namespace
 
 cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_groups, cudaStream_t stream) {
-    const StagePlan plan(p.K, p.k_tail);
-    dim3 grid(plan.S1, grid_groups);
+    dim3 grid((p.K + kAtomK - 1) / kAtomK, grid_groups);
     if (scale_perm) quant_act_kernel<true><<<grid, kQuantThreads, 0, stream>>>(p);
     else quant_act_kernel<false><<<grid, kQuantThreads, 0, stream>>>(p);
     return cudaGetLastError();
