@@ -145,16 +145,21 @@ prq_status prq_quantize_act(const prq_weights *w, prq_act_mode mode, const void 
                             const int32_t *expert_offsets, void *codes, void *scales_row, void *scales_sf,
                             prq_stream_t stream);
 
-/* Scratch the GEMM needs for M rows (split-K partial sums and tile counters); may be 0. */
+/* Scratch prq_linear needs for M rows: 0 for M <= 128 (the split-K partial sums of the decode kernel meet
+ * in distributed shared memory); for larger M the stream-K prefill kernel needs one flag per output tile
+ * and one fp32 partial tile per SM (about 17 MB on a B200).  Calls on different streams that may overlap
+ * need separate workspaces. */
 size_t prq_linear_workspace_bytes(const prq_weights *w, int M);
 
 /* Eq. (3): y = [Q(x) | Q(x)_tail] [Q(W D P) | Q(R)]^T, one block-scaled FP4 GEMM over K + k with fp32
  * accumulation.  Reads activation columns [0, K) and then [K - k, K) again; no M x (K + k) buffer exists.
  *   codes, scales_sf  device, as written by prq_quantize_act for the same w and M
  *   y                 device out, M x N, row stride ldy elements, dtype y_dtype (fp32 for parity)
- *   workspace         device, at least prq_linear_workspace_bytes(w, M) bytes, 16-byte aligned; its first
- *                     use must be zero-filled by the caller, the kernels leave it zeroed again
- * M <= 128 takes the weight-streaming split-K path, larger M the persistent prefill path. */
+ *   workspace         device, at least prq_linear_workspace_bytes(w, M) bytes, 16-byte aligned (may be NULL
+ *                     when that is 0); zero-filled by the caller before its first use, the kernel leaves
+ *                     its flags zeroed again
+ * M <= 128 takes the weight-streaming cluster split-K kernel, larger M the stream-K prefill kernel.
+ * Errors: INVALID_ARG, ALIGNMENT (y, ldy, workspace), WORKSPACE (too small), CUDA (launch failed). */
 prq_status prq_linear(const prq_weights *w, const void *codes, const void *scales_sf, int M, void *y, int ldy,
                       prq_dtype y_dtype, void *workspace, size_t workspace_bytes, prq_stream_t stream);
 

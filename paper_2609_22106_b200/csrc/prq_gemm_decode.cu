@@ -122,6 +122,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // set-up done: let the next kernel of the stream be scheduled (its launch latency then overlaps this
+    // kernel), and wait until the activation codes an earlier kernel wrote are settled (and nobody
+    // still reads y)
+    grid_launch_dependents();
+    grid_dependency_wait();
     const uint32_t tmem_base = tmem_slot;
     long long* trace = (p.trace && blockIdx.x < 4) ? p.trace + blockIdx.x * 512 : nullptr;
     if (trace && threadIdx.x == 0) trace[500] = clock64();
@@ -304,13 +309,15 @@ cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = p.splits;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, decode_kernel<BN>, tm_act, tm_w, p);
 }
 

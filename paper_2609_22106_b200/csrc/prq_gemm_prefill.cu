@@ -151,6 +151,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant
     const int G = gridDim.x, g = blockIdx.x;
     const uint32_t W = static_cast<uint32_t>(p.m_tiles) * p.n_tiles * S;
 
+    if (p.trace && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p.trace[2048 + 2 * blockIdx.x] = static_cast<long long>(t);
+    }
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
         for (int i = 0; i < 2; ++i) {
@@ -170,6 +175,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // set-up done: let the next kernel of the stream be scheduled (its launch latency then overlaps this
+    // kernel), and wait until everything earlier kernels wrote (activation codes, workspace flags) or
+    // still read (y) is settled
+    grid_launch_dependents();
+    grid_dependency_wait();
     const uint32_t tmem_base = tmem_slot;
     const int trace_cta0 = p.dbg >> 16;  // developer aid: first of the four traced CTAs
     long long* trace = (p.trace && static_cast<int>(blockIdx.x) >= trace_cta0 && static_cast<int>(blockIdx.x) < trace_cta0 + 4)
@@ -394,6 +404,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant
     tc_fence_before_sync();
     __syncthreads();
     if (trace && threadIdx.x == 0) trace[501] = clock64();
+    if (p.trace && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p.trace[2049 + 2 * blockIdx.x] = static_cast<long long>(t);
+    }
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();
@@ -412,8 +427,17 @@ cudaError_t launch_prefill(const CUtensorMap& tm_act, const CUtensorMap& tm_w, c
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    prefill_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tm_act, tm_w, tm_y, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_kernel, tm_act, tm_w, tm_y, p);
 }
 
 }  // namespace prq

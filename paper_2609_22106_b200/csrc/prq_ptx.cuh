@@ -21,6 +21,15 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of the library is launched with programmatic stream serialisation: it may start while
+// the previous kernel of the stream is still running, so that launch latency and its own set-up overlap
+// that kernel's tail.  It must pass grid_dependency_wait() before it reads or writes any global memory
+// that an earlier kernel may still touch, and it calls grid_launch_dependents() once its own CTAs are
+// running so that the next kernel can be scheduled.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");

@@ -15,6 +15,7 @@
 
 #include "prq_internal.h"
 #include "prq_kernels.h"
+#include "prq_ptx.cuh"
 
 namespace prq {
 namespace {
@@ -60,6 +61,12 @@ __global__ void __launch_bounds__(kQuantThreads)
 quant_act_kernel(QuantParams p) {
     __shared__ __align__(16) uint8_t sf_atom[512];
     __shared__ int s_tile_start[kMaxExperts + 1];
+
+    // Launched with programmatic stream serialisation: this CTA may be running while the previous kernel
+    // of the stream still is.  Nothing global is touched before the wait (x may be that kernel's output,
+    // and it may still be reading the buffers written here).
+    grid_launch_dependents();
+    grid_dependency_wait();
 
     const int atom = blockIdx.x;                  // 128-column slice of the reduction axis
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -240,10 +247,16 @@ quant_act_kernel(QuantParams p) {
 }  // namespace
 
 cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_groups, cudaStream_t stream) {
-    dim3 grid((p.K + kAtomK - 1) / kAtomK, grid_groups);
-    if (scale_perm) quant_act_kernel<true><<<grid, kQuantThreads, 0, stream>>>(p);
-    else quant_act_kernel<false><<<grid, kQuantThreads, 0, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((p.K + kAtomK - 1) / kAtomK, grid_groups);
+    cfg.blockDim = dim3(kQuantThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return scale_perm ? cudaLaunchKernelEx(&cfg, quant_act_kernel<true>, p) : cudaLaunchKernelEx(&cfg, quant_act_kernel<false>, p);
 }
 
 }  // namespace prq

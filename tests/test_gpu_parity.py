@@ -252,9 +252,15 @@ def test_empty_batch_and_errors(prq, oracle):
         buf = torch.empty(4 * 128 + 1, dtype=torch.float32, device="cuda")
         prq.linear(w, codes, sf, 4, out=buf[1:].view(4, 128))
     assert e.value.code == 2
-    with pytest.raises(prq.PrqError) as e:  # workspace too small for the split-K path
-        prq.linear(w, codes, sf, 4, workspace=torch.zeros(16, dtype=torch.uint8, device="cuda"))
-    assert e.value.code in (8, 0) or True
+    # the prefill path needs its stream-K workspace; the decode path needs none
+    L2 = synth.layer(96, 128, 256, 200, T_cal=32)
+    codes2, _, sf2 = prq.quantize_act(w, to_dev_bf16(L2["x"]), prq.ACT_IDENTITY)
+    with pytest.raises(prq.PrqError) as e:
+        prq.linear(w, codes2, sf2, 200, workspace=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == 8
+    assert prq.linear_workspace_bytes(w, 4) == 0 and prq.linear_workspace_bytes(w, 200) > 0
+    y = prq.linear(w, codes, sf, 4, workspace=torch.zeros(16, dtype=torch.uint8, device="cuda"))
+    assert y.shape == (4, 128)
     w.free()
 
 
