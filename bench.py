@@ -27,6 +27,9 @@ if ROOT not in sys.path:
 METRIC = "PRQuant W4A4 GEMM µs & TFLOP/s, Qwen3-4B down_proj; % of FP4/HBM roofline"
 N_OUT, K_IN, K_TAIL, M_TOK = 2560, 9728, 256, 2048
 FP4_OVER_BF16 = 4.0  # nominal dense tensor ratio (9 vs 2.25 PFLOP/s)
+# DRAM bytes of one prefill GEMM launch at this workload from the ncu capture summarised in
+# profiles/prefill_M2048.txt (dram__bytes_read.sum + dram__bytes_write.sum; the outputs were still in L2).
+NCU_PREFILL_DRAM_BYTES = 24.37e6 + 0.63e6
 
 
 def peaks():
@@ -374,7 +377,7 @@ def main():
                "bf16_matmul": bf16_us[M_TOK], "gemm_speedup_vs_bf16": bf16_us[M_TOK] / main_t["gemm_us"]},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": fp4_peak, "unit": "TFLOP/s",
                      "frac": achieved / fp4_peak, "frac_of_sustained": achieved / (pk["bf16_tflops_sustained"] * FP4_OVER_BF16),
-                     "traffic": None,
+                     "traffic": NCU_PREFILL_DRAM_BYTES, "algorithmic_bytes": gemm_bytes(M_TOK, K_TAIL),
                      "kernel": "prefill_kernel (stream-K, 128x224 tiles)", "launch_us": gemm_us,
                      "peak_source": f"4 x bf16 burst, of {pk['source']}"},
         "cpu_baseline": cpu,
