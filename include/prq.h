@@ -45,7 +45,8 @@ typedef enum {
     PRQ_ERR_OOM = 5,
     PRQ_ERR_TIMEOUT = 6,
     PRQ_ERR_NONFINITE = 7,
-    PRQ_ERR_WORKSPACE = 8
+    PRQ_ERR_WORKSPACE = 8,
+    PRQ_ERR_STATIC_SCRATCH = 9
 } prq_status;
 
 typedef struct prq_weights prq_weights; /* opaque: prepared weights of one layer (or of E stacked experts) */
@@ -162,6 +163,27 @@ size_t prq_linear_workspace_bytes(const prq_weights *w, int M);
  * Errors: INVALID_ARG, ALIGNMENT (y, ldy, workspace), WORKSPACE (too small), CUDA (launch failed). */
 prq_status prq_linear(const prq_weights *w, const void *codes, const void *scales_sf, int M, void *y, int ldy,
                       prq_dtype y_dtype, void *workspace, size_t workspace_bytes, prq_stream_t stream);
+
+/* prq_linear for callers that can neither allocate device memory nor hand over a workspace.  (The paper
+ * has no counterpart to this call; it exists for deployment.)  Think of an inference server whose memory
+ * pool already owns the whole GPU, so that a later cudaMalloc would fail, or of a plugin that runs inside
+ * a host application which forbids allocation calls on its threads.  The product is the same as
+ * prq_linear's; the stream-K scratch (tile flags and fp32 partial tiles) lives in an array that is part
+ * of the library image instead of in caller memory.
+ *   - Arguments as for prq_linear, minus the workspace.  The handle's device must be the current device.
+ *   - Limits: at most 16384 output tiles (ceil(M/128) * ceil(N/224)) and at most 160 SMs; beyond that the
+ *     call returns PRQ_ERR_STATIC_SCRATCH and launches nothing.  M <= 128 needs no scratch and is passed on.
+ *   - Cost: the array is 18,415,616 bytes (64 KB of flags + 160 partial tiles of 112 KB) on every GPU that
+ *     loads the library, until the process exits.
+ *   - The call itself performs no allocation (no cudaMalloc / cudaFree, no allocating library routine); it
+ *     enqueues one small memset of the flags and the kernel.  The first call on a device also looks up the
+ *     array's device address; make that first call outside any stream capture.
+ *   - All calls share the one array, which keeps the previous call's contents (the flags are cleared on
+ *     every call, the partial tiles are written before they are read).  Two calls that can overlap on the
+ *     GPU -- different streams, or one stream per thread -- race on it: serialise them, or give the
+ *     overlapping callers prq_linear with workspaces of their own. */
+prq_status prq_linear_static_scratch(const prq_weights *w, const void *codes, const void *scales_sf, int M, void *y,
+                                     int ldy, prq_dtype y_dtype, prq_stream_t stream);
 
 /* The same product for stacked experts (MoE): rows [expert_offsets[e], expert_offsets[e+1]) of the
  * activation use expert e's weights.  expert_offsets: device, n_experts + 1 int32, non-decreasing,

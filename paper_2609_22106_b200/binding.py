@@ -23,7 +23,7 @@ BUF_CODES, BUF_SCALES_ROW, BUF_SCALES_SF = range(3)
 EXPORTS = [
     "prq_prepare_weights", "prq_prepare_weights_host", "prq_prepare_weights_search", "prq_weights_free",
     "prq_weights_clone", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
-    "prq_linear", "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
+    "prq_linear", "prq_linear_static_scratch", "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count",
 ]
 
@@ -60,6 +60,7 @@ def lib():
         L.prq_linear_workspace_bytes.argtypes = [vp, ci]
         L.prq_linear_workspace_bytes.restype = cs
         L.prq_linear.argtypes = [vp, vp, vp, ci, vp, ci, ci, vp, cs, vp]
+        L.prq_linear_static_scratch.argtypes = [vp, vp, vp, ci, vp, ci, ci, vp]
         L.prq_linear_grouped.argtypes = [vp, vp, vp, vp, ci, vp, ci, ci, vp]
         L.prq_forward_host_scratch_bytes.argtypes = [vp, ci]
         L.prq_forward_host_scratch_bytes.restype = cs
@@ -229,6 +230,20 @@ def linear(w: Weights, codes, scales_sf, M: int, y_dtype: int = F32, workspace=N
         workspace = new_workspace(w, M, codes.device)
     _check(lib().prq_linear(w.handle, _dptr(codes), _dptr(scales_sf), M, _dptr(out), out.stride(0) if M else w.N,
                             y_dtype, _dptr(workspace), workspace.numel(), _stream_ptr(stream)), "prq_linear")
+    return out
+
+
+def linear_static_scratch(w: Weights, codes, scales_sf, M: int, y_dtype: int = F32, out=None, stream=None):
+    """prq_linear without a caller workspace: the scratch is an array inside the library (see include/prq.h
+    for the size limits and the rule that overlapping calls race).  `out` must be supplied by callers that
+    may not allocate; it is created here only as a convenience for tests."""
+    import torch
+
+    if out is None:
+        out = torch.empty((M, w.N), dtype=torch.float32 if y_dtype == F32 else torch.bfloat16, device=codes.device)
+    _check(lib().prq_linear_static_scratch(w.handle, _dptr(codes), _dptr(scales_sf), M, _dptr(out),
+                                           out.stride(0) if M else w.N, y_dtype, _stream_ptr(stream)),
+           "prq_linear_static_scratch")
     return out
 
 

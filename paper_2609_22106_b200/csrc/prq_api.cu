@@ -187,6 +187,7 @@ const char* prq_status_string(prq_status s) {
         case PRQ_ERR_TIMEOUT: return "a device-side wait expired";
         case PRQ_ERR_NONFINITE: return "non-finite input";
         case PRQ_ERR_WORKSPACE: return "workspace too small";
+        case PRQ_ERR_STATIC_SCRATCH: return "problem exceeds the library's built-in scratch (too many output tiles or SMs)";
     }
     return "unknown status";
 }
@@ -720,3 +721,67 @@ prq_status prq_forward_host(const prq_weights* w, prq_act_mode mode, const uint1
 }
 
 }  // extern "C"
+
+// ---- prq_linear_static_scratch: the GEMM for callers that cannot hand over (or allocate) a workspace ----
+namespace prq {
+namespace {
+
+// Built-in scratch of the stream-K prefill kernel: one flag per output tile, then one fp32 partial tile
+// per CTA.  It is part of the library image, so every GPU that loads the library carries it until the
+// process exits: 64 KB of flags + 160 x 112 KB of partial tiles = 18,415,616 bytes.
+constexpr int kStaticMaxTiles = 16384;
+constexpr int kStaticMaxCtas = 160;
+constexpr size_t kStaticFlagBytes = static_cast<size_t>(kStaticMaxTiles) * sizeof(int);
+constexpr size_t kStaticScratchBytes = kStaticFlagBytes + static_cast<size_t>(kStaticMaxCtas) * kPrefillSlotBytes;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticScratchDev {
+    bool ready = false;
+    void* ptr = nullptr;
+};
+StaticScratchDev g_static_dev[64];
+
+// Device address of the array on device `dev` (which must be current).  In host code the array's name
+// is only a handle for the runtime, not an address a kernel could use, so the address is looked up
+// once per device and cached.
+prq_status static_scratch_address(int dev, void** out) {
+    if (dev < 0 || dev >= 64) return PRQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_dev_mutex);
+    StaticScratchDev& d = g_static_dev[dev];
+    if (!d.ready) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) {
+            cudaGetLastError();
+            return PRQ_ERR_CUDA;
+        }
+        d.ptr = p;
+        d.ready = true;
+    }
+    *out = d.ptr;
+    return PRQ_OK;
+}
+
+}  // namespace
+}  // namespace prq
+
+extern "C" prq_status prq_linear_static_scratch(const prq_weights* w, const void* codes, const void* scales_sf, int M,
+                                                void* y, int ldy, prq_dtype y_dtype, prq_stream_t stream) {
+    if (!w || M < 0) return PRQ_ERR_INVALID_ARG;
+    if (M <= 128) return prq_linear(w, codes, scales_sf, M, y, ldy, y_dtype, nullptr, 0, stream);  // needs no scratch
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PRQ_ERR_CUDA;
+    if (dev != w->device) return PRQ_ERR_INVALID_ARG;  // the handle's device must be current
+    DeviceInfo* di;
+    prq_status st = device_info(dev, &di);
+    if (st != PRQ_OK) return st;
+    const size_t tiles = static_cast<size_t>((M + 127) / 128) * ((w->N + kPrefillTileN - 1) / kPrefillTileN);
+    if (tiles > static_cast<size_t>(kStaticMaxTiles) || di->num_sms > kStaticMaxCtas) return PRQ_ERR_STATIC_SCRATCH;
+    void* scratch = nullptr;
+    st = static_scratch_address(dev, &scratch);
+    if (st != PRQ_OK) return st;
+    // The array still holds whatever the previous call left there.  The partial tiles are always written
+    // before they are read; the tile flags must start at zero.
+    if (cudaMemsetAsync(scratch, 0, prefill_flag_bytes(w, M), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return PRQ_ERR_CUDA;
+    return prq_linear(w, codes, scales_sf, M, y, ldy, y_dtype, scratch, kStaticScratchBytes, stream);
+}
