@@ -108,6 +108,143 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+class GraphTimer:
+    """Replays calls from CUDA graphs between one pair of events (device time, launching stream)."""
+
+    def __init__(self, torch, dev):
+        self.torch = torch
+        self.side = torch.cuda.Stream(device=dev)
+
+    def capture(self, fns):
+        torch = self.torch
+        for f in fns:
+            f()  # first calls configure the kernels; must precede capture
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=self.side):
+            for f in fns:
+                f()
+        return g
+
+    def run(self, fns, n, warm):
+        """Exactly n calls, round-robin over `fns`, between one pair of events; returns seconds.  The calls
+        are replayed from two CUDA graphs (one whole rotation, one remainder) so that the host-side cost
+        of a call (ctypes, tensor-map encoding) cannot starve the GPU inside the timed region."""
+        torch = self.torch
+        R = len(fns)
+        g_full = self.capture(fns)
+        g_rem = self.capture(fns[: n % R]) if n % R else None
+        for _ in range(max(1, warm // R)):
+            g_full.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n // R):
+            g_full.replay()
+        if g_rem is not None:
+            g_rem.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e-3
+
+
+def rotation_count(bytes_per_set, lo=2, hi=24, l2_bytes=126e6):
+    """How many independent operand sets make one rotation larger than twice the L2."""
+    return int(min(hi, max(lo, np.ceil(2.2 * l2_bytes / bytes_per_set))))
+
+
+# Shapes of one Qwen3-4B-shaped decoder block's linears (BASELINE configs[2]): name -> (N, K, k_tail).
+BLOCK_LINEARS = {"q": (4096, 2560, 128), "k": (1024, 2560, 128), "v": (1024, 2560, 128), "o": (2560, 4096, 128),
+                 "gate": (9728, 2560, 128), "up": (9728, 2560, 128), "down": (2560, 9728, 256)}
+
+
+def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_layers=1, tag="block"):
+    """configs[2] / configs[4]: the seven linears of a decoder block at M tokens (n_layers distinct weight
+    sets, cycled).  A step = for every linear: prq_quantize_act (online scale + permute, identity for down_proj)
+    + prq_linear with bf16 output.  Returns per-linear device times and the whole-step time."""
+    timer = GraphTimer(torch, dev)
+    fp4_peak = pk["bf16_tflops"] * FP4_OVER_BF16
+    layers = []
+    for li in range(n_layers):
+        lin = {}
+        for j, (name, (N, K, k)) in enumerate(BLOCK_LINEARS.items()):
+            k = k if k_override is None else k_override
+            L = synth.layer(2, N, K, M, T_cal=128, tag=10 * li + j)
+            amax = np.abs(synth.bf16_to_f32(L["zcal"])).max(axis=0)
+            w = prq.prepare_weights(L["W"], amax, 0.5, k)
+            x = torch.from_numpy(L["x"].view(np.int16)).to(dev).view(torch.bfloat16)
+            codes = torch.empty(prq.act_bytes(M, K, k, 1, prq.BUF_CODES), dtype=torch.uint8, device=dev)
+            sf = torch.empty(prq.act_bytes(M, K, k, 1, prq.BUF_SCALES_SF), dtype=torch.uint8, device=dev)
+            y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+            lin[name] = dict(w=w, x=x, codes=codes, sf=sf, y=y, ws=prq.new_workspace(w, M, dev), N=N, K=K, k=k,
+                             mode=prq.ACT_IDENTITY if name == "down" else prq.ACT_SCALE_PERM,
+                             Wb=torch.from_numpy(L["W"].view(np.int16)).to(dev).view(torch.bfloat16))
+        layers.append(lin)
+
+    def q(d):
+        return lambda: prq.quantize_act(d["w"], d["x"], d["mode"], out=(d["codes"], None, d["sf"]))
+
+    def g(d):
+        return lambda: prq.linear(d["w"], d["codes"], d["sf"], M, prq.BF16, workspace=d["ws"], out=d["y"])
+
+    rows = {}
+    n = max(n_layers, 20)
+    for name in BLOCK_LINEARS:
+        ds = [lin[name] for lin in layers]
+        tq = timer.run([q(d) for d in ds], n, n_layers) / n * 1e6
+        tg = timer.run([g(d) for d in ds], n, n_layers) / n * 1e6
+        tb = timer.run([(lambda d=d: torch.matmul(d["x"], d["Wb"].t())) for d in ds], n, n_layers) / n * 1e6
+        N, K, k = ds[0]["N"], ds[0]["K"], ds[0]["k"]
+        fl = 2.0 * M * N * (K + k)
+        by = 0.53125 * N * (K + k) + 0.53125 * M * K + 2.0 * M * N
+        t_roof = max(fl / fp4_peak / 1e6, by / pk["hbm_gbs"] / 1e3)
+        rows[name] = dict(N=N, K=K, k=k, quant_us=tq, gemm_us=tg, bf16_matmul_us=tb, gemm_tflops=fl / tg / 1e6,
+                          gemm_gbs=by / tg / 1e3, gemm_roofline_frac=t_roof / tg,
+                          bound="tensor" if fl / fp4_peak / 1e6 > by / pk["hbm_gbs"] / 1e3 else "hbm")
+    step_fns = [(lambda lin=lin: [f() for name in BLOCK_LINEARS for f in (q(lin[name]), g(lin[name]))]) for lin in layers]
+    t_step = timer.run(step_fns, n, n_layers) / n
+    total_flops = sum(2.0 * M * N * (K + (k if k_override is None else k_override)) for N, K, k in BLOCK_LINEARS.values())
+    status = prq.last_device_status()
+    for lin in layers:
+        for d in lin.values():
+            d["w"].free()
+    return dict(workload=tag, M=M, layers=n_layers, step_us=t_step * 1e6, step_tflops=total_flops / t_step / 1e12,
+                gemm_us_sum=sum(r["gemm_us"] for r in rows.values()), quant_us_sum=sum(r["quant_us"] for r in rows.values()),
+                bf16_us_sum=sum(r["bf16_matmul_us"] for r in rows.values()), device_status=status, linears=rows)
+
+
+def run_moe_workload(args, torch, prq, synth, dev, pk, T):
+    """configs[3]: Qwen3-30B-A3B-shaped expert down_proj, 128 experts of 2048 x 768, tail 64, T tokens routed
+    top-8 with Zipf popularity.  A step = grouped quantise + grouped GEMM (bf16 output)."""
+    timer = GraphTimer(torch, dev)
+    E, N, K, k = 128, 2048, 768, 64
+    Ws = np.stack([synth.weights(3000 + e, N, K) for e in range(E)])
+    ch = synth.HeavyTailChannels(3005, K)
+    amax = np.stack([np.abs(synth.bf16_to_f32(ch.rows(3100 + e, 64))).max(axis=0) for e in range(E)])
+    w = prq.prepare_weights(Ws, amax, 0.5, k)
+    _, offsets, _ = synth.zipf_routing(3004, T, E)
+    M = int(offsets[-1])
+    x = torch.from_numpy(ch.rows(3001, M).view(np.int16)).to(dev).view(torch.bfloat16)
+    d_off = torch.from_numpy(offsets).to(dev)
+    codes = torch.empty(prq.act_bytes(M, K, k, E, prq.BUF_CODES), dtype=torch.uint8, device=dev)
+    sf = torch.empty(prq.act_bytes(M, K, k, E, prq.BUF_SCALES_SF), dtype=torch.uint8, device=dev)
+    y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
+    q = lambda: prq.quantize_act(w, x, prq.ACT_SCALE_PERM, expert_offsets=d_off, out=(codes, None, sf))
+    g = lambda: prq.linear_grouped(w, codes, sf, d_off, M, prq.BF16, out=y)
+    n = 20
+    tq = timer.run([q], n, 3) / n * 1e6
+    tg = timer.run([g], n, 3) / n * 1e6
+    active = int((np.diff(offsets) > 0).sum())
+    fl = 2.0 * M * N * (K + k)
+    by = 0.53125 * active * N * (K + k) + 0.53125 * M * K + 2.0 * M * N
+    t_roof = max(fl / (pk["bf16_tflops"] * FP4_OVER_BF16) / 1e6, by / pk["hbm_gbs"] / 1e3)
+    status = prq.last_device_status()
+    w.free()
+    return dict(workload="moe", T=T, rows=M, active_experts=active, quant_us=tq, gemm_us=tg, gemm_tflops=fl / tg / 1e6,
+                gemm_gbs=by / tg / 1e3, gemm_roofline_frac=t_roof / tg, device_status=status,
+                note="weights (116 MB for 128 experts) are re-read every launch; they nearly fit the 126 MB L2")
+
+
 def physical_gpu_index(local_rank):
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -161,6 +298,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--full", action="store_true", help="also time every (M, k) of the down_proj config")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="down_proj", choices=["down_proj", "block", "moe", "stack"],
+                    help="down_proj = the headline config (default); block / moe / stack = BASELINE configs 2, 3, 4")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -192,6 +331,26 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.workload != "down_proj":
+        # context workloads: one JSON line each, same peaks; rank 0 only (they are not the headline metric)
+        if rank == 0:
+            if args.workload == "block":
+                res = [run_block_workload(args, torch, prq, synth, dev, pk, 4096)]
+            elif args.workload == "moe":
+                res = [run_moe_workload(args, torch, prq, synth, dev, pk, T) for T in (64, 1024, 8192)]
+            else:
+                res = [run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=k, n_layers=3, tag="stack")
+                       for M in (64, 4096) for k in (256, 0)]
+                for r in res:
+                    r["stack_36_layers_us"] = 36 * r["step_us"]
+                    r["stack_36_layers_bf16_us"] = 36 * r["bf16_us_sum"]
+            print(json.dumps({"metric": METRIC, "workload": args.workload, "unit": "us / TFLOP/s", "n_gpus": 1,
+                              "dtype": "mxfp4 (e2m1 x e8m0), f32 accumulate, bf16 output", "data": "synthetic",
+                              "results": res}))
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
     # ---- inputs (seeded, synthetic, Qwen3-4B down_proj shape, heavy-tailed activations) ----
     L = synth.layer(1, N_OUT, K_IN, M_TOK, T_cal=512)
     amax = np.abs(synth.bf16_to_f32(L["zcal"])).max(axis=0)
@@ -199,7 +358,6 @@ def main():
     base = {k: prq.prepare_weights(L["W"], amax, 0.5, k) for k in ks}
     x_src = torch.from_numpy(L["x"].view(np.int16)).to(dev).view(torch.bfloat16)
     W_bf16 = torch.from_numpy(L["W"].view(np.int16)).to(dev).view(torch.bfloat16)
-    L2_BYTES = 126e6
     clones = {k: [base[k]] for k in ks}
 
     def weight_copies(k, n):
@@ -212,7 +370,7 @@ def main():
         """Enough independent (weights, x, codes, scales, y, workspace) sets that one pass over all of them
         touches more than twice the L2: every launch then finds its operands in HBM, without any flush."""
         per_set = 2.0 * M * K_IN + 0.53125 * M * K_IN + 0.53125 * N_OUT * (K_IN + k) + 4.0 * M * N_OUT
-        R = int(min(24, max(2, np.ceil(2.2 * L2_BYTES / per_set))))
+        R = rotation_count(per_set)
         sets = []
         for w in weight_copies(k, R):
             x = x_src[:M].clone()
@@ -222,37 +380,8 @@ def main():
             sets.append(dict(w=w, x=x, codes=codes, sf=sf, y=y, ws=prq.new_workspace(w, M, dev)))
         return sets
 
-    side = torch.cuda.Stream(device=dev)
-
-    def capture(fns):
-        for f in fns:
-            f()  # first calls configure the kernels; must precede capture
-        torch.cuda.synchronize()
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g, stream=side):
-            for f in fns:
-                f()
-        return g
-
-    def run_timed(fns, n, warm):
-        """Exactly n calls, round-robin over `fns`, between one pair of events; returns seconds.  The calls
-        are replayed from two CUDA graphs (one whole rotation, one remainder) so that the host-side cost
-        of a call (ctypes, tensor-map encoding) cannot starve the GPU inside the timed region."""
-        R = len(fns)
-        g_full = capture(fns)
-        g_rem = capture(fns[: n % R]) if n % R else None
-        for _ in range(max(1, warm // R)):
-            g_full.replay()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for _ in range(n // R):
-            g_full.replay()
-        if g_rem is not None:
-            g_rem.replay()
-        b.record()
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) * 1e-3
+    timer = GraphTimer(torch, dev)
+    run_timed = timer.run
 
     def build_graphs(M, k, y_dtype=prq.F32):
         sets = operand_sets(M, k, y_dtype)
@@ -271,7 +400,7 @@ def main():
                     step_total_s=t_step, rotation_sets=gs["R"], timed_launches=2 * steps)
 
     def time_bf16(M, steps):
-        R = int(min(12, max(2, np.ceil(2.2 * L2_BYTES / (2.0 * N_OUT * K_IN + 2.0 * M * K_IN + 2.0 * M * N_OUT)))))
+        R = rotation_count(2.0 * N_OUT * K_IN + 2.0 * M * K_IN + 2.0 * M * N_OUT, hi=12)
         Ws = [W_bf16.clone() for _ in range(R)]
         xs = [x_src[:M].clone() for _ in range(R)]
         ys = [torch.empty((M, N_OUT), dtype=torch.bfloat16, device=dev) for _ in range(R)]
@@ -293,12 +422,11 @@ def main():
                   rotation_sets=main_graphs["R"], timed_launches=2 * args.steps)
     launches = main_t["timed_launches"]  # K replays of a (quantise, GEMM) graph
     status = prq.last_device_status()
-    if dist is not None:
-        t = torch.tensor([total_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_s = float(t.item())
+    from paper_2609_22106_b200.replicas import job_time_and_throughput
+
+    total_s, flops_per_s = job_time_and_throughput(total_s, args.steps * flops(M_TOK, K_TAIL), dist, dev)
     ms_per_step = total_s / args.steps * 1e3
-    value = world * flops(M_TOK, K_TAIL) / (ms_per_step * 1e-3) / 1e12
+    value = flops_per_s / 1e12
 
     # ---- end to end from host buffers (H2D of x, D2H of y inside the timed region) ----
     xh = torch.from_numpy(L["x"].view(np.int16).copy()).view(torch.bfloat16).pin_memory()
@@ -315,11 +443,8 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     e2e_s = e0.elapsed_time(e1) * 1e-3
-    if dist is not None:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_val = world * flops(M_TOK, K_TAIL) * e2e_steps / e2e_s / 1e12
+    e2e_s, e2e_flops_per_s = job_time_and_throughput(e2e_s, e2e_steps * flops(M_TOK, K_TAIL), dist, dev)
+    e2e_val = e2e_flops_per_s / 1e12
 
     if rank != 0:
         if dist is not None:

@@ -107,6 +107,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     const int s_end = static_cast<int>(static_cast<long long>(S) * (split + 1) / splits);
     const int n0 = tile * 128;
 
+    const long long t_entry = clock64();
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
         mbar_init(smem_u32(&bar_acc_full), 1);
@@ -125,11 +126,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     // set-up done: let the next kernel of the stream be scheduled (its launch latency then overlaps this
     // kernel), and wait until the activation codes an earlier kernel wrote are settled (and nobody
     // still reads y)
+    const long long t_setup = clock64();
     grid_launch_dependents();
     grid_dependency_wait();
     const uint32_t tmem_base = tmem_slot;
     long long* trace = (p.trace && blockIdx.x < 4) ? p.trace + blockIdx.x * 512 : nullptr;
-    if (trace && threadIdx.x == 0) trace[500] = clock64();
+    if (trace && threadIdx.x == 0) { trace[500] = clock64(); trace[502] = t_entry; trace[503] = t_setup; }
     const uint32_t lo_base = ((smem_base & 0x3FFFF) >> 4) | (1u << 16);
 
     if (warp == 0) {
