@@ -28,6 +28,7 @@ struct DeviceInfo {
     int num_sms = 0;
     int* status_ptr = nullptr;
     int max_clusters[4][9] = {};  // decode kernel: [token-tile index][cluster size], 0 = not queried yet
+    int max_pairs = 0;            // prefill pair kernel: co-resident CTA pairs, 0 = not queried yet
 };
 std::mutex g_dev_mutex;
 DeviceInfo g_dev[64];
@@ -78,6 +79,21 @@ prq_status make_code_map(CUtensorMap* map, const void* base, uint64_t row_bytes,
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
+// Scale bytes in the tensor-core layout are a flat array of 1024-byte groups; seen as rows of 256 bytes,
+// a box of 4 rows is one group.  No swizzle: the bytes land in shared memory in array order.
+prq_status make_sf_map(CUtensorMap* map, const void* base, uint64_t total_bytes, uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return PRQ_ERR_CUDA;
+    cuuint64_t dims[2] = {256, total_bytes / 256};
+    cuuint64_t strides[1] = {256};
+    cuuint32_t box[2] = {256, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? PRQ_OK : PRQ_ERR_CUDA;
 }
@@ -164,9 +180,12 @@ constexpr int kNumAlt = 3;
 constexpr int kAltTileRows[kNumAlt] = {160, 192, 224};  // weight tile widths with their own scale layout
 constexpr size_t kPrefillSlotBytes = 128 * kPrefillTileN * sizeof(float);
 
+// One flag per 128-row half of a 256 x 224 pair tile.
+size_t prefill_flag_count(const prq_weights* w, int M) {
+    return 2 * static_cast<size_t>((M + 255) / 256) * ((w->N + kPrefillTileN - 1) / kPrefillTileN);
+}
 size_t prefill_flag_bytes(const prq_weights* w, int M) {
-    const size_t tiles = static_cast<size_t>((M + 127) / 128) * ((w->N + kPrefillTileN - 1) / kPrefillTileN);
-    return (tiles * sizeof(int) + 255) & ~static_cast<size_t>(255);
+    return (prefill_flag_count(w, M) * sizeof(int) + 255) & ~static_cast<size_t>(255);
 }
 
 }  // namespace
@@ -594,6 +613,37 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         cudaError_t e = launch_decode(bn, tm_act, tm_w, q, (w->N + 127) / 128, static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+    } else if (env_int("PRQ_PREFILL_BN", 0) == 0 && env_int("PRQ_PAIR", 1) != 0) {
+        // stream-K kernel on CTA pairs with 256 x 224 tiles (scale bytes grouped per 224-row weight tile)
+        PrefillParams q;
+        std::memset(&q, 0, sizeof(q));
+        q.M = M; q.N = w->N; q.K = w->K; q.k_tail = w->k_tail;
+        q.m_tiles = (M + 255) / 256; q.n_tiles = (w->N + kPrefillTileN - 1) / kPrefillTileN;
+        q.act_groups = p.act_groups; q.w_groups = w->w_groups_alt[2];
+        q.act_sf = p.act_sf; q.w_sf = w->d_sf_alt[2];
+        q.y_bf16 = p.y_bf16; q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
+        const size_t flag_bytes = prefill_flag_bytes(w, M);
+        const long long units = static_cast<long long>(q.m_tiles) * q.n_tiles * w->plan.S;
+        if (di->max_pairs == 0) di->max_pairs = std::min(prefill_pair_max_clusters(), di->num_sms / 2);
+        const int max_pairs = std::min(di->max_pairs, env_int("PRQ_GRID", 1 << 20));
+        const int pairs = static_cast<int>(std::min<long long>(units, max_pairs));
+        if (pairs < 1) return PRQ_ERR_CUDA;
+        if (units * pairs >= (1ll << 32)) return PRQ_ERR_INVALID_ARG;  // the kernel's range arithmetic is 32-bit
+        if (!workspace || workspace_bytes < flag_bytes + static_cast<size_t>(2 * pairs) * kPrefillSlotBytes) return PRQ_ERR_WORKSPACE;
+        if (!aligned16(workspace)) return PRQ_ERR_ALIGNMENT;
+        q.flags = static_cast<int*>(workspace);
+        q.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + flag_bytes);
+        CUtensorMap tm_y, tm_sfa, tm_sfw;
+        const uint64_t Sg = static_cast<uint64_t>(w->plan.S);
+        st = make_code_map(&tm_act, codes, w->K / 2, M, 128);
+        if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, kPrefillTileN / 2);
+        if (st == PRQ_OK) st = make_sf_map(&tm_sfa, p.act_sf, Sg * p.act_groups * kSfGroupBytes, 4);
+        if (st == PRQ_OK) st = make_sf_map(&tm_sfw, q.w_sf, Sg * q.w_groups * kSfGroupBytes, 8);
+        if (st == PRQ_OK) st = make_out_map(&tm_y, y, M, w->N, ldy, y_dtype == PRQ_BF16);
+        if (st != PRQ_OK) return st;
+        cudaError_t e = launch_prefill_pair(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, q, pairs, static_cast<cudaStream_t>(stream));
+        g_launches.fetch_add(1);
+        return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     } else if (env_int("PRQ_PREFILL_BN", 0) == 0) {
         // stream-K kernel with 128 x 224 tiles (scale bytes grouped per 224-row weight tile)
         PrefillParams q;
@@ -605,7 +655,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         q.y_bf16 = p.y_bf16; q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
         const size_t flag_bytes = prefill_flag_bytes(w, M);
         const long long units = static_cast<long long>(q.m_tiles) * q.n_tiles * w->plan.S;
-        const int g = static_cast<int>(std::min<long long>(units, di->num_sms));
+        const int g = static_cast<int>(std::min<long long>(units, env_int("PRQ_GRID", di->num_sms)));
         if (units * g >= (1ll << 32)) return PRQ_ERR_INVALID_ARG;  // the kernel's range arithmetic is 32-bit
         if (!workspace || workspace_bytes < flag_bytes + static_cast<size_t>(g) * kPrefillSlotBytes) return PRQ_ERR_WORKSPACE;
         if (!aligned16(workspace)) return PRQ_ERR_ALIGNMENT;
@@ -774,8 +824,7 @@ extern "C" prq_status prq_linear_static_scratch(const prq_weights* w, const void
     DeviceInfo* di;
     prq_status st = device_info(dev, &di);
     if (st != PRQ_OK) return st;
-    const size_t tiles = static_cast<size_t>((M + 127) / 128) * ((w->N + kPrefillTileN - 1) / kPrefillTileN);
-    if (tiles > static_cast<size_t>(kStaticMaxTiles) || di->num_sms > kStaticMaxCtas) return PRQ_ERR_STATIC_SCRATCH;
+    if (prefill_flag_count(w, M) > static_cast<size_t>(kStaticMaxTiles) || di->num_sms > kStaticMaxCtas) return PRQ_ERR_STATIC_SCRATCH;
     void* scratch = nullptr;
     st = static_scratch_address(dev, &scratch);
     if (st != PRQ_OK) return st;

@@ -93,4 +93,14 @@ struct PrefillParams {
 cudaError_t launch_prefill(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_y,
                            const PrefillParams& p, int grid, cudaStream_t stream);
 
+// Stream-K prefill kernel on CTA pairs (256 x 224 tiles, two CTAs of a cluster per tile).  Here
+// `m_tiles` counts 256-row tiles, `flags` holds one counter per 128-row half of a tile
+// (index 2 * tile + half) and `partial` one slot per CTA.  `tm_w` has boxes of 112 rows; `tm_sfa` /
+// `tm_sfw` view the scale bytes as rows of 256 bytes with boxes of 4 / 8 rows (one / two 128-row groups).
+cudaError_t launch_prefill_pair(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
+                                const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
+                                int pairs, cudaStream_t stream);
+// How many pairs of the pair kernel can be resident at once on the current device.
+int prefill_pair_max_clusters();
+
 }  // namespace prq
