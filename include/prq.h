@@ -147,9 +147,9 @@ prq_status prq_quantize_act(const prq_weights *w, prq_act_mode mode, const void 
                             prq_stream_t stream);
 
 /* Scratch prq_linear needs for M rows: 0 for M <= 128 (the split-K partial sums of the decode kernel meet
- * in distributed shared memory); for larger M the stream-K prefill kernel needs one flag per output tile
- * and one fp32 partial tile per SM (about 17 MB on a B200).  Calls on different streams that may overlap
- * need separate workspaces. */
+ * in distributed shared memory); for larger M the stream-K prefill kernel needs two counters per 128-row
+ * half of an output tile and two fp32 partial tiles per SM (about 34 MB on a B200).  Calls on different
+ * streams that may overlap need separate workspaces. */
 size_t prq_linear_workspace_bytes(const prq_weights *w, int M);
 
 /* Eq. (3): y = [Q(x) | Q(x)_tail] [Q(W D P) | Q(R)]^T, one block-scaled FP4 GEMM over K + k with fp32
@@ -171,10 +171,11 @@ prq_status prq_linear(const prq_weights *w, const void *codes, const void *scale
  * prq_linear's; the stream-K scratch (tile flags and fp32 partial tiles) lives in an array that is part
  * of the library image instead of in caller memory.
  *   - Arguments as for prq_linear, minus the workspace.  The handle's device must be the current device.
- *   - Limits: at most 16384 output tiles (ceil(M/128) * ceil(N/224)) and at most 160 SMs; beyond that the
- *     call returns PRQ_ERR_STATIC_SCRATCH and launches nothing.  M <= 128 needs no scratch and is passed on.
- *   - Cost: the array is 18,415,616 bytes (64 KB of flags + 160 partial tiles of 112 KB) on every GPU that
- *     loads the library, until the process exits.
+ *   - Limits: at most 8192 output half-tiles (2 * ceil(M/256) * ceil(N/224)) and at most 160 SMs; beyond
+ *     that the call returns PRQ_ERR_STATIC_SCRATCH and launches nothing.  M <= 128 needs no scratch and is
+ *     passed on.
+ *   - Cost: the array is 36,765,696 bytes (64 KB of counters + 2 x 160 partial tiles of 112 KB) on every
+ *     GPU that loads the library, until the process exits.
  *   - The call itself performs no allocation (no cudaMalloc / cudaFree, no allocating library routine); it
  *     enqueues one small memset of the flags and the kernel.  The first call on a device also looks up the
  *     array's device address; make that first call outside any stream capture.

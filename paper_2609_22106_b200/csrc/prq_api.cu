@@ -180,12 +180,13 @@ constexpr int kNumAlt = 3;
 constexpr int kAltTileRows[kNumAlt] = {160, 192, 224};  // weight tile widths with their own scale layout
 constexpr size_t kPrefillSlotBytes = 128 * kPrefillTileN * sizeof(float);
 
-// One flag per 128-row half of a 256 x 224 pair tile.
+// Two counters ("arrived", "finished") per 128-row half of a 256 x 224 pair tile: first all the "arrived"
+// counters, then all the "finished" ones.
 size_t prefill_flag_count(const prq_weights* w, int M) {
     return 2 * static_cast<size_t>((M + 255) / 256) * ((w->N + kPrefillTileN - 1) / kPrefillTileN);
 }
 size_t prefill_flag_bytes(const prq_weights* w, int M) {
-    return (prefill_flag_count(w, M) * sizeof(int) + 255) & ~static_cast<size_t>(255);
+    return (2 * prefill_flag_count(w, M) * sizeof(int) + 255) & ~static_cast<size_t>(255);
 }
 
 }  // namespace
@@ -553,7 +554,7 @@ size_t prq_linear_workspace_bytes(const prq_weights* w, int M) {
         // stream-K prefill: one flag per 128 x 256 tile, one fp32 partial tile per CTA (at most one CTA per SM)
         DeviceInfo* di;
         if (device_info(w->device, &di) != PRQ_OK) return 0;
-        return prefill_flag_bytes(w, M) + static_cast<size_t>(di->num_sms) * kPrefillSlotBytes;
+        return prefill_flag_bytes(w, M) + 2 * static_cast<size_t>(di->num_sms) * kPrefillSlotBytes;
     }
     return 0;  // decode: the split-K partial sums meet in distributed shared memory
 }
@@ -623,13 +624,26 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         q.act_sf = p.act_sf; q.w_sf = w->d_sf_alt[2];
         q.y_bf16 = p.y_bf16; q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
         const size_t flag_bytes = prefill_flag_bytes(w, M);
-        const long long units = static_cast<long long>(q.m_tiles) * q.n_tiles * w->plan.S;
+        const long long tiles = static_cast<long long>(q.m_tiles) * q.n_tiles;
+        const long long units = tiles * w->plan.S;
         if (di->max_pairs == 0) di->max_pairs = std::min(prefill_pair_max_clusters(), di->num_sms / 2);
         const int max_pairs = std::min(di->max_pairs, env_int("PRQ_GRID", 1 << 20));
         const int pairs = static_cast<int>(std::min<long long>(units, max_pairs));
         if (pairs < 1) return PRQ_ERR_CUDA;
-        if (units * pairs >= (1ll << 32)) return PRQ_ERR_INVALID_ARG;  // the kernel's range arithmetic is 32-bit
-        if (!workspace || workspace_bytes < flag_bytes + static_cast<size_t>(2 * pairs) * kPrefillSlotBytes) return PRQ_ERR_WORKSPACE;
+        // every pair gets `whole` whole tiles; the rest is shared out stream-K: each left-over tile cut into
+        // equal pieces for 2..8 consecutive pairs when there are at least two pairs per tile, else the
+        // (tile, stage) space cut into equal contiguous ranges
+        long long whole = tiles / pairs, sk = tiles - whole * pairs;
+        if (env_int("PRQ_PURE_SK", 0)) { whole = 0; sk = tiles; }
+        if (sk > 0 && pairs / sk >= 2 && !env_int("PRQ_SK_RANGES", 0)) {
+            q.sk_aligned = 1;
+            q.sk_base = static_cast<int>(std::min<long long>(pairs / sk, 8));
+            q.sk_extra = q.sk_base < 8 ? static_cast<int>(pairs % sk) : 0;
+        }
+        q.sk_tiles = static_cast<int>(sk); q.whole_tiles = static_cast<int>(whole);
+        if (sk * w->plan.S * pairs >= (1ll << 32) || tiles >= (1ll << 30)) return PRQ_ERR_INVALID_ARG;  // 32-bit range arithmetic
+        if (!workspace || workspace_bytes < flag_bytes + static_cast<size_t>(4 * pairs) * kPrefillSlotBytes) return PRQ_ERR_WORKSPACE;
+        q.flag_stride = static_cast<int>(prefill_flag_count(w, M));
         if (!aligned16(workspace)) return PRQ_ERR_ALIGNMENT;
         q.flags = static_cast<int*>(workspace);
         q.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + flag_bytes);
@@ -776,13 +790,13 @@ prq_status prq_forward_host(const prq_weights* w, prq_act_mode mode, const uint1
 namespace prq {
 namespace {
 
-// Built-in scratch of the stream-K prefill kernel: one flag per output tile, then one fp32 partial tile
-// per CTA.  It is part of the library image, so every GPU that loads the library carries it until the
-// process exits: 64 KB of flags + 160 x 112 KB of partial tiles = 18,415,616 bytes.
-constexpr int kStaticMaxTiles = 16384;
+// Built-in scratch of the stream-K prefill kernel: two counters per 128-row half of an output tile, then
+// two fp32 partial tiles per CTA.  It is part of the library image, so every GPU that loads the library
+// carries it until the process exits: 64 KB of counters + 2 x 160 x 112 KB of partial tiles = 36,765,696 bytes.
+constexpr int kStaticMaxFlags = 8192;   // tile halves
 constexpr int kStaticMaxCtas = 160;
-constexpr size_t kStaticFlagBytes = static_cast<size_t>(kStaticMaxTiles) * sizeof(int);
-constexpr size_t kStaticScratchBytes = kStaticFlagBytes + static_cast<size_t>(kStaticMaxCtas) * kPrefillSlotBytes;
+constexpr size_t kStaticFlagBytes = 2 * static_cast<size_t>(kStaticMaxFlags) * sizeof(int);
+constexpr size_t kStaticScratchBytes = kStaticFlagBytes + 2 * static_cast<size_t>(kStaticMaxCtas) * kPrefillSlotBytes;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 struct StaticScratchDev {
@@ -824,7 +838,7 @@ extern "C" prq_status prq_linear_static_scratch(const prq_weights* w, const void
     DeviceInfo* di;
     prq_status st = device_info(dev, &di);
     if (st != PRQ_OK) return st;
-    if (prefill_flag_count(w, M) > static_cast<size_t>(kStaticMaxTiles) || di->num_sms > kStaticMaxCtas) return PRQ_ERR_STATIC_SCRATCH;
+    if (prefill_flag_count(w, M) > static_cast<size_t>(kStaticMaxFlags) || di->num_sms > kStaticMaxCtas) return PRQ_ERR_STATIC_SCRATCH;
     void* scratch = nullptr;
     st = static_scratch_address(dev, &scratch);
     if (st != PRQ_OK) return st;

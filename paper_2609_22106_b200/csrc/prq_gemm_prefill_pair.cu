@@ -7,14 +7,16 @@
 // each CTA loads its own 128 activation rows and only 112 of the 224 weight rows, the tensor cores read
 // the other half from the peer's shared memory, and the bytes per SM and stage drop by 30 %.
 //
-// Why stream-K.  2048 tokens x 2560 features are 8 x 12 = 96 pair tiles on 74 pairs; tile-per-pair
-// scheduling would leave a third of the machine idle in its second wave.  The (tile, reduction-stage)
-// space is cut into equal contiguous ranges, one per pair.  A range covers the tail of one tile, whole
-// tiles, and the head of another.  The pair that holds a tile's first stage owns it; any other pair
-// working on it writes its fp32 partial accumulators to workspace slots (one per CTA) and raises the
-// flags of the tile's two halves.  Every pair processes its leading (contributed) segment first and its
-// trailing (owned) segment last, so an owner finds the contributions long finished and no pair ever
-// waits on work that is queued behind its own.
+// Schedule.  2048 tokens x 2560 features are 8 x 12 = 96 pair tiles on 74 pairs; tile-per-pair
+// scheduling would leave a third of the machine idle in its second wave.  So every pair gets the same
+// number of whole tiles (one here), and the tiles left over (22) are processed stream-K: their (tile,
+// reduction-stage) space is cut into equal contiguous ranges, one per pair, which the pairs work off
+// FIRST.  A range is a piece of one tile or the tail of one and the head of the next.  The pair that
+// holds a tile's first stage owns it; the others write their fp32 partial accumulators to workspace
+// slots (one per CTA) and raise the flags of the tile's two halves; the owner adds them in a fixed
+// order.  All of this fix-up traffic and waiting happens while the pairs' main loops are busy with
+// their whole tiles; what is exposed at the end of every pair is one plain tile epilogue, the same
+// for all of them.
 //
 // Roles (6 warps per CTA):
 //   warp 0    TMA producer (both CTAs): per 256-element reduction stage its own activation tile, its
@@ -67,16 +69,6 @@ __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src_smem
                  ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(src_smem), "r"(x), "r"(y)
                  : "memory");
 }
-// y[tile] += staging tile, performed by the memory system (one fp32 add per element, so the sum of two
-// contributions does not depend on their order).
-__device__ __forceinline__ void tma_reduce_add_2d(const void* tmap, uint32_t src_smem, int x, int y) {
-    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(reinterpret_cast<uint64_t>(tmap)), "r"(src_smem), "r"(x), "r"(y)
-                 : "memory");
-}
-// All bulk stores of this thread are complete (written, not only read from shared memory).
-__device__ __forceinline__ void bulk_wait_all_done() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() {
@@ -93,26 +85,78 @@ struct Segment {
     int tile, s0, s1;   // reduction stages [s0, s1) of `tile`
 };
 
-// The contiguous range of (tile, stage) units of one pair, walked segment by segment.
+// The work of one pair, walked segment by segment: first its contiguous range of (tile, stage) units of
+// the stream-K tiles, then its whole tiles (tile ids sk_tiles + wave * G + pair).
 // All of this is 32-bit arithmetic (the host checks that W * G fits): 64-bit divisions cost hundreds of
 // cycles each and sit on the critical path of every role's first instruction.
 struct Range {
     uint32_t cur, end;
     int S;
+    int next_whole, whole_left, G;
     __device__ __forceinline__ bool next(Segment& g) {
-        if (cur >= end) return false;
-        g.tile = static_cast<int>(cur / static_cast<uint32_t>(S));
-        g.s0 = static_cast<int>(cur - static_cast<uint32_t>(g.tile) * S);
-        const uint32_t left = end - cur;
-        g.s1 = left < static_cast<uint32_t>(S - g.s0) ? g.s0 + static_cast<int>(left) : S;
-        cur += g.s1 - g.s0;
-        return true;
+        if (cur < end) {
+            g.tile = static_cast<int>(cur / static_cast<uint32_t>(S));
+            g.s0 = static_cast<int>(cur - static_cast<uint32_t>(g.tile) * S);
+            const uint32_t left = end - cur;
+            g.s1 = left < static_cast<uint32_t>(S - g.s0) ? g.s0 + static_cast<int>(left) : S;
+            cur += g.s1 - g.s0;
+            return true;
+        }
+        if (whole_left > 0) {
+            g.tile = next_whole;
+            g.s0 = 0;
+            g.s1 = S;
+            next_whole += G;
+            --whole_left;
+            return true;
+        }
+        return false;
     }
 };
 
 __device__ __forceinline__ uint32_t range_begin(uint32_t W, int g, int G) {
     return W * static_cast<uint32_t>(g) / static_cast<uint32_t>(G);
 }
+
+// How the stream-K tiles are shared out.
+//   aligned: tile t is cut into P(t) equal pieces for P(t) consecutive pairs (sk_base + 1 pairs for the
+//            first sk_extra tiles, sk_base for the others), so that every pair has one piece at most and
+//            publishes once;
+//   ranges:  the (tile, stage) units are cut into G equal contiguous ranges; a range may hold the tail of
+//            one tile and the head of the next (two pieces).  Used when the aligned split would be too
+//            coarse to balance (fewer than two pairs per tile).
+struct SkPlan {
+    int aligned, base, extra, S, G;
+    uint32_t W;
+    // the pairs that work on `tile`: first pair and count
+    __device__ __forceinline__ void participants(int tile, int g, int& first, int& P) const {
+        if (aligned) {
+            if (tile < extra) { first = tile * (base + 1); P = base + 1; }
+            else { first = extra * (base + 1) + (tile - extra) * base; P = base; }
+        } else {
+            const uint32_t u0 = static_cast<uint32_t>(tile) * S, u1 = u0 + S - 1;
+            int gf = g, gl = g;
+            while (gf > 0 && range_begin(W, gf, G) > u0) --gf;
+            while (gl + 1 < G && range_begin(W, gl + 1, G) <= u1) ++gl;
+            first = gf; P = gl - gf + 1;
+        }
+    }
+    // which of its two workspace slots pair `pair` uses for its piece of `tile`
+    __device__ __forceinline__ int slot_index(int pair, int tile) const {
+        return (!aligned && range_begin(W, pair, G) < static_cast<uint32_t>(tile) * S) ? 1 : 0;
+    }
+    // the stream-K units [b, e) of pair g
+    __device__ __forceinline__ void range(int g, uint32_t& b, uint32_t& e) const {
+        if (!aligned) { b = range_begin(W, g, G); e = range_begin(W, g + 1, G); return; }
+        int tile, j, P;
+        const int cut = extra * (base + 1);
+        if (g < cut) { tile = g / (base + 1); j = g - tile * (base + 1); P = base + 1; }
+        else { const int h = g - cut; tile = extra + h / base; j = h - (tile - extra) * base; P = base; }
+        if (static_cast<uint32_t>(tile) * S >= W) { b = e = 0; return; }   // more pairs than pieces
+        b = static_cast<uint32_t>(tile) * S + static_cast<uint32_t>(S * j) / P;
+        e = static_cast<uint32_t>(tile) * S + static_cast<uint32_t>(S * (j + 1)) / P;
+    }
+};
 
 constexpr uint32_t kHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);  // SBO 1024, version 1, 128B swizzle
 constexpr uint32_t kHiPlain = (128u >> 4) | (1u << 14);                // SBO 128, version 1, no swizzle
@@ -167,7 +211,10 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     const StagePlan plan(p.K, p.k_tail);
     const int S = plan.S, S1 = plan.S1;
     const int G = gridDim.x >> 1, g = blockIdx.x >> 1;   // pairs
-    const uint32_t W = static_cast<uint32_t>(p.m_tiles) * p.n_tiles * S;
+    const uint32_t W = static_cast<uint32_t>(p.sk_tiles) * S;   // stream-K units, shared out over all pairs
+    const SkPlan plan_sk{p.sk_aligned, p.sk_base, p.sk_extra, S, G, W};
+    uint32_t sk_b, sk_e;
+    plan_sk.range(g, sk_b, sk_e);
 
     if (p.trace && threadIdx.x == 0) {
         unsigned long long t;
@@ -200,8 +247,18 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     // set-up done: let the next kernel of the stream be scheduled (its launch latency then overlaps this
     // kernel), and wait until everything earlier kernels wrote (activation codes, workspace flags) or
     // still read (y) is settled
+    if (p.trace && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p.trace[2048 + 400 + 2 * blockIdx.x] = static_cast<long long>(t);
+    }
     grid_launch_dependents();
     grid_dependency_wait();
+    if (p.trace && threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p.trace[2048 + 401 + 2 * blockIdx.x] = static_cast<long long>(t);
+    }
     const uint32_t tmem_base = tmem_slot;
     const int trace_cta0 = p.dbg >> 16;  // developer aid: first of the four traced CTAs
     long long* trace = (p.trace && static_cast<int>(blockIdx.x) >= trace_cta0 && static_cast<int>(blockIdx.x) < trace_cta0 + 4)
@@ -211,7 +268,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer (both CTAs)
-        Range r{range_begin(W, g, G), range_begin(W, g + 1, G), S};
+        Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G};
         Segment sg;
         int st = 0, it = 0;
         uint32_t ph = 0;
@@ -246,7 +303,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (rank == 0) {
-            Range r{range_begin(W, g, G), range_begin(W, g + 1, G), S};
+            Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G};
             Segment sg;
             const bool leader = elect_one();
             int it = 0, st = 0, seg_it = 0;
@@ -294,156 +351,167 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         const int row_in_tile = q4 * 32 + lane;  // row of this CTA's 128-row half
         const uint32_t stage_smem = staging_base + (warp - 2) * kStagingPerWarp;
         const uint32_t leader_acc_empty0 = cluster_map(smem_u32(&bar_acc_empty[0]), 0);
-        Range r{range_begin(W, g, G), range_begin(W, g + 1, G), S};
+        Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G};
         Segment sg;
         int seg_it = 0, store_it = 0;
         bool ok = true;
+
+        // 32 accumulator columns of this warp's 32 rows -> y: swizzled shared staging, then one TMA store
+        // (rows and columns outside M x N are clipped by the tensor map)
+        auto store_chunk = [&](const uint32_t (&v)[32], int x, int y_row) {
+            const uint32_t sbuf = stage_smem + (store_it & 1) * 4096;
+            // the store issued two chunks ago has finished reading this buffer
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+            if (!p.y_bf16) {
+                // 128-byte staging rows, 16-byte unit index ^= row % 8
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    st_shared_v4(sbuf + lane * 128 + ((u ^ (lane & 7)) << 4), v[4 * u], v[4 * u + 1], v[4 * u + 2], v[4 * u + 3]);
+            } else {
+                // 64-byte staging rows (32 bf16), unit index ^= (row / 2) % 4
+                uint32_t h[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                    h[i] = *reinterpret_cast<uint32_t*>(&t2);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    st_shared_v4(sbuf + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4), h[4 * u], h[4 * u + 1], h[4 * u + 2], h[4 * u + 3]);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(&tm_y, sbuf, x, y_row);
+                bulk_commit();
+            }
+            ++store_it;
+        };
+
+        // A stream-K tile is finished in two steps.  Publish: every pair that computed a piece of it writes
+        // its fp32 partial tile to a workspace slot and counts itself on the "arrived" counter of its
+        // 128-row half.  Fix up: once all P pieces have arrived, participant i sums, always in piece order,
+        // the column chunks c = i, i + P, ... over all pieces and stores them to y; the last participant to
+        // finish clears the counters for the next launch.  The fix-ups are deferred until all of the pair's
+        // own pieces are published (a fix-up waits for other pairs; a publication must never wait), and
+        // they run while the main loop works on the pair's whole tiles.
+        struct Fixup { int tile, first_pair, P; };
+        Fixup fix[2];
+        int n_fix = 0;
+        auto slot_of = [&](int pair, int tile) -> const float4* {
+            const int k = plan_sk.slot_index(pair, tile);
+            return reinterpret_cast<const float4*>(p.partial) +
+                   static_cast<size_t>(2 * (2 * pair + static_cast<int>(rank)) + k) * (kChunks * 8 * 128);
+        };
+        auto run_fixups = [&]() {
+            for (int f = 0; f < n_fix && ok; ++f) {
+                const Fixup fx = fix[f];
+                int* arrived = p.flags + 2 * fx.tile + rank;
+                int* finished = arrived + p.flag_stride;
+                if (lane == 0) {
+                    volatile int* a = arrived;
+                    const long long t0 = clock64();
+                    while (*a < fx.P) {
+                        if (*abort_flag) break;
+                        if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
+                    }
+                }
+                __syncwarp();
+                if (*abort_flag) { ok = false; break; }
+                __threadfence();
+                const int mi = fx.tile % p.m_tiles, ni = fx.tile / p.m_tiles;
+                const int y_row = mi * 256 + static_cast<int>(rank) * 128 + q4 * 32;
+                for (int c = g - fx.first_pair; c < kChunks; c += fx.P) {
+                    // unit (c, u) of row r sits at float4 index (c * 8 + u) * 128 + r of a slot
+                    const size_t off = static_cast<size_t>(c) * 8 * 128 + row_in_tile;
+                    float4 a4[8], b4[8];
+                    const float4* s0p = slot_of(fx.first_pair, fx.tile) + off;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) a4[u] = __ldcg(s0p + u * 128);
+                    for (int j = 1; j < fx.P; ++j) {
+                        const float4* sp = slot_of(fx.first_pair + j, fx.tile) + off;
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) b4[u] = __ldcg(sp + u * 128);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            a4[u].x += b4[u].x; a4[u].y += b4[u].y; a4[u].z += b4[u].z; a4[u].w += b4[u].w;
+                        }
+                    }
+                    uint32_t v[32];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        v[4 * u] = __float_as_uint(a4[u].x); v[4 * u + 1] = __float_as_uint(a4[u].y);
+                        v[4 * u + 2] = __float_as_uint(a4[u].z); v[4 * u + 3] = __float_as_uint(a4[u].w);
+                    }
+                    store_chunk(v, ni * BN + c * kChunkCols, y_row);
+                }
+                // all four warps have read what they need of this half
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (row_in_tile == 0) {
+                    if (atomicAdd(finished, 1) == fx.P - 1) { *finished = 0; *arrived = 0; }
+                }
+                if (trace && row_in_tile == 0 && f < 2) trace[208 + f] = clock64();
+            }
+            n_fix = 0;
+        };
+
         while (ok && r.next(sg)) {
             const int mi = sg.tile % p.m_tiles, ni = sg.tile / p.m_tiles;
             const int buf = seg_it & 1;
-            const bool contributor = sg.s0 > 0;
-            int* flag = p.flags + 2 * sg.tile + rank;   // one flag per 128-row half of the tile
-            int n_contrib = 0;
-            if (!contributor && sg.s1 < S) {
-                // owner of a tile that other pairs finish: they are the next pairs in order
-                const uint32_t last_unit = static_cast<uint32_t>(sg.tile + 1) * S - 1;
-                int gl = g + 1;
-                while (gl + 1 < G && range_begin(W, gl + 1, G) <= last_unit) ++gl;
-                n_contrib = gl - g;
-            }
-            // Direct fix-up (fp32 output, tile shared by exactly two pairs): the contributor stores its partial
-            // tile straight into y and the owner adds its own on top with a TMA reduction; no workspace
-            // round trip, and x + y is the same in either order.  Otherwise (bf16, or three and more pairs,
-            // whose order of addition must stay fixed) the partials go through the workspace.
-            const bool direct = !p.y_bf16 &&
-                (contributor ? (sg.s1 == S && range_begin(W, g - 1, G) <= static_cast<uint32_t>(sg.tile) * S)
-                             : n_contrib == 1);
+            const bool piece = sg.s1 - sg.s0 < S;
+            // all of this pair's pieces are published: fix up now, overlapping the main loop of this whole tile
+            if (!piece && n_fix > 0 && r.cur >= r.end) run_fixups();
+            if (!ok) break;
             if (!mbar_wait(smem_u32(&bar_acc_full[buf]), (seg_it >> 1) & 1, abort_flag)) { ok = false; break; }
             if (trace && row_in_tile == 0 && seg_it < 8) trace[192 + 2 * seg_it] = clock64();
             tc_fence_after_sync();
             const uint32_t acc_t = tmem_base + buf * BN + (static_cast<uint32_t>(q4 * 32) << 16);
-            if (contributor && !direct) {
-                // partial accumulator -> this CTA's slot, stored column-major so that warps write full lines
-                float* slot = p.partial + static_cast<size_t>(blockIdx.x) * (128 * BN) + row_in_tile;
+            if (piece) {
+                // publish this piece: partial accumulator -> workspace slot (one 512-byte line per warp store)
+                const int k = plan_sk.slot_index(g, sg.tile);
+                float4* slot = reinterpret_cast<float4*>(p.partial) +
+                               static_cast<size_t>(2 * blockIdx.x + k) * (kChunks * 8 * 128) + row_in_tile;
 #pragma unroll 1
                 for (int c = 0; c < kChunks; ++c) {
                     uint32_t v[32];
                     tmem_ld_32x32(acc_t + c * kChunkCols, v);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) __stcg(slot + (c * kChunkCols + i) * 128, __uint_as_float(v[i]));
+                    for (int u = 0; u < 8; ++u)
+                        __stcg(slot + (c * 8 + u) * 128,
+                               make_float4(__uint_as_float(v[4 * u]), __uint_as_float(v[4 * u + 1]),
+                                           __uint_as_float(v[4 * u + 2]), __uint_as_float(v[4 * u + 3])));
                 }
                 tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(leader_acc_empty0 + buf * 8);
-                // publish: all four warps' stores, then one count on the flag of this half
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (row_in_tile == 0) atomicAdd(flag, 1);
+                if (row_in_tile == 0) atomicAdd(p.flags + 2 * sg.tile + rank, 1);
+                int first, P;
+                plan_sk.participants(sg.tile, g, first, P);
+                fix[n_fix++] = Fixup{sg.tile, first, P};
             } else {
-                const bool add_ws = n_contrib > 0 && !direct;     // owner: add the partials parked in the workspace
-                const bool reduce = n_contrib > 0 && direct;      // owner: add onto the contributor's values in y
-                if (n_contrib > 0) {
-                    // wait (bounded) until every contribution to this half has been published
-                    if (lane == 0) {
-                        volatile int* f = flag;
-                        const long long t0 = clock64();
-                        while (*f < n_contrib) {
-                            if (*abort_flag) break;
-                            if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
-                        }
-                    }
-                    __syncwarp();
-                    if (*abort_flag) { ok = false; break; }
-                    __threadfence();
-                    fence_proxy_async_all();
-                    if (trace && row_in_tile == 0 && seg_it < 8) trace[208 + seg_it] = clock64();
-                }
-                // the contributors are the CTAs of the same rank in the following pairs
-                const float* slot = p.partial + static_cast<size_t>(blockIdx.x + 2) * (128 * BN) + row_in_tile;
                 const int y_row = mi * 256 + static_cast<int>(rank) * 128 + q4 * 32;
-                // Contributions are fetched one chunk ahead (32 independent, coalesced loads in flight while
-                // the current chunk is staged and stored); further contributors of the same tile are rare
-                // (only when a tile is shared by more than two pairs) and are read in place.
-                float nx[32];
-                if (add_ws) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) nx[i] = __ldcg(slot + i * 128);
-                }
 #pragma unroll 1
                 for (int c = 0; c < kChunks; ++c) {
                     uint32_t v[32];
                     tmem_ld_32x32(acc_t + c * kChunkCols, v);
                     tmem_ld_wait();
-                    if (add_ws) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + nx[i]);
-                        if (c + 1 < kChunks) {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) nx[i] = __ldcg(slot + ((c + 1) * kChunkCols + i) * 128);
-                        }
-                        for (int cidx = 1; cidx < n_contrib; ++cidx) {
-                            float t2[32];
-                            const float* src = slot + static_cast<size_t>(2 * cidx) * (128 * BN) + c * kChunkCols * 128;
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) t2[i] = __ldcg(src + i * 128);
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) + t2[i]);
-                        }
-                    }
-                    const uint32_t sbuf = stage_smem + (store_it & 1) * 4096;
-                    // the store issued two chunks ago has finished reading this buffer
-                    if (lane == 0) bulk_wait_read<1>();
-                    __syncwarp();
-                    if (!p.y_bf16) {
-                        // 128-byte staging rows, 16-byte unit index ^= row % 8
-#pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            st_shared_v4(sbuf + lane * 128 + ((u ^ (lane & 7)) << 4), v[4 * u], v[4 * u + 1], v[4 * u + 2], v[4 * u + 3]);
-                    } else {
-                        // 64-byte staging rows (32 bf16), unit index ^= (row / 2) % 4
-                        uint32_t h[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-                            h[i] = *reinterpret_cast<uint32_t*>(&t2);
-                        }
-#pragma unroll
-                        for (int u = 0; u < 4; ++u)
-                            st_shared_v4(sbuf + lane * 64 + ((u ^ ((lane >> 1) & 3)) << 4), h[4 * u], h[4 * u + 1], h[4 * u + 2], h[4 * u + 3]);
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        if (reduce) tma_reduce_add_2d(&tm_y, sbuf, ni * BN + c * kChunkCols, y_row);
-                        else tma_store_2d(&tm_y, sbuf, ni * BN + c * kChunkCols, y_row);
-                        bulk_commit();
-                    }
-                    ++store_it;
                     if (c == kChunks - 1) {
                         // the accumulator has been read completely: hand it back before the stores drain
                         tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(leader_acc_empty0 + buf * 8);
                     }
-                }
-                if (contributor) {
-                    // direct contribution: publish once all four warps' stores have been written
-                    if (lane == 0) bulk_wait_all_done();
-                    fence_proxy_async_all();
-                    __threadfence();
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    if (row_in_tile == 0) atomicAdd(flag, 1);
-                } else if (n_contrib > 0) {
-                    // everyone has seen (and, through the workspace, read) the contributions: clear the flag
-                    // for the next launch
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    if (row_in_tile == 0) *flag = 0;
+                    store_chunk(v, ni * BN + c * kChunkCols, y_row);
                 }
             }
             if (trace && row_in_tile == 0 && seg_it < 8) trace[193 + 2 * seg_it] = clock64();
             ++seg_it;
         }
+        if (ok && n_fix > 0) run_fixups();   // no whole tiles: the fix-ups come last
         // shared staging must not be released while a store is still reading it
         if (lane == 0) bulk_wait_read<0>();
         __syncwarp();

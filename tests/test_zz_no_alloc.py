@@ -47,7 +47,7 @@ def test_static_scratch_matches_prq_linear_twice(prq, oracle):
 
 
 def test_static_scratch_rejects_oversized_problems(prq, oracle):
-    # 16385 row tiles x 1 column tile exceed the 16384 flags of the built-in scratch: clear error, no launch
+    # 2 * 8193 half-tiles x 1 column tile exceed the 8192 counters of the built-in scratch: clear error, no launch
     W = synth.weights(5, 32, 64)
     w = prq.prepare_weights(W, np.ones(64, np.float32), 0.0, 0)
     M = 128 * 16384 + 1
