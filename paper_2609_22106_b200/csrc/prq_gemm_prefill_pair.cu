@@ -245,20 +245,14 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     cluster_wait();
     tc_fence_after_sync();
     // set-up done: let the next kernel of the stream be scheduled (its launch latency then overlaps this
-    // kernel), and wait until everything earlier kernels wrote (activation codes, workspace flags) or
-    // still read (y) is settled
+    // kernel).  Each role that touches global memory which earlier kernels wrote (activation codes,
+    // workspace counters) or still read (y) passes grid_dependency_wait() first; the issuer touches none.
     if (p.trace && threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
         p.trace[2048 + 400 + 2 * blockIdx.x] = static_cast<long long>(t);
     }
     grid_launch_dependents();
-    grid_dependency_wait();
-    if (p.trace && threadIdx.x == 0) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        p.trace[2048 + 401 + 2 * blockIdx.x] = static_cast<long long>(t);
-    }
     const uint32_t tmem_base = tmem_slot;
     const int trace_cta0 = p.dbg >> 16;  // developer aid: first of the four traced CTAs
     long long* trace = (p.trace && static_cast<int>(blockIdx.x) >= trace_cta0 && static_cast<int>(blockIdx.x) < trace_cta0 + 4)
@@ -274,6 +268,31 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         uint32_t ph = 0;
         bool ok = true;
         const uint32_t leader_full0 = cluster_map(smem_u32(&bar_full[0]), 0);
+        // The weights do not depend on earlier kernels of the stream: the weight tiles and weight scales of
+        // the first ring pass are requested before the dependency wait, so that their latency overlaps the
+        // tail of the previous kernel.
+        int pre = 0;
+        {
+            Range rr = r;
+            while (pre < kStages && rr.next(sg)) {
+                const int ni = sg.tile / p.m_tiles;
+                for (int s = sg.s0; s < sg.s1 && pre < kStages; ++s, ++pre) {
+                    if (elect_one()) {
+                        const uint32_t full = leader_full0 + pre * 8;
+                        const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
+                        const uint32_t sb = smem_base + pre * kStageBytes;
+                        tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * kHalfN, full);
+                        tma_load_2d_pair(sb + kPTile + kQTile + kSfp, &tm_sfw, 0, ni * 8 + s * p.w_groups * 4, full);
+                    }
+                }
+            }
+        }
+        grid_dependency_wait();
+        if (p.trace && threadIdx.x == 0) {
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+            p.trace[2048 + 401 + 2 * blockIdx.x] = static_cast<long long>(t);
+        }
         while (ok && r.next(sg)) {
             const int mi = sg.tile % p.m_tiles, ni = sg.tile / p.m_tiles;
             // scale bytes: rows of 256 bytes, 4 per 128-row group
@@ -289,9 +308,11 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                     const int xa = s < S1 ? s * 128 : (p.K - p.k_tail) / 2 + (s - S1) * 128;
                     const uint32_t sb = smem_base + st * kStageBytes;
                     tma_load_2d_pair(sb, &tm_act, xa, mi * 256 + static_cast<int>(rank) * 128, full);
-                    tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * kHalfN, full);
                     tma_load_2d_pair(sb + kPTile + kQTile, &tm_sfa, 0, sfa_row0 + s * sfa_stride, full);
-                    tma_load_2d_pair(sb + kPTile + kQTile + kSfp, &tm_sfw, 0, sfw_row0 + s * sfw_stride, full);
+                    if (it >= pre) {
+                        tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * kHalfN, full);
+                        tma_load_2d_pair(sb + kPTile + kQTile + kSfp, &tm_sfw, 0, sfw_row0 + s * sfw_stride, full);
+                    }
                 }
                 if (++st == kStages) { st = 0; ph ^= 1; }
             }
@@ -347,6 +368,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
+        grid_dependency_wait();
         const int q4 = warp & 3;                 // tensor-memory lane quarter of this warp
         const int row_in_tile = q4 * 32 + lane;  // row of this CTA's 128-row half
         const uint32_t stage_smem = staging_base + (warp - 2) * kStagingPerWarp;
