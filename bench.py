@@ -28,8 +28,8 @@ METRIC = "PRQuant W4A4 GEMM µs & TFLOP/s, Qwen3-4B down_proj; % of FP4/HBM roof
 N_OUT, K_IN, K_TAIL, M_TOK = 2560, 9728, 256, 2048
 FP4_OVER_BF16 = 4.0  # nominal dense tensor ratio (9 vs 2.25 PFLOP/s)
 # DRAM bytes of one prefill GEMM launch at this workload from the ncu capture summarised in
-# profiles/prefill_M2048.txt (dram__bytes_read.sum + dram__bytes_write.sum; the outputs were still in L2).
-NCU_PREFILL_DRAM_BYTES = 24.37e6 + 0.63e6
+# profiles/prefill_pair_M2048.txt (dram__bytes_read.sum + dram__bytes_write.sum; the outputs were still in L2).
+NCU_PREFILL_DRAM_BYTES = 24.39e6 + 1.14e6
 
 
 def peaks():
@@ -503,7 +503,7 @@ def main():
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": fp4_peak, "unit": "TFLOP/s",
                      "frac": achieved / fp4_peak, "frac_of_sustained": achieved / (pk["bf16_tflops_sustained"] * FP4_OVER_BF16),
                      "traffic": NCU_PREFILL_DRAM_BYTES, "algorithmic_bytes": gemm_bytes(M_TOK, K_TAIL),
-                     "kernel": "prefill_kernel (stream-K, 128x224 tiles)", "launch_us": gemm_us,
+                     "kernel": "prefill_pair_kernel (CTA pairs, 256x224 tiles, whole tiles + stream-K pieces)", "launch_us": gemm_us,
                      "peak_source": f"4 x bf16 burst, of {pk['source']}"},
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": M_TOK * K_IN * 2, "d2h_bytes_per_step": M_TOK * N_OUT * 4},

@@ -614,7 +614,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         cudaError_t e = launch_decode(bn, tm_act, tm_w, q, (w->N + 127) / 128, static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
-    } else if (env_int("PRQ_PREFILL_BN", 0) == 0 && env_int("PRQ_PAIR", 1) != 0) {
+    } else if (env_int("PRQ_PREFILL_BN", 0) == 0) {
         // stream-K kernel on CTA pairs with 256 x 224 tiles (scale bytes grouped per 224-row weight tile)
         PrefillParams q;
         std::memset(&q, 0, sizeof(q));
@@ -656,31 +656,6 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         if (st == PRQ_OK) st = make_out_map(&tm_y, y, M, w->N, ldy, y_dtype == PRQ_BF16);
         if (st != PRQ_OK) return st;
         cudaError_t e = launch_prefill_pair(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, q, pairs, static_cast<cudaStream_t>(stream));
-        g_launches.fetch_add(1);
-        return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
-    } else if (env_int("PRQ_PREFILL_BN", 0) == 0) {
-        // stream-K kernel with 128 x 224 tiles (scale bytes grouped per 224-row weight tile)
-        PrefillParams q;
-        std::memset(&q, 0, sizeof(q));
-        q.M = M; q.N = w->N; q.K = w->K; q.k_tail = w->k_tail;
-        q.m_tiles = (M + 127) / 128; q.n_tiles = (w->N + kPrefillTileN - 1) / kPrefillTileN;
-        q.act_groups = p.act_groups; q.w_groups = w->w_groups_alt[2];
-        q.act_sf = p.act_sf; q.w_sf = w->d_sf_alt[2];
-        q.y_bf16 = p.y_bf16; q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
-        const size_t flag_bytes = prefill_flag_bytes(w, M);
-        const long long units = static_cast<long long>(q.m_tiles) * q.n_tiles * w->plan.S;
-        const int g = static_cast<int>(std::min<long long>(units, env_int("PRQ_GRID", di->num_sms)));
-        if (units * g >= (1ll << 32)) return PRQ_ERR_INVALID_ARG;  // the kernel's range arithmetic is 32-bit
-        if (!workspace || workspace_bytes < flag_bytes + static_cast<size_t>(g) * kPrefillSlotBytes) return PRQ_ERR_WORKSPACE;
-        if (!aligned16(workspace)) return PRQ_ERR_ALIGNMENT;
-        q.flags = static_cast<int*>(workspace);
-        q.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + flag_bytes);
-        CUtensorMap tm_y;
-        st = make_code_map(&tm_act, codes, w->K / 2, M, 128);
-        if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, kPrefillTileN);
-        if (st == PRQ_OK) st = make_out_map(&tm_y, y, M, w->N, ldy, y_dtype == PRQ_BF16);
-        if (st != PRQ_OK) return st;
-        cudaError_t e = launch_prefill(tm_act, tm_w, tm_y, q, g, static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     } else {

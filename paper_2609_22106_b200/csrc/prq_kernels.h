@@ -75,33 +75,27 @@ cudaError_t launch_decode(int bn, const CUtensorMap& tm_act, const CUtensorMap& 
 // How many clusters of `splits` CTAs of the decode kernel can be resident at once on the current device.
 int decode_max_active_clusters(int bn, int splits);
 
-// Stream-K prefill kernel (128 x 224 tiles).
+// Prefill kernel (M > 128): 256 x 224 output tiles, each computed by two CTAs of a cluster.
 constexpr int kPrefillTileN = 224;
 struct PrefillParams {
     int M, N, K, k_tail;
-    int m_tiles, n_tiles;
-    int sk_tiles, whole_tiles;  // pair kernel: tiles 0 .. sk_tiles-1 are split stream-K over all pairs, then
-                                // pair g computes the whole tiles sk_tiles + wave * pairs + g, wave < whole_tiles
-    int sk_aligned, sk_base, sk_extra;  // pair kernel: how the stream-K tiles are cut (see SkPlan in the kernel)
+    int m_tiles, n_tiles;       // 256-row x 224-column tiles
+    int sk_tiles, whole_tiles;  // tiles 0 .. sk_tiles-1 are split stream-K over all pairs, then pair g
+                                // computes the whole tiles sk_tiles + wave * pairs + g, wave < whole_tiles
+    int sk_aligned, sk_base, sk_extra;  // how the stream-K tiles are cut (see SkPlan in the kernel)
     int act_groups, w_groups;   // 128-row scale groups per stage in act_sf / w_sf
     const uint8_t* act_sf;
     const uint8_t* w_sf;
-    float* partial;             // one 128 x 224 fp32 slot per CTA (column-major inside a slot)
-    int* flags;                 // one arrival counter per tile, zero between launches
-    int flag_stride;            // pair kernel: "finished" counters start this many ints behind `flags`
+    float* partial;             // two 128 x 224 fp32 slots per CTA
+    int* flags;                 // "arrived" counter per 128-row half of a tile (index 2 * tile + half) ...
+    int flag_stride;            // ... and, this many ints further, its "finished" counter; all zero between launches
     int y_bf16;
     int* status;
     long long* trace;
     int dbg;
 };
-cudaError_t launch_prefill(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_y,
-                           const PrefillParams& p, int grid, cudaStream_t stream);
-
-// Stream-K prefill kernel on CTA pairs (256 x 224 tiles, two CTAs of a cluster per tile).  Here
-// `m_tiles` counts 256-row tiles, `flags` holds an "arrived" and (flag_stride further) a "finished" counter
-// per 128-row half of a tile (index 2 * tile + half), all zero between launches, and `partial` two
-// 128 x 224 fp32 slots per CTA.  `tm_w` has boxes of 112 rows; `tm_sfa` /
-// `tm_sfw` view the scale bytes as rows of 256 bytes with boxes of 4 / 8 rows (one / two 128-row groups).
+// `tm_w` has boxes of 112 rows; `tm_sfa` / `tm_sfw` view the scale bytes as rows of 256 bytes with boxes of
+// 4 / 8 rows (one / two 128-row groups); `tm_y` has 32 x 32 boxes.
 cudaError_t launch_prefill_pair(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
                                 const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
                                 int pairs, cudaStream_t stream);

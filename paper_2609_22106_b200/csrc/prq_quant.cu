@@ -57,7 +57,7 @@ __device__ __forceinline__ uint32_t encode8(const float (&v)[8], uint32_t byte) 
 }
 
 template <bool kScalePerm>
-__global__ void __launch_bounds__(kQuantThreads)
+__global__ void __launch_bounds__(kQuantThreads, 5)
 quant_act_kernel(QuantParams p) {
     __shared__ __align__(16) uint8_t sf_atom[512];
     __shared__ int s_tile_start[kMaxExperts + 1];
