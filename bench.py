@@ -486,6 +486,20 @@ def main():
         cpu = {"value": flops(rows, K_TAIL) / dt / 1e12, "unit": "TFLOP/s", "cores": orc.num_threads(),
                "kind": "oracle", "sample": f"{rows} of {M_TOK} token rows, one pass (quantise + tail + FP64 product), {dt:.1f} s"}
 
+    # ---- what the FP4 tensor pipe itself sustains here: operands resident in shared memory, no loads ----
+    def probe(n_mma):
+        ts = []
+        for _ in range(3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            ctas = prq.mxf4_peak_probe(n_mma)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b) * 1e-3)
+        return ctas * n_mma * prq.MXF4_PROBE_FLOP_PER_MMA / sorted(ts)[1] / 1e12
+    mxf4_probe = {"burst_1.5ms": probe(20000), "sustained_17ms": probe(200000), "unit": "TFLOP/s",
+                  "what": "one CTA per SM issuing tcgen05.mma kind::mxf4 128x256x64 back to back from shared memory"}
+
     gemm_us = main_t["gemm_us"]
     achieved = flops(M_TOK, K_TAIL) / gemm_us / 1e6
     out = {
@@ -504,7 +518,10 @@ def main():
                      "frac": achieved / fp4_peak, "frac_of_sustained": achieved / (pk["bf16_tflops_sustained"] * FP4_OVER_BF16),
                      "traffic": NCU_PREFILL_DRAM_BYTES, "algorithmic_bytes": gemm_bytes(M_TOK, K_TAIL),
                      "kernel": "prefill_pair_kernel (CTA pairs, 256x224 tiles, whole tiles + stream-K pieces)", "launch_us": gemm_us,
-                     "peak_source": f"4 x bf16 burst, of {pk['source']}"},
+                     "peak_source": f"4 x bf16 burst, of {pk['source']}",
+                     "frac_of_measured_mxf4_probe": achieved / mxf4_probe["burst_1.5ms"],
+                     "frac_of_nominal_9pf": achieved / 9000.0},
+        "mxf4_probe": mxf4_probe,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": M_TOK * K_IN * 2, "d2h_bytes_per_step": M_TOK * N_OUT * 4},
         "gpu_launches": int(launches),

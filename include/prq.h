@@ -213,6 +213,14 @@ prq_status prq_last_device_status(prq_stream_t stream);
 /* Number of kernels this library has launched in this process (for benchmark bookkeeping). */
 unsigned long long prq_kernel_launch_count(void);
 
+/* Benchmark utility (the paper has no counterpart): launches, on `stream`, one CTA per SM that issues
+ * n_mma back-to-back block-scaled FP4 tensor-core instructions (M = 128, N = 256, K = 64, i.e.
+ * 2 * 128 * 256 * 64 flop each) on operands resident in shared memory -- no loads, no epilogue.  The
+ * caller times the launch; SMs * n_mma * 4,194,304 flop / time is the FP4 tensor rate this GPU sustains
+ * at the clocks it holds under that load.  n_mma: multiple of 4, 4 .. 2^24.  *n_ctas (nullable) receives
+ * the number of CTAs launched.  Errors: INVALID_ARG, CUDA. */
+prq_status prq_mxf4_peak_probe(int n_mma, int *n_ctas, prq_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

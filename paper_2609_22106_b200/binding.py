@@ -24,7 +24,7 @@ EXPORTS = [
     "prq_prepare_weights", "prq_prepare_weights_host", "prq_prepare_weights_search", "prq_weights_free",
     "prq_weights_clone", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
     "prq_linear", "prq_linear_static_scratch", "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
-    "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count",
+    "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
 ]
 
 
@@ -69,6 +69,7 @@ def lib():
         L.prq_status_string.restype = ctypes.c_char_p
         L.prq_last_device_status.argtypes = [vp]
         L.prq_kernel_launch_count.restype = ctypes.c_ulonglong
+        L.prq_mxf4_peak_probe.argtypes = [ci, ctypes.POINTER(ci), vp]
         _lib = L
     return _lib
 
@@ -277,3 +278,13 @@ def last_device_status(stream=None) -> int:
 
 def kernel_launch_count() -> int:
     return int(lib().prq_kernel_launch_count())
+
+
+MXF4_PROBE_FLOP_PER_MMA = 2 * 128 * 256 * 64
+
+
+def mxf4_peak_probe(n_mma: int, stream=None) -> int:
+    """Launches the tensor-pipe probe (n_mma instructions per CTA, one CTA per SM); returns the CTA count."""
+    n = ctypes.c_int()
+    _check(lib().prq_mxf4_peak_probe(int(n_mma), ctypes.byref(n), _stream_ptr(stream)), "prq_mxf4_peak_probe")
+    return n.value

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libprq.so")
-SOURCES = ["prq_api.cu", "prq_prep.cu", "prq_quant.cu", "prq_gemm.cu", "prq_gemm_prefill_pair.cu", "prq_gemm_decode.cu"]
+SOURCES = ["prq_api.cu", "prq_prep.cu", "prq_quant.cu", "prq_gemm.cu", "prq_gemm_prefill_pair.cu", "prq_gemm_decode.cu", "prq_peak_probe.cu"]
 
 
 def _newest_source_mtime() -> float:

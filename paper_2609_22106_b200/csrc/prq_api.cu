@@ -214,6 +214,19 @@ const char* prq_status_string(prq_status s) {
 
 unsigned long long prq_kernel_launch_count(void) { return g_launches.load(); }
 
+prq_status prq_mxf4_peak_probe(int n_mma, int* n_ctas, prq_stream_t stream) {
+    if (n_mma < 4 || n_mma > (1 << 24) || n_mma % 4) return PRQ_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PRQ_ERR_CUDA;
+    DeviceInfo* di;
+    prq_status st = device_info(dev, &di);
+    if (st != PRQ_OK) return st;
+    if (n_ctas) *n_ctas = di->num_sms;
+    cudaError_t e = launch_mxf4_peak_probe(n_mma, di->num_sms, di->status_ptr, static_cast<cudaStream_t>(stream));
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
 prq_status prq_last_device_status(prq_stream_t stream) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return PRQ_ERR_CUDA;

@@ -102,4 +102,7 @@ cudaError_t launch_prefill_pair(const CUtensorMap& tm_act, const CUtensorMap& tm
 // How many pairs of the pair kernel can be resident at once on the current device.
 int prefill_pair_max_clusters();
 
+// Benchmark utility: `grid` CTAs each issuing n_mma block-scaled FP4 MMAs (128 x 256 x 64) from shared memory.
+cudaError_t launch_mxf4_peak_probe(int n_mma, int grid, int* status, cudaStream_t stream);
+
 }  // namespace prq
