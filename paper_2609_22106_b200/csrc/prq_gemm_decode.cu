@@ -3,10 +3,13 @@
 // With few tokens the layer is bound by reading its 4-bit weights once.  The weight rows sit on the MMA
 // M axis (128-row tiles), the tokens on the N axis (16, 32, 64 or 128 columns), and the reduction axis
 // K + k is split over the CTAs of a thread-block cluster so that every SM streams a share of the
-// weights.  Each CTA of a cluster accumulates its K-range in tensor memory, parks the fp32 partial tile
-// in its own shared memory, and after one cluster barrier every CTA sums, over its peers' shared memory
-// (distributed shared memory), the tokens assigned to it and writes them to y.  No global scratch, no
-// atomics, and the summation order is fixed (peer 0, 1, ...), so the result is reproducible.
+// weights.  Each CTA of a cluster accumulates its K-range in tensor memory and then pushes, through
+// distributed shared memory, the partial sums of token t into a receive buffer of the CTA that owns
+// token t (t mod cluster size); after one cluster barrier every CTA adds up what it received and writes
+// its tokens to y.  No global scratch, no atomics, one barrier, and the summation order is fixed (peer
+// 0, 1, ...), so the result is reproducible.  For up to 32 tokens two CTAs fit on an SM, so that the
+// CTAs of the next kernel of the stream (the next layer's GEMM) are resident and streaming their weights
+// while this one finishes.
 //
 // Roles per CTA (6 warps): warp 0 TMA producer, warp 1 tcgen05 issuer (scale copies + MMAs), warps 2-5
 // epilogue and reduction.  The activation tail is re-read: stages past the K main columns load the
@@ -26,7 +29,6 @@ namespace {
 constexpr int kThreads = 192;
 constexpr int kPTile = 128 * 128;   // weight tile bytes: 128 rows x 256 codes
 constexpr int kSf = kSfGroupBytes;  // one 128-row scale group per operand and stage
-constexpr int kStages = 6;
 
 constexpr uint32_t kHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 constexpr uint32_t kHiPlain = (128u >> 4) | (1u << 14);
@@ -37,12 +39,19 @@ template <int BN>
 struct DCfg {
     static constexpr int kQTile = BN * 128;
     static constexpr int kStageBytes = kPTile + kQTile + 2 * kSf;
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024;
+    // ring depth: 5 / 4 stages leave room for two CTAs per SM at 16 / 32 tokens
+    static constexpr int kStages = BN == 16 ? 5 : BN == 32 ? 4 : BN == 64 ? 6 : 4;
+    static constexpr int kCtasPerSm = BN <= 32 ? 2 : 1;
+    // receive buffer of the split-K exchange: [peer][token slot][128 rows] fp32, ceil(BN / splits) token
+    // slots per peer, i.e. at most BN + 7 token rows of 512 bytes
+    static constexpr int kRecvBytes = (BN + 7) * 512;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kRecvBytes + 1024;
     static constexpr int kAccCols = BN < 32 ? 32 : BN;
     static constexpr int kSfCol = kAccCols;          // 8 weight-scale + 8 token-scale columns behind the accumulator
     static constexpr int kTmemCols = pow2_cols(kAccCols + 16);
     static_assert(kStageBytes % 1024 == 0, "stage slots must keep 1024-byte alignment");
     static_assert(BN * 128 * 4 <= kStages * kStageBytes, "the partial tile is parked in the pipeline buffers");
+    static_assert(kCtasPerSm * (kSmemBytes + 256) <= 232448, "shared memory budget");
 };
 
 __device__ __forceinline__ void cluster_sync_all() {
@@ -54,12 +63,6 @@ __device__ __forceinline__ uint32_t peer_addr(uint32_t local_addr, uint32_t peer
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(peer));
     return ra;
 }
-__device__ __forceinline__ float4 ld_cluster_f32x4(uint32_t addr) {
-    float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
-    return v;
-}
-
 // One reduction stage issued by the elected thread, ring slot Q known at compile time.
 template <int BN, int Q>
 __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, uint32_t sf_t, int rem,
@@ -85,11 +88,12 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
 }
 
 template <int BN>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, DCfg<BN>::kCtasPerSm)
 decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
               const DecodeParams p) {
     using C = DCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
+    constexpr int kStages = C::kStages;
     __shared__ __align__(8) uint64_t bar_full[kStages], bar_empty[kStages], bar_acc_full;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag_s;
@@ -124,11 +128,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     __syncthreads();
     tc_fence_after_sync();
     // set-up done: let the next kernel of the stream be scheduled (its launch latency then overlaps this
-    // kernel), and wait until the activation codes an earlier kernel wrote are settled (and nobody
-    // still reads y)
+    // kernel).  The roles that touch what earlier kernels wrote (activation codes and scales) or may
+    // still read (y) pass grid_dependency_wait() first; the weights depend on no kernel, so the producer
+    // requests them before it waits and they stream in while the previous kernel (normally the
+    // activation quantiser) is still running.
     const long long t_setup = clock64();
     grid_launch_dependents();
-    grid_dependency_wait();
     const uint32_t tmem_base = tmem_slot;
     long long* trace = (p.trace && blockIdx.x < 4) ? p.trace + blockIdx.x * 512 : nullptr;
     if (trace && threadIdx.x == 0) { trace[500] = clock64(); trace[502] = t_entry; trace[503] = t_setup; }
@@ -142,18 +147,35 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
         int st = 0, it = 0;
         uint32_t ph = 0;
         bool ok = true;
+        // first ring pass: weight tile and weight scales now, the token side after the dependency wait
+        const int pre = min(kStages, s_end - s_begin);
+        if (elect_one()) {
+            for (int i = 0; i < pre; ++i) {
+                const int s = s_begin + i;
+                const uint32_t full = smem_u32(&bar_full[i]);
+                mbar_arrive_expect_tx(full, C::kStageBytes);
+                const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
+                const uint32_t sb = smem_base + i * C::kStageBytes;
+                tma_load_2d(sb, &tm_w, xw, n0, full);
+                bulk_load(sb + kPTile + C::kQTile, sfp + s * sfp_stride, kSf, full);
+            }
+        }
+        __syncwarp();
+        grid_dependency_wait();
         for (int s = s_begin; s < s_end; ++s, ++it) {
-            if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
+            if (it >= pre && !mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
             if (trace && lane == 0 && it < 64) trace[it] = clock64();
             if (elect_one()) {
                 const uint32_t full = smem_u32(&bar_full[st]);
-                mbar_arrive_expect_tx(full, C::kStageBytes);
                 const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
                 const int xa = s < S1 ? s * 128 : (p.K - p.k_tail) / 2 + (s - S1) * 128;
                 const uint32_t sb = smem_base + st * C::kStageBytes;
-                tma_load_2d(sb, &tm_w, xw, n0, full);
+                if (it >= pre) {
+                    mbar_arrive_expect_tx(full, C::kStageBytes);
+                    tma_load_2d(sb, &tm_w, xw, n0, full);
+                    bulk_load(sb + kPTile + C::kQTile, sfp + s * sfp_stride, kSf, full);
+                }
                 tma_load_2d(sb + kPTile, &tm_act, xa, 0, full);
-                bulk_load(sb + kPTile + C::kQTile, sfp + s * sfp_stride, kSf, full);
                 bulk_load(sb + kPTile + C::kQTile + kSf, p.act_sf + s * sfq_stride, kSf, full);
             }
             if (++st == kStages) { st = 0; ph ^= 1; }
@@ -174,23 +196,27 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
         int st = 0, it = 0;
         uint32_t ph = 0, accumulate = 0;
         bool ok = true;
+        bool ready = false;   // the next slot was already seen full by the probe issued one stage earlier
         for (int s = s_begin; s < s_end; ++s, ++it) {
-            if (!mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
+            if (!ready && !mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
             if (trace && lane == 0 && it < 64) trace[64 + it] = clock64();
             const int rem = s < S1 ? p.K - s * kStageK : p.k_tail - (s - S1) * kStageK;
+            const int nst = st + 1 == kStages ? 0 : st + 1;
+            const uint32_t nph = nst == 0 ? ph ^ 1 : ph;
+            ready = mbar_test_wait(smem_u32(&bar_full[nst]), nph);
             if (leader) {
                 switch (st) {
                     case 0: issue_stage<BN, 0>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
                     case 1: issue_stage<BN, 1>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
                     case 2: issue_stage<BN, 2>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
                     case 3: issue_stage<BN, 3>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                    case 4: issue_stage<BN, 4>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                    default: issue_stage<BN, 5>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                    case 4: issue_stage<BN, (kStages > 4 ? 4 : 0)>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                    default: issue_stage<BN, (kStages > 5 ? 5 : 0)>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
                 }
             }
             accumulate = 1;
             if (trace && lane == 0 && it < 64) trace[128 + it] = clock64();
-            if (++st == kStages) { st = 0; ph ^= 1; }
+            st = nst; ph = nph;
         }
         if (ok && leader) tc_commit(smem_u32(&bar_acc_full));
     } else {
@@ -200,6 +226,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
         const int row = q4 * 32 + lane;              // weight row inside the tile
         const int n = n0 + row;
         const uint32_t acc_t = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
+        grid_dependency_wait();   // y may still be read by an earlier kernel
         if (mbar_wait(smem_u32(&bar_acc_full), 0, abort_flag)) {
             if (trace && row == 0) trace[192] = clock64();
             tc_fence_after_sync();
@@ -236,26 +263,45 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     }
 
     if (splits > 1) {
-        // ------------------------------------------------------------ meeting point of the cluster
-        // (all threads of all CTAs; orders the partial tiles before the peers' reads)
+        // ------------------------------------------------------------ split-K exchange
+        // Token t belongs to CTA t mod splits; its slot there is t / splits.  Every CTA pushes its partial
+        // sums (16-byte pieces of 4 weight rows, read back from the token-major tile parked above) into
+        // the owners' receive buffers [peer][slot][row]; one cluster barrier later the owner has all of
+        // them in its own shared memory.
+        const uint32_t recv_base = smem_base + kStages * C::kStageBytes;
+        const int slots = (p.M + splits - 1) / splits;        // token slots per peer in a receive buffer
+        const int et = threadIdx.x - 64;                        // 0..127 for the epilogue warps
+        const int j = et & 31, tq = et >> 5;
+        if (warp >= 2 && !abort_flag_s) {
+            asm volatile("bar.sync 1, 128;" ::: "memory");       // the parked tile is complete
+            for (int tok = tq; tok < p.M; tok += 4) {
+                const int owner = tok % splits, slot = tok / splits;
+                float4 v;
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(smem_base + tok * 512 + j * 16));
+                const uint32_t dst = peer_addr(recv_base + ((split * slots + slot) * 128 + 4 * j) * 4, owner);
+                asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};"
+                             ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+            }
+            if (trace && et == 0) trace[195] = clock64();
+        }
+        // all threads of all CTAs: orders the pushes before the owners' reads, and nobody leaves before
+        // everything addressed to its peers has been delivered
         __syncthreads();
         cluster_sync_all();
         if (warp >= 2 && !abort_flag_s) {
-            // epilogue, part 2: this CTA adds up tokens split, split + splits, ... over all peers.  A thread
-            // owns 4 consecutive weight rows (one 16-byte piece of the token-major partial tiles) and every
-            // fourth of the CTA's tokens; the loads from all peers are issued together, the sum runs
-            // in peer order.
-            const int et = threadIdx.x - 64;                 // 0..127
-            const int j = et & 31, tq = et >> 5;
+            // this CTA's tokens: split, split + splits, ...; a thread owns 4 consecutive weight rows and
+            // every fourth slot; the sum runs in peer order
             const int n = n0 + 4 * j;
-            uint32_t base[8];
-#pragma unroll
-            for (int peer = 0; peer < 8; ++peer) base[peer] = peer_addr(smem_base + j * 16, peer < splits ? peer : 0);
-            for (int tok = split + splits * tq; tok < p.M; tok += splits * 4) {
+            for (int slot = tq; split + slot * splits < p.M; slot += 4) {
+                const int tok = split + slot * splits;
                 float4 v[8];
 #pragma unroll
                 for (int peer = 0; peer < 8; ++peer)
-                    if (peer < splits) v[peer] = ld_cluster_f32x4(base[peer] + tok * 512);
+                    if (peer < splits)
+                        asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                                     : "=f"(v[peer].x), "=f"(v[peer].y), "=f"(v[peer].z), "=f"(v[peer].w)
+                                     : "r"(recv_base + ((peer * slots + slot) * 128 + 4 * j) * 4));
                 float4 sum = v[0];
 #pragma unroll
                 for (int peer = 1; peer < 8; ++peer)
@@ -280,8 +326,6 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
             }
             if (trace && et == 0) trace[194] = clock64();
         }
-        // nobody leaves while a peer may still be reading its shared memory
-        cluster_sync_all();
     }
 
     // ------------------------------------------------------------ teardown (normal and aborted)
