@@ -23,6 +23,7 @@ namespace {
 constexpr int kQuantThreads = 256;
 constexpr int kAtomK = 128;    // columns per CTA (4 blocks = one scale atom)
 constexpr int kSteps = kGroupRows / (2 * (kQuantThreads / 32));  // 8 steps of 16 rows
+constexpr int kPermBatch = 4;   // scale + permute mode: steps whose loads are in flight together
 
 // E2M1 conversion: round to nearest even, saturating; the sign of values that round to zero (and of
 // negative zero) is kept.
@@ -57,7 +58,7 @@ __device__ __forceinline__ uint32_t encode8(const float (&v)[8], uint32_t byte) 
 }
 
 template <bool kScalePerm>
-__global__ void __launch_bounds__(kQuantThreads, 5)
+__global__ void __launch_bounds__(kQuantThreads, kScalePerm ? 3 : 5)
 quant_act_kernel(QuantParams p) {
     __shared__ __align__(16) uint8_t sf_atom[512];
     __shared__ int s_tile_start[kMaxExperts + 1];
@@ -189,32 +190,43 @@ quant_act_kernel(QuantParams p) {
         }
     } else {
         // ---- scale + permute: gathered 2-byte loads (the head of the permutation is nearly the identity,
-        // so they coalesce), multiply by the stored reciprocal scale in fp32 ----
-#pragma unroll 2
-        for (int i = 0; i < kSteps; ++i) {
-            const int r = row_of(i);
-            const int rc = min(r, n_rows - 1);
-            float v[8];
-            const uint16_t* xrow = p.x + static_cast<size_t>(row0 + rc) * p.ldx;
+        // so they coalesce), multiply by the stored reciprocal scale in fp32.  The loads of four steps
+        // (32 per lane) are issued before any arithmetic.  (Fetching each row's source window with
+        // 16-byte loads and gathering from shared memory was no faster: this mode is bound by its fp32
+        // arithmetic, not by the gathers.) ----
+#pragma unroll 1
+        for (int i0 = 0; i0 < kSteps; i0 += kPermBatch) {
+            uint32_t raw[kPermBatch][8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
-                v[e] = col_ok ? __uint_as_float(static_cast<uint32_t>(__ldg(xrow + src[e])) << 16) * inv_s[e] : 0.f;
-            uint32_t am = 0;
+            for (int ii = 0; ii < kPermBatch; ++ii) {
+                const int rc = min(row_of(i0 + ii), n_rows - 1);
+                const uint16_t* xrow = p.x + static_cast<size_t>(row0 + rc) * p.ldx;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) am = max(am, __float_as_uint(v[e]) & 0x7fffffffu);
-            am = max(am, __shfl_xor_sync(0xffffffffu, am, 1));
-            am = max(am, __shfl_xor_sync(0xffffffffu, am, 2));
-            const uint32_t byte = scale_byte(am);
-            const uint32_t packed = encode8(v, byte);
-            if (col_ok && r < n_rows) {
-                const int row = row0 + r;
-                *reinterpret_cast<uint32_t*>(p.codes + static_cast<size_t>(row) * (K / 2) + col0 / 2) = packed;
-                if ((hl & 3) == 0) {
-                    sf_atom[(r & 31) * 16 + (r >> 5) * 4 + blk_in_atom] = static_cast<uint8_t>(byte);
-                    if (p.scales_row) p.scales_row[static_cast<size_t>(row) * (K / kBlock) + gblk] = static_cast<uint8_t>(byte);
-                    if (gblk >= tail_blk0) {
-                        const int t = gblk - tail_blk0;
-                        sf_group[(plan.S1 + t / 8) * sf_stage_stride + sf_offset_in_group(r, t % 8)] = static_cast<uint8_t>(byte);
+                for (int e = 0; e < 8; ++e) raw[ii][e] = col_ok ? static_cast<uint32_t>(__ldg(xrow + src[e])) : 0u;
+            }
+#pragma unroll
+            for (int ii = 0; ii < kPermBatch; ++ii) {
+                const int r = row_of(i0 + ii);
+                float v[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) v[e] = col_ok ? __uint_as_float(raw[ii][e] << 16) * inv_s[e] : 0.f;
+                uint32_t am = 0;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) am = max(am, __float_as_uint(v[e]) & 0x7fffffffu);
+                am = max(am, __shfl_xor_sync(0xffffffffu, am, 1));
+                am = max(am, __shfl_xor_sync(0xffffffffu, am, 2));
+                const uint32_t byte = scale_byte(am);
+                const uint32_t packed = encode8(v, byte);
+                if (col_ok && r < n_rows) {
+                    const int row = row0 + r;
+                    *reinterpret_cast<uint32_t*>(p.codes + static_cast<size_t>(row) * (K / 2) + col0 / 2) = packed;
+                    if ((hl & 3) == 0) {
+                        sf_atom[(r & 31) * 16 + (r >> 5) * 4 + blk_in_atom] = static_cast<uint8_t>(byte);
+                        if (p.scales_row) p.scales_row[static_cast<size_t>(row) * (K / kBlock) + gblk] = static_cast<uint8_t>(byte);
+                        if (gblk >= tail_blk0) {
+                            const int t = gblk - tail_blk0;
+                            sf_group[(plan.S1 + t / 8) * sf_stage_stride + sf_offset_in_group(r, t % 8)] = static_cast<uint8_t>(byte);
+                        }
                     }
                 }
             }
