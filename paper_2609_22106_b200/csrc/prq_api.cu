@@ -713,15 +713,19 @@ prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const voi
     p.y = y; p.ldy = ldy; p.y_bf16 = y_dtype == PRQ_BF16;
     p.status = di->status_ptr;
     p.splits = 1;
+    // Default: output features on the MMA M axis, one 128-token group of an expert on the N axis (coalesced
+    // stores straight from the accumulator, cheap for experts with few tokens).  PRQ_GROUPED_BN selects the
+    // tokens-on-M variant with that weight-tile width instead.
     int bn = env_int("PRQ_GROUPED_BN", 0);
-    if (!bn) bn = (M_total >= 8192 && w->N % 256 == 0) ? 256 : 128;
+    const bool swap = bn == 0;
+    if (swap) bn = 128;
     CUtensorMap tm_act, tm_w;
     st = make_code_map(&tm_act, codes, w->K / 2, M_total, 128);
     if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, static_cast<uint64_t>(w->n_experts) * w->N, bn);
     if (st != PRQ_OK) return st;
     bool unsupported = false;
-    cudaError_t e = launch_gemm(GemmKind::kGrouped, bn, tm_act, tm_w, p, di->num_sms, static_cast<cudaStream_t>(stream),
-                                &unsupported);
+    cudaError_t e = launch_gemm(swap ? GemmKind::kGroupedSwap : GemmKind::kGrouped, bn, tm_act, tm_w, p, di->num_sms,
+                                static_cast<cudaStream_t>(stream), &unsupported);
     if (unsupported) return PRQ_ERR_INVALID_ARG;
     g_launches.fetch_add(1);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;

@@ -33,7 +33,7 @@ namespace {
 
 constexpr int kThreads = 192;
 constexpr int kPTileBytes = 128 * 128;
-constexpr int kKindPrefill = 0, kKindDecode = 1, kKindGrouped = 2;
+constexpr int kKindPrefill = 0, kKindDecode = 1, kKindGrouped = 2, kKindGroupedSwap = 3;
 
 constexpr int cgcd(int a, int b) { return b == 0 ? a : cgcd(b, a % b); }
 constexpr int cmin(int a, int b) { return a < b ? a : b; }
@@ -42,7 +42,7 @@ constexpr int pow2_at_least(int x) { int p = 32; while (p < x) p *= 2; return p;
 
 template <int BN, int KIND>
 struct Cfg {
-    static constexpr bool kSwap = KIND == kKindDecode;
+    static constexpr bool kSwap = KIND == kKindDecode || KIND == kKindGroupedSwap;
     // 128-row scale groups of a Q tile; the weight scale buffer is laid out per BN-row tile, so a
     // tile's groups are contiguous and start at the tile's first row
     static constexpr int kNgq = (BN + 127) / 128;
@@ -56,7 +56,7 @@ struct Cfg {
     static constexpr int kSfpCols = 8;              // 2 atoms x 4 columns
     static constexpr int kSfqCols = 8 * kNgq;       // 2 atoms x 4 columns x groups
     static constexpr int kSfCols = kSfpCols + kSfqCols;
-    static constexpr int kAcc = (!kSwap && 2 * kAccStride + kSfCols <= 512) ? 2 : 1;
+    static constexpr int kAcc = (KIND != kKindDecode && 2 * kAccStride + kSfCols <= 512) ? 2 : 1;
     static constexpr int kTmemCols = pow2_at_least(kAcc * kAccStride + kSfCols);
     static constexpr int kSfpCol = kAcc * kAccStride;
     static constexpr int kSfqCol = kSfpCol + kSfpCols;
@@ -81,6 +81,7 @@ template <int BN, int KIND>
 __device__ __forceinline__ int unit_count(const GemmParams& p, const int* tile_start) {
     if (KIND == kKindPrefill) return ((p.M + 127) / 128) * ((p.N + BN - 1) / BN);
     if (KIND == kKindDecode) return ((p.N + 127) / 128) * p.splits;
+    if (KIND == kKindGroupedSwap) return tile_start[p.n_experts] * ((p.N + 127) / 128);
     return tile_start[p.n_experts] * ((p.N + BN - 1) / BN);
 }
 
@@ -113,6 +114,26 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
         t.row0 = 0; t.row_end = p.M;
         t.n0 = ni * 128;
         t.tile = ni; t.split = sp;
+    } else if (KIND == kKindGroupedSwap) {
+        // weights on the MMA M axis (128 output features), a 128-row group of one expert's tokens on N
+        const int total_mt = tile_start[p.n_experts];
+        const int mt = u % total_mt, ni = u / total_mt;
+        int lo = 0, hi = p.n_experts - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (tile_start[mid] <= mt) lo = mid; else hi = mid - 1;
+        }
+        const int e = lo;
+        t.p_row = e * p.N + ni * 128;
+        t.q_row = p.expert_offsets[e] + (mt - tile_start[e]) * 128;
+        t.sfp = p.w_sf + (static_cast<size_t>(e) * S * p.w_groups + ni) * kSfGroupBytes;
+        t.sfp_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
+        t.sfq = p.act_sf + static_cast<size_t>(mt) * kSfGroupBytes;
+        t.sfq_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
+        t.s_begin = 0; t.s_end = S;
+        t.row0 = t.q_row; t.row_end = min(p.expert_offsets[e + 1], t.q_row + 128);
+        t.n0 = ni * 128;
+        t.tile = u; t.split = 0;
     } else {
         const int total_mt = tile_start[p.n_experts];
         const int mt = u % total_mt, ni = u / total_mt;
@@ -148,7 +169,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag_s;
     __shared__ int is_last_s;
-    __shared__ int tile_start[KIND == kKindGrouped ? kMaxExperts + 1 : 1];
+    __shared__ int tile_start[(KIND == kKindGrouped || KIND == kKindGroupedSwap) ? kMaxExperts + 1 : 1];
     volatile int* abort_flag = &abort_flag_s;
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -166,7 +187,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
         tma_prefetch_desc(&tm_act);
         tma_prefetch_desc(&tm_w);
     }
-    if (KIND == kKindGrouped && threadIdx.x == 64) {
+    if ((KIND == kKindGrouped || KIND == kKindGroupedSwap) && threadIdx.x == 64) {
         int acc = 0;
         for (int e = 0; e < p.n_experts; ++e) {
             tile_start[e] = acc;
@@ -336,6 +357,62 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                         }
                     }
                 }
+            } else if (KIND == kKindGroupedSwap) {
+                // accumulator row = output feature n, column = token of this expert's 128-row group.  Sixteen
+                // tokens at a time, every warp parks its 32 features per token in a small shared tile (one
+                // contiguous row per token) and writes the rows out in 16-byte pieces: 64 (bf16) or 128 (fp32)
+                // contiguous bytes per token and warp.  A group with few tokens costs few stores.
+                const int n_tok = t.row_end - t.row0;
+                const int nw = t.n0 + q * 32;                   // first feature of this warp
+                const uint32_t stg = smem_base + C::kStages * C::kStageBytes + q * 2048;
+#pragma unroll 1
+                for (int c = 0; c * 16 < n_tok; ++c) {
+                    uint32_t r[16];
+                    tmem_ld_32x16(acc_t + c * 16, r);
+                    tmem_ld_wait();
+                    if (p.y_bf16) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const __nv_bfloat16 h = __float2bfloat16_rn(__uint_as_float(r[i]));
+                            asm volatile("st.shared.u16 [%0], %1;" ::"r"(stg + i * 64 + lane * 2), "h"(*reinterpret_cast<const uint16_t*>(&h)) : "memory");
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            const int tok = c * 16 + j * 8 + (lane >> 2), col = nw + (lane & 3) * 8;
+                            uint4 v;
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg + j * 512 + lane * 16));
+                            if (tok < n_tok && col < p.N) {
+                                __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<size_t>(t.row0 + tok) * p.ldy + col;
+                                if (col + 8 <= p.N) *reinterpret_cast<uint4*>(yp) = v;
+                                else {
+                                    const __nv_bfloat16* e = reinterpret_cast<const __nv_bfloat16*>(&v);
+                                    for (int i = 0; i < 8 && col + i < p.N; ++i) yp[i] = e[i];
+                                }
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + i * 128 + lane * 4), "r"(r[i]) : "memory");
+                        __syncwarp();
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int tok = c * 16 + j * 4 + (lane >> 3), col = nw + (lane & 7) * 4;
+                            uint4 v;
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg + j * 512 + lane * 16));
+                            if (tok < n_tok && col < p.N) {
+                                float* yp = reinterpret_cast<float*>(p.y) + static_cast<size_t>(t.row0 + tok) * p.ldy + col;
+                                if (col + 4 <= p.N) *reinterpret_cast<uint4*>(yp) = v;
+                                else {
+                                    const float* e = reinterpret_cast<const float*>(&v);
+                                    for (int i = 0; i < 4 && col + i < p.N; ++i) yp[i] = e[i];
+                                }
+                            }
+                        }
+                    }
+                    __syncwarp();   // the tile is read before the next chunk overwrites it
+                }
             } else {
                 // decode: accumulator row = weight row n, column = token
                 const int n = t.n0 + et;
@@ -441,7 +518,7 @@ template <int BN, int KIND>
 cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
                        cudaStream_t stream) {
     using C = Cfg<BN, KIND>;
-    constexpr int smem = C::kStages * C::kStageBytes + 1024;
+    constexpr int smem = C::kStages * C::kStageBytes + 1024 + (KIND == kKindGroupedSwap ? 8192 : 0);  // + store staging
     static bool configured = false;  // per template instance; the attribute is per function, setting it twice is harmless
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BN, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
@@ -467,6 +544,8 @@ cudaError_t launch_gemm(GemmKind kind, int bn, const CUtensorMap& tm_act, const 
     } else if (kind == GemmKind::kGrouped) {
         PRQ_CASE(kKindGrouped, 128)
         PRQ_CASE(kKindGrouped, 256)
+    } else if (kind == GemmKind::kGroupedSwap) {
+        PRQ_CASE(kKindGroupedSwap, 128)
     }
 #undef PRQ_CASE
     *unsupported = true;

@@ -26,7 +26,8 @@ cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_gro
 enum class GemmKind {
     kPrefill,  // tokens on the MMA M axis (128-row tiles), weights on the N axis, persistent CTAs
     kDecode,   // weights on the MMA M axis, tokens on the N axis, split-K with a workspace reduction
-    kGrouped   // prefill layout with per-expert row ranges
+    kGrouped,  // prefill layout with per-expert row ranges
+    kGroupedSwap  // per-expert row ranges with the weights on the MMA M axis and a 128-token group on N
 };
 
 struct GemmParams {

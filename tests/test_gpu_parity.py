@@ -294,10 +294,15 @@ def grouped_case(prq, oracle, E, N, K, k, counts, seed):
     w.free()
 
 
-@pytest.mark.parametrize("bn", [128, 256])
+@pytest.mark.parametrize("bn", [0, 128, 256])
 def test_grouped_experts(prq, oracle, bn, monkeypatch):
-    """MoE variant: ragged expert row ranges including empty experts and ranges that cross 128-row tiles."""
-    monkeypatch.setenv("PRQ_GROUPED_BN", str(bn))
+    """MoE variant: ragged expert row ranges including empty experts and ranges that cross 128-row tiles.
+    bn = 0 is the default kernel (output features on the MMA M axis); 128 / 256 force the tokens-on-M
+    variant with that weight-tile width."""
+    if bn:
+        monkeypatch.setenv("PRQ_GROUPED_BN", str(bn))
+    else:
+        monkeypatch.delenv("PRQ_GROUPED_BN", raising=False)
     grouped_case(prq, oracle, E=6, N=512, K=768, k=64, counts=[5, 0, 130, 1, 0, 300], seed=11)
     grouped_case(prq, oracle, E=3, N=256, K=512, k=0, counts=[0, 0, 7], seed=12)
 
