@@ -713,6 +713,7 @@ prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const voi
     p.y = y; p.ldy = ldy; p.y_bf16 = y_dtype == PRQ_BF16;
     p.status = di->status_ptr;
     p.splits = 1;
+    p.trace = trace_ptr();
     // Default: output features on the MMA M axis, one 128-token group of an expert on the N axis (coalesced
     // stores straight from the accumulator, cheap for experts with few tokens).  PRQ_GROUPED_BN selects the
     // tokens-on-M variant with that weight-tile width instead.

@@ -31,7 +31,7 @@
 namespace prq {
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kMainWarps = 2;   // producer + issuer; the epilogue warps follow
 constexpr int kPTileBytes = 128 * 128;
 constexpr int kKindPrefill = 0, kKindDecode = 1, kKindGrouped = 2, kKindGroupedSwap = 3;
 
@@ -43,6 +43,10 @@ constexpr int pow2_at_least(int x) { int p = 32; while (p < x) p *= 2; return p;
 template <int BN, int KIND>
 struct Cfg {
     static constexpr bool kSwap = KIND == kKindDecode || KIND == kKindGroupedSwap;
+    // epilogue warps: four (one per tensor-memory lane quarter), or eight taking alternate column chunks
+    // where the epilogue is what the main loop waits for (short reductions, many outputs)
+    static constexpr int kEpiWarps = KIND == kKindGroupedSwap ? 8 : 4;
+    static constexpr int kThreads = 32 * (kMainWarps + kEpiWarps);
     // 128-row scale groups of a Q tile; the weight scale buffer is laid out per BN-row tile, so a
     // tile's groups are contiguous and start at the tile's first row
     static constexpr int kNgq = (BN + 127) / 128;
@@ -50,7 +54,7 @@ struct Cfg {
     static constexpr int kSfpBytes = kSfGroupBytes;
     static constexpr int kSfqBytes = kNgq * kSfGroupBytes;
     static constexpr int kStageBytes = kPTileBytes + kQTileBytes + kSfpBytes + kSfqBytes;
-    static constexpr int kStages = cmin(8, (232448 - 1024 - 8192) / kStageBytes);
+    static constexpr int kStages = cmin(8, (232448 - 1024 - 16384 - 2048) / kStageBytes);
     // tensor memory columns: accumulators first, then scale words
     static constexpr int kAccStride = cmax(BN, 32);
     static constexpr int kSfpCols = 8;              // 2 atoms x 4 columns
@@ -160,7 +164,7 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
 template <int BN, int KIND>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(Cfg<BN, KIND>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
             const GemmParams p) {
     using C = Cfg<BN, KIND>;
@@ -180,7 +184,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < C::kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_empty[i]), 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_empty[i]), C::kEpiWarps); }
         abort_flag_s = 0;
         is_last_s = 0;
         fence_mbar_init();
@@ -254,6 +258,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
         int it = 0, acc_it = 0, st = 0;
         uint32_t ph = 0;
         bool ok = true;
+        bool ready = false;   // the next slot was already seen full by the probe issued one stage earlier
+        const bool leader = elect_one();
         const uint32_t sfp_t = tmem_base + C::kSfpCol;
         const uint32_t sfq_t = tmem_base + C::kSfqCol;
         for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
@@ -265,11 +271,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
             const uint32_t d_tmem = tmem_base + buf * C::kAccStride;
             uint32_t accumulate = 0;
             for (int s = t.s_begin; s < t.s_end; ++s, ++it) {
-                if (!mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
+                if (!ready && !mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
                 if (trace && lane == 0 && it < 64) trace[64 + it] = clock64();
                 const int rem = s < S1 ? p.K - s * kStageK : p.k_tail - (s - S1) * kStageK;
                 const int ksteps = min(4, (rem + 63) / 64);
-                if (elect_one()) {
+                // probe the next slot now: the probe's latency hides behind this stage's tcgen05 instructions
+                const int nst = st + 1 == C::kStages ? 0 : st + 1;
+                const uint32_t nph = nst == 0 ? ph ^ 1 : ph;
+                ready = mbar_test_wait(smem_u32(&bar_full[nst]), nph);
+                if (leader) {
                     const uint32_t sb = smem_base + st * C::kStageBytes;
                     const uint32_t sfp_s = sb + kPTileBytes + C::kQTileBytes;
                     const uint32_t sfq_s = sfp_s + C::kSfpBytes;
@@ -298,10 +308,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                 }
                 accumulate = 1;
                 if (trace && lane == 0 && it < 64) trace[128 + it] = clock64();
-                if (++st == C::kStages) { st = 0; ph ^= 1; }
+                st = nst; ph = nph;
             }
             if (!ok) break;
-            if (elect_one()) tc_commit(smem_u32(&bar_acc_full[buf]));
+            if (leader) tc_commit(smem_u32(&bar_acc_full[buf]));
             __syncwarp();
         }
     } else {
@@ -364,9 +374,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                 // contiguous bytes per token and warp.  A group with few tokens costs few stores.
                 const int n_tok = t.row_end - t.row0;
                 const int nw = t.n0 + q * 32;                   // first feature of this warp
-                const uint32_t stg = smem_base + C::kStages * C::kStageBytes + q * 2048;
+                const uint32_t stg = smem_base + C::kStages * C::kStageBytes + (warp - kMainWarps) * 2048;
+                constexpr int kPerQuarter = C::kEpiWarps / 4;   // warps sharing a lane quarter take alternate chunks
 #pragma unroll 1
-                for (int c = 0; c * 16 < n_tok; ++c) {
+                for (int c = (warp - kMainWarps) >> 2; c * 16 < n_tok; c += kPerQuarter) {
                     uint32_t r[16];
                     tmem_ld_32x16(acc_t + c * 16, r);
                     tmem_ld_wait();
@@ -518,14 +529,14 @@ template <int BN, int KIND>
 cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
                        cudaStream_t stream) {
     using C = Cfg<BN, KIND>;
-    constexpr int smem = C::kStages * C::kStageBytes + 1024 + (KIND == kKindGroupedSwap ? 8192 : 0);  // + store staging
+    constexpr int smem = C::kStages * C::kStageBytes + 1024 + (KIND == kKindGroupedSwap ? C::kEpiWarps * 2048 : 0);  // + store staging
     static bool configured = false;  // per template instance; the attribute is per function, setting it twice is harmless
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BN, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    gemm_kernel<BN, KIND><<<grid, kThreads, smem, stream>>>(tm_act, tm_w, p);
+    gemm_kernel<BN, KIND><<<grid, C::kThreads, smem, stream>>>(tm_act, tm_w, p);
     return cudaGetLastError();
 }
 
