@@ -2,13 +2,14 @@
 // Kernel design paragraph; Eq. (1) activation side when the scale and permutation are applied online).
 //
 // One CTA owns 128 rows x 128 columns: exactly one 512-byte scale atom of the GEMM's layout.  In
-// identity mode a lane takes 16 elements (a row of the tile is 8 lanes, a warp covers four rows per
-// step, four steps), with all eight 16-byte loads of a lane issued first, so that about 100 KB per SM
-// are in flight -- the kernel is HBM-bound (2 bytes read + 0.5 + 1/32 written per element), latency is
-// hidden by loads in flight rather than by occupancy, and the instruction count per element is what
-// decides how close it gets.  A 32-element block is 2 adjacent lanes: amax by packed 16-bit maxima and
-// one shuffle, E8M0 byte from the exponent field, sixteen round-to-nearest-even E2M1 conversions per
-// lane, one 8-byte packed store per lane.  (Scale + permute mode keeps 8 elements per lane.)  The atom's scale bytes are collected in shared memory and
+// identity mode a lane takes one whole 32-element block (a row of the tile is 4 lanes, a warp covers
+// eight rows per step, two steps), with all eight 16-byte loads of a lane issued first, so that about
+// 100 KB per SM are in flight -- the kernel is HBM-bound (2 bytes read + 0.5 + 1/32 written per element),
+// latency is hidden by loads in flight rather than by occupancy, and the instruction count per element
+// is what decides how close it gets (8 elements per lane: 11.3 us, 16: 10.3 us, 32: 9.8 us at 2048 x
+// 9728).  Block amax by packed 16-bit maxima without any shuffle, E8M0 byte from the exponent field, 32
+// round-to-nearest-even E2M1 conversions per lane, one 16-byte packed store per lane.  (Scale +
+// permute mode keeps 8 elements per lane and 4 lanes per block.)  The atom's scale bytes are collected in shared memory and
 // written out as one coalesced 512-byte piece; the bytes of tail blocks are also duplicated into the
 // residual stages, which is all the "tail copy" this design needs (the GEMM re-reads the tail codes).
 #include <cuda_bf16.h>
@@ -135,50 +136,51 @@ quant_act_kernel(QuantParams p) {
     auto row_of = [&](int i) { return i * 16 + warp * 2 + half; };
 
     if (!kScalePerm) {
-        // ---- identity.  Here a lane takes 16 elements (32 contiguous bytes, two 16-byte loads), so a
-        // row of the tile is 8 lanes, a warp covers 4 rows and the tile is done in 4 steps of 32 rows; a
-        // 32-element block is 2 lanes (one shuffle).  All eight loads are issued first, then the
-        // arithmetic runs on packed bf16 pairs.  Pointers advance by a constant per step. ----
-        const int l8 = lane & 7, rw = lane >> 3;
-        const int c4 = warp * 4 + rw;                        // row inside a 32-row step
-        const int col16 = atom * kAtomK + l8 * 16;           // first of this lane's 16 columns
-        const bool ok16 = col16 < K;                         // K % 32 == 0: a lane is all in or all out
-        const int blk = l8 >> 1;                             // block inside the atom
-        const int gb = atom * (kAtomK / kBlock) + blk;
-        const uint16_t* xp = p.x + static_cast<size_t>(row0 + c4) * p.ldx + col16;
-        const size_t x_step = static_cast<size_t>(32) * p.ldx;
-        uint4 q[4][2];
+        // ---- identity.  Here a lane takes one whole 32-element block (64 contiguous bytes, four 16-byte
+        // loads): no shuffle at all, a row of the tile is 4 lanes, a warp covers 8 rows and the tile is
+        // done in 2 steps of 64 rows.  All eight loads are issued first, then the arithmetic runs on
+        // packed bf16 pairs. ----
+        const int l4 = lane & 3, rw = lane >> 2;
+        const int c8 = warp * 8 + rw;                        // row inside a 64-row step
+        const int colb = atom * kAtomK + l4 * 32;            // first of this lane's 32 columns
+        const bool okb = colb < K;                           // K % 32 == 0: a lane is all in or all out
+        const int gb = atom * (kAtomK / kBlock) + l4;        // this lane's block
+        const uint16_t* xp = p.x + static_cast<size_t>(row0 + c8) * p.ldx + colb;
+        const size_t x_step = static_cast<size_t>(64) * p.ldx;
+        uint4 q[2][4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            q[i][0] = q[i][1] = make_uint4(0, 0, 0, 0);
-            if (ok16 && i * 32 + c4 < n_rows) {
-                q[i][0] = __ldg(reinterpret_cast<const uint4*>(xp + i * x_step));
-                q[i][1] = __ldg(reinterpret_cast<const uint4*>(xp + i * x_step + 8));
+        for (int i = 0; i < 2; ++i) {
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                q[i][h] = make_uint4(0, 0, 0, 0);
+                if (okb && i * 64 + c8 < n_rows) q[i][h] = __ldg(reinterpret_cast<const uint4*>(xp + i * x_step + 8 * h));
             }
         }
-        uint8_t* cp = p.codes + static_cast<size_t>(row0 + c4) * (K / 2) + col16 / 2;
-        const size_t c_step = static_cast<size_t>(32) * (K / 2);
-        uint8_t* rp = p.scales_row ? p.scales_row + static_cast<size_t>(row0 + c4) * (K / kBlock) + gb : nullptr;
-        const size_t r_step = static_cast<size_t>(32) * (K / kBlock);
-        const bool sf_lane = ok16 && (l8 & 1) == 0;
-        const bool tail_lane = sf_lane && gb >= tail_blk0;
+        uint8_t* cp = p.codes + static_cast<size_t>(row0 + c8) * (K / 2) + colb / 2;
+        const size_t c_step = static_cast<size_t>(64) * (K / 2);
+        uint8_t* rp = p.scales_row ? p.scales_row + static_cast<size_t>(row0 + c8) * (K / kBlock) + gb : nullptr;
+        const size_t r_step = static_cast<size_t>(64) * (K / kBlock);
+        const bool tail_lane = okb && gb >= tail_blk0;
         uint8_t* tp = nullptr;                                // this lane's duplicate slot in the residual stages
         if (tail_lane) {
             const int t = gb - tail_blk0;
             tp = sf_group + (plan.S1 + t / 8) * sf_stage_stride + ((t % 8) >> 2) * 512 + ((t % 8) & 3);
         }
-        // row r = 32 i + c4 of the group: atom offset (r % 32) * 16 + (r / 32) * 4 + block
-        uint8_t* ap = sf_atom + c4 * 16 + blk;
+        // row r = 64 i + c8 of the group: atom offset (r % 32) * 16 + (r / 32) * 4 + block
+        const int in_atom0 = (c8 & 31) * 16 + (c8 >> 5) * 4;
+        uint8_t* ap = sf_atom + in_atom0 + l4;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            // block amax: packed bf16 |.| and max over the lane's eight pairs, the two halves, the other lane
-            const __nv_bfloat162 a0 = __hmax2(__habs2(as_bf162(q[i][0].x)), __habs2(as_bf162(q[i][0].y)));
-            const __nv_bfloat162 a1 = __hmax2(__habs2(as_bf162(q[i][0].z)), __habs2(as_bf162(q[i][0].w)));
-            const __nv_bfloat162 a2 = __hmax2(__habs2(as_bf162(q[i][1].x)), __habs2(as_bf162(q[i][1].y)));
-            const __nv_bfloat162 a3 = __hmax2(__habs2(as_bf162(q[i][1].z)), __habs2(as_bf162(q[i][1].w)));
-            const uint32_t mm = as_u32(__hmax2(__hmax2(a0, a1), __hmax2(a2, a3)));
-            uint32_t m = max(mm & 0xffffu, mm >> 16);
-            m = max(m, __shfl_xor_sync(0xffffffffu, m, 1));
+        for (int i = 0; i < 2; ++i) {
+            // block amax: packed bf16 |.| and max over the lane's sixteen pairs, then the two halves
+            __nv_bfloat162 am = __floats2bfloat162_rn(0.f, 0.f);
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                const __nv_bfloat162 a0 = __hmax2(__habs2(as_bf162(q[i][h].x)), __habs2(as_bf162(q[i][h].y)));
+                const __nv_bfloat162 a1 = __hmax2(__habs2(as_bf162(q[i][h].z)), __habs2(as_bf162(q[i][h].w)));
+                am = __hmax2(am, __hmax2(a0, a1));
+            }
+            const uint32_t mm = as_u32(am);
+            const uint32_t m = max(mm & 0xffffu, mm >> 16);
             // E8M0 byte = biased exponent - 2 (floored at 0); 2^(127 - byte) as a packed bf16 pair.
             // Multiplying bf16 by a power of two is exact (results too small for bf16 round to code 0
             // in any case), so the scaling is done on pairs before widening to fp32.
@@ -186,9 +188,9 @@ quant_act_kernel(QuantParams p) {
             const uint32_t byte = eb < 0 ? 0u : static_cast<uint32_t>(eb);
             const uint32_t inv1 = (254u - byte) << 7;
             const __nv_bfloat162 inv2 = as_bf162(inv1 | (inv1 << 16));
-            uint32_t pk[2];
+            uint32_t pk[4];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
+            for (int h = 0; h < 4; ++h) {
                 const uint32_t s0 = as_u32(__hmul2(as_bf162(q[i][h].x), inv2)), s1 = as_u32(__hmul2(as_bf162(q[i][h].y), inv2));
                 const uint32_t s2 = as_u32(__hmul2(as_bf162(q[i][h].z), inv2)), s3 = as_u32(__hmul2(as_bf162(q[i][h].w), inv2));
                 pk[h] = cvt_e2m1x8(__uint_as_float(s0 << 16), __uint_as_float(s0 & 0xffff0000u),
@@ -196,12 +198,12 @@ quant_act_kernel(QuantParams p) {
                                    __uint_as_float(s2 << 16), __uint_as_float(s2 & 0xffff0000u),
                                    __uint_as_float(s3 << 16), __uint_as_float(s3 & 0xffff0000u));
             }
-            const bool row_ok = i * 32 + c4 < n_rows;
-            if (ok16 && row_ok) *reinterpret_cast<uint2*>(cp + i * c_step) = make_uint2(pk[0], pk[1]);
-            if (sf_lane && row_ok) {
-                ap[i * 4] = static_cast<uint8_t>(byte);
+            const bool row_ok = i * 64 + c8 < n_rows;
+            if (okb && row_ok) {
+                *reinterpret_cast<uint4*>(cp + i * c_step) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                ap[i * 8] = static_cast<uint8_t>(byte);
                 if (rp) rp[i * r_step] = static_cast<uint8_t>(byte);
-                if (tail_lane) tp[c4 * 16 + i * 4] = static_cast<uint8_t>(byte);
+                if (tail_lane) tp[in_atom0 + i * 8] = static_cast<uint8_t>(byte);
             }
         }
     } else {
