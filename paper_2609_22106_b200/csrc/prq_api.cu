@@ -143,6 +143,15 @@ int decode_splits(const prq_weights* w, int M, DeviceInfo* di) {
     const int forced = env_int("PRQ_DECODE_SPLITS", 0);
     const int limit = std::min(8, w->plan.S);
     if (forced > 0) return std::min(forced, limit);
+    if (bn <= 32) {
+        // Up to 32 tokens two CTAs share an SM, and a few clusters more than fit at once cost less than
+        // a longer reduction per CTA does (measured at 20 tiles: 8 splits beat 6 at every token count):
+        // the largest cluster that oversubscribes the SMs by at most a fifth.
+        int best = 1;
+        for (int s = 1; s <= limit; ++s)
+            if (static_cast<long long>(n_tiles) * s * 5 <= static_cast<long long>(di->num_sms) * 6) best = s;
+        return best;
+    }
     int best = 1, best_ctas = 0;
     for (int s = 1; s <= limit; ++s) {
         int mc;
