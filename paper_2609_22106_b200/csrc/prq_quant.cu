@@ -118,6 +118,11 @@ quant_act_kernel(QuantParams p) {
     const size_t sf_stage_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
     uint8_t* sf_group = sf_base + static_cast<size_t>(group) * kSfGroupBytes;
     const int n_rows = row_end - row0;            // 1..128
+    // With few groups the rows of a group are split over gridDim.z CTAs (1, 2, 4 or 8 parts of whole
+    // 16-row steps) so that a small batch still fills the GPU; only the scale + permute mode is split.
+    const int n_parts = kScalePerm ? static_cast<int>(gridDim.z) : 1;
+    const int part = kScalePerm ? static_cast<int>(blockIdx.z) : 0;
+    const int part_steps = kSteps / n_parts;
 
     float inv_s[8];
     int src[8];
@@ -213,10 +218,12 @@ quant_act_kernel(QuantParams p) {
         // 16-byte loads and gathering from shared memory was no faster: this mode is bound by its fp32
         // arithmetic, not by the gathers.) ----
 #pragma unroll 1
-        for (int i0 = 0; i0 < kSteps; i0 += kPermBatch) {
+        for (int i0 = part * part_steps; i0 < (part + 1) * part_steps; i0 += kPermBatch) {
+            if (i0 * 16 >= n_rows) break;   // nothing but padding rows from here on (their scale bytes are zero already)
             uint32_t raw[kPermBatch][8];
 #pragma unroll
             for (int ii = 0; ii < kPermBatch; ++ii) {
+                if (ii >= part_steps) break;
                 const int rc = min(row_of(i0 + ii), n_rows - 1);
                 const uint16_t* xrow = p.x + static_cast<size_t>(row0 + rc) * p.ldx;
 #pragma unroll
@@ -224,6 +231,7 @@ quant_act_kernel(QuantParams p) {
             }
 #pragma unroll
             for (int ii = 0; ii < kPermBatch; ++ii) {
+                if (ii >= part_steps) break;
                 const int r = row_of(i0 + ii);
                 float v[8];
 #pragma unroll
@@ -252,10 +260,19 @@ quant_act_kernel(QuantParams p) {
     }
     __syncthreads();
     // the atom's scale bytes, coalesced (rows past the end and blocks past K stay zero = 2^-127)
-    if (threadIdx.x < 32) {
-        reinterpret_cast<uint4*>(sf_group + stage * sf_stage_stride + (atom & 1) * 512)[threadIdx.x] =
-            reinterpret_cast<const uint4*>(sf_atom)[threadIdx.x];
+    if (n_parts == 1) {
+        if (threadIdx.x < 32) {
+            reinterpret_cast<uint4*>(sf_group + stage * sf_stage_stride + (atom & 1) * 512)[threadIdx.x] =
+                reinterpret_cast<const uint4*>(sf_atom)[threadIdx.x];
+        }
+    } else if (threadIdx.x < kGroupRows / n_parts) {
+        // this part's rows only: the four scale bytes of row r sit at (r % 32) * 16 + (r / 32) * 4
+        const int r = part * (kGroupRows / n_parts) + threadIdx.x;
+        const int off = (r & 31) * 16 + (r >> 5) * 4;
+        *reinterpret_cast<uint32_t*>(sf_group + stage * sf_stage_stride + (atom & 1) * 512 + off) =
+            *reinterpret_cast<const uint32_t*>(sf_atom + off);
     }
+    if (part != 0) return;
     const int n_atoms = gridDim.x;
     // An odd atom count leaves the second half of the last main stage without an owner: zero it.
     if (atom == n_atoms - 1 && (n_atoms & 1) && threadIdx.x >= 32 && threadIdx.x < 64)
@@ -278,7 +295,22 @@ quant_act_kernel(QuantParams p) {
 
 cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_groups, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((p.K + kAtomK - 1) / kAtomK, grid_groups);
+    const int n_atoms = (p.K + kAtomK - 1) / kAtomK;
+    int parts = 1;
+    if (scale_perm) {
+        // split the rows of a group until there are about four CTAs per SM
+        static int sm_count[64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+        if (sm_count[dev] == 0) {
+            int n = 0;
+            cudaError_t e = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess) return e;
+            sm_count[dev] = n;
+        }
+        while (parts < 8 && static_cast<long long>(n_atoms) * grid_groups * parts < 4LL * sm_count[dev]) parts *= 2;
+    }
+    cfg.gridDim = dim3(n_atoms, grid_groups, parts);
     cfg.blockDim = dim3(kQuantThreads);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
