@@ -15,6 +15,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <cstdlib>
+
 #include "prq_internal.h"
 #include "prq_kernels.h"
 #include "prq_ptx.cuh"
@@ -217,42 +219,61 @@ quant_act_kernel(QuantParams p) {
         // (32 per lane) are issued before any arithmetic.  (Fetching each row's source window with
         // 16-byte loads and gathering from shared memory was no faster: this mode is bound by its fp32
         // arithmetic, not by the gathers.) ----
+        // Everything that does not depend on the row is computed once: per-lane pointers that advance by
+        // a fixed stride per 16-row step, the lane's slot in the residual stages, and -- for lanes past K --
+        // zero sources and factors so that the arithmetic below needs no per-element select.
+        const int w2h = warp * 2 + half;                       // row inside a 16-row step
+        const size_t x_step = static_cast<size_t>(16) * p.ldx;
+        const size_t c_step = static_cast<size_t>(16) * (K / 2);
+        const size_t r_step = static_cast<size_t>(16) * (K / kBlock);
+        const bool sf_lane = col_ok && (hl & 3) == 0;          // the lane that writes the block's scale byte
+        const bool tail_lane = sf_lane && gblk >= tail_blk0;
+        uint8_t* tp = nullptr;
+        if (tail_lane) {
+            const int t = gblk - tail_blk0;
+            tp = sf_group + (plan.S1 + t / 8) * sf_stage_stride + ((t % 8) >> 2) * 512 + ((t % 8) & 3);
+        }
+        if (!col_ok) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { src[e] = 0; inv_s[e] = 0.f; }
+        }
 #pragma unroll 1
         for (int i0 = part * part_steps; i0 < (part + 1) * part_steps; i0 += kPermBatch) {
             if (i0 * 16 >= n_rows) break;   // nothing but padding rows from here on (their scale bytes are zero already)
+            const int rb = i0 * 16 + w2h;   // this lane's row in the batch's first step
+            const uint16_t* xb = p.x + static_cast<size_t>(row0 + rb) * p.ldx;
+            uint8_t* cp = p.codes + static_cast<size_t>(row0 + rb) * (K / 2) + col0 / 2;
+            uint8_t* rp = p.scales_row ? p.scales_row + static_cast<size_t>(row0 + rb) * (K / kBlock) + gblk : nullptr;
             uint32_t raw[kPermBatch][8];
 #pragma unroll
             for (int ii = 0; ii < kPermBatch; ++ii) {
                 if (ii >= part_steps) break;
-                const int rc = min(row_of(i0 + ii), n_rows - 1);
-                const uint16_t* xrow = p.x + static_cast<size_t>(row0 + rc) * p.ldx;
+                const bool ld_ok = col_ok && rb + 16 * ii < n_rows;
+                const uint16_t* xrow = xb + ii * x_step;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) raw[ii][e] = col_ok ? static_cast<uint32_t>(__ldg(xrow + src[e])) : 0u;
+                for (int e = 0; e < 8; ++e) raw[ii][e] = ld_ok ? static_cast<uint32_t>(__ldg(xrow + src[e])) : 0u;
             }
 #pragma unroll
             for (int ii = 0; ii < kPermBatch; ++ii) {
                 if (ii >= part_steps) break;
-                const int r = row_of(i0 + ii);
+                const int r = rb + 16 * ii;
                 float v[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) v[e] = col_ok ? __uint_as_float(raw[ii][e] << 16) * inv_s[e] : 0.f;
-                uint32_t am = 0;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) am = max(am, __float_as_uint(v[e]) & 0x7fffffffu);
+                for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(raw[ii][e] << 16) * inv_s[e];
+                const float a01 = fmaxf(fabsf(v[0]), fabsf(v[1])), a23 = fmaxf(fabsf(v[2]), fabsf(v[3]));
+                const float a45 = fmaxf(fabsf(v[4]), fabsf(v[5])), a67 = fmaxf(fabsf(v[6]), fabsf(v[7]));
+                uint32_t am = __float_as_uint(fmaxf(fmaxf(a01, a23), fmaxf(a45, a67)));
                 am = max(am, __shfl_xor_sync(0xffffffffu, am, 1));
                 am = max(am, __shfl_xor_sync(0xffffffffu, am, 2));
                 const uint32_t byte = scale_byte(am);
                 const uint32_t packed = encode8(v, byte);
                 if (col_ok && r < n_rows) {
-                    const int row = row0 + r;
-                    *reinterpret_cast<uint32_t*>(p.codes + static_cast<size_t>(row) * (K / 2) + col0 / 2) = packed;
-                    if ((hl & 3) == 0) {
-                        sf_atom[(r & 31) * 16 + (r >> 5) * 4 + blk_in_atom] = static_cast<uint8_t>(byte);
-                        if (p.scales_row) p.scales_row[static_cast<size_t>(row) * (K / kBlock) + gblk] = static_cast<uint8_t>(byte);
-                        if (gblk >= tail_blk0) {
-                            const int t = gblk - tail_blk0;
-                            sf_group[(plan.S1 + t / 8) * sf_stage_stride + sf_offset_in_group(r, t % 8)] = static_cast<uint8_t>(byte);
-                        }
+                    *reinterpret_cast<uint32_t*>(cp + ii * c_step) = packed;
+                    if (sf_lane) {
+                        const int in_atom = (r & 31) * 16 + (r >> 5) * 4;
+                        sf_atom[in_atom + blk_in_atom] = static_cast<uint8_t>(byte);
+                        if (rp) rp[ii * r_step] = static_cast<uint8_t>(byte);
+                        if (tail_lane) tp[in_atom] = static_cast<uint8_t>(byte);
                     }
                 }
             }
@@ -298,7 +319,7 @@ cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_gro
     const int n_atoms = (p.K + kAtomK - 1) / kAtomK;
     int parts = 1;
     if (scale_perm) {
-        // split the rows of a group until there are about four CTAs per SM
+        // split the rows of a group (a CTA has a fixed cost of about a microsecond, so no further than needed)
         static int sm_count[64] = {};
         int dev = 0;
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
@@ -308,7 +329,10 @@ cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_gro
             if (e != cudaSuccess) return e;
             sm_count[dev] = n;
         }
-        while (parts < 8 && static_cast<long long>(n_atoms) * grid_groups * parts < 4LL * sm_count[dev]) parts *= 2;
+        const long long tiles = static_cast<long long>(n_atoms) * grid_groups;
+        while (parts < 4 && tiles * parts < 8LL * sm_count[dev]) parts *= 2;   // 3 CTAs per SM: keep the last wave short
+        if (parts == 4 && tiles * parts < 4LL * sm_count[dev]) parts = 8;
+        if (const char* ev = getenv("PRQ_QUANT_PARTS")) { const int v = atoi(ev); if (v == 1 || v == 2 || v == 4 || v == 8) parts = v; }
     }
     cfg.gridDim = dim3(n_atoms, grid_groups, parts);
     cfg.blockDim = dim3(kQuantThreads);
