@@ -186,6 +186,20 @@ prq_status prq_linear(const prq_weights *w, const void *codes, const void *scale
 prq_status prq_linear_static_scratch(const prq_weights *w, const void *codes, const void *scales_sf, int M, void *y,
                                      int ldy, prq_dtype y_dtype, prq_stream_t stream);
 
+/* Decode step in one launch (Kernel design paragraph: the kernel quantises the reordered activation once
+ * and multiplies): y = prq_linear(prq_quantize_act(x)) for up to PRQ_FUSED_MAX_M tokens, with the
+ * activation quantised inside the GEMM kernel -- no code or scale buffer exists.  The result is bit-for-bit
+ * the one of the two calls.
+ *   mode   PRQ_ACT_IDENTITY only (the scale and the permutation were folded into x's producer, Eq. (1));
+ *          PRQ_ACT_SCALE_PERM returns INVALID_ARG -- use the two calls
+ *   x      device, M x K bf16, row stride ldx elements (multiple of 8), 16-byte aligned
+ *   M      1 .. PRQ_FUSED_MAX_M (0 is a no-op); larger M returns INVALID_ARG
+ *   y      device out, M x N, row stride ldy elements, dtype y_dtype
+ * Dense layers only.  Needs no workspace.  Errors: INVALID_ARG, ALIGNMENT, CUDA. */
+#define PRQ_FUSED_MAX_M 16
+prq_status prq_linear_fused(const prq_weights *w, prq_act_mode mode, const void *x, int M, int ldx, void *y,
+                            int ldy, prq_dtype y_dtype, prq_stream_t stream);
+
 /* The same product for stacked experts (MoE): rows [expert_offsets[e], expert_offsets[e+1]) of the
  * activation use expert e's weights.  expert_offsets: device, n_experts + 1 int32, non-decreasing,
  * last = M_total. */

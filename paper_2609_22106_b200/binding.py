@@ -23,7 +23,7 @@ BUF_CODES, BUF_SCALES_ROW, BUF_SCALES_SF = range(3)
 EXPORTS = [
     "prq_prepare_weights", "prq_prepare_weights_host", "prq_prepare_weights_search", "prq_weights_free",
     "prq_weights_clone", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
-    "prq_linear", "prq_linear_static_scratch", "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
+    "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
 ]
 
@@ -61,6 +61,7 @@ def lib():
         L.prq_linear_workspace_bytes.restype = cs
         L.prq_linear.argtypes = [vp, vp, vp, ci, vp, ci, ci, vp, cs, vp]
         L.prq_linear_static_scratch.argtypes = [vp, vp, vp, ci, vp, ci, ci, vp]
+        L.prq_linear_fused.argtypes = [vp, ci, vp, ci, ci, vp, ci, ci, vp]
         L.prq_linear_grouped.argtypes = [vp, vp, vp, vp, ci, vp, ci, ci, vp]
         L.prq_forward_host_scratch_bytes.argtypes = [vp, ci]
         L.prq_forward_host_scratch_bytes.restype = cs
@@ -245,6 +246,21 @@ def linear_static_scratch(w: Weights, codes, scales_sf, M: int, y_dtype: int = F
     _check(lib().prq_linear_static_scratch(w.handle, _dptr(codes), _dptr(scales_sf), M, _dptr(out),
                                            out.stride(0) if M else w.N, y_dtype, _stream_ptr(stream)),
            "prq_linear_static_scratch")
+    return out
+
+
+FUSED_MAX_M = 16
+
+
+def linear_fused(w: Weights, x, mode: int = ACT_IDENTITY, y_dtype: int = F32, out=None, stream=None):
+    """Quantise x (M x K bf16 on the device, M <= FUSED_MAX_M) and multiply, in one launch."""
+    import torch
+
+    M = x.shape[0]
+    if out is None:
+        out = torch.empty((M, w.N), dtype=torch.float32 if y_dtype == F32 else torch.bfloat16, device=x.device)
+    _check(lib().prq_linear_fused(w.handle, mode, _dptr(x), M, x.stride(0) if M else w.K, _dptr(out),
+                                  out.stride(0) if M else w.N, y_dtype, _stream_ptr(stream)), "prq_linear_fused")
     return out
 
 

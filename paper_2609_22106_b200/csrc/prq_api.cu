@@ -706,6 +706,34 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
 }
 
+prq_status prq_linear_fused(const prq_weights* w, prq_act_mode mode, const void* x, int M, int ldx, void* y, int ldy,
+                            prq_dtype y_dtype, prq_stream_t stream) {
+    if (!w || M < 0 || M > PRQ_FUSED_MAX_M || mode != PRQ_ACT_IDENTITY || w->n_experts != 1) return PRQ_ERR_INVALID_ARG;
+    if (M == 0) return PRQ_OK;
+    if (!x || !y || ldx < w->K || ldy < w->N) return PRQ_ERR_INVALID_ARG;
+    if (y_dtype != PRQ_F32 && y_dtype != PRQ_BF16) return PRQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(y) || ldx % 8 || ldy % (y_dtype == PRQ_F32 ? 4 : 8)) return PRQ_ERR_ALIGNMENT;
+    DeviceInfo* di;
+    prq_status st = device_info(w->device, &di);
+    if (st != PRQ_OK) return st;
+    DecodeParams q;
+    std::memset(&q, 0, sizeof(q));
+    q.M = M; q.N = w->N; q.K = w->K; q.k_tail = w->k_tail;
+    q.w_groups = w->w_groups;
+    q.w_sf = w->d_sf;
+    q.x = static_cast<const uint16_t*>(x); q.ldx = ldx;
+    q.y = y; q.ldy = ldy; q.y_bf16 = y_dtype == PRQ_BF16;
+    q.status = di->status_ptr; q.trace = trace_ptr();
+    q.splits = decode_splits(w, M, di);
+    CUtensorMap tm_w;
+    st = make_code_map(&tm_w, w->d_codes, (static_cast<size_t>(w->K) + w->k_tail) / 2, w->N, 128);
+    if (st != PRQ_OK) return st;
+    // the kernel takes no activation tensor map in this mode; the weight map fills the parameter
+    cudaError_t e = launch_decode(decode_bn(M), tm_w, tm_w, q, (w->N + 127) / 128, static_cast<cudaStream_t>(stream));
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
 prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const void* scales_sf,
                               const int32_t* expert_offsets, int M_total, void* y, int ldy, prq_dtype y_dtype,
                               prq_stream_t stream) {

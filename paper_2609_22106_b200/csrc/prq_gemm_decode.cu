@@ -16,12 +16,22 @@
 // token tile from column K - k and the weight tile from column K onwards (Kernel design paragraph).
 // Every wait is bounded; the cluster barriers sit on the common path so that a CTA that gave up still
 // arrives and its peers are released.
+//
+// Fused variant (up to 16 tokens, activation already scaled and reordered by its producer): the kernel
+// takes the bf16 activation itself.  The four epilogue warps first act as the activation quantiser of
+// their CTA -- one 32-element block per thread and stage, codes written straight into the 128-byte-
+// swizzled token tile of the pipeline slot, scale bytes into the slot's scale atom -- so that the
+// separate quantiser launch, its round trip through global memory and one kernel-to-kernel hand-over
+// leave the decode step ("the kernel quantizes the reordered activation once", Kernel design paragraph).
+// Every cluster quantises the K-range it reduces over, i.e. the bf16 activation is read once per 128-row
+// weight tile; that extra L2 traffic grows with the token count and is why the variant stops at 16 tokens.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include "prq_kernels.h"
 #include "prq_ptx.cuh"
+#include "prq_quant_block.cuh"
 
 namespace prq {
 namespace {
@@ -87,7 +97,7 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
     tc_commit(empty_bar0 + Q * 8);
 }
 
-template <int BN>
+template <int BN, bool kFused>
 __global__ void __launch_bounds__(kThreads, DCfg<BN>::kCtasPerSm)
 decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
               const DecodeParams p) {
@@ -113,7 +123,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
 
     const long long t_entry = clock64();
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
+        // a slot is full when its TMA bytes have landed and, fused, when the four quantiser warps are done
+        for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), kFused ? 5 : 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
         mbar_init(smem_u32(&bar_acc_full), 1);
         abort_flag_s = 0;
         fence_mbar_init();
@@ -153,7 +164,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
             for (int i = 0; i < pre; ++i) {
                 const int s = s_begin + i;
                 const uint32_t full = smem_u32(&bar_full[i]);
-                mbar_arrive_expect_tx(full, C::kStageBytes);
+                mbar_arrive_expect_tx(full, kFused ? kPTile + kSf : C::kStageBytes);
                 const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
                 const uint32_t sb = smem_base + i * C::kStageBytes;
                 tma_load_2d(sb, &tm_w, xw, n0, full);
@@ -161,7 +172,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
             }
         }
         __syncwarp();
-        grid_dependency_wait();
+        if (!kFused) grid_dependency_wait();
         for (int s = s_begin; s < s_end; ++s, ++it) {
             if (it >= pre && !mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
             if (trace && lane == 0 && it < 64) trace[it] = clock64();
@@ -171,12 +182,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
                 const int xa = s < S1 ? s * 128 : (p.K - p.k_tail) / 2 + (s - S1) * 128;
                 const uint32_t sb = smem_base + st * C::kStageBytes;
                 if (it >= pre) {
-                    mbar_arrive_expect_tx(full, C::kStageBytes);
+                    mbar_arrive_expect_tx(full, kFused ? kPTile + kSf : C::kStageBytes);
                     tma_load_2d(sb, &tm_w, xw, n0, full);
                     bulk_load(sb + kPTile + C::kQTile, sfp + s * sfp_stride, kSf, full);
                 }
-                tma_load_2d(sb + kPTile, &tm_act, xa, 0, full);
-                bulk_load(sb + kPTile + C::kQTile + kSf, p.act_sf + s * sfq_stride, kSf, full);
+                if (!kFused) {
+                    tma_load_2d(sb + kPTile, &tm_act, xa, 0, full);
+                    bulk_load(sb + kPTile + C::kQTile + kSf, p.act_sf + s * sfq_stride, kSf, full);
+                }
             }
             if (++st == kStages) { st = 0; ph ^= 1; }
         }
@@ -226,7 +239,63 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
         const int row = q4 * 32 + lane;              // weight row inside the tile
         const int n = n0 + row;
         const uint32_t acc_t = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
-        grid_dependency_wait();   // y may still be read by an earlier kernel
+        if constexpr (kFused) {
+            // ---- activation quantiser of this CTA: thread = (token, 32-column block) of a stage ----
+            const int et = threadIdx.x - 64;
+            const int tok0 = et >> 3, blk = et & 7;
+            // token-scale atoms of all slots start as zeros (rows past M and the unused atom rows stay so)
+            for (int i = 0; i < kStages; ++i)
+                *reinterpret_cast<uint2*>(smem + i * C::kStageBytes + kPTile + C::kQTile + kSf + et * 8) = make_uint2(0, 0);
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            grid_dependency_wait();   // x is the previous kernel's output
+            if (trace && et == 0) trace[200] = clock64();
+            bool qok = true;
+#pragma unroll 1
+            for (int base = s_begin; base < s_end && qok; base += kStages) {
+                const int n = min(kStages, s_end - base);
+                // the loads of all stages of a ring pass are in flight together
+                uint4 q[kStages][BN / 16][4];
+#pragma unroll
+                for (int i = 0; i < kStages; ++i) {
+                    const int s = base + i;
+                    const int col = (s < S1 ? s * kStageK : p.K - p.k_tail + (s - S1) * kStageK) + blk * kBlock;
+#pragma unroll
+                    for (int h = 0; h < BN / 16; ++h) {
+                        const int tok = tok0 + 16 * h;
+                        const bool live = i < n && tok < p.M && col < p.K;
+                        const uint16_t* xp = p.x + static_cast<size_t>(tok) * p.ldx + col;
+#pragma unroll
+                        for (int w4 = 0; w4 < 4; ++w4)
+                            q[i][h][w4] = live ? __ldg(reinterpret_cast<const uint4*>(xp + 8 * w4)) : make_uint4(0, 0, 0, 0);
+                    }
+                }
+                const int pass = (base - s_begin) / kStages;
+#pragma unroll
+                for (int i = 0; i < kStages; ++i) {
+                    if (i < n && qok) {
+                        // a reused slot must have been drained by the tensor core
+                        if (pass > 0 && !mbar_wait(smem_u32(&bar_empty[i]), (pass - 1) & 1, abort_flag)) { qok = false; break; }
+                        uint8_t* slot = smem + i * C::kStageBytes;
+#pragma unroll
+                        for (int h = 0; h < BN / 16; ++h) {
+                            const int tok = tok0 + 16 * h;
+                            uint4 codes;
+                            const uint32_t byte = quant_block32(q[i][h], codes);
+                            // token tile: rows of 128 bytes, 16-byte piece c of row r at piece c ^ (r % 8)
+                            *reinterpret_cast<uint4*>(slot + kPTile + tok * 128 + ((blk ^ (tok & 7)) << 4)) = codes;
+                            if (tok < p.M)
+                                slot[kPTile + C::kQTile + kSf + (blk >> 2) * 512 + tok * 16 + (blk & 3)] = static_cast<uint8_t>(byte);
+                        }
+                        fence_proxy_async_smem();   // the tensor core reads the slot through the async proxy
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bar_full[i]));
+                        if (trace && et == 0 && pass == 0) trace[201 + i] = clock64();
+                    }
+                }
+            }
+        } else {
+            grid_dependency_wait();   // y may still be read by an earlier kernel
+        }
         if (mbar_wait(smem_u32(&bar_acc_full), 0, abort_flag)) {
             if (trace && row == 0) trace[192] = clock64();
             tc_fence_after_sync();
@@ -340,13 +409,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     if (threadIdx.x == 0 && abort_flag_s) atomicExch(p.status, static_cast<int>(PRQ_ERR_TIMEOUT));
 }
 
-template <int BN>
+template <int BN, bool kFused>
 cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const DecodeParams& p, int n_tiles,
                        cudaStream_t stream) {
     using C = DCfg<BN>;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(decode_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel<BN, kFused>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -364,13 +433,13 @@ cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, decode_kernel<BN>, tm_act, tm_w, p);
+    return cudaLaunchKernelEx(&cfg, decode_kernel<BN, kFused>, tm_act, tm_w, p);
 }
 
 template <int BN>
 int max_clusters(int splits) {
     using C = DCfg<BN>;
-    cudaFuncSetAttribute(decode_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    cudaFuncSetAttribute(decode_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(splits);
     cfg.blockDim = dim3(kThreads);
@@ -383,7 +452,7 @@ int max_clusters(int splits) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<BN>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<BN, false>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
     return n;
 }
 
@@ -391,11 +460,13 @@ int max_clusters(int splits) {
 
 cudaError_t launch_decode(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const DecodeParams& p,
                           int n_tiles, cudaStream_t stream) {
+    if (p.x != nullptr)   // fused activation quantiser: the 16-token tile only
+        return bn == 16 ? launch_one<16, true>(tm_act, tm_w, p, n_tiles, stream) : cudaErrorInvalidValue;
     switch (bn) {
-        case 16: return launch_one<16>(tm_act, tm_w, p, n_tiles, stream);
-        case 32: return launch_one<32>(tm_act, tm_w, p, n_tiles, stream);
-        case 64: return launch_one<64>(tm_act, tm_w, p, n_tiles, stream);
-        default: return launch_one<128>(tm_act, tm_w, p, n_tiles, stream);
+        case 16: return launch_one<16, false>(tm_act, tm_w, p, n_tiles, stream);
+        case 32: return launch_one<32, false>(tm_act, tm_w, p, n_tiles, stream);
+        case 64: return launch_one<64, false>(tm_act, tm_w, p, n_tiles, stream);
+        default: return launch_one<128, false>(tm_act, tm_w, p, n_tiles, stream);
     }
 }
 

@@ -64,6 +64,8 @@ struct DecodeParams {
     int w_groups;               // 128-row scale groups per stage in w_sf
     const uint8_t* act_sf;      // one group per stage
     const uint8_t* w_sf;
+    const uint16_t* x;          // fused variant: bf16 activation M x K (leading dimension ldx), else null
+    int ldx;
     void* y;
     int ldy, y_bf16;
     int splits;                 // = cluster size, 1..8
