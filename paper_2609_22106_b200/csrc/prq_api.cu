@@ -627,7 +627,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         q.w_groups = w->w_groups;
         q.act_sf = p.act_sf; q.w_sf = w->d_sf;
         q.y = y; q.ldy = ldy; q.y_bf16 = p.y_bf16;
-        q.status = p.status; q.trace = p.trace;
+        q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
         q.splits = decode_splits(w, M, di);
         bn = decode_bn(M);
         st = make_code_map(&tm_act, codes, w->K / 2, M, bn);
@@ -723,7 +723,7 @@ prq_status prq_linear_fused(const prq_weights* w, prq_act_mode mode, const void*
     q.w_sf = w->d_sf;
     q.x = static_cast<const uint16_t*>(x); q.ldx = ldx;
     q.y = y; q.ldy = ldy; q.y_bf16 = y_dtype == PRQ_BF16;
-    q.status = di->status_ptr; q.trace = trace_ptr();
+    q.status = di->status_ptr; q.trace = trace_ptr(); q.dbg = env_int("PRQ_DBG", 0);
     q.splits = decode_splits(w, M, di);
     CUtensorMap tm_w;
     st = make_code_map(&tm_w, w->d_codes, (static_cast<size_t>(w->K) + w->k_tail) / 2, w->N, 128);

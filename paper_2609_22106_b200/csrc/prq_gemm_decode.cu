@@ -73,16 +73,17 @@ __device__ __forceinline__ uint32_t peer_addr(uint32_t local_addr, uint32_t peer
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(peer));
     return ra;
 }
-// One reduction stage issued by the elected thread, ring slot Q known at compile time.
-template <int BN, int Q>
-__device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, uint32_t sf_t, int rem,
+// One reduction stage issued by the elected thread.  The ring slot is a run-time value on purpose: a
+// CTA runs only a handful of stages, so one compact code path that stays in the instruction cache beats
+// a specialised copy per slot, each of which would be fetched cold.
+template <int BN>
+__device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, uint32_t sf_t, int slot, int rem,
                                             uint32_t accumulate, uint32_t empty_bar0) {
     using C = DCfg<BN>;
-    constexpr uint32_t so = (Q * C::kStageBytes) >> 4;
-    constexpr uint32_t sfo = so + ((kPTile + C::kQTile) >> 4);
     constexpr uint32_t idesc0 = (1u << 7) | (1u << 10) | ((BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
     constexpr uint32_t idesc2 = idesc0 | (2u << 4) | (2u << 29);
-    const uint32_t plo = lo_base + so, qlo = lo_base + so + (kPTile >> 4), slo = lo_base + sfo;
+    const uint32_t plo = lo_base + slot * (C::kStageBytes >> 4), qlo = plo + (kPTile >> 4);
+    const uint32_t slo = plo + ((kPTile + C::kQTile) >> 4);
     const uint32_t sfp_t = sf_t, sfq_t = sf_t + 8;
     tc_copy_sf_atom(sfp_t, desc64(kHiPlain, slo));
     tc_copy_sf_atom(sfq_t, desc64(kHiPlain, slo + (kSf >> 4)));
@@ -94,7 +95,7 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
     if (rem > 64) tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 2), desc64(kHiSw128, qlo + 2), idesc2, sfp_t, sfq_t, 1);
     if (rem > 128) tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 4), desc64(kHiSw128, qlo + 4), idesc0, sfp_t + 4, sfq_t + 4, 1);
     if (rem > 192) tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 6), desc64(kHiSw128, qlo + 6), idesc2, sfp_t + 4, sfq_t + 4, 1);
-    tc_commit(empty_bar0 + Q * 8);
+    tc_commit(empty_bar0 + slot * 8);
 }
 
 template <int BN, bool kFused>
@@ -218,14 +219,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
             const uint32_t nph = nst == 0 ? ph ^ 1 : ph;
             ready = mbar_test_wait(smem_u32(&bar_full[nst]), nph);
             if (leader) {
-                switch (st) {
-                    case 0: issue_stage<BN, 0>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                    case 1: issue_stage<BN, 1>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                    case 2: issue_stage<BN, 2>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                    case 3: issue_stage<BN, 3>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                    case 4: issue_stage<BN, (kStages > 4 ? 4 : 0)>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                    default: issue_stage<BN, (kStages > 5 ? 5 : 0)>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                }
+                issue_stage<BN>(lo_base, d_tmem, sf_t, st, rem, accumulate, eb);
             }
             accumulate = 1;
             if (trace && lane == 0 && it < 64) trace[128 + it] = clock64();

@@ -71,6 +71,7 @@ struct DecodeParams {
     int splits;                 // = cluster size, 1..8
     int* status;
     long long* trace;
+    int dbg;
 };
 // `bn` in {16, 32, 64, 128} is the token tile; the grid is n_tiles * splits CTAs in clusters of `splits`.
 cudaError_t launch_decode(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const DecodeParams& p,

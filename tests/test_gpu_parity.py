@@ -345,3 +345,61 @@ def test_full_size_down_proj_sampled_rows(prq, oracle, M, k):
     assert np.abs(y[rows] - y_ref).max() <= prq_ref.tolerance(y_ref)
     assert np.isfinite(y).all()
     w.free()
+
+
+@pytest.mark.parametrize("M,k,y_dtype", [(1, 256, "f32"), (16, 256, "f32"), (7, 128, "f32"), (16, 0, "f32"), (3, 256, "bf16")])
+def test_linear_fused_matches_two_calls_and_oracle(prq, oracle, M, k, y_dtype):
+    """The one-launch decode step (activation quantised inside the GEMM kernel) against the oracle and,
+    bit for bit, against prq_quantize_act + prq_linear."""
+    N, K = 2560, 9728
+    L = synth.layer(1, N, K, M, T_cal=64, tag=700 + M + k)
+    amax = oracle.channel_amax(L["zcal"])
+    w = prq.prepare_weights(L["W"], amax, 0.5, k)
+    o = oracle.prepare(L["W"], amax, float(np.float32(0.5)), k)
+    x = to_dev_bf16(L["x"])
+    dt = prq.F32 if y_dtype == "f32" else prq.BF16
+    y = prq.linear_fused(w, x, prq.ACT_IDENTITY, dt)
+    assert prq.last_device_status() == 0
+    codes, _, sf = prq.quantize_act(w, x, prq.ACT_IDENTITY)
+    y2 = prq.linear(w, codes, sf, M, dt)
+    assert torch.equal(y, y2)
+    oc, osc = oracle.quantize_act(L["x"])
+    ca, sa = oracle.augment_act(oc, osc, k)
+    y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+    got = y.float().cpu().numpy().astype(np.float64)
+    if y_dtype == "f32":
+        assert np.abs(got - y_ref).max() <= prq_ref.tolerance(y_ref)
+    else:
+        ulp = np.maximum(np.abs(y_ref), 2.0 ** -126) * 2.0 ** -7
+        assert np.all(np.abs(got - y_ref) <= ulp + prq_ref.tolerance(y_ref))
+    w.free()
+
+
+def test_linear_fused_small_shapes_and_strides(prq, oracle):
+    """Ragged N and K (K + k not a multiple of the 256-column stage), a row stride larger than K, and a
+    short reduction (one stage, hence no split)."""
+    for (N, K, k, M) in [(200, 416, 32, 5), (384, 1024, 64, 16), (128, 64, 32, 2)]:
+        L = synth.layer(0, N, K, M, T_cal=32, tag=900 + N)
+        amax = oracle.channel_amax(L["zcal"])
+        w = prq.prepare_weights(L["W"], amax, 0.25, k)
+        o = oracle.prepare(L["W"], amax, float(np.float32(0.25)), k)
+        xs = torch.zeros((M, K + 64), dtype=torch.bfloat16, device="cuda")
+        xs[:, :K] = to_dev_bf16(L["x"])
+        y = prq.linear_fused(w, xs[:, :K])
+        assert prq.last_device_status() == 0
+        oc, osc = oracle.quantize_act(L["x"])
+        ca, sa = oracle.augment_act(oc, osc, k)
+        y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+        assert np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max() <= prq_ref.tolerance(y_ref)
+        w.free()
+
+
+def test_linear_fused_rejects_what_it_does_not_cover(prq, oracle):
+    L = synth.layer(0, 128, 256, 4, T_cal=16, tag=950)
+    w = prq.prepare_weights(L["W"], oracle.channel_amax(L["zcal"]), 0.5, 32)
+    x = torch.zeros((prq.FUSED_MAX_M + 1, 256), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(prq.PrqError):
+        prq.linear_fused(w, x)
+    with pytest.raises(prq.PrqError):
+        prq.linear_fused(w, x[:4], prq.ACT_SCALE_PERM)
+    w.free()
