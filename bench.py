@@ -388,7 +388,10 @@ def main():
         q = lambda s: (lambda: prq.quantize_act(s["w"], s["x"], prq.ACT_IDENTITY, out=(s["codes"], None, s["sf"])))
         g = lambda s: (lambda: prq.linear(s["w"], s["codes"], s["sf"], M, y_dtype, workspace=s["ws"], out=s["y"]))
         step = [(lambda s=s: (q(s)(), g(s)())) for s in sets]
-        return dict(step=step, quant=[q(s) for s in sets], gemm=[g(s) for s in sets], R=len(sets))
+        # one-launch decode step (activation quantised inside the GEMM kernel), where the library offers it
+        f = lambda s: (lambda: prq.linear_fused(s["w"], s["x"], prq.ACT_IDENTITY, y_dtype, out=s["y"]))
+        fused = [f(s) for s in sets] if M <= prq.FUSED_MAX_M else None
+        return dict(step=step, quant=[q(s) for s in sets], gemm=[g(s) for s in sets], fused=fused, R=len(sets))
 
     def time_path(M, k, steps, warmup, y_dtype=prq.F32):
         gs = build_graphs(M, k, y_dtype)
@@ -396,8 +399,11 @@ def main():
         n_side = max(gs["R"], min(steps, 200))
         t_q = run_timed(gs["quant"], n_side, gs["R"])
         t_g = run_timed(gs["gemm"], n_side, gs["R"])
-        return dict(step_us=t_step / steps * 1e6, quant_us=t_q / n_side * 1e6, gemm_us=t_g / n_side * 1e6,
-                    step_total_s=t_step, rotation_sets=gs["R"], timed_launches=2 * steps)
+        out = dict(step_us=t_step / steps * 1e6, quant_us=t_q / n_side * 1e6, gemm_us=t_g / n_side * 1e6,
+                   step_total_s=t_step, rotation_sets=gs["R"], timed_launches=2 * steps)
+        if gs["fused"] is not None:
+            out["fused_step_us"] = run_timed(gs["fused"], n_side, gs["R"]) / n_side * 1e6
+        return out
 
     def time_bf16(M, steps):
         R = rotation_count(2.0 * N_OUT * K_IN + 2.0 * M * K_IN + 2.0 * M * N_OUT, hi=12)
@@ -471,6 +477,9 @@ def main():
         d["bound"] = "tensor" if t_fp4 > t_hbm else "hbm"
         d["gemm_roofline_frac"] = max(t_hbm, t_fp4) / d["gemm_us"]
         d["quant_roofline_frac"] = d["quant_gbs"] / pk["hbm_gbs"]
+        if "fused_step_us" in d:   # the whole step against the bytes it must move: weights, bf16 x, y
+            step_bytes = gemm_bytes(M, k, ob) - 0.53125 * M * K_IN + 2.0 * M * K_IN
+            d["fused_step_roofline_frac"] = step_bytes / pk["hbm_gbs"] / 1e3 / d["fused_step_us"]
     bf16_us = {M: time_bf16(M, side_steps) for M in (1, 16, 128, M_TOK)}
     k0 = detail[f"M{M_TOK}_k0"]
 
