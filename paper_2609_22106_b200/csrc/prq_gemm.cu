@@ -34,11 +34,18 @@ namespace {
 constexpr int kMainWarps = 2;   // producer + issuer; the epilogue warps follow
 constexpr int kPTileBytes = 128 * 128;
 constexpr int kKindPrefill = 0, kKindDecode = 1, kKindGrouped = 2, kKindGroupedSwap = 3;
+constexpr int kRowCache = 256;   // experts whose row ranges are cached in shared memory
 
 constexpr int cgcd(int a, int b) { return b == 0 ? a : cgcd(b, a % b); }
 constexpr int cmin(int a, int b) { return a < b ? a : b; }
 constexpr int cmax(int a, int b) { return a > b ? a : b; }
 constexpr int pow2_at_least(int x) { int p = 32; while (p < x) p *= 2; return p; }
+
+// high words of the shared-memory descriptors: stride between 8-row groups (1024 or 128 bytes, in 16-byte
+// units), descriptor version bit, swizzle mode (2 = 128-byte)
+constexpr uint32_t kHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
+constexpr uint32_t kHiPlain = (128u >> 4) | (1u << 14);
+__device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo) { return (static_cast<uint64_t>(hi) << 32) | lo; }
 
 template <int BN, int KIND>
 struct Cfg {
@@ -81,6 +88,9 @@ struct Unit {
     int tile, split;             // decode bookkeeping
 };
 
+// Where a grouped unit sits: expert, 128-row token tile (counted over all experts), feature tile.
+struct GroupPos { int e, mt, ni; };
+
 template <int BN, int KIND>
 __device__ __forceinline__ int unit_count(const GemmParams& p, const int* tile_start) {
     if (KIND == kKindPrefill) return ((p.M + 127) / 128) * ((p.N + BN - 1) / BN);
@@ -90,7 +100,8 @@ __device__ __forceinline__ int unit_count(const GemmParams& p, const int* tile_s
 }
 
 template <int BN, int KIND>
-__device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_start, int u, int S) {
+__device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_start, const int* row_start, int u, int S,
+                                           const GroupPos& g) {
     Unit t;
     if (KIND == kKindPrefill) {
         const int m_tiles = (p.M + 127) / 128;
@@ -120,46 +131,76 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
         t.tile = ni; t.split = sp;
     } else if (KIND == kKindGroupedSwap) {
         // weights on the MMA M axis (128 output features), a 128-row group of one expert's tokens on N
-        const int total_mt = tile_start[p.n_experts];
-        const int mt = u % total_mt, ni = u / total_mt;
-        int lo = 0, hi = p.n_experts - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (tile_start[mid] <= mt) lo = mid; else hi = mid - 1;
-        }
-        const int e = lo;
+        const int e = g.e, mt = g.mt, ni = g.ni;
         t.p_row = e * p.N + ni * 128;
-        t.q_row = p.expert_offsets[e] + (mt - tile_start[e]) * 128;
+        t.q_row = row_start[e] + (mt - tile_start[e]) * 128;
         t.sfp = p.w_sf + (static_cast<size_t>(e) * S * p.w_groups + ni) * kSfGroupBytes;
         t.sfp_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
         t.sfq = p.act_sf + static_cast<size_t>(mt) * kSfGroupBytes;
         t.sfq_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
         t.s_begin = 0; t.s_end = S;
-        t.row0 = t.q_row; t.row_end = min(p.expert_offsets[e + 1], t.q_row + 128);
+        t.row0 = t.q_row; t.row_end = min(row_start[e + 1], t.q_row + 128);
         t.n0 = ni * 128;
         t.tile = u; t.split = 0;
     } else {
-        const int total_mt = tile_start[p.n_experts];
-        const int mt = u % total_mt, ni = u / total_mt;
-        int lo = 0, hi = p.n_experts - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (tile_start[mid] <= mt) lo = mid; else hi = mid - 1;
-        }
-        const int e = lo;
-        t.p_row = p.expert_offsets[e] + (mt - tile_start[e]) * 128;
+        const int e = g.e, mt = g.mt, ni = g.ni;
+        t.p_row = row_start[e] + (mt - tile_start[e]) * 128;
         t.q_row = e * p.N + ni * BN;
         t.sfp = p.act_sf + static_cast<size_t>(mt) * kSfGroupBytes;
         t.sfp_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
         t.sfq = p.w_sf + (static_cast<size_t>(e) * S * p.w_groups + static_cast<size_t>(ni) * Cfg<BN, KIND>::kNgq) * kSfGroupBytes;
         t.sfq_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
         t.s_begin = 0; t.s_end = S;
-        t.row0 = t.p_row; t.row_end = min(p.expert_offsets[e + 1], t.p_row + 128);
+        t.row0 = t.p_row; t.row_end = min(row_start[e + 1], t.p_row + 128);
         t.n0 = ni * BN;
         t.tile = u; t.split = 0;
     }
     return t;
 }
+
+// The units of one CTA, in order.  Dense kinds: u = blockIdx.x, + gridDim.x, ...  Grouped kinds: a
+// contiguous range of units, so that stepping to the next one is a couple of shared-memory reads (the
+// next token tile, usually of the same expert) instead of a division and a search over the experts in
+// every role's critical path; consecutive units of an expert also reuse its weight tile from L2.
+template <int BN, int KIND>
+struct UnitIter {
+    static constexpr bool kGroupedKind = KIND == kKindGrouped || KIND == kKindGroupedSwap;
+    const GemmParams& p;
+    const int* tile_start;
+    const int* row_start;
+    int S, u, u_end, step;
+    GroupPos g;
+    __device__ __forceinline__ UnitIter(const GemmParams& p_, const int* ts, const int* rs, int S_, int n_units)
+        : p(p_), tile_start(ts), row_start(rs), S(S_), g{0, 0, 0} {
+        if (kGroupedKind) {
+            const int per = (n_units + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+            u = min(n_units, static_cast<int>(blockIdx.x) * per);
+            u_end = min(n_units, u + per);
+            step = 1;
+            if (u < u_end) {
+                const int total_mt = tile_start[p.n_experts];
+                g.mt = u % total_mt; g.ni = u / total_mt;
+                int lo = 0, hi = p.n_experts - 1;
+                while (lo < hi) {   // last expert whose first tile is <= mt
+                    const int mid = (lo + hi + 1) >> 1;
+                    if (tile_start[mid] <= g.mt) lo = mid; else hi = mid - 1;
+                }
+                g.e = lo;
+            }
+        } else {
+            u = blockIdx.x; u_end = n_units; step = gridDim.x;
+        }
+    }
+    __device__ __forceinline__ bool valid() const { return u < u_end; }
+    __device__ __forceinline__ Unit get() const { return make_unit<BN, KIND>(p, tile_start, row_start, u, S, g); }
+    __device__ __forceinline__ void next() {
+        u += step;
+        if (kGroupedKind && u < u_end) {
+            if (++g.mt == tile_start[p.n_experts]) { g.mt = 0; g.e = 0; ++g.ni; }
+            while (tile_start[g.e + 1] <= g.mt) ++g.e;   // experts without rows have no tile: skipped here
+        }
+    }
+};
 
 __device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
@@ -174,7 +215,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
     __shared__ int abort_flag_s;
     __shared__ int is_last_s;
     __shared__ int tile_start[(KIND == kKindGrouped || KIND == kKindGroupedSwap) ? kMaxExperts + 1 : 1];
+    __shared__ int row_cache[(KIND == kKindGrouped || KIND == kKindGroupedSwap) ? kRowCache + 1 : 1];
     volatile int* abort_flag = &abort_flag_s;
+    const int* row_start = ((KIND == kKindGrouped || KIND == kKindGroupedSwap) && p.n_experts <= kRowCache)
+                               ? row_cache : p.expert_offsets;
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
@@ -191,13 +235,20 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
         tma_prefetch_desc(&tm_act);
         tma_prefetch_desc(&tm_w);
     }
-    if ((KIND == kKindGrouped || KIND == kKindGroupedSwap) && threadIdx.x == 64) {
-        int acc = 0;
-        for (int e = 0; e < p.n_experts; ++e) {
-            tile_start[e] = acc;
-            acc += (p.expert_offsets[e + 1] - p.expert_offsets[e] + 127) / 128;
+    if (KIND == kKindGrouped || KIND == kKindGroupedSwap) {
+        // the expert row ranges are kept in shared memory (up to kRowCache experts): every role looks
+        // them up once per tile, and a dependent global load there sits on the producer's critical path
+        if (p.n_experts <= kRowCache)
+            for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x) row_cache[e] = p.expert_offsets[e];
+        __syncthreads();
+        if (threadIdx.x == 64) {
+            int acc = 0;
+            for (int e = 0; e < p.n_experts; ++e) {
+                tile_start[e] = acc;
+                acc += (row_start[e + 1] - row_start[e] + 127) / 128;
+            }
+            tile_start[p.n_experts] = acc;
         }
-        tile_start[p.n_experts] = acc;
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&tmem_slot), C::kTmemCols);
@@ -222,8 +273,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
         int it = 0, st = 0;
         uint32_t ph = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
-            const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
+        for (UnitIter<BN, KIND> ui(p, tile_start, row_start, S, n_units); ui.valid() && ok; ui.next()) {
+            const Unit t = ui.get();
             for (int s = t.s_begin; s < t.s_end; ++s, ++it) {
                 if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
                 if (trace && lane == 0 && it < 64) trace[it] = clock64();
@@ -262,8 +313,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
         const bool leader = elect_one();
         const uint32_t sfp_t = tmem_base + C::kSfpCol;
         const uint32_t sfq_t = tmem_base + C::kSfqCol;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
-            const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
+        const uint32_t lo_base = ((smem_base & 0x3FFFF) >> 4) | (1u << 16);
+        for (UnitIter<BN, KIND> ui(p, tile_start, row_start, S, n_units); ui.valid() && ok; ui.next(), ++acc_it) {
+            const Unit t = ui.get();
             const int buf = acc_it % C::kAcc;
             const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
             if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1, abort_flag)) { ok = false; break; }
@@ -280,27 +332,30 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                 const uint32_t nph = nst == 0 ? ph ^ 1 : ph;
                 ready = mbar_test_wait(smem_u32(&bar_full[nst]), nph);
                 if (leader) {
-                    const uint32_t sb = smem_base + st * C::kStageBytes;
-                    const uint32_t sfp_s = sb + kPTileBytes + C::kQTileBytes;
-                    const uint32_t sfq_s = sfp_s + C::kSfpBytes;
+                    // Descriptors as (constant high word, 32-bit low word): the low word is the shared
+                    // address in 16-byte units plus the leading-dimension field, so a stage's descriptors
+                    // cost one add each instead of a 64-bit shift-and-or chain.
+                    const uint32_t plo = lo_base + st * (C::kStageBytes >> 4);
+                    const uint32_t qlo = plo + (kPTileBytes >> 4);
+                    const uint32_t sfp_lo = qlo + (C::kQTileBytes >> 4), sfq_lo = sfp_lo + (C::kSfpBytes >> 4);
 #pragma unroll
                     for (int ka = 0; ka < 2; ++ka) {
                         if (ka * 2 < ksteps && !(p.dbg & 1)) {
-                            tc_copy_sf_atom(sfp_t + ka * 4, make_smem_desc(sfp_s + ka * 512, 16, 128, kSwizzleNone));
+                            tc_copy_sf_atom(sfp_t + ka * 4, desc64(kHiPlain, sfp_lo + ka * (512 >> 4)));
 #pragma unroll
                             for (int g = 0; g < C::kNgq; ++g)
                                 tc_copy_sf_atom(sfq_t + ka * 4 * C::kNgq + g * 4,
-                                                make_smem_desc(sfq_s + g * kSfGroupBytes + ka * 512, 16, 128, kSwizzleNone));
+                                                desc64(kHiPlain, sfq_lo + g * (kSfGroupBytes >> 4) + ka * (512 >> 4)));
                         }
                     }
-                    const uint64_t pd = make_smem_desc(sb, 16, 1024, kSwizzle128B);
-                    const uint64_t qd = make_smem_desc(sb + kPTileBytes, 16, 1024, kSwizzle128B);
+                    constexpr uint32_t idesc0 = (1u << 7) | (1u << 10) | ((BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+                    constexpr uint32_t idesc2 = idesc0 | (2u << 4) | (2u << 29);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         if (j < ksteps && !(p.dbg & 2)) {
-                            const uint32_t sf_id = (j & 1) * 2;
-                            tc_mma_mxf4(d_tmem, pd + 2 * j, qd + 2 * j, make_idesc_mxf4(BN, sf_id, sf_id),
-                                        sfp_t + (j >> 1) * 4, sfq_t + (j >> 1) * 4 * C::kNgq, accumulate);
+                            tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 2 * j), desc64(kHiSw128, qlo + 2 * j),
+                                        (j & 1) ? idesc2 : idesc0, sfp_t + (j >> 1) * 4,
+                                        sfq_t + (j >> 1) * 4 * C::kNgq, accumulate);
                             accumulate = 1;
                         }
                     }
@@ -320,8 +375,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
         const int et = q * 32 + lane;           // 0..127: accumulator row
         int acc_it = 0;
         bool ok = true;
-        for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x, ++acc_it) {
-            const Unit t = make_unit<BN, KIND>(p, tile_start, u, S);
+        for (UnitIter<BN, KIND> ui(p, tile_start, row_start, S, n_units); ui.valid() && ok; ui.next(), ++acc_it) {
+            const Unit t = ui.get();
             const int buf = acc_it % C::kAcc;
             const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
             if (!mbar_wait(smem_u32(&bar_acc_full[buf]), acc_ph, abort_flag)) { ok = false; break; }
