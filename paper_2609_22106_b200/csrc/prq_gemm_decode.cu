@@ -11,7 +11,7 @@
 // CTAs of the next kernel of the stream (the next layer's GEMM) are resident and streaming their weights
 // while this one finishes.
 //
-// Roles per CTA (6 warps): warp 0 TMA producer, warp 1 tcgen05 issuer (scale copies + MMAs), warps 2-5
+// Roles per CTA (6 warps, 10 from 64 tokens on): warp 0 TMA producer, warp 1 tcgen05 issuer (scale copies + MMAs), warps 2-5 (2-9)
 // epilogue and reduction.  The activation tail is re-read: stages past the K main columns load the
 // token tile from column K - k and the weight tile from column K onwards (Kernel design paragraph).
 // Every wait is bounded; the cluster barriers sit on the common path so that a CTA that gave up still
@@ -36,7 +36,6 @@
 namespace prq {
 namespace {
 
-constexpr int kThreads = 192;
 constexpr int kPTile = 128 * 128;   // weight tile bytes: 128 rows x 256 codes
 constexpr int kSf = kSfGroupBytes;  // one 128-row scale group per operand and stage
 
@@ -52,6 +51,10 @@ struct DCfg {
     // ring depth: 5 / 4 stages leave room for two CTAs per SM at 16 / 32 tokens
     static constexpr int kStages = BN == 16 ? 5 : BN == 32 ? 4 : BN == 64 ? 6 : 4;
     static constexpr int kCtasPerSm = BN <= 32 ? 2 : 1;
+    // epilogue warps: four (one per tensor-memory lane quarter); eight from 64 tokens on, where moving the
+    // partial sums is most of the kernel -- two warps per quarter then take alternate 16-token chunks
+    static constexpr int kEpiWarps = BN >= 64 ? 8 : 4;
+    static constexpr int kThreads = 64 + 32 * kEpiWarps;
     // receive buffer of the split-K exchange: [peer][token slot][128 rows] fp32, ceil(BN / splits) token
     // slots per peer, i.e. at most BN + 7 token rows of 512 bytes
     static constexpr int kRecvBytes = (BN + 7) * 512;
@@ -99,7 +102,7 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
 }
 
 template <int BN, bool kFused>
-__global__ void __launch_bounds__(kThreads, DCfg<BN>::kCtasPerSm)
+__global__ void __launch_bounds__(DCfg<BN>::kThreads, DCfg<BN>::kCtasPerSm)
 decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
               const DecodeParams p) {
     using C = DCfg<BN>;
@@ -230,10 +233,12 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
         // ------------------------------------------------------------ epilogue, part 1: accumulator -> registers
         // -> (splits == 1) y, or this CTA's partial tile in shared memory, token-major: partial[t][row]
         const int q4 = warp & 3;
+        const int chunk0 = (warp - 2) >> 2;          // which of the quarter's warps this is
         const int row = q4 * 32 + lane;              // weight row inside the tile
         const int n = n0 + row;
         const uint32_t acc_t = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
         if constexpr (kFused) {
+            static_assert(!kFused || C::kEpiWarps == 4, "the quantiser role is written for four warps");
             // ---- activation quantiser of this CTA: thread = (token, 32-column block) of a stage ----
             const int et = threadIdx.x - 64;
             const int tok0 = et >> 3, blk = et & 7;
@@ -295,7 +300,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
             tc_fence_after_sync();
             float* partial = reinterpret_cast<float*>(smem);
 #pragma unroll 1
-            for (int c = 0; c < (BN + 15) / 16; ++c) {
+            for (int c = chunk0; c < (BN + 15) / 16; c += C::kEpiWarps / 4) {
                 uint32_t v[16];
                 tmem_ld_32x16(acc_t + c * 16, v);
                 tmem_ld_wait();
@@ -336,8 +341,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
         const int et = threadIdx.x - 64;                        // 0..127 for the epilogue warps
         const int j = et & 31, tq = et >> 5;
         if (warp >= 2 && !abort_flag_s) {
-            asm volatile("bar.sync 1, 128;" ::: "memory");       // the parked tile is complete
-            for (int tok = tq; tok < p.M; tok += 4) {
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * C::kEpiWarps) : "memory");   // the parked tile is complete
+            for (int tok = tq; tok < p.M; tok += C::kEpiWarps) {
                 const int owner = tok % splits, slot = tok / splits;
                 float4 v;
                 asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
@@ -356,7 +361,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
             // this CTA's tokens: split, split + splits, ...; a thread owns 4 consecutive weight rows and
             // every fourth slot; the sum runs in peer order
             const int n = n0 + 4 * j;
-            for (int slot = tq; split + slot * splits < p.M; slot += 4) {
+            for (int slot = tq; split + slot * splits < p.M; slot += C::kEpiWarps) {
                 const int tok = split + slot * splits;
                 float4 v[8];
 #pragma unroll
@@ -415,7 +420,7 @@ cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_tiles * p.splits);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(C::kThreads);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
@@ -436,7 +441,7 @@ int max_clusters(int splits) {
     cudaFuncSetAttribute(decode_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(splits);
-    cfg.blockDim = dim3(kThreads);
+    cfg.blockDim = dim3(C::kThreads);
     cfg.dynamicSmemBytes = C::kSmemBytes;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
