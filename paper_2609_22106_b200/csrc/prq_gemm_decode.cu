@@ -126,6 +126,13 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     const int n0 = tile * 128;
 
     const long long t_entry = clock64();
+    __shared__ int trace_slot_s;
+    if (p.trace && blockIdx.x == 0 && threadIdx.x == 0) {
+        unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g));
+        const int sl = static_cast<int>(atomicAdd(reinterpret_cast<unsigned long long*>(p.trace + 2040), 1ull)) & 63;
+        trace_slot_s = sl;
+        p.trace[2048 + sl * 4] = static_cast<long long>(g);
+    }
     if (threadIdx.x == 0) {
         // a slot is full when its TMA bytes have landed and, fused, when the four quantiser warps are done
         for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), kFused ? 5 : 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
@@ -247,6 +254,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
                 *reinterpret_cast<uint2*>(smem + i * C::kStageBytes + kPTile + C::kQTile + kSf + et * 8) = make_uint2(0, 0);
             asm volatile("bar.sync 1, 128;" ::: "memory");
             grid_dependency_wait();   // x is the previous kernel's output
+            if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[2048 + trace_slot_s * 4 + 1] = static_cast<long long>(g); }
             if (trace && et == 0) trace[200] = clock64();
             bool qok = true;
 #pragma unroll 1
@@ -294,6 +302,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
             }
         } else {
             grid_dependency_wait();   // y may still be read by an earlier kernel
+            if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[2048 + trace_slot_s * 4 + 1] = static_cast<long long>(g); }
         }
         if (mbar_wait(smem_u32(&bar_acc_full), 0, abort_flag)) {
             if (trace && row == 0) trace[192] = clock64();
@@ -400,6 +409,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     tc_fence_before_sync();
     __syncthreads();
     if (trace && threadIdx.x == 0) trace[501] = clock64();
+    if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[2048 + trace_slot_s * 4 + 2] = static_cast<long long>(g); }
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();
