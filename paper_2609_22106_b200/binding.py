@@ -12,7 +12,8 @@ import os
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libprq.so")
+# PRQ_TRACE=1 selects the developer build with clock-stamp tracing compiled in (see build.py)
+LIB_PATH = os.path.join(_HERE, "libprq_trace.so" if os.environ.get("PRQ_TRACE") == "1" else "libprq.so")
 
 OK = 0
 F32, BF16 = 0, 1

@@ -8,7 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
-LIB = os.path.join(HERE, "libprq.so")
+TRACE = os.environ.get("PRQ_TRACE") == "1"   # developer build: clock-stamp tracing compiled into the kernels
+LIB = os.path.join(HERE, "libprq_trace.so" if TRACE else "libprq.so")
 SOURCES = ["prq_api.cu", "prq_prep.cu", "prq_quant.cu", "prq_gemm.cu", "prq_gemm_prefill_pair.cu", "prq_gemm_decode.cu", "prq_peak_probe.cu"]
 
 
@@ -29,6 +30,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     ] + [os.path.join(CSRC, s) for s in SOURCES] + ["-lpthread"]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
+    if TRACE:
+        cmd.insert(1, "-DPRQ_TRACE=1")
     subprocess.check_call(cmd)
     return LIB
 

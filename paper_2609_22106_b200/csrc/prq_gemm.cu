@@ -259,7 +259,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_slot;
     // optional developer trace: SM clock stamps of the first iterations of each role (CTA 0..3 only)
-    long long* trace = (p.trace && blockIdx.x < 4) ? p.trace + blockIdx.x * 512 : nullptr;
+    long long* const ptrace = kTraceBuild ? p.trace : nullptr;
+    long long* trace = (ptrace && blockIdx.x < 4) ? ptrace + blockIdx.x * 512 : nullptr;
     if (trace && threadIdx.x == 0) trace[500] = clock64();
     const int n_units = unit_count<BN, KIND>(p, tile_start);
 

@@ -5,9 +5,11 @@
 // K + k is split over the CTAs of a thread-block cluster so that every SM streams a share of the
 // weights.  Each CTA of a cluster accumulates its K-range in tensor memory and then pushes, through
 // distributed shared memory, the partial sums of token t into a receive buffer of the CTA that owns
-// token t (t mod cluster size); after one cluster barrier every CTA adds up what it received and writes
-// its tokens to y.  No global scratch, no atomics, one barrier, and the summation order is fixed (peer
-// 0, 1, ...), so the result is reproducible.  For up to 32 tokens two CTAs fit on an SM, so that the
+// token t (t mod cluster size); the owner adds up what it received and writes its tokens to y.  Up to 32
+// tokens the pushes are asynchronous stores whose bytes are counted on an mbarrier of the owner, which
+// therefore waits for exactly its own tokens; from 64 tokens on they are plain stores followed by one
+// cluster barrier.  No global scratch, no atomics, and the summation order is fixed (peer 0, 1, ...), so
+// the result is reproducible.  For up to 32 tokens two CTAs fit on an SM, so that the
 // CTAs of the next kernel of the stream (the next layer's GEMM) are resident and streaming their weights
 // while this one finishes.
 //
@@ -55,6 +57,10 @@ struct DCfg {
     // partial sums is most of the kernel -- two warps per quarter then take alternate 16-token chunks
     static constexpr int kEpiWarps = BN >= 64 ? 8 : 4;
     static constexpr int kThreads = 64 + 32 * kEpiWarps;
+    // split-K exchange: up to 32 tokens asynchronous stores counted on the owner's mbarrier (the owner waits
+    // only for its own tokens: 0.3 us less at M = 1 than a cluster barrier); from 64 tokens on plain stores and
+    // one cluster barrier (the per-store barrier update costs more than it saves: 9.4 against 9.6 us at M = 128)
+    static constexpr bool kAsyncExchange = BN <= 32;
     // receive buffer of the split-K exchange: [peer][token slot][128 rows] fp32, ceil(BN / splits) token
     // slots per peer, i.e. at most BN + 7 token rows of 512 bytes
     static constexpr int kRecvBytes = (BN + 7) * 512;
@@ -109,6 +115,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     constexpr int kStages = C::kStages;
     __shared__ __align__(8) uint64_t bar_full[kStages], bar_empty[kStages], bar_acc_full;
+    __shared__ __align__(8) uint64_t bar_recv;   // counts the bytes of partial sums that the peers deliver to this CTA
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag_s;
     volatile int* abort_flag = &abort_flag_s;
@@ -125,18 +132,20 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     const int s_end = static_cast<int>(static_cast<long long>(S) * (split + 1) / splits);
     const int n0 = tile * 128;
 
-    const long long t_entry = clock64();
+    long long* const ptrace = kTraceBuild ? p.trace : nullptr;
+    const long long t_entry = kTraceBuild ? clock64() : 0;
     __shared__ int trace_slot_s;
-    if (p.trace && blockIdx.x == 0 && threadIdx.x == 0) {
+    if (ptrace && blockIdx.x == 0 && threadIdx.x == 0) {
         unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g));
-        const int sl = static_cast<int>(atomicAdd(reinterpret_cast<unsigned long long*>(p.trace + 2040), 1ull)) & 63;
+        const int sl = static_cast<int>(atomicAdd(reinterpret_cast<unsigned long long*>(ptrace + 2040), 1ull)) & 63;
         trace_slot_s = sl;
-        p.trace[2048 + sl * 4] = static_cast<long long>(g);
+        ptrace[2048 + sl * 4] = static_cast<long long>(g);
     }
     if (threadIdx.x == 0) {
         // a slot is full when its TMA bytes have landed and, fused, when the four quantiser warps are done
         for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), kFused ? 5 : 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
         mbar_init(smem_u32(&bar_acc_full), 1);
+        mbar_init(smem_u32(&bar_recv), 1);
         abort_flag_s = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tm_act);
@@ -149,15 +158,24 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    // Split-K exchange, receiving side: this CTA owns tokens split, split + splits, ...; every CTA of the
+    // cluster (itself included) delivers 512 bytes per owned token, counted on bar_recv.  The cluster
+    // barrier only tells the peers that the barrier exists before they push: arrive here, wait just before
+    // the pushes, so that it costs nothing.
+    const int n_own = split < p.M ? (p.M - split + splits - 1) / splits : 0;
+    if (C::kAsyncExchange && splits > 1) {
+        if (threadIdx.x == 0) mbar_arrive_expect_tx(smem_u32(&bar_recv), static_cast<uint32_t>(n_own) * splits * 512u);
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    }
     // set-up done: let the next kernel of the stream be scheduled (its launch latency then overlaps this
     // kernel).  The roles that touch what earlier kernels wrote (activation codes and scales) or may
     // still read (y) pass grid_dependency_wait() first; the weights depend on no kernel, so the producer
     // requests them before it waits and they stream in while the previous kernel (normally the
     // activation quantiser) is still running.
-    const long long t_setup = clock64();
+    const long long t_setup = kTraceBuild ? clock64() : 0;
     grid_launch_dependents();
     const uint32_t tmem_base = tmem_slot;
-    long long* trace = (p.trace && blockIdx.x < 4) ? p.trace + blockIdx.x * 512 : nullptr;
+    long long* trace = (ptrace && blockIdx.x < 4) ? ptrace + blockIdx.x * 512 : nullptr;
     if (trace && threadIdx.x == 0) { trace[500] = clock64(); trace[502] = t_entry; trace[503] = t_setup; }
     const uint32_t lo_base = ((smem_base & 0x3FFFF) >> 4) | (1u << 16);
 
@@ -254,7 +272,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
                 *reinterpret_cast<uint2*>(smem + i * C::kStageBytes + kPTile + C::kQTile + kSf + et * 8) = make_uint2(0, 0);
             asm volatile("bar.sync 1, 128;" ::: "memory");
             grid_dependency_wait();   // x is the previous kernel's output
-            if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[2048 + trace_slot_s * 4 + 1] = static_cast<long long>(g); }
+            if (ptrace && blockIdx.x == 0 && threadIdx.x == 64) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); ptrace[2048 + trace_slot_s * 4 + 1] = static_cast<long long>(g); }
             if (trace && et == 0) trace[200] = clock64();
             bool qok = true;
 #pragma unroll 1
@@ -302,7 +320,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
             }
         } else {
             grid_dependency_wait();   // y may still be read by an earlier kernel
-            if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[2048 + trace_slot_s * 4 + 1] = static_cast<long long>(g); }
+            if (ptrace && blockIdx.x == 0 && threadIdx.x == 64) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); ptrace[2048 + trace_slot_s * 4 + 1] = static_cast<long long>(g); }
         }
         if (mbar_wait(smem_u32(&bar_acc_full), 0, abort_flag)) {
             if (trace && row == 0) trace[192] = clock64();
@@ -349,23 +367,36 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
         const int slots = (p.M + splits - 1) / splits;        // token slots per peer in a receive buffer
         const int et = threadIdx.x - 64;                        // 0..127 for the epilogue warps
         const int j = et & 31, tq = et >> 5;
+        if constexpr (C::kAsyncExchange)
+            asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every peer's bar_recv exists
         if (warp >= 2 && !abort_flag_s) {
             asm volatile("bar.sync 1, %0;" ::"n"(32 * C::kEpiWarps) : "memory");   // the parked tile is complete
             for (int tok = tq; tok < p.M; tok += C::kEpiWarps) {
                 const int owner = tok % splits, slot = tok / splits;
-                float4 v;
-                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                             : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(smem_base + tok * 512 + j * 16));
+                uint4 v;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(smem_base + tok * 512 + j * 16));
                 const uint32_t dst = peer_addr(recv_base + ((split * slots + slot) * 128 + 4 * j) * 4, owner);
-                asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};"
-                             ::"r"(dst), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+                if constexpr (C::kAsyncExchange) {
+                    const uint32_t rbar = peer_addr(smem_u32(&bar_recv), owner);
+                    // asynchronous store into the owner's receive buffer; its bytes are counted on the owner's barrier
+                    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                                 ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "r"(rbar) : "memory");
+                } else {
+                    asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};"
+                                 ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+                }
             }
             if (trace && et == 0) trace[195] = clock64();
+            // the owner's wait: all partial sums of its tokens have arrived (nobody writes to this CTA after that)
+            if (C::kAsyncExchange && n_own > 0) mbar_wait(smem_u32(&bar_recv), 0, abort_flag);
         }
-        // all threads of all CTAs: orders the pushes before the owners' reads, and nobody leaves before
-        // everything addressed to its peers has been delivered
-        __syncthreads();
-        cluster_sync_all();
+        if constexpr (!C::kAsyncExchange) {
+            // all threads of all CTAs: orders the pushes before the owners' reads, and nobody leaves before
+            // everything addressed to its peers has been delivered
+            __syncthreads();
+            cluster_sync_all();
+        }
         if (warp >= 2 && !abort_flag_s) {
             // this CTA's tokens: split, split + splits, ...; a thread owns 4 consecutive weight rows and
             // every fourth slot; the sum runs in peer order
@@ -409,7 +440,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     tc_fence_before_sync();
     __syncthreads();
     if (trace && threadIdx.x == 0) trace[501] = clock64();
-    if (p.trace && blockIdx.x == 0 && threadIdx.x == 64) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); p.trace[2048 + trace_slot_s * 4 + 2] = static_cast<long long>(g); }
+    if (ptrace && blockIdx.x == 0 && threadIdx.x == 64) { unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); ptrace[2048 + trace_slot_s * 4 + 2] = static_cast<long long>(g); }
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();

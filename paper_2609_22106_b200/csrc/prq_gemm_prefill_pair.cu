@@ -216,10 +216,11 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     uint32_t sk_b, sk_e;
     plan_sk.range(g, sk_b, sk_e);
 
-    if (p.trace && threadIdx.x == 0) {
+    long long* const ptrace = kTraceBuild ? p.trace : nullptr;
+    if (ptrace && threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        p.trace[2048 + 2 * blockIdx.x] = static_cast<long long>(t);
+        ptrace[2048 + 2 * blockIdx.x] = static_cast<long long>(t);
     }
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
@@ -247,16 +248,16 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     // set-up done: let the next kernel of the stream be scheduled (its launch latency then overlaps this
     // kernel).  Each role that touches global memory which earlier kernels wrote (activation codes,
     // workspace counters) or still read (y) passes grid_dependency_wait() first; the issuer touches none.
-    if (p.trace && threadIdx.x == 0) {
+    if (ptrace && threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        p.trace[2048 + 400 + 2 * blockIdx.x] = static_cast<long long>(t);
+        ptrace[2048 + 400 + 2 * blockIdx.x] = static_cast<long long>(t);
     }
     grid_launch_dependents();
     const uint32_t tmem_base = tmem_slot;
     const int trace_cta0 = p.dbg >> 16;  // developer aid: first of the four traced CTAs
-    long long* trace = (p.trace && static_cast<int>(blockIdx.x) >= trace_cta0 && static_cast<int>(blockIdx.x) < trace_cta0 + 4)
-                           ? p.trace + (blockIdx.x - trace_cta0) * 512 : nullptr;
+    long long* trace = (ptrace && static_cast<int>(blockIdx.x) >= trace_cta0 && static_cast<int>(blockIdx.x) < trace_cta0 + 4)
+                           ? ptrace + (blockIdx.x - trace_cta0) * 512 : nullptr;
     if (trace && threadIdx.x == 0) trace[500] = clock64();
     const uint32_t lo_base = ((smem_base & 0x3FFFF) >> 4) | (1u << 16);
 
@@ -288,10 +289,10 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             }
         }
         grid_dependency_wait();
-        if (p.trace && threadIdx.x == 0) {
+        if (ptrace && threadIdx.x == 0) {
             unsigned long long t;
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-            p.trace[2048 + 401 + 2 * blockIdx.x] = static_cast<long long>(t);
+            ptrace[2048 + 401 + 2 * blockIdx.x] = static_cast<long long>(t);
         }
         while (ok && r.next(sg)) {
             const int mi = sg.tile % p.m_tiles, ni = sg.tile / p.m_tiles;
@@ -546,10 +547,10 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     cluster_arrive();
     cluster_wait();
     if (trace && threadIdx.x == 0) trace[501] = clock64();
-    if (p.trace && threadIdx.x == 0) {
+    if (ptrace && threadIdx.x == 0) {
         unsigned long long t;
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        p.trace[2049 + 2 * blockIdx.x] = static_cast<long long>(t);
+        ptrace[2049 + 2 * blockIdx.x] = static_cast<long long>(t);
     }
     if (warp == 1) {
         __syncwarp();
