@@ -341,7 +341,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                     const uint32_t sfp_lo = qlo + (C::kQTileBytes >> 4), sfq_lo = sfp_lo + (C::kSfpBytes >> 4);
 #pragma unroll
                     for (int ka = 0; ka < 2; ++ka) {
-                        if (ka * 2 < ksteps && !(p.dbg & 1)) {
+                        if (ka * 2 < ksteps && !(kTraceBuild && (p.dbg & 1))) {
                             tc_copy_sf_atom(sfp_t + ka * 4, desc64(kHiPlain, sfp_lo + ka * (512 >> 4)));
 #pragma unroll
                             for (int g = 0; g < C::kNgq; ++g)
@@ -353,7 +353,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                     constexpr uint32_t idesc2 = idesc0 | (2u << 4) | (2u << 29);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        if (j < ksteps && !(p.dbg & 2)) {
+                        if (j < ksteps && !(kTraceBuild && (p.dbg & 2))) {
                             tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 2 * j), desc64(kHiSw128, qlo + 2 * j),
                                         (j & 1) ? idesc2 : idesc0, sfp_t + (j >> 1) * 4,
                                         sfq_t + (j >> 1) * 4 * C::kNgq, accumulate);
