@@ -403,3 +403,23 @@ def test_linear_fused_rejects_what_it_does_not_cover(prq, oracle):
     with pytest.raises(prq.PrqError):
         prq.linear_fused(w, x[:4], prq.ACT_SCALE_PERM)
     w.free()
+
+
+@pytest.mark.parametrize("M", [1, 16, 64, 128])
+def test_decode_split_k_is_reproducible(prq, oracle, M):
+    """The cluster split-K exchange sums the partial results in a fixed order: repeated launches of the same
+    problem give the same bits, for both forms of the exchange (asynchronous stores up to 32 tokens, plain
+    stores and a cluster barrier above) and for the fused entry."""
+    N, K, k = 2560, 9728, 256
+    L = synth.layer(1, N, K, M, T_cal=32, tag=800 + M)
+    w = prq.prepare_weights(L["W"], oracle.channel_amax(L["zcal"]), 0.5, k)
+    x = to_dev_bf16(L["x"])
+    codes, _, sf = prq.quantize_act(w, x, prq.ACT_IDENTITY)
+    ref = prq.linear(w, codes, sf, M).clone()
+    for _ in range(40):
+        assert torch.equal(prq.linear(w, codes, sf, M), ref)
+    if M <= prq.FUSED_MAX_M:
+        for _ in range(40):
+            assert torch.equal(prq.linear_fused(w, x), ref)
+    assert prq.last_device_status() == 0
+    w.free()
