@@ -115,7 +115,22 @@ prq_status make_out_map(CUtensorMap* map, void* y, int M, int N, int ldy, bool b
     return r == CUDA_SUCCESS ? PRQ_OK : PRQ_ERR_CUDA;
 }
 
+// Weight-side tensor maps of a dense handle, encoded once at creation (cloning re-encodes: other addresses).
+prq_status build_weight_maps(prq_weights* w) {
+    w->maps_ready = false;
+    if (w->n_experts != 1) return PRQ_OK;
+    const uint64_t Ka = static_cast<uint64_t>(w->K) + w->k_tail;
+    prq_status st = make_code_map(&w->tm_w_decode, w->d_codes, Ka / 2, w->N, 128);
+    if (st == PRQ_OK) st = make_code_map(&w->tm_w_pair, w->d_codes, Ka / 2, w->N, kPrefillTileN / 2);
+    if (st == PRQ_OK && w->d_sf_alt[2])
+        st = make_sf_map(&w->tm_sfw_pair, w->d_sf_alt[2],
+                         static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[2] * kSfGroupBytes, 8);
+    if (st == PRQ_OK) w->maps_ready = true;
+    return st;
+}
+
 int env_int(const char* name, int dflt) {
+    if (!dev_knobs_enabled()) return dflt;
     const char* v = std::getenv(name);
     return v && *v ? std::atoi(v) : dflt;
 }
@@ -123,6 +138,7 @@ int env_int(const char* name, int dflt) {
 // Developer aid: PRQ_TRACE_PTR holds the address of a device buffer (4 x 512 int64) that the GEMM
 // fills with clock stamps.  Unset in normal use.
 long long* trace_ptr() {
+    if (!dev_knobs_enabled()) return nullptr;
     const char* v = std::getenv("PRQ_TRACE_PTR");
     return v && *v ? reinterpret_cast<long long*>(std::strtoull(v, nullptr, 0)) : nullptr;
 }
@@ -353,6 +369,7 @@ prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, c
             ok = cudaMemcpy(w->d_sf_alt[a], sf_alt[a].data(), sf_alt[a].size(), cudaMemcpyHostToDevice) == cudaSuccess;
         }
         if (!ok) { prq_weights_free(w); return PRQ_ERR_CUDA; }
+        if (build_weight_maps(w) != PRQ_OK) { prq_weights_free(w); return PRQ_ERR_CUDA; }
     } catch (const std::bad_alloc&) {
         prq_weights_free(w);
         return PRQ_ERR_OOM;
@@ -495,6 +512,7 @@ prq_status prq_weights_clone(const prq_weights* w, prq_weights** out) {
     } catch (const std::bad_alloc&) {
         st = PRQ_ERR_OOM;
     }
+    if (st == PRQ_OK) st = build_weight_maps(c);
     if (cur != w->device) cudaSetDevice(cur);
     if (st != PRQ_OK) { prq_weights_free(c); return st; }
     *out = c;
@@ -596,7 +614,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
     if (w && M == 0) return PRQ_OK;
     prq_status st = check_linear_common(w, codes, scales_sf, y, ldy, y_dtype);
     if (st != PRQ_OK) return st;
-    if (M < 0 || w->n_experts != 1) return PRQ_ERR_INVALID_ARG;
+    if (M < 0 || w->n_experts != 1 || !w->maps_ready) return PRQ_ERR_INVALID_ARG;
     DeviceInfo* di;
     st = device_info(w->device, &di);
     if (st != PRQ_OK) return st;
@@ -631,9 +649,8 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         q.splits = decode_splits(w, M, di);
         bn = decode_bn(M);
         st = make_code_map(&tm_act, codes, w->K / 2, M, bn);
-        if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, 128);
         if (st != PRQ_OK) return st;
-        cudaError_t e = launch_decode(bn, tm_act, tm_w, q, (w->N + 127) / 128, static_cast<cudaStream_t>(stream));
+        cudaError_t e = launch_decode(bn, tm_act, w->tm_w_decode, q, (w->N + 127) / 128, static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     } else if (env_int("PRQ_PREFILL_BN", 0) == 0) {
@@ -677,15 +694,13 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         if (!aligned16(workspace)) return PRQ_ERR_ALIGNMENT;
         q.flags = static_cast<int*>(workspace);
         q.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + flag_bytes);
-        CUtensorMap tm_y, tm_sfa, tm_sfw;
+        CUtensorMap tm_y, tm_sfa;
         const uint64_t Sg = static_cast<uint64_t>(w->plan.S);
         st = make_code_map(&tm_act, codes, w->K / 2, M, 128);
-        if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, kPrefillTileN / 2);
         if (st == PRQ_OK) st = make_sf_map(&tm_sfa, p.act_sf, Sg * p.act_groups * kSfGroupBytes, 4);
-        if (st == PRQ_OK) st = make_sf_map(&tm_sfw, q.w_sf, Sg * q.w_groups * kSfGroupBytes, 8);
         if (st == PRQ_OK) st = make_out_map(&tm_y, y, M, w->N, ldy, y_dtype == PRQ_BF16);
         if (st != PRQ_OK) return st;
-        cudaError_t e = launch_prefill_pair(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, q, pairs, static_cast<cudaStream_t>(stream));
+        cudaError_t e = launch_prefill_pair(tm_act, w->tm_w_pair, tm_sfa, w->tm_sfw_pair, tm_y, q, pairs, static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     } else {
@@ -708,7 +723,8 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
 
 prq_status prq_linear_fused(const prq_weights* w, prq_act_mode mode, const void* x, int M, int ldx, void* y, int ldy,
                             prq_dtype y_dtype, prq_stream_t stream) {
-    if (!w || M < 0 || M > PRQ_FUSED_MAX_M || mode != PRQ_ACT_IDENTITY || w->n_experts != 1) return PRQ_ERR_INVALID_ARG;
+    if (!w || M < 0 || M > PRQ_FUSED_MAX_M || mode != PRQ_ACT_IDENTITY || w->n_experts != 1 || !w->maps_ready)
+        return PRQ_ERR_INVALID_ARG;
     if (M == 0) return PRQ_OK;
     if (!x || !y || ldx < w->K || ldy < w->N) return PRQ_ERR_INVALID_ARG;
     if (y_dtype != PRQ_F32 && y_dtype != PRQ_BF16) return PRQ_ERR_INVALID_ARG;
@@ -725,11 +741,8 @@ prq_status prq_linear_fused(const prq_weights* w, prq_act_mode mode, const void*
     q.y = y; q.ldy = ldy; q.y_bf16 = y_dtype == PRQ_BF16;
     q.status = di->status_ptr; q.trace = trace_ptr(); q.dbg = env_int("PRQ_DBG", 0);
     q.splits = decode_splits(w, M, di);
-    CUtensorMap tm_w;
-    st = make_code_map(&tm_w, w->d_codes, (static_cast<size_t>(w->K) + w->k_tail) / 2, w->N, 128);
-    if (st != PRQ_OK) return st;
     // the kernel takes no activation tensor map in this mode; the weight map fills the parameter
-    cudaError_t e = launch_decode(decode_bn(M), tm_w, tm_w, q, (w->N + 127) / 128, static_cast<cudaStream_t>(stream));
+    cudaError_t e = launch_decode(decode_bn(M), w->tm_w_decode, w->tm_w_decode, q, (w->N + 127) / 128, static_cast<cudaStream_t>(stream));
     g_launches.fetch_add(1);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
 }

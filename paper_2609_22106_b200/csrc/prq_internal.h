@@ -1,12 +1,24 @@
 // Internal declarations shared by the translation units of libprq.
 #pragma once
+#include <cstdlib>
 #include <cstddef>
 #include <cstdint>
 #include <vector>
 
+#include <cuda.h>
+
 #include "prq.h"
 
 namespace prq {
+
+// Developer switches (PRQ_DECODE_SPLITS, PRQ_GROUPED_BN, PRQ_TRACE_PTR, ...) are looked at only when the
+// process was started with PRQ_DEV=1; that one variable is read once, so that a normal call makes no
+// getenv at all.
+inline bool dev_knobs_enabled() {
+    static const bool on = [] { const char* v = std::getenv("PRQ_DEV"); return v && v[0] == '1'; }();
+    return on;
+}
+
 
 constexpr int kBlock = 32;        // MXFP4 block length
 constexpr int kStageK = 256;      // reduction elements per pipeline stage (one 128-byte swizzled row)
@@ -64,6 +76,11 @@ struct prq_weights {
     // 128-row groups per tile, the second partly empty) so that those tile widths need no re-alignment.
     uint8_t* d_sf_alt[3] = {nullptr, nullptr, nullptr};
     int w_groups_alt[3] = {0, 0, 0};
+    // tensor maps of the weight side, encoded once (dense layers; a handle is immutable afterwards):
+    // codes with 128-row boxes (decode kernel), codes with half-tile boxes and the scale bytes of the
+    // 224-row tiling (CTA-pair prefill kernel)
+    CUtensorMap tm_w_decode, tm_w_pair, tm_sfw_pair;
+    bool maps_ready = false;
     int32_t* d_perm = nullptr;       // E x K
     float* d_inv_s_perm = nullptr;   // E x K : inv_s[perm[j]] in the new channel order
     size_t d_codes_bytes = 0, d_sf_bytes = 0;

@@ -288,7 +288,7 @@ cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_gro
         const long long tiles = static_cast<long long>(n_atoms) * grid_groups;
         while (parts < 4 && tiles * parts < 8LL * sm_count[dev]) parts *= 2;   // 3 CTAs per SM: keep the last wave short
         if (parts == 4 && tiles * parts < 4LL * sm_count[dev]) parts = 8;
-        if (const char* ev = getenv("PRQ_QUANT_PARTS")) { const int v = atoi(ev); if (v == 1 || v == 2 || v == 4 || v == 8) parts = v; }
+        if (const char* ev = dev_knobs_enabled() ? getenv("PRQ_QUANT_PARTS") : nullptr) { const int v = atoi(ev); if (v == 1 || v == 2 || v == 4 || v == 8) parts = v; }
     }
     cfg.gridDim = dim3(n_atoms, grid_groups, parts);
     cfg.blockDim = dim3(kQuantThreads);

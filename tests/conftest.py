@@ -4,6 +4,9 @@ import sys
 import pytest
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+# some tests force a kernel variant through the library's developer switches; the library reads them only
+# in processes started with this variable (it is looked at once, at the first call)
+os.environ.setdefault("PRQ_DEV", "1")
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
