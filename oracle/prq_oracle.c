@@ -27,7 +27,15 @@
  *     accumulated in FP64 in ascending row order;
  *   - top-k ties break toward the lower channel index; the permutation lists the
  *     unselected channels in ascending order, then the selected ones ascending;
- *   - s_j = max(amax_j, 1e-5)^alpha.
+ *   - s_j = max(amax_j, 1e-5)^alpha;
+ *   - weight-side block-scale search (the "E8M0-W" variant of the ablation study, for which the
+ *     paper gives only the name "local block-scale search"): for every block of Q(W D P) and of
+ *     Q(R) the candidates are the floor-rule exponent e0 and its neighbours e0 - 1 and e0 + 1
+ *     (bytes kept in [0, 254]); the block is quantised with each, the squared error is summed in
+ *     FP64 in element order, and a neighbour replaces e0 only if its error is strictly smaller
+ *     (e0 - 1 is looked at before e0 + 1).  The column-error ranking of step 4 keeps the floor
+ *     rule, so the permutation does not depend on the option; R is the residual of the searched
+ *     quantisation.  An all-zero block keeps byte 0.
  *
  * Pins (see tests/test_oracle_*.py): hand-worked encodings, a brute-force
  * nearest-value quantiser in exact rational arithmetic, the worked prep example,
@@ -115,6 +123,49 @@ int orc_quantize_rows(const float *v, long rows, long cols, uint8_t *codes, uint
     return 0;
 }
 
+/* Squared error of one block quantised with the scale 2^e, FP64, element order. */
+static double orc_block_error(const float *blk, int e) {
+    double err = 0.0;
+    for (int i = 0; i < ORC_BLOCK; ++i) {
+        uint8_t c = orc_e2m1_code(blk[i], e);
+        double x = ldexp(orc_e2m1_value[c & 7], e);
+        double d = (double)blk[i] - ((c & 8) ? -x : x);
+        err += d * d;
+    }
+    return err;
+}
+
+/* Q with the weight-side block-scale search ("E8M0-W", Ablation study): like orc_quantize_rows,
+ * but every block takes the best of the floor-rule exponent and its two neighbours. */
+int orc_quantize_rows_search(const float *v, long rows, long cols, uint8_t *codes, uint8_t *scales) {
+    if (cols % ORC_BLOCK) return 1;
+    for (long r = 0; r < rows; ++r) {
+        for (long b = 0; b < cols / ORC_BLOCK; ++b) {
+            const float *blk = v + r * cols + b * ORC_BLOCK;
+            int byte0 = (int)orc_block_scale_byte(blk), best = byte0;
+            int zero = 1;
+            for (int i = 0; i < ORC_BLOCK; ++i) zero = zero && blk[i] == 0.0f;
+            if (!zero) {
+                double best_err = orc_block_error(blk, byte0 - 127);
+                const int cand[2] = {byte0 - 1, byte0 + 1};
+                for (int c = 0; c < 2; ++c) {
+                    if (cand[c] < 0 || cand[c] > 254) continue;
+                    double err = orc_block_error(blk, cand[c] - 127);
+                    if (err < best_err) { best_err = err; best = cand[c]; }
+                }
+            }
+            scales[r * (cols / ORC_BLOCK) + b] = (uint8_t)best;
+            int e = best - 127;
+            for (int i = 0; i < ORC_BLOCK; i += 2) {
+                uint8_t lo = orc_e2m1_code(blk[i], e);
+                uint8_t hi = orc_e2m1_code(blk[i + 1], e);
+                codes[(r * cols + b * ORC_BLOCK + i) / 2] = (uint8_t)(lo | (hi << 4));
+            }
+        }
+    }
+    return 0;
+}
+
 static double orc_dequant_one(const uint8_t *codes, const uint8_t *scales, long cols, long r, long j) {
     uint8_t byte = codes[(r * cols + j) / 2];
     uint8_t c = (j & 1) ? (uint8_t)(byte >> 4) : (uint8_t)(byte & 0xF);
@@ -184,9 +235,9 @@ static int orc_rank_cmp(const void *pa, const void *pb) {
  *   export [Qw | Q(R)]                                (step 11, right factor of Eq. (3))
  * Outputs: s, inv_s (K), col_err (K), perm (K, new -> old), wcodes N x (K+k)/2,
  * wscales N x (K+k)/32, R (N x k fp32, may be NULL). */
-int orc_prepare(const uint16_t *W_bf16, long N, long K, const float *amax, double alpha, long k,
-                float *s, float *inv_s, double *col_err, int32_t *perm,
-                uint8_t *wcodes, uint8_t *wscales, float *R_out) {
+int orc_prepare_ex(const uint16_t *W_bf16, long N, long K, const float *amax, double alpha, long k,
+                   int scale_search, float *s, float *inv_s, double *col_err, int32_t *perm,
+                   uint8_t *wcodes, uint8_t *wscales, float *R_out) {
     if (K % ORC_BLOCK || k % ORC_BLOCK || k < 0 || k > K) return 1;
     long Ka = K + k;
     orc_scales_from_amax(amax, K, alpha, s, inv_s);
@@ -225,7 +276,8 @@ int orc_prepare(const uint16_t *W_bf16, long N, long K, const float *amax, doubl
         for (long j = 0; j < K; ++j) Wt[n * K + j] = W0[n * K + perm[j]];
     uint8_t *c1 = (uint8_t *)malloc((size_t)N * K / 2);
     uint8_t *s1 = (uint8_t *)malloc((size_t)N * K / ORC_BLOCK);
-    orc_quantize_rows(Wt, N, K, c1, s1);
+    if (scale_search) orc_quantize_rows_search(Wt, N, K, c1, s1);
+    else orc_quantize_rows(Wt, N, K, c1, s1);
 
     float *R = (float *)malloc(sizeof(float) * (size_t)(N * (k ? k : 1)));
     for (long n = 0; n < N; ++n)
@@ -237,7 +289,10 @@ int orc_prepare(const uint16_t *W_bf16, long N, long K, const float *amax, doubl
         }
     uint8_t *cr = (uint8_t *)malloc((size_t)(N * (k ? k : ORC_BLOCK)) / 2);
     uint8_t *sr = (uint8_t *)malloc((size_t)(N * (k ? k : ORC_BLOCK)) / ORC_BLOCK);
-    if (k) orc_quantize_rows(R, N, k, cr, sr);
+    if (k) {
+        if (scale_search) orc_quantize_rows_search(R, N, k, cr, sr);
+        else orc_quantize_rows(R, N, k, cr, sr);
+    }
 
     for (long n = 0; n < N; ++n) {
         memcpy(wcodes + n * (Ka / 2), c1 + n * (K / 2), (size_t)K / 2);
@@ -251,6 +306,12 @@ int orc_prepare(const uint16_t *W_bf16, long N, long K, const float *amax, doubl
 
     free(W0); free(c0); free(s0); free(rank); free(selected); free(Wt); free(c1); free(s1); free(R); free(cr); free(sr);
     return 0;
+}
+
+int orc_prepare(const uint16_t *W_bf16, long N, long K, const float *amax, double alpha, long k,
+                float *s, float *inv_s, double *col_err, int32_t *perm,
+                uint8_t *wcodes, uint8_t *wscales, float *R_out) {
+    return orc_prepare_ex(W_bf16, N, K, amax, alpha, k, 0, s, inv_s, col_err, perm, wcodes, wscales, R_out);
 }
 
 /* Eq. (1), activation side: Zt = Z D^-1 P, i.e. xt[t,j'] = fl32(x[t,perm[j']] * inv_s[perm[j']]);

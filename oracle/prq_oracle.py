@@ -94,9 +94,21 @@ def scales_from_amax(amax, alpha: float):
     return s, inv_s
 
 
-def prepare(W_bf16, amax, alpha: float, k: int):
-    """Algorithm 1 steps 3-7, 11 for one alpha.  Returns a dict with s, inv_s, col_err,
-    perm (new -> old), topk (= perm[K-k:]), wcodes, wscales, R."""
+def quantize_rows_search(v):
+    """Q with the weight-side block-scale search (E8M0-W, Ablation study): best of the floor-rule
+    exponent and its two neighbours per block."""
+    v = _c(v, np.float32)
+    rows, cols = v.shape
+    codes = np.empty((rows, cols // 2), np.uint8)
+    scales = np.empty((rows, cols // BLOCK), np.uint8)
+    if _load().orc_quantize_rows_search(_p(v), ctypes.c_long(rows), ctypes.c_long(cols), _p(codes), _p(scales)):
+        raise ValueError("cols must be a multiple of 32")
+    return codes, scales
+
+
+def prepare(W_bf16, amax, alpha: float, k: int, scale_search: bool = False):
+    """Algorithm 1 steps 3-7, 11 for one alpha (scale_search: the E8M0-W variant).  Returns a dict with
+    s, inv_s, col_err, perm (new -> old), topk (= perm[K-k:]), wcodes, wscales, R."""
     W = _c(W_bf16, np.uint16)
     amax = _c(amax, np.float32)
     N, K = W.shape
@@ -108,8 +120,9 @@ def prepare(W_bf16, amax, alpha: float, k: int):
     wcodes = np.empty((N, Ka // 2), np.uint8)
     wscales = np.empty((N, Ka // BLOCK), np.uint8)
     R = np.empty((N, max(k, 1)), np.float32)
-    rc = _load().orc_prepare(
+    rc = _load().orc_prepare_ex(
         _p(W), ctypes.c_long(N), ctypes.c_long(K), _p(amax), ctypes.c_double(alpha), ctypes.c_long(k),
+        ctypes.c_int(1 if scale_search else 0),
         _p(s), _p(inv_s), _p(col_err), _p(perm), _p(wcodes), _p(wscales), _p(R),
     )
     if rc:
