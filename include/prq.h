@@ -91,6 +91,24 @@ typedef enum {
 prq_status prq_prepare_weights(const uint16_t *W, int n_experts, int N, int K, const float *act_amax,
                                float alpha, int k_tail, prq_weights **out);
 
+/* Options of the offline pipeline.  Set struct_size = sizeof(prq_prep_opts); NULL means all defaults.
+ *   weight_scale_search  0 (default): every weight block takes the floor-rule scale.
+ *                        1: the "E8M0-W" variant of the paper's ablation study (local block-scale search):
+ *                           every block of Q(W D P) and of Q(R) takes, of the floor-rule exponent and its
+ *                           two neighbours, the one with the smallest squared quantisation error (a
+ *                           neighbour only if strictly better).  Channel ranking, permutation and scales s
+ *                           are not affected; R is the residual of the searched quantisation.  The GEMM is
+ *                           untouched. */
+typedef struct prq_prep_opts {
+    size_t struct_size;
+    int weight_scale_search;
+} prq_prep_opts;
+
+/* prq_prepare_weights with options (opts may be NULL).  Errors as prq_prepare_weights, plus INVALID_ARG for a
+ * struct_size smaller than this header's. */
+prq_status prq_prepare_weights_opts(const uint16_t *W, int n_experts, int N, int K, const float *act_amax,
+                                    float alpha, int k_tail, const prq_prep_opts *opts, prq_weights **out);
+
 /* The same per-alpha pipeline as prq_prepare_weights, host buffers in and out, no device involved
  * (offline tooling, export, checks on machines without a GPU).  One layer.
  *   codes   host out, N x (K+k)/2    scales  host out, N x (K+k)/32    perm  host out, K int32
@@ -98,6 +116,11 @@ prq_status prq_prepare_weights(const uint16_t *W, int n_experts, int N, int K, c
 prq_status prq_prepare_weights_host(const uint16_t *W, int N, int K, const float *act_amax, float alpha,
                                     int k_tail, uint8_t *codes, uint8_t *scales, int32_t *perm, float *s,
                                     float *inv_s, double *col_err);
+
+/* prq_prepare_weights_host with options (opts may be NULL). */
+prq_status prq_prepare_weights_host_opts(const uint16_t *W, int N, int K, const float *act_amax, float alpha,
+                                         int k_tail, const prq_prep_opts *opts, uint8_t *codes, uint8_t *scales,
+                                         int32_t *perm, float *s, float *inv_s, double *col_err);
 
 /* Algorithm 1 steps 1-10: derive amax from the calibration rows, run the per-alpha pipeline for
  * every candidate, evaluate Eq. (3) on the calibration rows with the GPU kernels and keep the

@@ -22,7 +22,7 @@ FIELD_CODES, FIELD_SCALES, FIELD_PERM, FIELD_TOPK, FIELD_S, FIELD_INV_S, FIELD_C
 BUF_CODES, BUF_SCALES_ROW, BUF_SCALES_SF = range(3)
 
 EXPORTS = [
-    "prq_prepare_weights", "prq_prepare_weights_host", "prq_prepare_weights_search", "prq_weights_free",
+    "prq_prepare_weights", "prq_prepare_weights_opts", "prq_prepare_weights_host", "prq_prepare_weights_host_opts", "prq_prepare_weights_search", "prq_weights_free",
     "prq_weights_clone", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
     "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
@@ -48,6 +48,8 @@ def lib():
         vp, ci, cf, cs = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
         L.prq_prepare_weights.argtypes = [vp, ci, ci, ci, vp, cf, ci, ctypes.POINTER(vp)]
         L.prq_prepare_weights_host.argtypes = [vp, ci, ci, vp, cf, ci, vp, vp, vp, vp, vp, vp]
+        L.prq_prepare_weights_opts.argtypes = [vp, ci, ci, ci, vp, cf, ci, vp, ctypes.POINTER(vp)]
+        L.prq_prepare_weights_host_opts.argtypes = [vp, ci, ci, vp, cf, ci, vp, vp, vp, vp, vp, vp, vp]
         L.prq_prepare_weights_search.argtypes = [vp, ci, ci, vp, ci, vp, ci, ci, ctypes.POINTER(vp),
                                                  ctypes.POINTER(cf), vp]
         L.prq_weights_clone.argtypes = [vp, ctypes.POINTER(vp)]
@@ -148,8 +150,18 @@ class Weights:
             pass
 
 
-def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_tail: int) -> Weights:
-    """W_bf16: uint16 (N, K) or (E, N, K); act_amax: float32 (K,) or (E, K)."""
+class PrepOpts(ctypes.Structure):
+    _fields_ = [("struct_size", ctypes.c_size_t), ("weight_scale_search", ctypes.c_int)]
+
+
+def _opts(scale_search: bool):
+    return PrepOpts(ctypes.sizeof(PrepOpts), 1 if scale_search else 0)
+
+
+def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_tail: int,
+                    scale_search: bool = False) -> Weights:
+    """W_bf16: uint16 (N, K) or (E, N, K); act_amax: float32 (K,) or (E, K).  scale_search: the E8M0-W
+    variant (weight-side block-scale search)."""
     W = np.ascontiguousarray(W_bf16, np.uint16)
     amax = np.ascontiguousarray(act_amax, np.float32)
     if W.ndim == 2:
@@ -157,12 +169,15 @@ def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_ta
         amax = amax[None]
     E, N, K = W.shape
     h = ctypes.c_void_p()
-    _check(lib().prq_prepare_weights(_np_ptr(W), E, N, K, _np_ptr(amax), alpha, k_tail, ctypes.byref(h)),
-           "prq_prepare_weights")
+    o = _opts(scale_search)
+    _check(lib().prq_prepare_weights_opts(_np_ptr(W), E, N, K, _np_ptr(amax), alpha, k_tail,
+                                          ctypes.cast(ctypes.pointer(o), ctypes.c_void_p), ctypes.byref(h)),
+           "prq_prepare_weights_opts")
     return Weights(h)
 
 
-def prepare_weights_host(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_tail: int) -> dict:
+def prepare_weights_host(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_tail: int,
+                         scale_search: bool = False) -> dict:
     W = np.ascontiguousarray(W_bf16, np.uint16)
     amax = np.ascontiguousarray(act_amax, np.float32)
     N, K = W.shape
@@ -170,9 +185,12 @@ def prepare_weights_host(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float,
     out = dict(codes=np.empty((N, Ka // 2), np.uint8), scales=np.empty((N, Ka // 32), np.uint8),
                perm=np.empty(K, np.int32), s=np.empty(K, np.float32), inv_s=np.empty(K, np.float32),
                col_err=np.empty(K, np.float64))
-    _check(lib().prq_prepare_weights_host(_np_ptr(W), N, K, _np_ptr(amax), alpha, k_tail, _np_ptr(out["codes"]),
-                                          _np_ptr(out["scales"]), _np_ptr(out["perm"]), _np_ptr(out["s"]),
-                                          _np_ptr(out["inv_s"]), _np_ptr(out["col_err"])), "prq_prepare_weights_host")
+    o = _opts(scale_search)
+    _check(lib().prq_prepare_weights_host_opts(_np_ptr(W), N, K, _np_ptr(amax), alpha, k_tail,
+                                               ctypes.cast(ctypes.pointer(o), ctypes.c_void_p), _np_ptr(out["codes"]),
+                                               _np_ptr(out["scales"]), _np_ptr(out["perm"]), _np_ptr(out["s"]),
+                                               _np_ptr(out["inv_s"]), _np_ptr(out["col_err"])),
+           "prq_prepare_weights_host_opts")
     return out
 
 

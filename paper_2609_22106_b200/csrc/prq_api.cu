@@ -284,6 +284,13 @@ void prq_weights_free(prq_weights* w) {
 
 prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, const float* act_amax, float alpha,
                                int k_tail, prq_weights** out) {
+    return prq_prepare_weights_opts(W, n_experts, N, K, act_amax, alpha, k_tail, nullptr, out);
+}
+
+prq_status prq_prepare_weights_opts(const uint16_t* W, int n_experts, int N, int K, const float* act_amax, float alpha,
+                                    int k_tail, const prq_prep_opts* opts, prq_weights** out) {
+    if (opts && opts->struct_size < sizeof(prq_prep_opts)) return PRQ_ERR_INVALID_ARG;
+    const bool scale_search = opts && opts->weight_scale_search != 0;
     if (!W || !act_amax || !out) return PRQ_ERR_INVALID_ARG;
     if (n_experts < 1 || n_experts > kMaxExperts || N < 1 || K < kBlock) return PRQ_ERR_INVALID_ARG;
     if (K % kBlock || k_tail % kBlock || k_tail < 0 || k_tail > K) return PRQ_ERR_INVALID_ARG;
@@ -322,7 +329,7 @@ prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, c
         }
         PrepResult r;
         for (size_t e = 0; e < E; ++e) {
-            st = prepare_layer(W + e * N * K, N, K, act_amax + e * K, alpha, k_tail, r);
+            st = prepare_layer(W + e * N * K, N, K, act_amax + e * K, alpha, k_tail, r, scale_search);
             if (st != PRQ_OK) { delete w; return st; }
             std::memcpy(&w->h_codes[e * N * Ka / 2], r.codes.data(), r.codes.size());
             std::memcpy(&w->h_scales[e * N * Ka / kBlock], r.scales.data(), r.scales.size());
@@ -460,12 +467,21 @@ prq_status prq_prepare_weights_search(const uint16_t* W, int N, int K, const uin
 prq_status prq_prepare_weights_host(const uint16_t* W, int N, int K, const float* act_amax, float alpha, int k_tail,
                                     uint8_t* codes, uint8_t* scales, int32_t* perm, float* s_out, float* inv_s_out,
                                     double* col_err) {
+    return prq_prepare_weights_host_opts(W, N, K, act_amax, alpha, k_tail, nullptr, codes, scales, perm, s_out,
+                                         inv_s_out, col_err);
+}
+
+prq_status prq_prepare_weights_host_opts(const uint16_t* W, int N, int K, const float* act_amax, float alpha,
+                                         int k_tail, const prq_prep_opts* opts, uint8_t* codes, uint8_t* scales,
+                                         int32_t* perm, float* s_out, float* inv_s_out, double* col_err) {
+    if (opts && opts->struct_size < sizeof(prq_prep_opts)) return PRQ_ERR_INVALID_ARG;
+    const bool scale_search = opts && opts->weight_scale_search != 0;
     if (!W || !act_amax || !codes || !scales || !perm) return PRQ_ERR_INVALID_ARG;
     if (N < 1 || K < kBlock || K % kBlock || k_tail % kBlock || k_tail < 0 || k_tail > K) return PRQ_ERR_INVALID_ARG;
     if (!std::isfinite(alpha)) return PRQ_ERR_INVALID_ARG;
     PrepResult r;
     try {
-        prq_status st = prepare_layer(W, N, K, act_amax, alpha, k_tail, r);
+        prq_status st = prepare_layer(W, N, K, act_amax, alpha, k_tail, r, scale_search);
         if (st != PRQ_OK) return st;
     } catch (const std::bad_alloc&) {
         return PRQ_ERR_OOM;

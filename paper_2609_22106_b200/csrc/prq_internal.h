@@ -53,8 +53,10 @@ struct PrepResult {
 
 // Algorithm 1 steps 3-7 and 11 for one layer and one alpha, on the host.
 // Returns PRQ_ERR_NONFINITE if W or amax hold a NaN or an infinity.
+// scale_search: every weight block (main part and residual) takes the best of the floor-rule scale and its
+// two neighbours (the "E8M0-W" variant of the ablation study); ranking and permutation are unaffected.
 prq_status prepare_layer(const uint16_t* W, int N, int K, const float* amax, float alpha, int k_tail,
-                         PrepResult& out);
+                         PrepResult& out, bool scale_search = false);
 
 }  // namespace prq
 

@@ -84,6 +84,35 @@ inline uint8_t quantize_block(const float* v, uint8_t* codes) {
     return byte;
 }
 
+// The same with the weight-side block-scale search (the "E8M0-W" variant of the ablation study): the
+// block is quantised with the floor-rule byte and with its two neighbours; a neighbour wins only with a
+// strictly smaller sum of squared errors (FP64, element order; byte - 1 is looked at before byte + 1).
+inline double block_error(const float* v, uint8_t byte, uint8_t* codes) {
+    double err = 0.0;
+    for (int i = 0; i < kBlock; ++i) {
+        codes[i] = e2m1_code(v[i], byte);
+        const double d = static_cast<double>(v[i]) - static_cast<double>(e2m1_value(codes[i], byte));
+        err += d * d;
+    }
+    return err;
+}
+inline uint8_t quantize_block_search(const float* v, uint8_t* codes) {
+    uint8_t tmp[kBlock];
+    const uint8_t byte0 = quantize_block(v, codes);
+    bool zero = true;
+    for (int i = 0; i < kBlock; ++i) zero = zero && v[i] == 0.f;
+    if (zero) return byte0;
+    double best_err = block_error(v, byte0, tmp);
+    uint8_t best = byte0;
+    const int cand[2] = {static_cast<int>(byte0) - 1, static_cast<int>(byte0) + 1};
+    for (int c = 0; c < 2; ++c) {
+        if (cand[c] < 0 || cand[c] > 254) continue;
+        const double err = block_error(v, static_cast<uint8_t>(cand[c]), tmp);
+        if (err < best_err) { best_err = err; best = static_cast<uint8_t>(cand[c]); std::memcpy(codes, tmp, kBlock); }
+    }
+    return best;
+}
+
 template <class F>
 void parallel_for(long n, F&& body) {
     unsigned hw = std::thread::hardware_concurrency();
@@ -113,7 +142,7 @@ double scale_power(double a, float alpha) {
 }  // namespace
 
 prq_status prepare_layer(const uint16_t* W, int N, int K, const float* amax, float alpha, int k_tail,
-                         PrepResult& out) {
+                         PrepResult& out, bool scale_search) {
     const long Ka = static_cast<long>(K) + k_tail;
     const int nblk = K / kBlock;
     out.s.resize(K);
@@ -185,13 +214,13 @@ prq_status prepare_layer(const uint16_t* W, int N, int K, const float* amax, flo
             uint8_t* srow = &out.scales[n * (Ka / kBlock)];
             for (int b = 0; b < nblk; ++b) {
                 for (int i = 0; i < kBlock; ++i) v[i] = W0[n * K + out.perm[b * kBlock + i]];
-                uint8_t byte = quantize_block(v, codes);
+                uint8_t byte = scale_search ? quantize_block_search(v, codes) : quantize_block(v, codes);
                 srow[b] = byte;
                 for (int i = 0; i < kBlock; i += 2)
                     crow[(b * kBlock + i) / 2] = static_cast<uint8_t>(codes[i] | (codes[i + 1] << 4));
                 if (b >= tail_blk0) {
                     for (int i = 0; i < kBlock; ++i) r[i] = v[i] - e2m1_value(codes[i], byte);  // exact
-                    uint8_t rbyte = quantize_block(r, codes);
+                    uint8_t rbyte = scale_search ? quantize_block_search(r, codes) : quantize_block(r, codes);
                     const int rb = nblk + (b - tail_blk0);
                     srow[rb] = rbyte;
                     for (int i = 0; i < kBlock; i += 2)

@@ -423,3 +423,27 @@ def test_decode_split_k_is_reproducible(prq, oracle, M):
             assert torch.equal(prq.linear_fused(w, x), ref)
     assert prq.last_device_status() == 0
     w.free()
+
+
+def test_linear_with_weight_scale_search(prq, oracle):
+    """Weights prepared with the E8M0-W option: prep fields bit-exact against the oracle's, the product within
+    tolerance of the oracle's (decode and prefill kernels), and the synthetic reconstruction error of the
+    layer output is reported not to grow."""
+    N, K, k = 512, 2048, 128
+    L = synth.layer(1, N, K, 300, T_cal=64, tag=990)
+    amax = oracle.channel_amax(L["zcal"])
+    w = prq.prepare_weights(L["W"], amax, 0.5, k, scale_search=True)
+    o = oracle.prepare(L["W"], amax, float(np.float32(0.5)), k, scale_search=True)
+    assert np.array_equal(w.get(prq.FIELD_PERM), o["perm"])
+    assert np.array_equal(w.get(prq.FIELD_SCALES), o["wscales"])
+    assert np.array_equal(w.get(prq.FIELD_CODES), o["wcodes"])
+    for M in (16, 300):
+        x = to_dev_bf16(L["x"][:M])
+        codes, _, sf = prq.quantize_act(w, x, prq.ACT_SCALE_PERM)
+        y = prq.linear(w, codes, sf, M).cpu().numpy().astype(np.float64)
+        oc, osc = oracle.quantize_act(L["x"][:M], o["perm"], o["inv_s"])
+        ca, sa = oracle.augment_act(oc, osc, k)
+        y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+        assert np.abs(y - y_ref).max() <= prq_ref.tolerance(y_ref)
+    assert prq.last_device_status() == 0
+    w.free()

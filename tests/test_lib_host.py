@@ -71,9 +71,9 @@ def test_argument_validation_without_a_gpu(prq):
     L.prq_weights_free(None)  # no-op
 
 
-def host_vs_oracle(prq, oracle, W, amax, alpha, k):
-    got = prq.prepare_weights_host(W, amax, alpha, k)
-    want = oracle.prepare(W, amax, float(np.float32(alpha)), k)
+def host_vs_oracle(prq, oracle, W, amax, alpha, k, scale_search=False):
+    got = prq.prepare_weights_host(W, amax, alpha, k, scale_search=scale_search)
+    want = oracle.prepare(W, amax, float(np.float32(alpha)), k, scale_search=scale_search)
     assert np.array_equal(got["s"], want["s"])
     assert np.array_equal(got["inv_s"], want["inv_s"])
     assert np.array_equal(got["col_err"], want["col_err"])
@@ -103,6 +103,33 @@ def test_host_prep_bit_exact_heavy_tailed(prq, oracle):
     amax2[5:10] = 1e30
     amax2[10:15] = 1e-30
     host_vs_oracle(prq, oracle, L["W"], amax2, 1.0, 128)
+
+
+def test_host_prep_with_weight_scale_search_bit_exact(prq, oracle):
+    """The E8M0-W option (weight-side block-scale search): the library's prep against the oracle's, bit for
+    bit, and against its own result without the option (same ranking, some scales one step away)."""
+    cfg = synth.tiny_config(0)
+    amax = oracle.channel_amax(cfg["zcal"])
+    host_vs_oracle(prq, oracle, cfg["W"], amax, 0.5, cfg["k"], scale_search=True)
+    L = synth.layer(1, 96, 1024, 4, T_cal=64)
+    amax = oracle.channel_amax(L["zcal"])
+    changed = 0
+    for k in (0, 128):
+        on = host_vs_oracle(prq, oracle, L["W"], amax, 0.5, k, scale_search=True)
+        off = prq.prepare_weights_host(L["W"], amax, 0.5, k)
+        assert np.array_equal(on["perm"], off["perm"]) and np.array_equal(on["col_err"], off["col_err"])
+        # main part only: with the option R is the residual of a different quantisation
+        d = on["scales"][:, : 1024 // 32].astype(int) - off["scales"][:, : 1024 // 32].astype(int)
+        assert np.abs(d).max() <= 1
+        changed += int((d != 0).sum())
+    assert changed > 0
+    # a struct_size that is too small is refused
+    o = prq.PrepOpts(4, 1)
+    out = prq.prepare_weights_host(L["W"], amax, 0.5, 0)
+    rc = prq.lib().prq_prepare_weights_host_opts(
+        L["W"].ctypes.data, 96, 1024, amax.ctypes.data, 0.5, 0, ctypes.cast(ctypes.pointer(o), ctypes.c_void_p),
+        out["codes"].ctypes.data, out["scales"].ctypes.data, out["perm"].ctypes.data, None, None, None)
+    assert rc == 1
 
 
 def test_host_prep_worked_example(prq):
