@@ -646,7 +646,6 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
     p.w_sf = w->d_sf;
     p.y = y; p.ldy = ldy; p.y_bf16 = y_dtype == PRQ_BF16;
     p.status = di->status_ptr;
-    p.splits = 1;
     p.trace = trace_ptr();
     p.dbg = env_int("PRQ_DBG", 0);
 
@@ -786,7 +785,6 @@ prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const voi
     p.expert_offsets = expert_offsets;
     p.y = y; p.ldy = ldy; p.y_bf16 = y_dtype == PRQ_BF16;
     p.status = di->status_ptr;
-    p.splits = 1;
     p.trace = trace_ptr();
     // Default: output features on the MMA M axis, one 128-token group of an expert on the N axis (coalesced
     // stores straight from the accumulator, cheap for experts with few tokens).  PRQ_GROUPED_BN selects the

@@ -15,9 +15,11 @@
 // representation of the tail", Kernel design paragraph); only the tail's scale bytes were duplicated.
 //
 // Operand roles.  "P" is the operand on the MMA M axis (always 128 rows), "Q" the operand on the MMA N
-// axis (BN rows).  Prefill / grouped: P = activation tokens, Q = weight rows.  Decode (M <= 128): P =
-// weight rows, Q = tokens, and the reduction is split over CTAs so that all SMs stream weights; the
-// partial sums meet in a workspace and the last CTA of a tile adds them in a fixed order.
+// axis (BN rows).  Dense and grouped kinds: P = activation tokens, Q = weight rows.  Swapped grouped kind
+// (the default for stacked experts): P = 128 output features of one expert, Q = one 128-token group of
+// that expert, so that an expert with few tokens costs few stores.  (M <= 128 and the large dense shapes
+// have kernels of their own: prq_gemm_decode.cu, prq_gemm_prefill_pair.cu; this one serves the grouped
+// product and, behind a developer switch, dense prefill with one CTA per tile.)
 //
 // Every wait is bounded; on expiry the CTA raises an abort flag, all roles unwind, tensor memory is
 // freed and PRQ_ERR_TIMEOUT is recorded in the device status word.
@@ -33,7 +35,7 @@ namespace {
 
 constexpr int kMainWarps = 2;   // producer + issuer; the epilogue warps follow
 constexpr int kPTileBytes = 128 * 128;
-constexpr int kKindPrefill = 0, kKindDecode = 1, kKindGrouped = 2, kKindGroupedSwap = 3;
+constexpr int kKindPrefill = 0, kKindGrouped = 2, kKindGroupedSwap = 3;
 constexpr int kRowCache = 256;   // experts whose row ranges are cached in shared memory
 
 constexpr int cgcd(int a, int b) { return b == 0 ? a : cgcd(b, a % b); }
@@ -49,7 +51,7 @@ __device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo) { return (s
 
 template <int BN, int KIND>
 struct Cfg {
-    static constexpr bool kSwap = KIND == kKindDecode || KIND == kKindGroupedSwap;
+    static constexpr bool kSwap = KIND == kKindGroupedSwap;
     // epilogue warps: four (one per tensor-memory lane quarter), or eight taking alternate column chunks
     // where the epilogue is what the main loop waits for (short reductions, many outputs)
     static constexpr int kEpiWarps = KIND == kKindGroupedSwap ? 8 : 4;
@@ -67,7 +69,7 @@ struct Cfg {
     static constexpr int kSfpCols = 8;              // 2 atoms x 4 columns
     static constexpr int kSfqCols = 8 * kNgq;       // 2 atoms x 4 columns x groups
     static constexpr int kSfCols = kSfpCols + kSfqCols;
-    static constexpr int kAcc = (KIND != kKindDecode && 2 * kAccStride + kSfCols <= 512) ? 2 : 1;
+    static constexpr int kAcc = 2 * kAccStride + kSfCols <= 512 ? 2 : 1;
     static constexpr int kTmemCols = pow2_at_least(kAcc * kAccStride + kSfCols);
     static constexpr int kSfpCol = kAcc * kAccStride;
     static constexpr int kSfqCol = kSfpCol + kSfpCols;
@@ -85,7 +87,6 @@ struct Unit {
     int s_begin, s_end;          // reduction stages of this unit
     int row0, row_end;           // token rows covered / first row past the valid ones
     int n0;                      // first output feature
-    int tile, split;             // decode bookkeeping
 };
 
 // Where a grouped unit sits: expert, 128-row token tile (counted over all experts), feature tile.
@@ -94,7 +95,6 @@ struct GroupPos { int e, mt, ni; };
 template <int BN, int KIND>
 __device__ __forceinline__ int unit_count(const GemmParams& p, const int* tile_start) {
     if (KIND == kKindPrefill) return ((p.M + 127) / 128) * ((p.N + BN - 1) / BN);
-    if (KIND == kKindDecode) return ((p.N + 127) / 128) * p.splits;
     if (KIND == kKindGroupedSwap) return tile_start[p.n_experts] * ((p.N + 127) / 128);
     return tile_start[p.n_experts] * ((p.N + BN - 1) / BN);
 }
@@ -115,20 +115,6 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
         t.s_begin = 0; t.s_end = S;
         t.row0 = mi * 128; t.row_end = min(p.M, t.row0 + 128);
         t.n0 = ni * BN;
-        t.tile = u; t.split = 0;
-    } else if (KIND == kKindDecode) {
-        const int ni = u / p.splits, sp = u % p.splits;
-        t.p_row = ni * 128;
-        t.q_row = 0;
-        t.sfp = p.w_sf + static_cast<size_t>(ni) * kSfGroupBytes;
-        t.sfp_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
-        t.sfq = p.act_sf;
-        t.sfq_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
-        t.s_begin = static_cast<int>(static_cast<long long>(S) * sp / p.splits);
-        t.s_end = static_cast<int>(static_cast<long long>(S) * (sp + 1) / p.splits);
-        t.row0 = 0; t.row_end = p.M;
-        t.n0 = ni * 128;
-        t.tile = ni; t.split = sp;
     } else if (KIND == kKindGroupedSwap) {
         // weights on the MMA M axis (128 output features), a 128-row group of one expert's tokens on N
         const int e = g.e, mt = g.mt, ni = g.ni;
@@ -141,7 +127,6 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
         t.s_begin = 0; t.s_end = S;
         t.row0 = t.q_row; t.row_end = min(row_start[e + 1], t.q_row + 128);
         t.n0 = ni * 128;
-        t.tile = u; t.split = 0;
     } else {
         const int e = g.e, mt = g.mt, ni = g.ni;
         t.p_row = row_start[e] + (mt - tile_start[e]) * 128;
@@ -153,7 +138,6 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
         t.s_begin = 0; t.s_end = S;
         t.row0 = t.p_row; t.row_end = min(row_start[e + 1], t.p_row + 128);
         t.n0 = ni * BN;
-        t.tile = u; t.split = 0;
     }
     return t;
 }
@@ -202,8 +186,6 @@ struct UnitIter {
     }
 };
 
-__device__ __forceinline__ void epi_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
 template <int BN, int KIND>
 __global__ void __launch_bounds__(Cfg<BN, KIND>::kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
@@ -213,7 +195,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
     __shared__ __align__(8) uint64_t bar_full[C::kStages], bar_empty[C::kStages], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag_s;
-    __shared__ int is_last_s;
     __shared__ int tile_start[(KIND == kKindGrouped || KIND == kKindGroupedSwap) ? kMaxExperts + 1 : 1];
     __shared__ int row_cache[(KIND == kKindGrouped || KIND == kKindGroupedSwap) ? kRowCache + 1 : 1];
     volatile int* abort_flag = &abort_flag_s;
@@ -230,7 +211,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
         for (int i = 0; i < C::kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_acc_full[i]), 1); mbar_init(smem_u32(&bar_acc_empty[i]), C::kEpiWarps); }
         abort_flag_s = 0;
-        is_last_s = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tm_act);
         tma_prefetch_desc(&tm_w);
@@ -480,86 +460,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ 
                     }
                     __syncwarp();   // the tile is read before the next chunk overwrites it
                 }
-            } else {
-                // decode: accumulator row = weight row n, column = token
-                const int n = t.n0 + et;
-                const int n_pad = ((p.N + 127) / 128) * 128;
-                const bool direct = p.splits == 1;
-#pragma unroll 1
-                for (int c = 0; c < BN / 16; ++c) {
-                    uint32_t r[16];
-                    tmem_ld_32x16(acc_t + c * 16, r);
-                    tmem_ld_wait();
-                    if (c * 16 < p.M) {
-                        if (direct) {
-                            if (n < p.N) {
-#pragma unroll
-                                for (int i = 0; i < 16; ++i) {
-                                    const int tok = c * 16 + i;
-                                    if (tok < p.M) {
-                                        if (p.y_bf16)
-                                            reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] =
-                                                __float2bfloat16_rn(__uint_as_float(r[i]));
-                                        else
-                                            reinterpret_cast<float*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = __uint_as_float(r[i]);
-                                    }
-                                }
-                            }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const int tok = c * 16 + i;
-                                if (tok < p.M)
-                                    __stcg(&p.partial[(static_cast<size_t>(t.split) * BN + tok) * n_pad + n], __uint_as_float(r[i]));
-                            }
-                        }
-                    }
-                }
-                if (!direct) {
-                    // Split-K meeting point.  Every CTA of a tile publishes its partial sums, waits
-                    // (bounded) until all `splits` partials of the tile are there, then adds up its own
-                    // share of the tokens in a fixed order.  All CTAs of the launch are co-resident
-                    // (the host keeps the grid within one wave), so the wait cannot starve.
-                    __threadfence();
-                    epi_barrier();
-                    if (et == 0) {
-                        atomicAdd(&p.counters[t.tile], 1);
-                        const long long t0 = clock64();
-                        volatile int* cnt = p.counters + t.tile;
-                        while (*cnt < p.splits) {
-                            if (*abort_flag) break;
-                            if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
-                        }
-                    }
-                    epi_barrier();
-                    if (*abort_flag) { ok = false; break; }
-                    __threadfence();
-                    if (n < p.N) {
-                        for (int tok = t.split; tok < p.M; tok += p.splits) {
-                            const float* src = p.partial + static_cast<size_t>(tok) * n_pad + n;
-                            const size_t sp_stride = static_cast<size_t>(BN) * n_pad;
-                            float sum = 0.f;
-                            for (int sp0 = 0; sp0 < p.splits; sp0 += 8) {
-                                float v[8];
-#pragma unroll
-                                for (int i = 0; i < 8; ++i)
-                                    v[i] = sp0 + i < p.splits ? __ldcg(src + (sp0 + i) * sp_stride) : 0.f;
-#pragma unroll
-                                for (int i = 0; i < 8; ++i) sum += v[i];
-                            }
-                            if (p.y_bf16)
-                                reinterpret_cast<__nv_bfloat16*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = __float2bfloat16_rn(sum);
-                            else
-                                reinterpret_cast<float*>(p.y)[static_cast<size_t>(tok) * p.ldy + n] = sum;
-                        }
-                    }
-                    epi_barrier();
-                    // the last CTA to finish reading leaves the counter at zero for the next launch
-                    if (et == 0) {
-                        const int old = atomicAdd(&p.counters[t.tile], 1);
-                        if (old == 2 * p.splits - 1) p.counters[t.tile] = 0;
-                    }
-                }
             }
             // hand the accumulator back to the MMA issuer
             tc_fence_before_sync();
@@ -617,12 +517,6 @@ cudaError_t launch_gemm(GemmKind kind, int bn, const CUtensorMap& tm_act, const 
 #undef PRQ_CASE
     *unsupported = true;
     return cudaSuccess;
-}
-
-int gemm_smem_bytes(GemmKind kind, int bn) {
-    const int stage = kPTileBytes + bn * 128 + kSfGroupBytes + 2 * kSfGroupBytes;
-    (void)kind;
-    return stage;
 }
 
 }  // namespace prq

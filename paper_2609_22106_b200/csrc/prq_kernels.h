@@ -32,7 +32,6 @@ cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_gro
 // Which GEMM variant to run.
 enum class GemmKind {
     kPrefill,  // tokens on the MMA M axis (128-row tiles), weights on the N axis, persistent CTAs
-    kDecode,   // weights on the MMA M axis, tokens on the N axis, split-K with a workspace reduction
     kGrouped,  // prefill layout with per-expert row ranges
     kGroupedSwap  // per-expert row ranges with the weights on the MMA M axis and a 128-token group on N
 };
@@ -49,9 +48,6 @@ struct GemmParams {
     void* y;
     int ldy;
     int y_bf16;
-    float* partial;          // decode: splits x bn x N_pad fp32 partial sums
-    int* counters;           // decode: one arrival counter per 128-row weight tile
-    int splits;
     int* status;             // device status word
     long long* trace;        // developer trace buffer (nullptr in normal use)
     int dbg;                 // developer switches for timing experiments (0 in normal use)
@@ -63,7 +59,6 @@ struct GemmParams {
 cudaError_t launch_gemm(GemmKind kind, int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w,
                         const GemmParams& p, int grid, cudaStream_t stream, bool* unsupported);
 
-int gemm_smem_bytes(GemmKind kind, int bn);
 
 // Decode kernel (M <= 128): cluster split-K with a distributed-shared-memory reduction.
 struct DecodeParams {
