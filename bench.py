@@ -131,15 +131,18 @@ class GraphTimer:
         are replayed from two CUDA graphs (one whole rotation, one remainder) so that the host-side cost
         of a call (ctypes, tensor-map encoding) cannot starve the GPU inside the timed region."""
         torch = self.torch
-        R = len(fns)
-        g_full = self.capture(fns)
-        g_rem = self.capture(fns[: n % R]) if n % R else None
-        for _ in range(max(1, warm // R)):
+        # a graph holds at least eight calls: replays of a one-kernel graph would put a graph-launch gap
+        # after every short kernel
+        seq = list(fns) * max(1, -(-8 // len(fns)))
+        L = len(seq)
+        g_full = self.capture(seq)
+        g_rem = self.capture(seq[: n % L]) if n % L else None
+        for _ in range(max(1, warm // L)):
             g_full.replay()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        for _ in range(n // R):
+        for _ in range(n // L):
             g_full.replay()
         if g_rem is not None:
             g_rem.replay()
@@ -335,7 +338,9 @@ def main():
         # context workloads: one JSON line each, same peaks; rank 0 only (they are not the headline metric)
         if rank == 0:
             if args.workload == "block":
-                res = [run_block_workload(args, torch, prq, synth, dev, pk, 4096)]
+                # three weight / activation sets per linear, cycled, so that consecutive launches do not find
+                # their operands in L2 (one set of a block's operands is 366 MB, of one linear 15 - 100 MB)
+                res = [run_block_workload(args, torch, prq, synth, dev, pk, 4096, n_layers=3)]
             elif args.workload == "moe":
                 res = [run_moe_workload(args, torch, prq, synth, dev, pk, T) for T in (64, 1024, 8192)]
             else:
