@@ -29,7 +29,7 @@ N_OUT, K_IN, K_TAIL, M_TOK = 2560, 9728, 256, 2048
 FP4_OVER_BF16 = 4.0  # nominal dense tensor ratio (9 vs 2.25 PFLOP/s)
 # DRAM bytes of one prefill GEMM launch at this workload from the ncu capture summarised in
 # profiles/prefill_pair_M2048.txt (dram__bytes_read.sum + dram__bytes_write.sum; the outputs were still in L2).
-NCU_PREFILL_DRAM_BYTES = 24.39e6 + 1.43e6
+NCU_PREFILL_DRAM_BYTES = 24.39e6 + 1.24e6
 
 
 def peaks():
