@@ -156,7 +156,7 @@ def rotation_count(bytes_per_set, lo=2, hi=24, l2_bytes=126e6):
     return int(min(hi, max(lo, np.ceil(2.2 * l2_bytes / bytes_per_set))))
 
 
-# Shapes of one Qwen3-4B-shaped decoder block's linears (BASELINE configs[2]): name -> (N, K, k_tail).
+# Shapes of one Qwen3-4B-shaped decoder block's linears (benchmark configuration 2): name -> (N, K, k_tail).
 BLOCK_LINEARS = {"q": (4096, 2560, 128), "k": (1024, 2560, 128), "v": (1024, 2560, 128), "o": (2560, 4096, 128),
                  "gate": (9728, 2560, 128), "up": (9728, 2560, 128), "down": (2560, 9728, 256)}
 
@@ -302,7 +302,7 @@ def main():
     ap.add_argument("--full", action="store_true", help="also time every (M, k) of the down_proj config")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="down_proj", choices=["down_proj", "block", "moe", "stack"],
-                    help="down_proj = the headline config (default); block / moe / stack = BASELINE configs 2, 3, 4")
+                    help="down_proj = the headline config (default); block / moe / stack = the benchmark configurations 2, 3, 4")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
