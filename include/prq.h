@@ -223,6 +223,24 @@ prq_status prq_linear_static_scratch(const prq_weights *w, const void *codes, co
 prq_status prq_linear_fused(const prq_weights *w, prq_act_mode mode, const void *x, int M, int ldx, void *y,
                             int ldy, prq_dtype y_dtype, prq_stream_t stream);
 
+/* Several dense layers that read the same activation (q / k / v, gate / up), each with its own prepared
+ * weights, served by one launch each of the quantiser and of the GEMM instead of n.  (Not in the paper: it
+ * only saves launches; every layer's result is bit-for-bit the one of its own prq_quantize_act /
+ * prq_linear calls.)  At decode batch sizes a launch costs as much as the work in it.
+ *   n          1 .. PRQ_MULTI_MAX layers, all dense, on one device, with the same K
+ *   ws         host array of n handles
+ * prq_quantize_act_multi: x device, M x K bf16 (row stride ldx); codes[i], scales_sf[i] device out, sized by
+ *   prq_act_bytes for layer i (k_tail may differ between the layers).  No row-major scales.
+ * prq_linear_multi: M <= 128 only (the weight-streaming kernel); the layers must also share k_tail.
+ *   codes[i], scales_sf[i] as written by the quantiser for layer i; y[i] device out, M x N_i, row stride ldy[i].
+ * The pointer arrays are host arrays, read before the call returns.  Errors as for the single-layer calls. */
+#define PRQ_MULTI_MAX 4
+prq_status prq_quantize_act_multi(int n, const prq_weights *const *ws, prq_act_mode mode, const void *x, int M,
+                                  int ldx, void *const *codes, void *const *scales_sf, prq_stream_t stream);
+prq_status prq_linear_multi(int n, const prq_weights *const *ws, const void *const *codes,
+                            const void *const *scales_sf, int M, void *const *y, const int *ldy,
+                            prq_dtype y_dtype, prq_stream_t stream);
+
 /* The same product for stacked experts (MoE): rows [expert_offsets[e], expert_offsets[e+1]) of the
  * activation use expert e's weights.  expert_offsets: device, n_experts + 1 int32, non-decreasing,
  * last = M_total. */

@@ -24,7 +24,8 @@ BUF_CODES, BUF_SCALES_ROW, BUF_SCALES_SF = range(3)
 EXPORTS = [
     "prq_prepare_weights", "prq_prepare_weights_opts", "prq_prepare_weights_host", "prq_prepare_weights_host_opts", "prq_prepare_weights_search", "prq_weights_free",
     "prq_weights_clone", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
-    "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
+    "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_multi", "prq_quantize_act_multi",
+    "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
 ]
 
@@ -65,6 +66,8 @@ def lib():
         L.prq_linear.argtypes = [vp, vp, vp, ci, vp, ci, ci, vp, cs, vp]
         L.prq_linear_static_scratch.argtypes = [vp, vp, vp, ci, vp, ci, ci, vp]
         L.prq_linear_fused.argtypes = [vp, ci, vp, ci, ci, vp, ci, ci, vp]
+        L.prq_quantize_act_multi.argtypes = [ci, vp, ci, vp, ci, ci, vp, vp, vp]
+        L.prq_linear_multi.argtypes = [ci, vp, vp, vp, ci, vp, vp, ci, vp]
         L.prq_linear_grouped.argtypes = [vp, vp, vp, vp, ci, vp, ci, ci, vp]
         L.prq_forward_host_scratch_bytes.argtypes = [vp, ci]
         L.prq_forward_host_scratch_bytes.restype = cs
@@ -269,6 +272,46 @@ def linear_static_scratch(w: Weights, codes, scales_sf, M: int, y_dtype: int = F
 
 
 FUSED_MAX_M = 16
+MULTI_MAX = 4
+
+
+def _ptr_array(ptrs):
+    vals = [p.value if isinstance(p, ctypes.c_void_p) else p for p in ptrs]
+    return (ctypes.c_void_p * len(vals))(*vals)
+
+
+def quantize_act_multi(ws, x, mode: int = ACT_SCALE_PERM, out=None, stream=None):
+    """One quantiser launch for several dense layers that read the same x.  Returns [(codes, scales_sf), ...]."""
+    import torch
+
+    M = x.shape[0]
+    if out is None:
+        out = []
+        for w in ws:
+            out.append((torch.empty(act_bytes(M, w.K, w.k_tail, 1, BUF_CODES), dtype=torch.uint8, device=x.device),
+                        torch.empty(act_bytes(M, w.K, w.k_tail, 1, BUF_SCALES_SF), dtype=torch.uint8, device=x.device)))
+    hs = _ptr_array([w.handle for w in ws])
+    cs = _ptr_array([_dptr(c) for c, _ in out])
+    ss = _ptr_array([_dptr(s) for _, s in out])
+    _check(lib().prq_quantize_act_multi(len(ws), hs, mode, _dptr(x), M, x.stride(0) if M else ws[0].K, cs, ss,
+                                        _stream_ptr(stream)), "prq_quantize_act_multi")
+    return out
+
+
+def linear_multi(ws, acts, M: int, y_dtype: int = F32, out=None, stream=None):
+    """One GEMM launch (M <= 128) for several dense layers over the same tokens; acts = [(codes, scales_sf), ...]."""
+    import torch
+
+    if out is None:
+        out = [torch.empty((M, w.N), dtype=torch.float32 if y_dtype == F32 else torch.bfloat16, device=acts[0][0].device)
+               for w in ws]
+    hs = _ptr_array([w.handle for w in ws])
+    cs = _ptr_array([_dptr(c) for c, _ in acts])
+    ss = _ptr_array([_dptr(s) for _, s in acts])
+    ys = _ptr_array([_dptr(y) for y in out])
+    ld = (ctypes.c_int * len(ws))(*[y.stride(0) if M else w.N for y, w in zip(out, ws)])
+    _check(lib().prq_linear_multi(len(ws), hs, cs, ss, M, ys, ld, y_dtype, _stream_ptr(stream)), "prq_linear_multi")
+    return out
 
 
 def linear_fused(w: Weights, x, mode: int = ACT_IDENTITY, y_dtype: int = F32, out=None, stream=None):

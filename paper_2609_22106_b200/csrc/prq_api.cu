@@ -152,12 +152,11 @@ int decode_bn(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; 
 
 // Cluster size (= number of K-splits) of the decode kernel: the one that puts the most SMs to work in
 // the first wave, given how many clusters of each size the device can hold at once.
-int decode_splits(const prq_weights* w, int M, DeviceInfo* di) {
-    const int n_tiles = (w->N + 127) / 128;
+int decode_splits_for(int n_tiles, int S, int M, DeviceInfo* di) {
     const int bn = decode_bn(M);
     const int bi = bn == 16 ? 0 : bn == 32 ? 1 : bn == 64 ? 2 : 3;
     const int forced = env_int("PRQ_DECODE_SPLITS", 0);
-    const int limit = std::min(8, w->plan.S);
+    const int limit = std::min(8, S);
     if (forced > 0) return std::min(forced, limit);
     if (bn <= 32) {
         // Up to 32 tokens two CTAs share an SM, and a few clusters more than fit at once cost less than
@@ -183,6 +182,10 @@ int decode_splits(const prq_weights* w, int M, DeviceInfo* di) {
         if (score > best_ctas) { best_ctas = score; best = s; }
     }
     return best;
+}
+
+int decode_splits(const prq_weights* w, int M, DeviceInfo* di) {
+    return decode_splits_for((w->N + 127) / 128, w->plan.S, M, di);
 }
 
 int prefill_bn(const prq_weights* w, int M, int num_sms) {
@@ -604,6 +607,34 @@ prq_status prq_quantize_act(const prq_weights* w, prq_act_mode mode, const void*
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
 }
 
+prq_status prq_quantize_act_multi(int n, const prq_weights* const* ws, prq_act_mode mode, const void* x, int M, int ldx,
+                                  void* const* codes, void* const* scales_sf, prq_stream_t stream) {
+    if (n < 1 || n > PRQ_MULTI_MAX || !ws || !codes || !scales_sf || M < 0) return PRQ_ERR_INVALID_ARG;
+    if (mode != PRQ_ACT_IDENTITY && mode != PRQ_ACT_SCALE_PERM) return PRQ_ERR_INVALID_ARG;
+    for (int i = 0; i < n; ++i) {
+        if (!ws[i] || ws[i]->n_experts != 1 || ws[i]->K != ws[0]->K || ws[i]->device != ws[0]->device) return PRQ_ERR_INVALID_ARG;
+        if (M > 0 && (!codes[i] || !scales_sf[i])) return PRQ_ERR_INVALID_ARG;
+    }
+    if (M == 0) return PRQ_OK;
+    if (!x || ldx < ws[0]->K) return PRQ_ERR_INVALID_ARG;
+    if (!aligned16(x) || ldx % 8) return PRQ_ERR_ALIGNMENT;
+    for (int i = 0; i < n; ++i)
+        if (!aligned16(codes[i]) || !aligned16(scales_sf[i])) return PRQ_ERR_ALIGNMENT;
+    QuantBatch b = {};
+    b.x = static_cast<const uint16_t*>(x);
+    b.M = M; b.ldx = ldx; b.K = ws[0]->K;
+    b.n_experts = 1;
+    b.act_groups = dense_groups(M);
+    b.n_lin = n;
+    b.groups_per_lin = b.act_groups;
+    for (int i = 0; i < n; ++i)
+        b.lay[i] = QuantLayer{ws[i]->d_perm, ws[i]->d_inv_s_perm, static_cast<uint8_t*>(codes[i]), nullptr,
+                              static_cast<uint8_t*>(scales_sf[i]), ws[i]->k_tail};
+    cudaError_t e = launch_quant_act_batch(b, mode == PRQ_ACT_SCALE_PERM, static_cast<cudaStream_t>(stream));
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
 size_t prq_linear_workspace_bytes(const prq_weights* w, int M) {
     if (!w || M < 0) return 0;
     if (M > 128) {
@@ -732,6 +763,46 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
     bool unsupported = false;
     cudaError_t e = launch_gemm(kind, bn, tm_act, tm_w, p, grid, static_cast<cudaStream_t>(stream), &unsupported);
     if (unsupported) return PRQ_ERR_INVALID_ARG;
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
+prq_status prq_linear_multi(int n, const prq_weights* const* ws, const void* const* codes, const void* const* scales_sf,
+                            int M, void* const* y, const int* ldy, prq_dtype y_dtype, prq_stream_t stream) {
+    if (n < 1 || n > PRQ_MULTI_MAX || !ws || !codes || !scales_sf || !y || !ldy) return PRQ_ERR_INVALID_ARG;
+    if (M < 0 || M > 128) return PRQ_ERR_INVALID_ARG;
+    for (int i = 0; i < n; ++i) {
+        if (!ws[i]) return PRQ_ERR_INVALID_ARG;
+        if (M == 0) continue;
+        prq_status st = check_linear_common(ws[i], codes[i], scales_sf[i], y[i], ldy[i], y_dtype);
+        if (st != PRQ_OK) return st;
+        if (ws[i]->n_experts != 1 || !ws[i]->maps_ready) return PRQ_ERR_INVALID_ARG;
+        // one stage plan and one cluster size for the whole launch
+        if (ws[i]->K != ws[0]->K || ws[i]->k_tail != ws[0]->k_tail || ws[i]->device != ws[0]->device) return PRQ_ERR_INVALID_ARG;
+    }
+    if (M == 0) return PRQ_OK;
+    DeviceInfo* di;
+    prq_status st = device_info(ws[0]->device, &di);
+    if (st != PRQ_OK) return st;
+    const int bn = decode_bn(M);
+    DecodeMaps maps;
+    std::memset(&maps, 0, sizeof(maps));
+    DecodeBatch b = {};
+    b.status = di->status_ptr; b.trace = trace_ptr(); b.dbg = env_int("PRQ_DBG", 0);
+    b.M = M; b.K = ws[0]->K; b.k_tail = ws[0]->k_tail;
+    b.y_bf16 = y_dtype == PRQ_BF16;
+    b.n_lin = n;
+    int tiles = 0;
+    for (int i = 0; i < n; ++i) {
+        tiles += (ws[i]->N + 127) / 128;
+        st = make_code_map(&maps.act[i], codes[i], ws[i]->K / 2, M, bn);
+        if (st != PRQ_OK) return st;
+        maps.w[i] = ws[i]->tm_w_decode;
+        b.lay[i] = DecodeLayer{static_cast<const uint8_t*>(scales_sf[i]), ws[i]->d_sf, y[i], ws[i]->N, ws[i]->w_groups,
+                               ldy[i], tiles};
+    }
+    b.splits = decode_splits_for(tiles, ws[0]->plan.S, M, di);
+    cudaError_t e = launch_decode_batch(bn, maps, b, static_cast<cudaStream_t>(stream));
     g_launches.fetch_add(1);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
 }

@@ -31,6 +31,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <cstring>
+
 #include "prq_kernels.h"
 #include "prq_ptx.cuh"
 #include "prq_quant_block.cuh"
@@ -107,11 +109,25 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
     tc_commit(empty_bar0 + slot * 8);
 }
 
-template <int BN, bool kFused>
+template <int BN, bool kFused, bool kBatch>
 __global__ void __launch_bounds__(DCfg<BN>::kThreads, DCfg<BN>::kCtasPerSm)
-decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
-              const DecodeParams p) {
+decode_kernel(const __grid_constant__ DecodeMaps maps, const DecodeBatch b) {
     using C = DCfg<BN>;
+    // which of the batched layers this cluster works for (one launch may run several layers over the same
+    // tokens, each with its own weights, activation codes and output)
+    const int tile_all = static_cast<int>(blockIdx.x) / b.splits;
+    int lin = 0;   // (kBatch = false: a single layer, nothing to look up)
+    if (kBatch)
+        while (lin + 1 < b.n_lin && tile_all >= b.lay[lin].tile_end) ++lin;
+    DecodeParams p;
+    p.M = b.M; p.K = b.K; p.k_tail = b.k_tail; p.x = b.x; p.ldx = b.ldx; p.y_bf16 = b.y_bf16; p.splits = b.splits;
+    p.status = b.status; p.trace = b.trace; p.dbg = b.dbg;
+    {
+        const DecodeLayer& l = b.lay[lin];
+        p.N = l.N; p.w_groups = l.w_groups; p.act_sf = l.act_sf; p.w_sf = l.w_sf; p.y = l.y; p.ldy = l.ldy;
+    }
+    const CUtensorMap* const tm_act = &maps.act[lin];
+    const CUtensorMap* const tm_w = &maps.w[lin];
     extern __shared__ uint8_t smem_raw[];
     constexpr int kStages = C::kStages;
     __shared__ __align__(8) uint64_t bar_full[kStages], bar_empty[kStages], bar_acc_full;
@@ -126,8 +142,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     const StagePlan plan(p.K, p.k_tail);
     const int S = plan.S, S1 = plan.S1;
     const int splits = p.splits;
-    const int tile = blockIdx.x / splits;
-    const int split = blockIdx.x - tile * splits;   // = rank in the cluster
+    const int tile = tile_all - (lin ? b.lay[lin - 1].tile_end : 0);   // 128-row weight tile of this layer
+    const int split = static_cast<int>(blockIdx.x) - tile_all * splits;   // = rank in the cluster
     const int s_begin = static_cast<int>(static_cast<long long>(S) * split / splits);
     const int s_end = static_cast<int>(static_cast<long long>(S) * (split + 1) / splits);
     const int n0 = tile * 128;
@@ -148,8 +164,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
         mbar_init(smem_u32(&bar_recv), 1);
         abort_flag_s = 0;
         fence_mbar_init();
-        tma_prefetch_desc(&tm_act);
-        tma_prefetch_desc(&tm_w);
+        tma_prefetch_desc(tm_act);
+        tma_prefetch_desc(tm_w);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&tmem_slot), C::kTmemCols);
@@ -196,7 +212,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
                 mbar_arrive_expect_tx(full, kFused ? kPTile + kSf : C::kStageBytes);
                 const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
                 const uint32_t sb = smem_base + i * C::kStageBytes;
-                tma_load_2d(sb, &tm_w, xw, n0, full);
+                tma_load_2d(sb, tm_w, xw, n0, full);
                 bulk_load(sb + kPTile + C::kQTile, sfp + s * sfp_stride, kSf, full);
             }
         }
@@ -212,11 +228,11 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
                 const uint32_t sb = smem_base + st * C::kStageBytes;
                 if (it >= pre) {
                     mbar_arrive_expect_tx(full, kFused ? kPTile + kSf : C::kStageBytes);
-                    tma_load_2d(sb, &tm_w, xw, n0, full);
+                    tma_load_2d(sb, tm_w, xw, n0, full);
                     bulk_load(sb + kPTile + C::kQTile, sfp + s * sfp_stride, kSf, full);
                 }
                 if (!kFused) {
-                    tma_load_2d(sb + kPTile, &tm_act, xa, 0, full);
+                    tma_load_2d(sb + kPTile, tm_act, xa, 0, full);
                     bulk_load(sb + kPTile + C::kQTile + kSf, p.act_sf + s * sfq_stride, kSf, full);
                 }
             }
@@ -449,13 +465,14 @@ decode_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant_
     if (threadIdx.x == 0 && abort_flag_s) atomicExch(p.status, static_cast<int>(PRQ_ERR_TIMEOUT));
 }
 
-template <int BN, bool kFused>
-cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const DecodeParams& p, int n_tiles,
-                       cudaStream_t stream) {
+template <int BN, bool kFused, bool kBatch>
+cudaError_t launch_one(const DecodeMaps& maps, const DecodeBatch& b, cudaStream_t stream) {
+    const DecodeBatch& p = b;
+    const int n_tiles = b.lay[b.n_lin - 1].tile_end;
     using C = DCfg<BN>;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(decode_kernel<BN, kFused>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel<BN, kFused, kBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -473,13 +490,13 @@ cudaError_t launch_one(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, decode_kernel<BN, kFused>, tm_act, tm_w, p);
+    return cudaLaunchKernelEx(&cfg, decode_kernel<BN, kFused, kBatch>, maps, b);
 }
 
 template <int BN>
 int max_clusters(int splits) {
     using C = DCfg<BN>;
-    cudaFuncSetAttribute(decode_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    cudaFuncSetAttribute(decode_kernel<BN, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(splits);
     cfg.blockDim = dim3(C::kThreads);
@@ -492,22 +509,44 @@ int max_clusters(int splits) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<BN, false>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
+    if (cudaOccupancyMaxActiveClusters(&n, decode_kernel<BN, false, false>, &cfg) != cudaSuccess) { cudaGetLastError(); return 0; }
     return n;
 }
 
 }  // namespace
 
+cudaError_t launch_decode_batch(int bn, const DecodeMaps& maps, const DecodeBatch& b, cudaStream_t stream) {
+    if (b.n_lin < 1 || b.n_lin > kMaxBatch) return cudaErrorInvalidValue;
+    if (b.x != nullptr)   // fused activation quantiser: one layer, the 16-token tile only
+        return (bn == 16 && b.n_lin == 1) ? launch_one<16, true, false>(maps, b, stream) : cudaErrorInvalidValue;
+    if (b.n_lin > 1) {
+        switch (bn) {
+            case 16: return launch_one<16, false, true>(maps, b, stream);
+            case 32: return launch_one<32, false, true>(maps, b, stream);
+            case 64: return launch_one<64, false, true>(maps, b, stream);
+            default: return launch_one<128, false, true>(maps, b, stream);
+        }
+    }
+    switch (bn) {
+        case 16: return launch_one<16, false, false>(maps, b, stream);
+        case 32: return launch_one<32, false, false>(maps, b, stream);
+        case 64: return launch_one<64, false, false>(maps, b, stream);
+        default: return launch_one<128, false, false>(maps, b, stream);
+    }
+}
+
 cudaError_t launch_decode(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const DecodeParams& p,
                           int n_tiles, cudaStream_t stream) {
-    if (p.x != nullptr)   // fused activation quantiser: the 16-token tile only
-        return bn == 16 ? launch_one<16, true>(tm_act, tm_w, p, n_tiles, stream) : cudaErrorInvalidValue;
-    switch (bn) {
-        case 16: return launch_one<16, false>(tm_act, tm_w, p, n_tiles, stream);
-        case 32: return launch_one<32, false>(tm_act, tm_w, p, n_tiles, stream);
-        case 64: return launch_one<64, false>(tm_act, tm_w, p, n_tiles, stream);
-        default: return launch_one<128, false>(tm_act, tm_w, p, n_tiles, stream);
-    }
+    DecodeMaps maps;
+    std::memset(&maps, 0, sizeof(maps));
+    maps.act[0] = tm_act; maps.w[0] = tm_w;
+    DecodeBatch b = {};
+    b.x = p.x; b.status = p.status; b.trace = p.trace;
+    b.M = p.M; b.K = p.K; b.k_tail = p.k_tail; b.ldx = p.ldx;
+    b.y_bf16 = p.y_bf16; b.splits = p.splits; b.dbg = p.dbg;
+    b.n_lin = 1;
+    b.lay[0] = DecodeLayer{p.act_sf, p.w_sf, p.y, p.N, p.w_groups, p.ldy, n_tiles};
+    return launch_decode_batch(bn, maps, b, stream);
 }
 
 int decode_max_active_clusters(int bn, int splits) {

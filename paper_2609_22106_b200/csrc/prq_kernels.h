@@ -29,6 +29,31 @@ struct QuantParams {
 
 cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_groups, cudaStream_t stream);
 
+// Several dense layers that read the same activation (q / k / v, gate / up), quantised by one launch: the
+// fields that differ per layer; everything else comes from `base`.
+constexpr int kMaxBatch = 4;
+struct QuantLayer {                      // what differs per batched layer
+    const int32_t* perm;
+    const float* inv_s_perm;
+    uint8_t* codes;
+    uint8_t* scales_row;
+    uint8_t* scales_sf;
+    int k_tail;
+};
+// The common fields come first and layer 0 right behind them, so that a launch for a single layer reads
+// one 128-byte line of kernel parameters.
+struct QuantBatch {
+    const uint16_t* x;
+    const int32_t* expert_offsets;
+    int M, ldx, K;
+    int n_experts;
+    int act_groups;
+    int n_lin;                           // 1 .. kMaxBatch
+    int groups_per_lin;                  // blockIdx.y = layer * groups_per_lin + group
+    QuantLayer lay[kMaxBatch];
+};
+cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStream_t stream);
+
 // Which GEMM variant to run.
 enum class GemmKind {
     kPrefill,  // tokens on the MMA M axis (128-row tiles), weights on the N axis, persistent CTAs
@@ -75,6 +100,31 @@ struct DecodeParams {
     long long* trace;
     int dbg;
 };
+// Several dense layers over the same tokens (q / k / v, gate / up) in one launch.
+struct DecodeLayer {                 // what differs per batched layer
+    const uint8_t* act_sf;
+    const uint8_t* w_sf;
+    void* y;
+    int N, w_groups, ldy;
+    int tile_end;                    // 128-row weight tiles of layers 0 .. this one together
+};
+// The common fields come first and layer 0 right behind them, so that a launch for a single layer reads
+// one 128-byte line of kernel parameters.
+struct DecodeBatch {
+    const uint16_t* x;               // fused variant (one layer): bf16 activation, else null
+    int* status;
+    long long* trace;
+    int M, K, k_tail, ldx;
+    int y_bf16, splits, dbg;
+    int n_lin;                       // 1 .. kMaxBatch
+    DecodeLayer lay[kMaxBatch];
+};
+struct DecodeMaps {
+    CUtensorMap act[kMaxBatch];
+    CUtensorMap w[kMaxBatch];
+};
+// `bn` in {16, 32, 64, 128} is the token tile; the grid is (all tiles) * splits CTAs in clusters of `splits`.
+cudaError_t launch_decode_batch(int bn, const DecodeMaps& maps, const DecodeBatch& b, cudaStream_t stream);
 // `bn` in {16, 32, 64, 128} is the token tile; the grid is n_tiles * splits CTAs in clusters of `splits`.
 cudaError_t launch_decode(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const DecodeParams& p,
                           int n_tiles, cudaStream_t stream);

@@ -42,9 +42,9 @@ __device__ __forceinline__ uint32_t encode8(const float (&v)[8], uint32_t byte) 
     return cvt_e2m1x8(v[0] * inv, v[1] * inv, v[2] * inv, v[3] * inv, v[4] * inv, v[5] * inv, v[6] * inv, v[7] * inv);
 }
 
-template <bool kScalePerm>
+template <bool kScalePerm, bool kBatch>
 __global__ void __launch_bounds__(kQuantThreads, kScalePerm ? 3 : 4)
-quant_act_kernel(QuantParams p) {
+quant_act_kernel(const QuantBatch b) {
     __shared__ __align__(16) uint8_t sf_atom[512];
     __shared__ int s_tile_start[kMaxExperts + 1];
 
@@ -54,6 +54,19 @@ quant_act_kernel(QuantParams p) {
     grid_launch_dependents();
     grid_dependency_wait();
 
+    // which of the batched layers this CTA works for (one launch may quantise the same activation for
+    // several layers, each with its own scale, permutation and outputs)
+    // (kBatch = false: a single layer, nothing to look up -- the division alone costs the small-batch
+    // launches 0.2 us)
+    const int lin = kBatch ? static_cast<int>(blockIdx.y) / b.groups_per_lin : 0;
+    QuantParams p;
+    p.x = b.x; p.M = b.M; p.ldx = b.ldx; p.K = b.K; p.n_experts = b.n_experts; p.act_groups = b.act_groups;
+    p.expert_offsets = b.expert_offsets;
+    {
+        const QuantLayer& l = b.lay[lin];
+        p.k_tail = l.k_tail; p.perm = l.perm; p.inv_s_perm = l.inv_s_perm;
+        p.codes = l.codes; p.scales_row = l.scales_row; p.scales_sf = l.scales_sf;
+    }
     const int atom = blockIdx.x;                  // 128-column slice of the reduction axis
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = lane >> 4, hl = lane & 15;   // which of the warp's two rows, lane inside the row
@@ -61,7 +74,7 @@ quant_act_kernel(QuantParams p) {
     // Which rows does this CTA own?  Dense: group g covers rows [128 g, 128 g + 128).  Grouped: the
     // scale groups are padded per expert, so walk the expert offsets to find ours.
     int row0, row_end, expert = 0;
-    const int group = blockIdx.y;
+    const int group = static_cast<int>(blockIdx.y) - lin * b.groups_per_lin;
     if (p.expert_offsets == nullptr) {
         row0 = group * kGroupRows;
         row_end = min(p.M, row0 + kGroupRows);
@@ -270,7 +283,9 @@ quant_act_kernel(QuantParams p) {
 
 }  // namespace
 
-cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_groups, cudaStream_t stream) {
+cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStream_t stream) {
+    const QuantBatch& p = b;
+    const int grid_groups = b.groups_per_lin * b.n_lin;
     cudaLaunchConfig_t cfg = {};
     const int n_atoms = (p.K + kAtomK - 1) / kAtomK;
     int parts = 1;
@@ -298,7 +313,21 @@ cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_gro
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return scale_perm ? cudaLaunchKernelEx(&cfg, quant_act_kernel<true>, p) : cudaLaunchKernelEx(&cfg, quant_act_kernel<false>, p);
+    if (b.n_lin > 1)
+        return scale_perm ? cudaLaunchKernelEx(&cfg, quant_act_kernel<true, true>, b)
+                          : cudaLaunchKernelEx(&cfg, quant_act_kernel<false, true>, b);
+    return scale_perm ? cudaLaunchKernelEx(&cfg, quant_act_kernel<true, false>, b)
+                      : cudaLaunchKernelEx(&cfg, quant_act_kernel<false, false>, b);
+}
+
+cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_groups, cudaStream_t stream) {
+    QuantBatch b = {};
+    b.x = p.x; b.expert_offsets = p.expert_offsets; b.M = p.M; b.ldx = p.ldx; b.K = p.K;
+    b.n_experts = p.n_experts; b.act_groups = p.act_groups;
+    b.n_lin = 1;
+    b.groups_per_lin = grid_groups;
+    b.lay[0] = QuantLayer{p.perm, p.inv_s_perm, p.codes, p.scales_row, p.scales_sf, p.k_tail};
+    return launch_quant_act_batch(b, scale_perm, stream);
 }
 
 }  // namespace prq

@@ -447,3 +447,37 @@ def test_linear_with_weight_scale_search(prq, oracle):
         assert np.abs(y - y_ref).max() <= prq_ref.tolerance(y_ref)
     assert prq.last_device_status() == 0
     w.free()
+
+
+@pytest.mark.parametrize("M", [1, 16, 64, 128])
+def test_multi_layer_launches_match_single_layer_calls(prq, oracle, M):
+    """q / k / v-shaped layers over the same activation: one quantiser launch and one GEMM launch for all
+    three give, layer by layer, the bits of the single-layer calls (and hence the oracle's result)."""
+    K, k = 1024, 128
+    shapes = [384, 128, 200]
+    L0 = synth.layer(1, shapes[0], K, M, T_cal=32, tag=970)
+    x = to_dev_bf16(L0["x"])
+    ws, os_ = [], []
+    for i, N in enumerate(shapes):
+        Li = synth.layer(1, N, K, 4, T_cal=32, tag=971 + i)
+        amax = oracle.channel_amax(Li["zcal"])
+        ws.append(prq.prepare_weights(Li["W"], amax, 0.5, k))
+        os_.append(oracle.prepare(Li["W"], amax, float(np.float32(0.5)), k))
+    acts = prq.quantize_act_multi(ws, x, prq.ACT_SCALE_PERM)
+    ys = prq.linear_multi(ws, acts, M)
+    assert prq.last_device_status() == 0
+    for w, o, (codes, sf), y in zip(ws, os_, acts, ys):
+        c1, _, s1 = prq.quantize_act(w, x, prq.ACT_SCALE_PERM)
+        assert torch.equal(codes, c1) and torch.equal(sf, s1)
+        assert torch.equal(y, prq.linear(w, c1, s1, M))
+        oc, osc = oracle.quantize_act(L0["x"], o["perm"], o["inv_s"])
+        ca, sa = oracle.augment_act(oc, osc, k)
+        y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+        assert np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max() <= prq_ref.tolerance(y_ref)
+    # layers that do not share K (or k_tail for the GEMM) are refused
+    Lb = synth.layer(1, 128, 512, 4, T_cal=32, tag=979)
+    wb = prq.prepare_weights(Lb["W"], oracle.channel_amax(Lb["zcal"]), 0.5, 64)
+    with pytest.raises(prq.PrqError):
+        prq.quantize_act_multi([ws[0], wb], x, prq.ACT_SCALE_PERM, out=acts[:2])
+    for w in ws + [wb]:
+        w.free()
