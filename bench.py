@@ -206,12 +206,42 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
                           bound="tensor" if fl / fp4_peak / 1e6 > by / pk["hbm_gbs"] / 1e3 else "hbm")
     step_fns = [(lambda lin=lin: [f() for name in BLOCK_LINEARS for f in (q(lin[name]), g(lin[name]))]) for lin in layers]
     t_step = timer.run(step_fns, n, n_layers) / n
+    # At decode batch sizes a launch costs as much as the work in it: the layers that read the same activation
+    # (q / k / v and gate / up) also go through one quantiser launch and one GEMM launch per group.
+    t_step_multi = None
+    bf16_fused = None
+    if M <= 128:
+        def multi_step(lin):
+            def run():
+                for group in (("q", "k", "v"), ("o",), ("gate", "up"), ("down",)):
+                    ds = [lin[name] for name in group]
+                    if len(ds) == 1:
+                        q(ds[0])(); g(ds[0])()
+                    else:
+                        ws = [d["w"] for d in ds]
+                        acts = [(d["codes"], d["sf"]) for d in ds]
+                        prq.quantize_act_multi(ws, ds[0]["x"], ds[0]["mode"], out=acts)
+                        prq.linear_multi(ws, acts, M, prq.BF16, out=[d["y"] for d in ds])
+            return run
+        t_step_multi = timer.run([multi_step(lin) for lin in layers], n, n_layers) / n
+        # the BF16 baseline with the same launch fusion: q / k / v and gate / up weights concatenated
+        fused_w = [dict(qkv=torch.cat([lin[nm]["Wb"] for nm in ("q", "k", "v")]), gu=torch.cat([lin[nm]["Wb"] for nm in ("gate", "up")]))
+                   for lin in layers]
+        def bf16_step(lin, fw):
+            def run():
+                torch.matmul(lin["q"]["x"], fw["qkv"].t()); torch.matmul(lin["o"]["x"], lin["o"]["Wb"].t())
+                torch.matmul(lin["gate"]["x"], fw["gu"].t()); torch.matmul(lin["down"]["x"], lin["down"]["Wb"].t())
+            return run
+        bf16_fused = timer.run([bf16_step(lin, fw) for lin, fw in zip(layers, fused_w)], n, n_layers) / n
     total_flops = sum(2.0 * M * N * (K + (k if k_override is None else k_override)) for N, K, k in BLOCK_LINEARS.values())
     status = prq.last_device_status()
     for lin in layers:
         for d in lin.values():
             d["w"].free()
-    return dict(workload=tag, M=M, layers=n_layers, step_us=t_step * 1e6, step_tflops=total_flops / t_step / 1e12,
+    extra = {}
+    if t_step_multi is not None:
+        extra = dict(step_multi_launch_us=t_step_multi * 1e6, bf16_fused_qkv_gateup_us=bf16_fused * 1e6)
+    return dict(workload=tag, M=M, layers=n_layers, step_us=t_step * 1e6, step_tflops=total_flops / t_step / 1e12, **extra,
                 gemm_us_sum=sum(r["gemm_us"] for r in rows.values()), quant_us_sum=sum(r["quant_us"] for r in rows.values()),
                 bf16_us_sum=sum(r["bf16_matmul_us"] for r in rows.values()), device_status=status, linears=rows)
 
@@ -348,6 +378,9 @@ def main():
                        for M in (64, 4096) for k in (256, 0)]
                 for r in res:
                     r["stack_36_layers_us"] = 36 * r["step_us"]
+                    if "step_multi_launch_us" in r:
+                        r["stack_36_layers_multi_launch_us"] = 36 * r["step_multi_launch_us"]
+                        r["stack_36_layers_bf16_fused_us"] = 36 * r["bf16_fused_qkv_gateup_us"]
                     r["stack_36_layers_bf16_us"] = 36 * r["bf16_us_sum"]
             print(json.dumps({"metric": METRIC, "workload": args.workload, "unit": "us / TFLOP/s", "n_gpus": 1,
                               "dtype": "mxfp4 (e2m1 x e8m0), f32 accumulate, bf16 output", "data": "synthetic",
