@@ -49,10 +49,11 @@ quant_act_kernel(const QuantBatch b) {
     __shared__ int s_tile_start[kMaxExperts + 1];
 
     // Launched with programmatic stream serialisation: this CTA may be running while the previous kernel
-    // of the stream still is.  Nothing global is touched before the wait (x may be that kernel's output,
-    // and it may still be reading the buffers written here).
+    // of the stream still is.  Nothing that an earlier kernel may write or still read is touched before the
+    // wait (x may be that kernel's output, and it may still be reading the buffers written here); the
+    // layer's own permutation and reciprocal scales are constants of the prepared weights, and a dense
+    // launch requests them first so that their latency overlaps the wait.
     grid_launch_dependents();
-    grid_dependency_wait();
 
     // which of the batched layers this CTA works for (one launch may quantise the same activation for
     // several layers, each with its own scale, permutation and outputs)
@@ -70,6 +71,24 @@ quant_act_kernel(const QuantBatch b) {
     const int atom = blockIdx.x;                  // 128-column slice of the reduction axis
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = lane >> 4, hl = lane & 15;   // which of the warp's two rows, lane inside the row
+    float inv_s[8];
+    int src[8];
+    auto load_layer_constants = [&](int expert_) {
+        const int c0 = atom * kAtomK + hl * 8;
+        if (c0 < p.K) {
+            const int32_t* perm = p.perm + static_cast<size_t>(expert_) * p.K + c0;
+            const float* isp = p.inv_s_perm + static_cast<size_t>(expert_) * p.K + c0;
+            const int4 p0 = *reinterpret_cast<const int4*>(perm), p1 = *reinterpret_cast<const int4*>(perm + 4);
+            const float4 s0 = *reinterpret_cast<const float4*>(isp), s1 = *reinterpret_cast<const float4*>(isp + 4);
+            src[0] = p0.x; src[1] = p0.y; src[2] = p0.z; src[3] = p0.w;
+            src[4] = p1.x; src[5] = p1.y; src[6] = p1.z; src[7] = p1.w;
+            inv_s[0] = s0.x; inv_s[1] = s0.y; inv_s[2] = s0.z; inv_s[3] = s0.w;
+            inv_s[4] = s1.x; inv_s[5] = s1.y; inv_s[6] = s1.z; inv_s[7] = s1.w;
+        }
+    };
+    const bool dense = p.expert_offsets == nullptr;
+    if (kScalePerm && dense) load_layer_constants(0);
+    grid_dependency_wait();
 
     // Which rows does this CTA own?  Dense: group g covers rows [128 g, 128 g + 128).  Grouped: the
     // scale groups are padded per expert, so walk the expert offsets to find ours.
@@ -120,18 +139,7 @@ quant_act_kernel(const QuantBatch b) {
     const int part = kScalePerm ? static_cast<int>(blockIdx.z) : 0;
     const int part_steps = kSteps / n_parts;
 
-    float inv_s[8];
-    int src[8];
-    if (kScalePerm && col_ok) {
-        const int32_t* perm = p.perm + static_cast<size_t>(expert) * K + col0;
-        const float* isp = p.inv_s_perm + static_cast<size_t>(expert) * K + col0;
-        const int4 p0 = *reinterpret_cast<const int4*>(perm), p1 = *reinterpret_cast<const int4*>(perm + 4);
-        const float4 s0 = *reinterpret_cast<const float4*>(isp), s1 = *reinterpret_cast<const float4*>(isp + 4);
-        src[0] = p0.x; src[1] = p0.y; src[2] = p0.z; src[3] = p0.w;
-        src[4] = p1.x; src[5] = p1.y; src[6] = p1.z; src[7] = p1.w;
-        inv_s[0] = s0.x; inv_s[1] = s0.y; inv_s[2] = s0.z; inv_s[3] = s0.w;
-        inv_s[4] = s1.x; inv_s[5] = s1.y; inv_s[6] = s1.z; inv_s[7] = s1.w;
-    }
+    if (kScalePerm && !dense) load_layer_constants(expert);   // grouped: the expert is known only now
 
     // row of step i: 16 rows per step, 2 per warp
     auto row_of = [&](int i) { return i * 16 + warp * 2 + half; };
