@@ -707,6 +707,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         q.m_tiles = (M + 255) / 256; q.n_tiles = (w->N + kPrefillTileN - 1) / kPrefillTileN;
         q.act_groups = p.act_groups; q.w_groups = w->w_groups_alt[2];
         q.act_sf = p.act_sf; q.w_sf = w->d_sf_alt[2];
+        q.y = y; q.ldy = ldy;
         q.y_bf16 = p.y_bf16; q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
         const size_t flag_bytes = prefill_flag_bytes(w, M);
         const long long tiles = static_cast<long long>(q.m_tiles) * q.n_tiles;

@@ -381,7 +381,26 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
 
         // 32 accumulator columns of this warp's 32 rows -> y: swizzled shared staging, then one TMA store
         // (rows and columns outside M x N are clipped by the tensor map)
+        // first column of the 32-column chunk that holds a right edge narrower than 16 bytes (chunks start at
+        // multiples of 32), or -1 if N is a multiple of 16 bytes
+        const int ragged_x = (p.N % (p.y_bf16 ? 8 : 4)) ? (p.N / 32) * 32 : -1;
         auto store_chunk = [&](const uint32_t (&v)[32], int x, int y_row) {
+            // A tiled store clips at the tensor's edge in units of 16 bytes: where N is not a multiple of that,
+            // it would fill the last column group up with zeros, i.e. write into the caller's bytes between
+            // column N and the row stride.  That one chunk goes out with plain stores instead.
+            if (x == ragged_x) {
+                const int row = y_row + lane;
+                if (row < p.M) {
+                    if (p.y_bf16) {
+                        __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<size_t>(row) * p.ldy + x;
+                        for (int i = 0; i < 32 && x + i < p.N; ++i) yp[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                    } else {
+                        float* yp = reinterpret_cast<float*>(p.y) + static_cast<size_t>(row) * p.ldy + x;
+                        for (int i = 0; i < 32 && x + i < p.N; ++i) yp[i] = __uint_as_float(v[i]);
+                    }
+                }
+                return;
+            }
             const uint32_t sbuf = stage_smem + (store_it & 1) * 4096;
             // the store issued two chunks ago has finished reading this buffer
             if (lane == 0) bulk_wait_read<1>();

@@ -145,6 +145,8 @@ struct PrefillParams {
     float* partial;             // two 128 x 224 fp32 slots per CTA
     int* flags;                 // "arrived" counter per 128-row half of a tile (index 2 * tile + half) ...
     int flag_stride;            // ... and, this many ints further, its "finished" counter; all zero between launches
+    void* y;                    // output matrix and its row stride in elements: used only for the column group at
+    int ldy;                    // the right edge that is narrower than 16 bytes (the tiled stores cover the rest)
     int y_bf16;
     int* status;
     long long* trace;

@@ -1,0 +1,67 @@
+"""Random-shape parity sweep: seeded draws of (N, K, k, M, mode, output type, alpha, block-scale search) through
+every dense entry point -- quantiser, prq_linear (decode and prefill kernels by M), the fused decode step, the
+multi-layer launches -- against the oracle, with output row strides larger than N."""
+import numpy as np
+import pytest
+
+import prq_ref
+from paper_2609_22106_b200 import synth
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+def dev_bf16(x_u16):
+    return torch.from_numpy(np.ascontiguousarray(x_u16).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_shapes_against_oracle(prq, oracle, seed):
+    rng = np.random.default_rng(seed)
+    for case in range(12):
+        K = int(rng.integers(1, 40)) * 32
+        k = int(rng.integers(0, min(K // 32, 8) + 1)) * 32
+        N = int(rng.choice([8, 16, 24, 100, 128, 130, 224, 256, 300, 448, 500]))
+        M = int(rng.choice([1, 2, 5, 15, 16, 17, 31, 33, 64, 65, 127, 128, 129, 200, 255, 256, 257, 300, 511, 600]))
+        mode = int(rng.integers(0, 2))
+        dt = prq.F32 if rng.random() < 0.7 else prq.BF16
+        alpha = float(rng.choice([0.0, 0.25, 0.5, 1.0]))
+        search = bool(rng.random() < 0.3)
+        what = f"seed {seed} case {case}: N={N} K={K} k={k} M={M} mode={mode} dt={dt} alpha={alpha} search={search}"
+        L = synth.layer(7, N, K, M, T_cal=32, tag=int(rng.integers(0, 10000)))
+        amax = oracle.channel_amax(L["zcal"])
+        w = prq.prepare_weights(L["W"], amax, alpha, k, scale_search=search)
+        o = oracle.prepare(L["W"], amax, float(np.float32(alpha)), k, scale_search=search)
+        assert np.array_equal(w.get(prq.FIELD_PERM), o["perm"]), what
+        assert np.array_equal(w.get(prq.FIELD_SCALES), o["wscales"]), what
+        assert np.array_equal(w.get(prq.FIELD_CODES), o["wcodes"]), what
+        x = dev_bf16(L["x"])
+        codes, srow, sf = prq.quantize_act(w, x, mode, row_scales=True)
+        if mode == prq.ACT_IDENTITY:
+            oc, osc = oracle.quantize_act(L["x"])
+        else:
+            oc, osc = oracle.quantize_act(L["x"], o["perm"], o["inv_s"])
+        assert np.array_equal(codes.cpu().numpy()[: M * K // 2].reshape(M, K // 2), oc), what
+        assert np.array_equal(srow.cpu().numpy()[: M * K // 32].reshape(M, K // 32), osc), what
+        ca, sa = oracle.augment_act(oc, osc, k)
+        y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+        n_pad = (N + 7) // 8 * 8 + 8 * int(rng.integers(0, 3))
+        tdt = torch.float32 if dt == prq.F32 else torch.bfloat16
+
+        def ybuf():
+            return torch.full((M, n_pad), 7.0, dtype=tdt, device="cuda")
+
+        full = ybuf()
+        y = prq.linear(w, codes, sf, M, dt, out=full[:, :N])
+        assert prq.last_device_status() == 0, what
+        assert bool((full[:, N:] == 7.0).all()), what          # nothing written past column N
+        got = y.float().cpu().numpy().astype(np.float64)
+        slack = np.abs(y_ref).max() * 2.0 ** -7 if dt == prq.BF16 else 0.0
+        assert np.abs(got - y_ref).max() <= prq_ref.tolerance(y_ref) + slack, what
+        if M <= prq.FUSED_MAX_M and mode == prq.ACT_IDENTITY:
+            assert torch.equal(prq.linear_fused(w, x, mode, dt, out=ybuf()[:, :N]), y), what
+        if M <= 128:
+            acts = prq.quantize_act_multi([w, w], x, mode)
+            ys = prq.linear_multi([w, w], acts, M, dt, out=[ybuf()[:, :N], ybuf()[:, :N]])
+            assert torch.equal(acts[1][0], codes) and torch.equal(ys[0], y) and torch.equal(ys[1], y), what
+        w.free()
