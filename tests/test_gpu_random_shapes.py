@@ -65,3 +65,55 @@ def test_random_shapes_against_oracle(prq, oracle, seed):
             ys = prq.linear_multi([w, w], acts, M, dt, out=[ybuf()[:, :N], ybuf()[:, :N]])
             assert torch.equal(acts[1][0], codes) and torch.equal(ys[0], y) and torch.equal(ys[1], y), what
         w.free()
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_grouped_shapes_against_oracle(prq, oracle, seed):
+    """Stacked experts with random row counts (empty experts included), strided activations and outputs."""
+    rng = np.random.default_rng(seed)
+    for case in range(8):
+        E = int(rng.choice([2, 3, 5, 8, 16]))
+        K = int(rng.integers(1, 16)) * 32
+        k = int(rng.integers(0, min(K // 32, 4) + 1)) * 32
+        N = int(rng.choice([16, 100, 128, 136, 256, 300]))
+        counts = rng.choice([0, 0, 1, 3, 17, 64, 127, 128, 129, 200, 300], size=E)
+        if counts.sum() == 0:
+            counts[0] = 5
+        offsets = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+        M = int(offsets[-1])
+        mode = int(rng.integers(0, 2))
+        dt = prq.F32 if rng.random() < 0.5 else prq.BF16
+        what = f"seed {seed} case {case}: E={E} N={N} K={K} k={k} counts={counts.tolist()} mode={mode} dt={dt}"
+        ch = synth.HeavyTailChannels(int(rng.integers(0, 10000)), K)
+        Ws = np.stack([synth.weights(int(rng.integers(0, 10000)), N, K) for _ in range(E)])
+        amax = np.stack([oracle.channel_amax(ch.rows(int(rng.integers(0, 10000)), 32)) for _ in range(E)])
+        x = ch.rows(int(rng.integers(0, 10000)), M)
+        w = prq.prepare_weights(Ws, amax, 0.5, k)
+        ldx = K + 8 * int(rng.integers(0, 3))
+        xs = torch.zeros((M, ldx), dtype=torch.bfloat16, device="cuda")
+        xs[:, :K] = dev_bf16(x)
+        d_off = torch.from_numpy(offsets).cuda()
+        codes, srow, sf = prq.quantize_act(w, xs[:, :K], mode, expert_offsets=d_off, row_scales=True)
+        n_pad = (N + 7) // 8 * 8 + 8 * int(rng.integers(0, 3))
+        full = torch.full((M, n_pad), 7.0, dtype=torch.float32 if dt == prq.F32 else torch.bfloat16, device="cuda")
+        y = prq.linear_grouped(w, codes, sf, d_off, M, dt, out=full[:, :N])
+        assert prq.last_device_status() == 0, what
+        assert bool((full[:, N:] == 7.0).all()), what
+        got_c = codes.cpu().numpy()[: M * K // 2].reshape(M, K // 2)
+        got_s = srow.cpu().numpy()[: M * K // 32].reshape(M, K // 32)
+        for e in range(E):
+            r0, r1 = int(offsets[e]), int(offsets[e + 1])
+            if r1 == r0:
+                continue
+            o = oracle.prepare(Ws[e], amax[e], float(np.float32(0.5)), k)
+            if mode == prq.ACT_IDENTITY:
+                oc, osc = oracle.quantize_act(x[r0:r1])
+            else:
+                oc, osc = oracle.quantize_act(x[r0:r1], o["perm"], o["inv_s"])
+            assert np.array_equal(got_c[r0:r1], oc) and np.array_equal(got_s[r0:r1], osc), what
+            ca, sa = oracle.augment_act(oc, osc, k)
+            y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+            got = y[r0:r1].float().cpu().numpy().astype(np.float64)
+            slack = np.abs(y_ref).max() * 2.0 ** -7 if dt == prq.BF16 else 0.0
+            assert np.abs(got - y_ref).max() <= prq_ref.tolerance(y_ref) + slack, what
+        w.free()
