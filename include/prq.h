@@ -179,6 +179,7 @@ size_t prq_linear_workspace_bytes(const prq_weights *w, int M);
  * accumulation.  Reads activation columns [0, K) and then [K - k, K) again; no M x (K + k) buffer exists.
  *   codes, scales_sf  device, as written by prq_quantize_act for the same w and M
  *   y                 device out, M x N, row stride ldy elements, dtype y_dtype (fp32 for parity)
+ *                     (only columns [0, N) of a row are written: y may be a column slice of a wider matrix)
  *   workspace         device, at least prq_linear_workspace_bytes(w, M) bytes, 16-byte aligned (may be NULL
  *                     when that is 0); zero-filled by the caller before its first use, the kernel leaves
  *                     its flags zeroed again
