@@ -198,7 +198,7 @@ prq_status prq_linear(const prq_weights *w, const void *codes, const void *scale
  *   - Limits: at most 8192 output half-tiles (2 * ceil(M/256) * ceil(N/224)) and at most 160 SMs; beyond
  *     that the call returns PRQ_ERR_STATIC_SCRATCH and launches nothing.  M <= 128 needs no scratch and is
  *     passed on.
- *   - Cost: the array is 36,765,696 bytes (64 KB of counters + 2 x 160 partial tiles of 112 KB) on every
+ *   - Cost: the array is 42,008,576 bytes (64 KB of counters + 2 x 160 partial tiles of 128 KB) on every
  *     GPU that loads the library, until the process exits.
  *   - The call itself performs no allocation (no cudaMalloc / cudaFree, no allocating library routine); it
  *     enqueues one small memset of the flags and the kernel.  The first call on a device also looks up the

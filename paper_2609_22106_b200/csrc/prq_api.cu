@@ -121,10 +121,12 @@ prq_status build_weight_maps(prq_weights* w) {
     if (w->n_experts != 1) return PRQ_OK;
     const uint64_t Ka = static_cast<uint64_t>(w->K) + w->k_tail;
     prq_status st = make_code_map(&w->tm_w_decode, w->d_codes, Ka / 2, w->N, 128);
-    if (st == PRQ_OK) st = make_code_map(&w->tm_w_pair, w->d_codes, Ka / 2, w->N, kPrefillTileN / 2);
-    if (st == PRQ_OK && w->d_sf_alt[2])
-        st = make_sf_map(&w->tm_sfw_pair, w->d_sf_alt[2],
-                         static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[2] * kSfGroupBytes, 8);
+    for (int v = 0; v < 2; ++v) {   // 224- and 240-row tilings: scale layouts 2 and 3
+        if (st == PRQ_OK) st = make_code_map(&w->tm_w_pair[v], w->d_codes, Ka / 2, w->N, (v ? kPrefillTileWide : kPrefillTileN) / 2);
+        if (st == PRQ_OK && w->d_sf_alt[2 + v])
+            st = make_sf_map(&w->tm_sfw_pair[v], w->d_sf_alt[2 + v],
+                             static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[2 + v] * kSfGroupBytes, 8);
+    }
     if (st == PRQ_OK) w->maps_ready = true;
     return st;
 }
@@ -204,9 +206,56 @@ int prefill_bn(const prq_weights* w, int M, int num_sms) {
     return best;
 }
 
-constexpr int kNumAlt = 3;
-constexpr int kAltTileRows[kNumAlt] = {160, 192, 224};  // weight tile widths with their own scale layout
-constexpr size_t kPrefillSlotBytes = 128 * kPrefillTileN * sizeof(float);
+constexpr int kNumAlt = 4;
+constexpr int kAltTileRows[kNumAlt] = {160, 192, 224, 240};  // weight tile widths with their own scale layout
+
+// How the pair kernel shares out the tiles of one call: every pair gets `whole` whole tiles; the `sk`
+// tiles left over are each cut into equal pieces for `base` (the first `extra` tiles: base + 1)
+// consecutive pairs.
+struct PairSchedule {
+    int bn, pairs;
+    long long tiles, whole, sk;
+    int base, extra;
+    long long stages_per_pair;   // reduction stages of the busiest pair
+};
+
+PairSchedule pair_schedule(int bn, int M, int N, int S, int max_pairs) {
+    PairSchedule ps = {};
+    ps.bn = bn;
+    ps.tiles = static_cast<long long>((M + 255) / 256) * ((N + bn - 1) / bn);
+    ps.pairs = static_cast<int>(std::min<long long>(ps.tiles * S, max_pairs));
+    if (ps.pairs < 1) return ps;
+    ps.whole = ps.tiles / ps.pairs;
+    ps.sk = ps.tiles - ps.whole * ps.pairs;
+    if (env_int("PRQ_PURE_SK", 0)) { ps.whole = 0; ps.sk = ps.tiles; }
+    // Pieces have at least `min_piece` stages: a piece costs a whole partial tile of traffic whatever its
+    // length, so short reductions are cut into few pieces or not at all (the left-over tiles then go whole
+    // to as many pairs) and the pairs left over sit that phase out.  (Cutting the unit space into equal
+    // contiguous ranges, two pieces per pair, balances better on paper and measured worse: 47.7 vs 45.5 us
+    // on the 4096-token down projection, 28.3 vs 20.0 us with 1024 tokens; PRQ_SK_RANGES=1 still selects it.)
+    const long long min_piece = std::max(1, env_int("PRQ_SK_MIN_PIECE", 9));
+    const long long cap = std::max<long long>(1, std::min<long long>(8, S / min_piece));
+    ps.base = 1;
+    if (ps.sk > 0) {
+        ps.base = static_cast<int>(std::max<long long>(1, std::min<long long>(ps.pairs / ps.sk, cap)));
+        ps.extra = ps.base >= 2 && ps.base == ps.pairs / ps.sk && ps.base < cap ? static_cast<int>(ps.pairs % ps.sk) : 0;
+    }
+    ps.stages_per_pair = ps.whole * S + (ps.sk > 0 ? (S + ps.base - 1) / ps.base : 0);
+    return ps;
+}
+
+// Tile width of the pair kernel: the main loop is bound by the operand bytes an SM takes in per stage
+// (33792 with 224-column tiles, 34816 with 240-column ones), so the width whose busiest pair takes in
+// fewer bytes wins; 224 on a tie.  With the paper's down projection that is 240 from 2048 tokens on
+// (11 instead of 12 column tiles) and 224 below (the tile counts do not fill the pairs either way).
+PairSchedule choose_pair_schedule(int M, int N, int S, int max_pairs) {
+    const PairSchedule narrow = pair_schedule(kPrefillTileN, M, N, S, max_pairs);
+    const PairSchedule wide = pair_schedule(kPrefillTileWide, M, N, S, max_pairs);
+    const int forced = env_int("PRQ_PAIR_BN", 0);
+    if (forced == kPrefillTileN) return narrow;
+    if (forced == kPrefillTileWide) return wide;
+    return wide.stages_per_pair * 34816 < narrow.stages_per_pair * 33792 ? wide : narrow;
+}
 
 // Two counters ("arrived", "finished") per 128-row half of a 256 x 224 pair tile: first all the "arrived"
 // counters, then all the "finished" ones.
@@ -700,39 +749,27 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     } else if (env_int("PRQ_PREFILL_BN", 0) == 0) {
-        // stream-K kernel on CTA pairs with 256 x 224 tiles (scale bytes grouped per 224-row weight tile)
+        // stream-K kernel on CTA pairs with 256 x 224 or 256 x 240 tiles (scale bytes grouped per weight tile)
         PrefillParams q;
         std::memset(&q, 0, sizeof(q));
+        if (di->max_pairs == 0)
+            di->max_pairs = std::min(std::min(prefill_pair_max_clusters(kPrefillTileN), prefill_pair_max_clusters(kPrefillTileWide)),
+                                     di->num_sms / 2);
+        const PairSchedule ps = choose_pair_schedule(M, w->N, w->plan.S, std::min(di->max_pairs, env_int("PRQ_GRID", 1 << 20)));
+        const int pair_bn = ps.bn, variant = pair_bn == kPrefillTileWide ? 1 : 0, pairs = ps.pairs;
+        if (pairs < 1) return PRQ_ERR_CUDA;
         q.M = M; q.N = w->N; q.K = w->K; q.k_tail = w->k_tail;
-        q.m_tiles = (M + 255) / 256; q.n_tiles = (w->N + kPrefillTileN - 1) / kPrefillTileN;
-        q.act_groups = p.act_groups; q.w_groups = w->w_groups_alt[2];
-        q.act_sf = p.act_sf; q.w_sf = w->d_sf_alt[2];
+        q.m_tiles = (M + 255) / 256; q.n_tiles = (w->N + pair_bn - 1) / pair_bn;
+        q.act_groups = p.act_groups; q.w_groups = w->w_groups_alt[2 + variant];
+        q.act_sf = p.act_sf; q.w_sf = w->d_sf_alt[2 + variant];
         q.y = y; q.ldy = ldy;
         q.y_bf16 = p.y_bf16; q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
         const size_t flag_bytes = prefill_flag_bytes(w, M);
-        const long long tiles = static_cast<long long>(q.m_tiles) * q.n_tiles;
-        const long long units = tiles * w->plan.S;
-        if (di->max_pairs == 0) di->max_pairs = std::min(prefill_pair_max_clusters(), di->num_sms / 2);
-        const int max_pairs = std::min(di->max_pairs, env_int("PRQ_GRID", 1 << 20));
-        const int pairs = static_cast<int>(std::min<long long>(units, max_pairs));
-        if (pairs < 1) return PRQ_ERR_CUDA;
-        // every pair gets `whole` whole tiles; the rest is shared out stream-K: each left-over tile cut into
-        // equal pieces for 2..8 consecutive pairs when there are at least two pairs per tile, else the
-        // (tile, stage) space cut into equal contiguous ranges
-        long long whole = tiles / pairs, sk = tiles - whole * pairs;
-        if (env_int("PRQ_PURE_SK", 0)) { whole = 0; sk = tiles; }
-        // Each left-over tile is cut into equal pieces for 1 .. 8 consecutive pairs.  Pieces have at least
-        // `min_piece` stages: a piece costs a whole partial tile of traffic whatever its length, so short
-        // reductions are cut into few pieces or not at all (the left-over tiles then go whole to as many
-        // pairs) and the pairs left over sit that phase out.  (Cutting the unit space into equal contiguous
-        // ranges, two pieces per pair, balances better on paper and measured worse: 47.7 vs 45.5 us on the
-        // 4096-token down projection; PRQ_SK_RANGES=1 still selects it.)
-        const long long min_piece = std::max(1, env_int("PRQ_SK_MIN_PIECE", 9));
-        const long long cap = std::max<long long>(1, std::min<long long>(8, w->plan.S / min_piece));
+        const long long tiles = ps.tiles, whole = ps.whole, sk = ps.sk;
         if (sk > 0 && !env_int("PRQ_SK_RANGES", 0)) {
             q.sk_aligned = 1;
-            q.sk_base = static_cast<int>(std::max<long long>(1, std::min<long long>(pairs / sk, cap)));
-            q.sk_extra = q.sk_base >= 2 && q.sk_base == pairs / sk && q.sk_base < cap ? static_cast<int>(pairs % sk) : 0;
+            q.sk_base = ps.base;
+            q.sk_extra = ps.extra;
         }
         q.sk_tiles = static_cast<int>(sk); q.whole_tiles = static_cast<int>(whole);
         if (sk * w->plan.S * pairs >= (1ll << 32) || tiles >= (1ll << 30)) return PRQ_ERR_INVALID_ARG;  // 32-bit range arithmetic
@@ -747,7 +784,8 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         if (st == PRQ_OK) st = make_sf_map(&tm_sfa, p.act_sf, Sg * p.act_groups * kSfGroupBytes, 4);
         if (st == PRQ_OK) st = make_out_map(&tm_y, y, M, w->N, ldy, y_dtype == PRQ_BF16);
         if (st != PRQ_OK) return st;
-        cudaError_t e = launch_prefill_pair(tm_act, w->tm_w_pair, tm_sfa, w->tm_sfw_pair, tm_y, q, pairs, static_cast<cudaStream_t>(stream));
+        cudaError_t e = launch_prefill_pair(pair_bn, tm_act, w->tm_w_pair[variant], tm_sfa, w->tm_sfw_pair[variant], tm_y, q, pairs,
+                                            static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     } else {
@@ -929,7 +967,7 @@ namespace {
 
 // Built-in scratch of the stream-K prefill kernel: two counters per 128-row half of an output tile, then
 // two fp32 partial tiles per CTA.  It is part of the library image, so every GPU that loads the library
-// carries it until the process exits: 64 KB of counters + 2 x 160 x 112 KB of partial tiles = 36,765,696 bytes.
+// carries it until the process exits: 64 KB of counters + 2 x 160 x 128 KB of partial tiles = 42,008,576 bytes.
 constexpr int kStaticMaxFlags = 8192;   // tile halves
 constexpr int kStaticMaxCtas = 160;
 constexpr size_t kStaticFlagBytes = 2 * static_cast<size_t>(kStaticMaxFlags) * sizeof(int);

@@ -1,5 +1,7 @@
-// Prefill GEMM (M > 128) on CTA pairs: the block-scaled FP4 product of Eq. (3) with 256 x 224 output
-// tiles computed by two CTAs of a cluster as one tcgen05 cta_group::2 unit, under a stream-K schedule.
+// Prefill GEMM (M > 128) on CTA pairs: the block-scaled FP4 product of Eq. (3) with 256 x 224 (or
+// 256 x 240) output tiles computed by two CTAs of a cluster as one tcgen05 cta_group::2 unit, under a
+// stream-K schedule.  The text below speaks of the 224-column tile; the 240-column variant differs in the
+// constants only (120 weight rows per CTA, a 16-column chunk closing the epilogue).
 //
 // Why pairs.  With one CTA per 128 x 224 tile every SM pulls (128 + 224) operand rows per reduction
 // stage from L2, and at the paper's down-projection shape the 148 SMs together ask for more than the
@@ -45,24 +47,34 @@ namespace prq {
 namespace {
 
 constexpr int kThreads = 192;
-constexpr int BN = kPrefillTileN;                 // 224 weight rows per tile
-constexpr int kHalfN = BN / 2;                    // weight rows each CTA of the pair loads
 constexpr int kPTile = 128 * 128;                 // activation tile bytes (128 rows x 256 codes)
-constexpr int kQTile = kHalfN * 128;              // half weight tile bytes
 constexpr int kSfp = kSfGroupBytes;               // 1 group of 128 activation rows
-constexpr int kSfq = 2 * kSfGroupBytes;           // 2 groups (128 + 96 weight rows)
-constexpr int kStageBytes = kPTile + kQTile + kSfp + kSfq;  // 33792
+constexpr int kSfq = 2 * kSfGroupBytes;           // 2 groups (128 + up to 128 weight rows)
 constexpr int kStages = 5;
 constexpr int kStagingPerWarp = 2 * 4096;         // two 32-row x 128-byte chunks per epilogue warp
-constexpr int kSmemBytes = kStages * kStageBytes + 4 * kStagingPerWarp + 1024;
 constexpr int kTmemCols = 512;
-constexpr int kSfCol = 2 * BN;                    // scale columns start behind the two accumulators
 constexpr int kSfSetCols = 24;                    // 8 activation + 16 weight scale columns
 constexpr int kChunkCols = 32;                    // accumulator columns per epilogue chunk
-constexpr int kChunks = BN / kChunkCols;          // 7
-static_assert(kQTile % 1024 == 0 && kStageBytes % 1024 == 0, "operand tiles must keep 1024-byte alignment");
-static_assert(kSmemBytes <= 232448 - 256, "shared memory budget");
-static_assert(kSfCol + kSfSetCols <= kTmemCols, "tensor memory budget");
+
+// Everything that depends on the tile width BN (weight rows per tile): 224 or 240.  Two accumulators of
+// BN columns and the scale columns must fit the 512 columns of tensor memory, which 240 still does; the
+// wider tile needs fewer operand bytes per multiply-add and pads N = 2560 less (11 x 240 against 12 x 224).
+template <int BN>
+struct PCfg {
+    static constexpr int kHalfN = BN / 2;                    // weight rows each CTA of the pair loads
+    static constexpr int kQTile = kHalfN * 128;              // half weight tile bytes
+    static constexpr int kStageBytes = kPTile + kQTile + kSfp + kSfq;  // 33792 / 34816
+    static constexpr int kSmemBytes = kStages * kStageBytes + 4 * kStagingPerWarp + 1024;
+    static constexpr int kSfCol = 2 * BN;                    // scale columns start behind the two accumulators
+    static constexpr int kChunks = (BN + kChunkCols - 1) / kChunkCols;   // 7, or 7 and a 16-column one
+    static constexpr int kLastCols = BN - (kChunks - 1) * kChunkCols;    // 32 or 16
+    static constexpr int kSlotUnits = kChunks * 8 * 128;     // float4 per workspace slot (128 rows)
+    static_assert(kQTile % 1024 == 0 && kStageBytes % 1024 == 0, "operand tiles must keep 1024-byte alignment");
+    static_assert(kSmemBytes <= 232448 - 256, "shared memory budget");
+    static_assert(kSfCol + kSfSetCols <= kTmemCols, "tensor memory budget");
+    static_assert(kLastCols == 32 || kLastCols == 16, "epilogue chunks are 32 columns, the last one 32 or 16");
+    static_assert(static_cast<size_t>(kSlotUnits) * 16 <= kPrefillSlotBytes, "workspace slot");
+};
 
 __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src_smem, int x, int y) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
@@ -168,12 +180,13 @@ __device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo) { return (s
 // -- then up to four K = 64 MMAs, then the commit that frees the slot in both CTAs.  The copies and
 // the MMAs are issued by one thread, so tensor memory sees them in order and one set of scale columns
 // is enough.  `rem` = reduction elements this stage still covers.
-template <int Q>
+template <int BN, int Q>
 __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, uint32_t sf_t, int rem,
                                             uint32_t accumulate, uint32_t empty_bar0) {
+    constexpr int kStageBytes = PCfg<BN>::kStageBytes, kQTile = PCfg<BN>::kQTile;
     constexpr uint32_t so = (Q * kStageBytes) >> 4;  // stage offset in 16-byte units
     constexpr uint32_t sfo = so + ((kPTile + kQTile) >> 4);
-    // E2M1 x E2M1, E8M0 scales, both operands K-major, N = 224, M = 256 (two CTAs)
+    // E2M1 x E2M1, E8M0 scales, both operands K-major, N = BN, M = 256 (two CTAs)
     constexpr uint32_t idesc0 = (1u << 7) | (1u << 10) | ((BN >> 3) << 17) | (1u << 23) | ((256u >> 4) << 24);
     constexpr uint32_t idesc2 = idesc0 | (2u << 4) | (2u << 29);
     const uint32_t plo = lo_base + so, qlo = lo_base + so + (kPTile >> 4), slo = lo_base + sfo;
@@ -193,10 +206,14 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
     tc_commit_pair(empty_bar0 + Q * 8, 3);
 }
 
+template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
                     const __grid_constant__ CUtensorMap tm_sfa, const __grid_constant__ CUtensorMap tm_sfw,
                     const __grid_constant__ CUtensorMap tm_y, const PrefillParams p) {
+    using C = PCfg<BN>;
+    constexpr int kHalfN = C::kHalfN, kQTile = C::kQTile, kStageBytes = C::kStageBytes, kSfCol = C::kSfCol;
+    constexpr int kChunks = C::kChunks, kLastCols = C::kLastCols;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[kStages], bar_empty[kStages], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_slot;
@@ -351,11 +368,11 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                     if (leader) {
                         const uint32_t eb = smem_u32(&bar_empty[0]);
                         switch (st) {
-                            case 0: issue_stage<0>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                            case 1: issue_stage<1>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                            case 2: issue_stage<2>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                            case 3: issue_stage<3>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
-                            default: issue_stage<4>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                            case 0: issue_stage<BN, 0>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                            case 1: issue_stage<BN, 1>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                            case 2: issue_stage<BN, 2>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                            case 3: issue_stage<BN, 3>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
+                            default: issue_stage<BN, 4>(lo_base, d_tmem, sf_t, rem, accumulate, eb); break;
                         }
                     }
                     accumulate = 1;
@@ -381,22 +398,49 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
 
         // 32 accumulator columns of this warp's 32 rows -> y: swizzled shared staging, then one TMA store
         // (rows and columns outside M x N are clipped by the tensor map)
-        // first column of the 32-column chunk that holds a right edge narrower than 16 bytes (chunks start at
-        // multiples of 32), or -1 if N is a multiple of 16 bytes
-        const int ragged_x = (p.N % (p.y_bf16 ? 8 : 4)) ? (p.N / 32) * 32 : -1;
-        auto store_chunk = [&](const uint32_t (&v)[32], int x, int y_row) {
+        // first column of a right edge narrower than 16 bytes, or -1 if N is a multiple of 16 bytes
+        const int ragged_col = (p.N % (p.y_bf16 ? 8 : 4)) ? p.N - p.N % (p.y_bf16 ? 8 : 4) : -1;
+        auto store_chunk = [&](const uint32_t (&v)[32], int x, int y_row, int cols) {
             // A tiled store clips at the tensor's edge in units of 16 bytes: where N is not a multiple of that,
             // it would fill the last column group up with zeros, i.e. write into the caller's bytes between
             // column N and the row stride.  That one chunk goes out with plain stores instead.
-            if (x == ragged_x) {
+            if (ragged_col >= x && ragged_col < x + cols) {
                 const int row = y_row + lane;
                 if (row < p.M) {
                     if (p.y_bf16) {
                         __nv_bfloat16* yp = reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<size_t>(row) * p.ldy + x;
-                        for (int i = 0; i < 32 && x + i < p.N; ++i) yp[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                        for (int i = 0; i < cols && x + i < p.N; ++i) yp[i] = __float2bfloat16_rn(__uint_as_float(v[i]));
                     } else {
                         float* yp = reinterpret_cast<float*>(p.y) + static_cast<size_t>(row) * p.ldy + x;
-                        for (int i = 0; i < 32 && x + i < p.N; ++i) yp[i] = __uint_as_float(v[i]);
+                        for (int i = 0; i < cols && x + i < p.N; ++i) yp[i] = __uint_as_float(v[i]);
+                    }
+                }
+                return;
+            }
+            // The 16-column chunk that closes a 240-column tile: 64 (32) contiguous bytes per row, written with
+            // 16-byte stores (y and its row stride are 16-byte aligned -- the tensor map demands it -- and chunks
+            // start at multiples of 16 columns).  Columns from N on are dropped 16 bytes at a time; a narrower
+            // rest is the ragged chunk above.
+            if (kLastCols == 16 && cols == 16) {
+                const int row = y_row + lane;
+                if (row < p.M) {
+                    if (p.y_bf16) {
+                        uint4* yp = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(p.y) + static_cast<size_t>(row) * p.ldy + x);
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            uint32_t h[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(v[8 * u + 2 * i]), __uint_as_float(v[8 * u + 2 * i + 1]));
+                                h[i] = *reinterpret_cast<uint32_t*>(&t2);
+                            }
+                            if (x + 8 * u + 8 <= p.N) yp[u] = make_uint4(h[0], h[1], h[2], h[3]);
+                        }
+                    } else {
+                        uint4* yp = reinterpret_cast<uint4*>(reinterpret_cast<float*>(p.y) + static_cast<size_t>(row) * p.ldy + x);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+                            if (x + 4 * u + 4 <= p.N) yp[u] = make_uint4(v[4 * u], v[4 * u + 1], v[4 * u + 2], v[4 * u + 3]);
                     }
                 }
                 return;
@@ -444,7 +488,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         auto slot_of = [&](int pair, int tile) -> const float4* {
             const int k = plan_sk.slot_index(pair, tile);
             return reinterpret_cast<const float4*>(p.partial) +
-                   static_cast<size_t>(2 * (2 * pair + static_cast<int>(rank)) + k) * (kChunks * 8 * 128);
+                   static_cast<size_t>(2 * (2 * pair + static_cast<int>(rank)) + k) * C::kSlotUnits;
         };
         auto run_fixups = [&]() {
             for (int f = 0; f < n_fix && ok; ++f) {
@@ -467,14 +511,16 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 for (int c = g - fx.first_pair; c < kChunks; c += fx.P) {
                     // unit (c, u) of row r sits at float4 index (c * 8 + u) * 128 + r of a slot
                     const size_t off = static_cast<size_t>(c) * 8 * 128 + row_in_tile;
+                    const int cols = c == kChunks - 1 ? kLastCols : kChunkCols;
+                    const int nu = cols >> 2;   // 16-byte units per row of this chunk
                     float4 a4[8], b4[8];
                     const float4* s0p = slot_of(fx.first_pair, fx.tile) + off;
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) a4[u] = __ldcg(s0p + u * 128);
+                    for (int u = 0; u < 8; ++u) a4[u] = u < nu ? __ldcg(s0p + u * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
                     for (int j = 1; j < fx.P; ++j) {
                         const float4* sp = slot_of(fx.first_pair + j, fx.tile) + off;
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) b4[u] = __ldcg(sp + u * 128);
+                        for (int u = 0; u < 8; ++u) b4[u] = u < nu ? __ldcg(sp + u * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                         for (int u = 0; u < 8; ++u) {
                             a4[u].x += b4[u].x; a4[u].y += b4[u].y; a4[u].z += b4[u].z; a4[u].w += b4[u].w;
@@ -486,7 +532,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                         v[4 * u] = __float_as_uint(a4[u].x); v[4 * u + 1] = __float_as_uint(a4[u].y);
                         v[4 * u + 2] = __float_as_uint(a4[u].z); v[4 * u + 3] = __float_as_uint(a4[u].w);
                     }
-                    store_chunk(v, ni * BN + c * kChunkCols, y_row);
+                    store_chunk(v, ni * BN + c * kChunkCols, y_row, cols);
                 }
                 // all four warps have read what they need of this half
                 asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -496,6 +542,21 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 if (trace && row_in_tile == 0 && f < 2) trace[208 + f] = clock64();
             }
             n_fix = 0;
+        };
+
+        // accumulator columns [c * 32, c * 32 + cols) of this warp's rows -> v (waits for the data)
+        auto load_chunk = [&](uint32_t acc_t, int c, uint32_t (&v)[32]) -> int {
+            if (kLastCols == 16 && c == kChunks - 1) {
+                uint32_t h[16];
+                tmem_ld_32x16(acc_t + c * kChunkCols, h);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 16; ++i) { v[i] = h[i]; v[16 + i] = 0; }
+                return 16;
+            }
+            tmem_ld_32x32(acc_t + c * kChunkCols, v);
+            tmem_ld_wait();
+            return kChunkCols;
         };
 
         while (ok && r.next(sg)) {
@@ -513,17 +574,17 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 // publish this piece: partial accumulator -> workspace slot (one 512-byte line per warp store)
                 const int k = plan_sk.slot_index(g, sg.tile);
                 float4* slot = reinterpret_cast<float4*>(p.partial) +
-                               static_cast<size_t>(2 * blockIdx.x + k) * (kChunks * 8 * 128) + row_in_tile;
+                               static_cast<size_t>(2 * blockIdx.x + k) * C::kSlotUnits + row_in_tile;
 #pragma unroll 1
                 for (int c = 0; c < kChunks; ++c) {
                     uint32_t v[32];
-                    tmem_ld_32x32(acc_t + c * kChunkCols, v);
-                    tmem_ld_wait();
+                    const int nu = load_chunk(acc_t, c, v) >> 2;
 #pragma unroll
                     for (int u = 0; u < 8; ++u)
-                        __stcg(slot + (c * 8 + u) * 128,
-                               make_float4(__uint_as_float(v[4 * u]), __uint_as_float(v[4 * u + 1]),
-                                           __uint_as_float(v[4 * u + 2]), __uint_as_float(v[4 * u + 3])));
+                        if (u < nu)
+                            __stcg(slot + (c * 8 + u) * 128,
+                                   make_float4(__uint_as_float(v[4 * u]), __uint_as_float(v[4 * u + 1]),
+                                               __uint_as_float(v[4 * u + 2]), __uint_as_float(v[4 * u + 3])));
                 }
                 tc_fence_before_sync();
                 __syncwarp();
@@ -539,15 +600,14 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
 #pragma unroll 1
                 for (int c = 0; c < kChunks; ++c) {
                     uint32_t v[32];
-                    tmem_ld_32x32(acc_t + c * kChunkCols, v);
-                    tmem_ld_wait();
+                    const int cols = load_chunk(acc_t, c, v);
                     if (c == kChunks - 1) {
                         // the accumulator has been read completely: hand it back before the stores drain
                         tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(leader_acc_empty0 + buf * 8);
                     }
-                    store_chunk(v, ni * BN + c * kChunkCols, y_row);
+                    store_chunk(v, ni * BN + c * kChunkCols, y_row, cols);
                 }
             }
             if (trace && row_in_tile == 0 && seg_it < 8) trace[193 + 2 * seg_it] = clock64();
@@ -579,12 +639,12 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     if (threadIdx.x == 0 && abort_flag_s) atomicExch(p.status, static_cast<int>(PRQ_ERR_TIMEOUT));
 }
 
-}  // namespace
-
-int prefill_pair_max_clusters() {
+template <int BN>
+int max_clusters_bn() {
+    constexpr int kSmemBytes = PCfg<BN>::kSmemBytes;
     static int cached = -1;
     if (cached >= 0) return cached;
-    if (cudaFuncSetAttribute(prefill_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return 0;
+    if (cudaFuncSetAttribute(prefill_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2);
     cfg.blockDim = dim3(kThreads);
@@ -597,17 +657,19 @@ int prefill_pair_max_clusters() {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, prefill_pair_kernel, &cfg) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveClusters(&n, prefill_pair_kernel<BN>, &cfg) != cudaSuccess) return 0;
     cached = n;
     return n;
 }
 
-cudaError_t launch_prefill_pair(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
-                                const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
-                                int pairs, cudaStream_t stream) {
+template <int BN>
+cudaError_t launch_bn(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
+                      const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
+                      int pairs, cudaStream_t stream) {
+    constexpr int kSmemBytes = PCfg<BN>::kSmemBytes;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(prefill_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -625,7 +687,21 @@ cudaError_t launch_prefill_pair(const CUtensorMap& tm_act, const CUtensorMap& tm
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel, tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p);
+    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BN>, tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p);
+}
+
+}  // namespace
+
+int prefill_pair_max_clusters(int bn) {
+    return bn == kPrefillTileWide ? max_clusters_bn<kPrefillTileWide>() : max_clusters_bn<kPrefillTileN>();
+}
+
+cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
+                                const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
+                                int pairs, cudaStream_t stream) {
+    if (bn == kPrefillTileWide) return launch_bn<kPrefillTileWide>(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+    if (bn == kPrefillTileN) return launch_bn<kPrefillTileN>(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace prq

@@ -131,18 +131,20 @@ cudaError_t launch_decode(int bn, const CUtensorMap& tm_act, const CUtensorMap& 
 // How many clusters of `splits` CTAs of the decode kernel can be resident at once on the current device.
 int decode_max_active_clusters(int bn, int splits);
 
-// Prefill kernel (M > 128): 256 x 224 output tiles, each computed by two CTAs of a cluster.
+// Prefill kernel (M > 128): 256 x 224 or 256 x 240 output tiles, each computed by two CTAs of a cluster.
 constexpr int kPrefillTileN = 224;
+constexpr int kPrefillTileWide = 240;
+constexpr size_t kPrefillSlotBytes = 128 * 256 * sizeof(float);   // workspace per partial tile of one CTA
 struct PrefillParams {
     int M, N, K, k_tail;
-    int m_tiles, n_tiles;       // 256-row x 224-column tiles
+    int m_tiles, n_tiles;       // 256-row x 224- (240-) column tiles
     int sk_tiles, whole_tiles;  // tiles 0 .. sk_tiles-1 are split stream-K over all pairs, then pair g
                                 // computes the whole tiles sk_tiles + wave * pairs + g, wave < whole_tiles
     int sk_aligned, sk_base, sk_extra;  // how the stream-K tiles are cut (see SkPlan in the kernel)
     int act_groups, w_groups;   // 128-row scale groups per stage in act_sf / w_sf
     const uint8_t* act_sf;
     const uint8_t* w_sf;
-    float* partial;             // two 128 x 224 fp32 slots per CTA
+    float* partial;             // two fp32 slots (128 rows x tile width, rounded up to 32 columns) per CTA
     int* flags;                 // "arrived" counter per 128-row half of a tile (index 2 * tile + half) ...
     int flag_stride;            // ... and, this many ints further, its "finished" counter; all zero between launches
     void* y;                    // output matrix and its row stride in elements: used only for the column group at
@@ -152,13 +154,13 @@ struct PrefillParams {
     long long* trace;
     int dbg;
 };
-// `tm_w` has boxes of 112 rows; `tm_sfa` / `tm_sfw` view the scale bytes as rows of 256 bytes with boxes of
+// `bn` = tile width (kPrefillTileN or kPrefillTileWide).  `tm_w` has boxes of bn / 2 rows; `tm_sfa` / `tm_sfw` view the scale bytes as rows of 256 bytes with boxes of
 // 4 / 8 rows (one / two 128-row groups); `tm_y` has 32 x 32 boxes.
-cudaError_t launch_prefill_pair(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
+cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
                                 const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
                                 int pairs, cudaStream_t stream);
 // How many pairs of the pair kernel can be resident at once on the current device.
-int prefill_pair_max_clusters();
+int prefill_pair_max_clusters(int bn);
 
 // Benchmark utility: `grid` CTAs each issuing n_mma block-scaled FP4 MMAs (128 x 256 x 64) from shared memory.
 cudaError_t launch_mxf4_peak_probe(int n_mma, int grid, int* status, cudaStream_t stream);

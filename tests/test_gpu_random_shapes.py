@@ -117,3 +117,39 @@ def test_random_grouped_shapes_against_oracle(prq, oracle, seed):
             slack = np.abs(y_ref).max() * 2.0 ** -7 if dt == prq.BF16 else 0.0
             assert np.abs(got - y_ref).max() <= prq_ref.tolerance(y_ref) + slack, what
         w.free()
+
+
+@pytest.mark.parametrize("bn", [224, 240])
+@pytest.mark.parametrize("seed", [31, 32])
+def test_prefill_tile_widths_against_oracle(prq, oracle, monkeypatch, bn, seed):
+    """Both tile widths of the CTA-pair prefill kernel on shapes whose last column tile is ragged in every way
+    (narrower than the closing 16-column chunk, inside it, an odd number of 16-byte groups, not a multiple of
+    16 bytes), with fp32 and bf16 outputs in padded rows."""
+    monkeypatch.setenv("PRQ_PAIR_BN", str(bn))
+    rng = np.random.default_rng(seed)
+    for case in range(8):
+        K = int(rng.integers(2, 24)) * 32
+        k = int(rng.integers(0, min(K // 32, 4) + 1)) * 32
+        N = int(rng.choice([100, 224, 228, 232, 236, 240, 250, 256, 464, 472, 476, 480, 490, 500, 730]))
+        M = int(rng.choice([129, 256, 300, 520, 700, 1100]))
+        dt = prq.F32 if rng.random() < 0.5 else prq.BF16
+        if dt == prq.BF16 and N % 2:
+            N += 1
+        what = f"bn {bn} seed {seed} case {case}: N={N} K={K} k={k} M={M} dt={dt}"
+        L = synth.layer(9, N, K, M, T_cal=32, tag=int(rng.integers(0, 10000)))
+        amax = oracle.channel_amax(L["zcal"])
+        w = prq.prepare_weights(L["W"], amax, 0.5, k)
+        o = oracle.prepare(L["W"], amax, 0.5, k)
+        codes, srow, sf = prq.quantize_act(w, dev_bf16(L["x"]), prq.ACT_SCALE_PERM, row_scales=True)
+        oc, osc = oracle.quantize_act(L["x"], o["perm"], o["inv_s"])
+        ca, sa = oracle.augment_act(oc, osc, k)
+        y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+        n_pad = (N + 7) // 8 * 8 + 8 * int(rng.integers(0, 3))
+        full = torch.full((M, n_pad), 7.0, dtype=torch.float32 if dt == prq.F32 else torch.bfloat16, device="cuda")
+        y = prq.linear(w, codes, sf, M, dt, out=full[:, :N])
+        assert prq.last_device_status() == 0, what
+        assert bool((full[:, N:] == 7.0).all()), what
+        got = y.float().cpu().numpy().astype(np.float64)
+        slack = np.abs(y_ref).max() * 2.0 ** -7 if dt == prq.BF16 else 0.0
+        assert np.abs(got - y_ref).max() <= prq_ref.tolerance(y_ref) + slack, what
+        w.free()
