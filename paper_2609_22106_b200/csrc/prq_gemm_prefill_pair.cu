@@ -20,7 +20,7 @@
 // their whole tiles; what is exposed at the end of every pair is one plain tile epilogue, the same
 // for all of them.
 //
-// Roles (10 warps per CTA):
+// Roles (6 warps per CTA):
 //   warp 0    TMA producer (both CTAs): per 256-element reduction stage its own activation tile, its
 //             half of the weight tile, the scale bytes of its activation rows and of all 224 weight rows;
 //             all four copies of both CTAs are counted on the LEADER's "full" mbarrier;
@@ -28,12 +28,9 @@
 //             copies from its own shared memory), up to four K = 64 MMAs, one commit that arrives on
 //             the "empty" barrier of both CTAs.  In the other CTA this warp only allocates and frees
 //             tensor memory;
-//   warps 2-9 epilogue (both CTAs): tcgen05.ld of their 32-lane quarter of the CTA's 128 accumulator
+//   warps 2-5 epilogue (both CTAs): tcgen05.ld of their 32-lane quarter of the CTA's 128 accumulator
 //             rows, 32 columns at a time, into swizzled shared staging, then one TMA store per warp and
-//             chunk (rows and columns outside M x N are clipped by the tensor map).  Two warps share a
-//             lane quarter and take alternate chunks: a chunk is a serial chain (load from tensor memory,
-//             stage, fence, store) and the last tile's epilogue is exposed at the end of the kernel, so
-//             halving the chain per warp shortens the kernel.
+//             chunk (rows and columns outside M x N are clipped by the tensor map).
 //
 // The activation tail is re-read, not copied: stages past the K main columns load the activation tile
 // from column K - k and the weight tile from column K onwards (Kernel design paragraph).
@@ -49,14 +46,12 @@
 namespace prq {
 namespace {
 
-constexpr int kEpiWarps = 8;                      // two per tensor-memory lane quarter, alternating chunks
-constexpr int kPerQuarter = kEpiWarps / 4;        // warps per lane quarter
-constexpr int kThreads = (2 + kEpiWarps) * 32;
+constexpr int kThreads = 192;
 constexpr int kPTile = 128 * 128;                 // activation tile bytes (128 rows x 256 codes)
 constexpr int kSfp = kSfGroupBytes;               // 1 group of 128 activation rows
 constexpr int kSfq = 2 * kSfGroupBytes;           // 2 groups (128 + up to 128 weight rows)
 constexpr int kStages = 5;
-constexpr int kStagingPerWarp = 4096;             // one 32-row x 128-byte chunk per epilogue warp
+constexpr int kStagingPerWarp = 2 * 4096;         // two 32-row x 128-byte chunks per epilogue warp
 constexpr int kTmemCols = 512;
 constexpr int kSfSetCols = 24;                    // 8 activation + 16 weight scale columns
 constexpr int kChunkCols = 32;                    // accumulator columns per epilogue chunk
@@ -69,7 +64,7 @@ struct PCfg {
     static constexpr int kHalfN = BN / 2;                    // weight rows each CTA of the pair loads
     static constexpr int kQTile = kHalfN * 128;              // half weight tile bytes
     static constexpr int kStageBytes = kPTile + kQTile + kSfp + kSfq;  // 33792 / 34816
-    static constexpr int kSmemBytes = kStages * kStageBytes + kEpiWarps * kStagingPerWarp + 1024;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 4 * kStagingPerWarp + 1024;
     static constexpr int kSfCol = 2 * BN;                    // scale columns start behind the two accumulators
     static constexpr int kChunks = (BN + kChunkCols - 1) / kChunkCols;   // 7, or 7 and a 16-column one
     static constexpr int kLastCols = BN - (kChunks - 1) * kChunkCols;    // 32 or 16
@@ -248,7 +243,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         for (int i = 0; i < kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bar_acc_full[i]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[i]), 2 * kEpiWarps);   // the epilogue warps of both CTAs
+            mbar_init(smem_u32(&bar_acc_empty[i]), 8);   // four epilogue warps of each CTA
         }
         abort_flag_s = 0;
         fence_mbar_init();
@@ -390,16 +385,15 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..9, both CTAs)
+        // ------------------------------------------------------------ epilogue (warps 2..5, both CTAs)
         grid_dependency_wait();
         const int q4 = warp & 3;                 // tensor-memory lane quarter of this warp
-        const int h = (warp - 2) >> 2;           // which of the quarter's two warps: it takes every other chunk
         const int row_in_tile = q4 * 32 + lane;  // row of this CTA's 128-row half
         const uint32_t stage_smem = staging_base + (warp - 2) * kStagingPerWarp;
         const uint32_t leader_acc_empty0 = cluster_map(smem_u32(&bar_acc_empty[0]), 0);
         Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G};
         Segment sg;
-        int seg_it = 0;
+        int seg_it = 0, store_it = 0;
         bool ok = true;
 
         // 32 accumulator columns of this warp's 32 rows -> y: swizzled shared staging, then one TMA store
@@ -451,9 +445,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 }
                 return;
             }
-            const uint32_t sbuf = stage_smem;
-            // the previous store of this warp has finished reading the buffer
-            if (lane == 0) bulk_wait_read<0>();
+            const uint32_t sbuf = stage_smem + (store_it & 1) * 4096;
+            // the store issued two chunks ago has finished reading this buffer
+            if (lane == 0) bulk_wait_read<1>();
             __syncwarp();
             if (!p.y_bf16) {
                 // 128-byte staging rows, 16-byte unit index ^= row % 8
@@ -478,6 +472,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 tma_store_2d(&tm_y, sbuf, x, y_row);
                 bulk_commit();
             }
+            ++store_it;
         };
 
         // A stream-K tile is finished in two steps.  Publish: every pair that computed a piece of it writes
@@ -513,7 +508,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 __threadfence();
                 const int mi = fx.tile % p.m_tiles, ni = fx.tile / p.m_tiles;
                 const int y_row = mi * 256 + static_cast<int>(rank) * 128 + q4 * 32;
-                for (int c = g - fx.first_pair + h * fx.P; c < kChunks; c += kPerQuarter * fx.P) {
+                for (int c = g - fx.first_pair; c < kChunks; c += fx.P) {
                     // unit (c, u) of row r sits at float4 index (c * 8 + u) * 128 + r of a slot
                     const size_t off = static_cast<size_t>(c) * 8 * 128 + row_in_tile;
                     const int cols = c == kChunks - 1 ? kLastCols : kChunkCols;
@@ -539,12 +534,12 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                     }
                     store_chunk(v, ni * BN + c * kChunkCols, y_row, cols);
                 }
-                // all epilogue warps have read what they need of this half
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-                if (row_in_tile == 0 && h == 0) {
+                // all four warps have read what they need of this half
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (row_in_tile == 0) {
                     if (atomicAdd(finished, 1) == fx.P - 1) { *finished = 0; *arrived = 0; }
                 }
-                if (trace && row_in_tile == 0 && h == 0 && f < 2) trace[208 + f] = clock64();
+                if (trace && row_in_tile == 0 && f < 2) trace[208 + f] = clock64();
             }
             n_fix = 0;
         };
@@ -581,7 +576,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 float4* slot = reinterpret_cast<float4*>(p.partial) +
                                static_cast<size_t>(2 * blockIdx.x + k) * C::kSlotUnits + row_in_tile;
 #pragma unroll 1
-                for (int c = h; c < kChunks; c += kPerQuarter) {
+                for (int c = 0; c < kChunks; ++c) {
                     uint32_t v[32];
                     const int nu = load_chunk(acc_t, c, v) >> 2;
 #pragma unroll
@@ -595,19 +590,19 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(leader_acc_empty0 + buf * 8);
                 __threadfence();
-                asm volatile("bar.sync 1, %0;" ::"n"(kEpiWarps * 32) : "memory");
-                if (row_in_tile == 0 && h == 0) atomicAdd(p.flags + 2 * sg.tile + rank, 1);
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (row_in_tile == 0) atomicAdd(p.flags + 2 * sg.tile + rank, 1);
                 int first, P;
                 plan_sk.participants(sg.tile, g, first, P);
                 fix[n_fix++] = Fixup{sg.tile, first, P};
             } else {
                 const int y_row = mi * 256 + static_cast<int>(rank) * 128 + q4 * 32;
 #pragma unroll 1
-                for (int c = h; c < kChunks; c += kPerQuarter) {
+                for (int c = 0; c < kChunks; ++c) {
                     uint32_t v[32];
                     const int cols = load_chunk(acc_t, c, v);
-                    if (c + kPerQuarter >= kChunks) {
-                        // this warp has read its part of the accumulator: hand it back before the stores drain
+                    if (c == kChunks - 1) {
+                        // the accumulator has been read completely: hand it back before the stores drain
                         tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster(leader_acc_empty0 + buf * 8);
