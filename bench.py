@@ -29,7 +29,7 @@ N_OUT, K_IN, K_TAIL, M_TOK = 2560, 9728, 256, 2048
 FP4_OVER_BF16 = 4.0  # nominal dense tensor ratio (9 vs 2.25 PFLOP/s)
 # DRAM bytes of one prefill GEMM launch at this workload from the ncu capture summarised in
 # profiles/prefill_pair_M2048.txt (dram__bytes_read.sum + dram__bytes_write.sum; the outputs were still in L2).
-NCU_PREFILL_DRAM_BYTES = 24.39e6 + 1.24e6
+NCU_PREFILL_DRAM_BYTES = 24.34e6 + 2.18e6
 
 
 def peaks():
@@ -584,7 +584,7 @@ def main():
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": fp4_peak, "unit": "TFLOP/s",
                      "frac": achieved / fp4_peak, "frac_of_sustained": achieved / (pk["bf16_tflops_sustained"] * FP4_OVER_BF16),
                      "traffic": NCU_PREFILL_DRAM_BYTES, "algorithmic_bytes": gemm_bytes(M_TOK, K_TAIL),
-                     "kernel": "prefill_pair_kernel (CTA pairs, 256x224 tiles, whole tiles + stream-K pieces)", "launch_us": gemm_us,
+                     "kernel": "prefill_pair_kernel<240> (CTA pairs, 256x240 tiles, whole tiles + stream-K pieces)", "launch_us": gemm_us,
                      "peak_source": f"4 x bf16 burst, of {pk['source']}",
                      "frac_of_measured_mxf4_probe": achieved / mxf4_probe["burst_1.5ms"],
                      "frac_of_nominal_9pf": achieved / 9000.0},
