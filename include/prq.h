@@ -109,6 +109,19 @@ typedef struct prq_prep_opts {
 prq_status prq_prepare_weights_opts(const uint16_t *W, int n_experts, int N, int K, const float *act_amax,
                                     float alpha, int k_tail, const prq_prep_opts *opts, prq_weights **out);
 
+/* prq_prepare_weights_opts for weights that already sit in DEVICE memory (Algorithm 1 steps 3-7 and 11 with
+ * the heavy steps as kernels on the current device; the K channel scales and the ranking of the K column
+ * errors stay on the host).  The handle is bit-for-bit the one prq_prepare_weights_opts builds from a host
+ * copy of the same W.
+ *   W_device  device, n_experts x N x K bf16 row-major (read only; not kept)
+ *   act_amax  HOST, n_experts x K fp32          opts  may be NULL
+ *   stream    the kernels and copies run there; the call synchronises it before it returns
+ * Allocates temporaries on the device (codes, scale bytes and a few arrays of K elements) and frees them.
+ * Errors as prq_prepare_weights; a NaN or an infinity in W * s gives NONFINITE. */
+prq_status prq_prepare_weights_device(const uint16_t *W_device, int n_experts, int N, int K, const float *act_amax,
+                                      float alpha, int k_tail, const prq_prep_opts *opts, prq_stream_t stream,
+                                      prq_weights **out);
+
 /* The same per-alpha pipeline as prq_prepare_weights, host buffers in and out, no device involved
  * (offline tooling, export, checks on machines without a GPU).  One layer.
  *   codes   host out, N x (K+k)/2    scales  host out, N x (K+k)/32    perm  host out, K int32

@@ -22,7 +22,7 @@ FIELD_CODES, FIELD_SCALES, FIELD_PERM, FIELD_TOPK, FIELD_S, FIELD_INV_S, FIELD_C
 BUF_CODES, BUF_SCALES_ROW, BUF_SCALES_SF = range(3)
 
 EXPORTS = [
-    "prq_prepare_weights", "prq_prepare_weights_opts", "prq_prepare_weights_host", "prq_prepare_weights_host_opts", "prq_prepare_weights_search", "prq_weights_free",
+    "prq_prepare_weights", "prq_prepare_weights_opts", "prq_prepare_weights_device", "prq_prepare_weights_host", "prq_prepare_weights_host_opts", "prq_prepare_weights_search", "prq_weights_free",
     "prq_weights_clone", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
     "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_multi", "prq_quantize_act_multi",
     "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
@@ -51,6 +51,7 @@ def lib():
         L.prq_prepare_weights_host.argtypes = [vp, ci, ci, vp, cf, ci, vp, vp, vp, vp, vp, vp]
         L.prq_prepare_weights_opts.argtypes = [vp, ci, ci, ci, vp, cf, ci, vp, ctypes.POINTER(vp)]
         L.prq_prepare_weights_host_opts.argtypes = [vp, ci, ci, vp, cf, ci, vp, vp, vp, vp, vp, vp, vp]
+        L.prq_prepare_weights_device.argtypes = [vp, ci, ci, ci, vp, cf, ci, vp, vp, ctypes.POINTER(vp)]
         L.prq_prepare_weights_search.argtypes = [vp, ci, ci, vp, ci, vp, ci, ci, ctypes.POINTER(vp),
                                                  ctypes.POINTER(cf), vp]
         L.prq_weights_clone.argtypes = [vp, ctypes.POINTER(vp)]
@@ -176,6 +177,26 @@ def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_ta
     _check(lib().prq_prepare_weights_opts(_np_ptr(W), E, N, K, _np_ptr(amax), alpha, k_tail,
                                           ctypes.cast(ctypes.pointer(o), ctypes.c_void_p), ctypes.byref(h)),
            "prq_prepare_weights_opts")
+    return Weights(h)
+
+
+def prepare_weights_device(W, act_amax: np.ndarray, alpha: float, k_tail: int, scale_search: bool = False,
+                           stream=None) -> Weights:
+    """W: torch CUDA tensor, bf16 (or its uint16 / int16 bit pattern), (N, K) or (E, N, K), contiguous.  The prep
+    runs on the GPU; the handle equals the one prepare_weights builds from a host copy."""
+    assert W.is_cuda and W.is_contiguous() and W.element_size() == 2
+    amax = np.ascontiguousarray(act_amax, np.float32)
+    shape = tuple(W.shape)
+    if len(shape) == 2:
+        shape = (1,) + shape
+        amax = amax[None]
+    E, N, K = shape
+    h = ctypes.c_void_p()
+    o = _opts(scale_search)
+    _check(lib().prq_prepare_weights_device(W.data_ptr(), E, N, K, _np_ptr(amax), alpha, k_tail,
+                                            ctypes.cast(ctypes.pointer(o), ctypes.c_void_p), _stream_ptr(stream),
+                                            ctypes.byref(h)),
+           "prq_prepare_weights_device")
     return Weights(h)
 
 

@@ -329,7 +329,7 @@ void prq_weights_free(prq_weights* w) {
     cudaFree(w->d_sf);
     cudaFree(w->d_perm);
     cudaFree(w->d_inv_s_perm);
-    for (int a = 0; a < 3; ++a) cudaFree(w->d_sf_alt[a]);
+    for (uint8_t* p : w->d_sf_alt) cudaFree(p);
     if (w->device >= 0 && w->device != cur) cudaSetDevice(cur);
     delete w;
 }
@@ -339,8 +339,22 @@ prq_status prq_prepare_weights(const uint16_t* W, int n_experts, int N, int K, c
     return prq_prepare_weights_opts(W, n_experts, N, K, act_amax, alpha, k_tail, nullptr, out);
 }
 
+static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_t stream, int n_experts, int N, int K,
+                                const float* act_amax, float alpha, int k_tail, const prq_prep_opts* opts, prq_weights** out);
+
 prq_status prq_prepare_weights_opts(const uint16_t* W, int n_experts, int N, int K, const float* act_amax, float alpha,
                                     int k_tail, const prq_prep_opts* opts, prq_weights** out) {
+    return create_handle(W, false, nullptr, n_experts, N, K, act_amax, alpha, k_tail, opts, out);
+}
+
+prq_status prq_prepare_weights_device(const uint16_t* W_device, int n_experts, int N, int K, const float* act_amax,
+                                      float alpha, int k_tail, const prq_prep_opts* opts, prq_stream_t stream,
+                                      prq_weights** out) {
+    return create_handle(W_device, true, stream, n_experts, N, K, act_amax, alpha, k_tail, opts, out);
+}
+
+static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_t stream, int n_experts, int N, int K,
+                                const float* act_amax, float alpha, int k_tail, const prq_prep_opts* opts, prq_weights** out) {
     if (opts && opts->struct_size < sizeof(prq_prep_opts)) return PRQ_ERR_INVALID_ARG;
     const bool scale_search = opts && opts->weight_scale_search != 0;
     if (!W || !act_amax || !out) return PRQ_ERR_INVALID_ARG;
@@ -381,7 +395,9 @@ prq_status prq_prepare_weights_opts(const uint16_t* W, int n_experts, int N, int
         }
         PrepResult r;
         for (size_t e = 0; e < E; ++e) {
-            st = prepare_layer(W + e * N * K, N, K, act_amax + e * K, alpha, k_tail, r, scale_search);
+            st = w_on_device ? prepare_layer_device(W + e * N * K, N, K, act_amax + e * K, alpha, k_tail, r, scale_search,
+                                                     static_cast<cudaStream_t>(stream))
+                             : prepare_layer(W + e * N * K, N, K, act_amax + e * K, alpha, k_tail, r, scale_search);
             if (st != PRQ_OK) { delete w; return st; }
             std::memcpy(&w->h_codes[e * N * Ka / 2], r.codes.data(), r.codes.size());
             std::memcpy(&w->h_scales[e * N * Ka / kBlock], r.scales.data(), r.scales.size());

@@ -6,6 +6,7 @@
 #include <vector>
 
 #include <cuda.h>
+#include <cuda_runtime.h>
 
 #include "prq.h"
 
@@ -57,6 +58,17 @@ struct PrepResult {
 // two neighbours (the "E8M0-W" variant of the ablation study); ranking and permutation are unaffected.
 prq_status prepare_layer(const uint16_t* W, int N, int K, const float* amax, float alpha, int k_tail,
                          PrepResult& out, bool scale_search = false);
+// The pieces of it that stay on the host when the rest runs on the GPU:
+// s_j = max(amax_j, 1e-5)^alpha and its reciprocal (FP64, stored fp32; PRQ_ERR_NONFINITE on a bad amax) ...
+prq_status channel_scales(const float* amax, int K, float alpha, std::vector<float>& s, std::vector<float>& inv_s);
+// ... and the error-ranked top-k with its permutation [unselected ascending | selected ascending]
+// (ties: the lower channel index ranks first).
+void rank_and_permute(const std::vector<double>& col_err, int K, int k_tail, std::vector<int32_t>& perm);
+// The same result computed on the current device from a DEVICE copy of W (column errors, permuted
+// quantisation, residual and packing as kernels; scales and ranking on the host in between).  Allocates its
+// temporaries, runs on `stream` and synchronises it.
+prq_status prepare_layer_device(const uint16_t* W_dev, int N, int K, const float* amax, float alpha, int k_tail,
+                                PrepResult& out, bool scale_search, cudaStream_t stream);
 
 }  // namespace prq
 

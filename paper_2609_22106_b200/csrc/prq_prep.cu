@@ -141,23 +141,40 @@ double scale_power(double a, float alpha) {
 
 }  // namespace
 
+prq_status channel_scales(const float* amax, int K, float alpha, std::vector<float>& s, std::vector<float>& inv_s) {
+    s.resize(K);
+    inv_s.resize(K);
+    for (int j = 0; j < K; ++j) {
+        if (!std::isfinite(amax[j])) return PRQ_ERR_NONFINITE;
+        double a = std::max(static_cast<double>(amax[j]), 1e-5);
+        s[j] = static_cast<float>(scale_power(a, alpha));
+        inv_s[j] = static_cast<float>(1.0 / static_cast<double>(s[j]));
+    }
+    return PRQ_OK;
+}
+
+void rank_and_permute(const std::vector<double>& col_err, int K, int k_tail, std::vector<int32_t>& perm) {
+    perm.resize(K);
+    std::vector<int32_t> order(K);
+    for (int j = 0; j < K; ++j) order[j] = j;
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return col_err[a] > col_err[b]; });
+    std::vector<uint8_t> sel(K, 0);
+    for (int i = 0; i < k_tail; ++i) sel[order[i]] = 1;
+    int head = 0, tail = K - k_tail;
+    for (int j = 0; j < K; ++j) {
+        if (sel[j]) perm[tail++] = j;
+        else perm[head++] = j;
+    }
+}
+
 prq_status prepare_layer(const uint16_t* W, int N, int K, const float* amax, float alpha, int k_tail,
                          PrepResult& out, bool scale_search) {
     const long Ka = static_cast<long>(K) + k_tail;
     const int nblk = K / kBlock;
-    out.s.resize(K);
-    out.inv_s.resize(K);
     out.col_err.assign(K, 0.0);
-    out.perm.resize(K);
     out.codes.assign(static_cast<size_t>(N) * Ka / 2, 0);
     out.scales.assign(static_cast<size_t>(N) * Ka / kBlock, 0);
-
-    for (int j = 0; j < K; ++j) {
-        if (!std::isfinite(amax[j])) return PRQ_ERR_NONFINITE;
-        double a = std::max(static_cast<double>(amax[j]), 1e-5);
-        out.s[j] = static_cast<float>(scale_power(a, alpha));
-        out.inv_s[j] = static_cast<float>(1.0 / static_cast<double>(out.s[j]));
-    }
+    if (channel_scales(amax, K, alpha, out.s, out.inv_s) != PRQ_OK) return PRQ_ERR_NONFINITE;
 
     // scaled weight, fp32 (one rounding of the exact product)
     std::vector<float> W0(static_cast<size_t>(N) * K);
@@ -190,19 +207,7 @@ prq_status prepare_layer(const uint16_t* W, int N, int K, const float* amax, flo
     });
 
     // error-ranked top-k and the permutation
-    std::vector<int32_t> order(K);
-    for (int j = 0; j < K; ++j) order[j] = j;
-    std::stable_sort(order.begin(), order.end(),
-                     [&](int32_t a, int32_t b) { return out.col_err[a] > out.col_err[b]; });
-    std::vector<uint8_t> sel(K, 0);
-    for (int i = 0; i < k_tail; ++i) sel[order[i]] = 1;
-    {
-        int head = 0, tail = K - k_tail;
-        for (int j = 0; j < K; ++j) {
-            if (sel[j]) out.perm[tail++] = j;
-            else out.perm[head++] = j;
-        }
-    }
+    rank_and_permute(out.col_err, K, k_tail, out.perm);
 
     // permuted quantisation, residual and its quantisation, packed export
     const int tail_blk0 = (K - k_tail) / kBlock;

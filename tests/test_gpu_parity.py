@@ -481,3 +481,58 @@ def test_multi_layer_launches_match_single_layer_calls(prq, oracle, M):
         prq.quantize_act_multi([ws[0], wb], x, prq.ACT_SCALE_PERM, out=acts[:2])
     for w in ws + [wb]:
         w.free()
+
+
+@pytest.mark.parametrize("N,K,k,alpha,search", [
+    (256, 256, 32, 0.5, False),      # the tiny configuration's shape
+    (100, 96, 0, 0.0, False),        # k = 0, alpha = 0: plain MXFP4 of W
+    (132, 1024, 1024, 1.0, False),   # every channel in the tail
+    (512, 2048, 128, 0.5, True),     # weight-side block-scale search
+    (300, 640, 64, 0.3, True),       # an alpha off the closed-form grid (pow), ragged N
+])
+def test_device_prep_is_bit_exact(prq, oracle, N, K, k, alpha, search):
+    """prq_prepare_weights_device (Algorithm 1 steps 3-7 and 11 as kernels on a device copy of W): every field of
+    the handle equals the oracle's, bit for bit -- scales s and 1/s, the FP64 column errors, the permutation,
+    codes and scale bytes of [Q(W D P) | Q(R)] -- and the handle runs the product like a host-prepared one."""
+    L = synth.layer(3, N, K, 40, T_cal=32, tag=N + K + k)
+    amax = oracle.channel_amax(L["zcal"])
+    amax[3] = 0.0                                     # a dead channel takes the 1e-5 floor
+    Wd = torch.from_numpy(L["W"].view(np.int16)).cuda()
+    w = prq.prepare_weights_device(Wd, amax, alpha, k, scale_search=search)
+    o = oracle.prepare(L["W"], amax, float(np.float32(alpha)), k, scale_search=search)
+    assert np.array_equal(w.get(prq.FIELD_S), o["s"])
+    assert np.array_equal(w.get(prq.FIELD_INV_S), o["inv_s"])
+    assert np.array_equal(w.get(prq.FIELD_COL_ERR), o["col_err"])
+    assert np.array_equal(w.get(prq.FIELD_PERM), o["perm"])
+    assert np.array_equal(w.get(prq.FIELD_TOPK), o["topk"])
+    assert np.array_equal(w.get(prq.FIELD_SCALES), o["wscales"])
+    assert np.array_equal(w.get(prq.FIELD_CODES), o["wcodes"])
+    x = to_dev_bf16(L["x"])
+    codes, _, sf = prq.quantize_act(w, x, prq.ACT_SCALE_PERM)
+    y = prq.linear(w, codes, sf, 40).cpu().numpy().astype(np.float64)
+    oc, osc = oracle.quantize_act(L["x"], o["perm"], o["inv_s"])
+    ca, sa = oracle.augment_act(oc, osc, k)
+    y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+    assert np.abs(y - y_ref).max() <= prq_ref.tolerance(y_ref)
+    assert prq.last_device_status() == 0
+    w.free()
+
+
+def test_device_prep_experts_and_errors(prq, oracle):
+    """Stacked experts through the device prep equal the host prep expert by expert; a non-finite weight is
+    reported, not encoded."""
+    E, N, K, k = 3, 64, 128, 32
+    Ws = np.stack([synth.weights(40 + e, N, K) for e in range(E)])
+    amax = np.stack([np.abs(np.random.default_rng(50 + e).standard_normal(K)).astype(np.float32) + 0.05 for e in range(E)])
+    wd = prq.prepare_weights_device(torch.from_numpy(Ws.view(np.int16)).cuda(), amax, 0.5, k)
+    wh = prq.prepare_weights(Ws, amax, 0.5, k)
+    for e in range(E):
+        for f in (prq.FIELD_S, prq.FIELD_INV_S, prq.FIELD_COL_ERR, prq.FIELD_PERM, prq.FIELD_SCALES, prq.FIELD_CODES):
+            assert np.array_equal(wd.get(f, e), wh.get(f, e)), (e, f)
+    wd.free()
+    wh.free()
+    bad = Ws[0].copy()
+    bad[5, 7] = 0x7F80                                # +infinity in bf16
+    with pytest.raises(prq.PrqError) as ei:
+        prq.prepare_weights_device(torch.from_numpy(bad.view(np.int16)).cuda(), amax[0], 0.5, k)
+    assert ei.value.code == 7                        # PRQ_ERR_NONFINITE
