@@ -294,6 +294,40 @@ def oracle_step(orc, x_rows, prep):
     return y
 
 
+def run_prep_workload(args, torch, prq, synth, dev):
+    """Offline prep of the block's linears (Algorithm 1 steps 3-7 and 11, alpha fixed): wall time of one whole call of
+    the device path (W already in HBM; includes the host's share -- scales, ranking, scale-byte layout -- and all
+    copies) and of the host path, and whether the two handles are identical."""
+    shapes = [("q", 4096, 2560, 128), ("k/v", 1024, 2560, 128), ("o", 2560, 4096, 128), ("gate/up", 9728, 2560, 128),
+              ("down", 2560, 9728, 256)]
+    out = []
+    for name, N, K, k in shapes:
+        W = synth.weights(5, N, K)
+        amax = np.abs(np.random.default_rng(6).standard_normal(K)).astype(np.float32) + 0.05
+        Wd = torch.from_numpy(W.view(np.int16)).to(dev)
+        row = {"linear": name, "N": N, "K": K, "k": k}
+        for search in (False, True):
+            td, th, same = [], [], True
+            for it in range(3):
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                wd = prq.prepare_weights_device(Wd, amax, 0.5, k, scale_search=search)
+                td.append(time.perf_counter() - t0)
+                t0 = time.perf_counter()
+                wh = prq.prepare_weights(W, amax, 0.5, k, scale_search=search)
+                th.append(time.perf_counter() - t0)
+                if it == 0:
+                    same = all(np.array_equal(wd.get(f), wh.get(f)) for f in range(7))
+                wd.free()
+                wh.free()
+            tag = "_scale_search" if search else ""
+            row["device_prep_ms" + tag] = 1e3 * min(td)
+            row["host_prep_ms" + tag] = 1e3 * min(th)
+            row["identical" + tag] = bool(same)
+        out.append(row)
+    return out
+
+
 def run_reference(args, rank, world):
     """--impl reference: the CPU oracle as it stands, timed on the host cores on a bounded row sample."""
     if rank != 0:
@@ -331,8 +365,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--full", action="store_true", help="also time every (M, k) of the down_proj config")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="down_proj", choices=["down_proj", "block", "moe", "stack"],
-                    help="down_proj = the headline config (default); block / moe / stack = the benchmark configurations 2, 3, 4")
+    ap.add_argument("--workload", default="down_proj", choices=["down_proj", "block", "moe", "stack", "prep"],
+                    help="down_proj = the headline config (default); block / moe / stack = the benchmark configurations 2, 3, 4; "
+                         "prep = offline weight preparation on the device against the host path")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -373,6 +408,8 @@ def main():
                 res = [run_block_workload(args, torch, prq, synth, dev, pk, 4096, n_layers=3)]
             elif args.workload == "moe":
                 res = [run_moe_workload(args, torch, prq, synth, dev, pk, T) for T in (64, 1024, 8192)]
+            elif args.workload == "prep":
+                res = run_prep_workload(args, torch, prq, synth, dev)
             else:
                 res = [run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=k, n_layers=3, tag="stack")
                        for M in (64, 4096) for k in (256, 0)]

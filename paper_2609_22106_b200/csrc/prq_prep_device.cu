@@ -58,23 +58,35 @@ __device__ __forceinline__ float e2m1_value(uint32_t code, uint32_t byte) {
 }
 
 // ---------------------------------------------------------------------------------------------- column errors
-__global__ void __launch_bounds__(128) col_err_kernel(const uint16_t* __restrict__ W, const float* __restrict__ s, int N, int K,
+constexpr int kRowsInFlight = 16;   // rows whose loads are issued before the first of them is consumed
+
+__global__ void __launch_bounds__(32) col_err_kernel(const uint16_t* __restrict__ W, const float* __restrict__ s, int N, int K,
                                                       double* __restrict__ err, int* __restrict__ nonfinite) {
-    const int warp = static_cast<int>((blockIdx.x * blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
-    if (warp >= K / kBlock) return;
-    const int j = warp * kBlock + lane;
+    // one warp per CTA: a layer has only K / 32 of these warps (80 - 304 at the paper's shapes), each bound
+    // by the latency of its own loads, so they are spread over as many SMs as there are
+    const int lane = threadIdx.x;
+    const int j = static_cast<int>(blockIdx.x) * kBlock + lane;
     const float sj = s[j];
     const uint16_t* p = W + j;
     double acc = 0.0;
     bool ok = true;
-#pragma unroll 8
-    for (int n = 0; n < N; ++n) {
-        const float v = __fmul_rn(bf16_to_float(__ldg(p + static_cast<size_t>(n) * K)), sj);
-        const uint32_t mag = __float_as_uint(v) & 0x7fffffffu;
-        ok = ok && mag < 0x7f800000u;
-        const uint32_t byte = scale_byte(__reduce_max_sync(0xffffffffu, mag));
-        const double d = static_cast<double>(v) - static_cast<double>(e2m1_value(e2m1_code(v, byte), byte));
-        acc = __dadd_rn(acc, __dmul_rn(d, d));
+    for (int n0 = 0; n0 < N; n0 += kRowsInFlight) {
+        // the warp reduction below orders memory operations, so the loads of a batch of rows are issued
+        // explicitly before any of them is used (one DRAM latency per batch instead of one per row)
+        uint16_t h[kRowsInFlight];
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) h[u] = n0 + u < N ? __ldg(p + static_cast<size_t>(n0 + u) * K) : uint16_t(0);
+#pragma unroll
+        for (int u = 0; u < kRowsInFlight; ++u) {
+            if (n0 + u < N) {
+                const float v = __fmul_rn(bf16_to_float(h[u]), sj);
+                const uint32_t mag = __float_as_uint(v) & 0x7fffffffu;
+                ok = ok && mag < 0x7f800000u;
+                const uint32_t byte = scale_byte(__reduce_max_sync(0xffffffffu, mag));
+                const double d = static_cast<double>(v) - static_cast<double>(e2m1_value(e2m1_code(v, byte), byte));
+                acc = __dadd_rn(acc, __dmul_rn(d, d));
+            }
+        }
     }
     err[j] = acc;
     if (!ok) atomicExch(nonfinite, 1);
@@ -205,7 +217,7 @@ prq_status prepare_layer_device(const uint16_t* W_dev, int N, int K, const float
     if (!ok) return PRQ_ERR_CUDA;
 
     const int nblk = K / kBlock;
-    col_err_kernel<<<(nblk + 3) / 4, 128, 0, stream>>>(W_dev, d_s.as<float>(), N, K, d_err.as<double>(), d_flag.as<int>());
+    col_err_kernel<<<nblk, 32, 0, stream>>>(W_dev, d_s.as<float>(), N, K, d_err.as<double>(), d_flag.as<int>());
     int nonfinite = 0;
     ok = cudaGetLastError() == cudaSuccess;
     ok = ok && cudaMemcpyAsync(out.col_err.data(), d_err.p, sizeof(double) * K, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
