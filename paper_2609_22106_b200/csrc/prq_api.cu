@@ -497,9 +497,14 @@ prq_status prq_prepare_weights_search(const uint16_t* W, int N, int K, const uin
     prq_weights* best = nullptr;
     double best_err = 0.0;
     prq_status st = PRQ_OK;
+    // the per-alpha pipeline runs on the device from one upload of W (bit-identical to the host path)
+    uint16_t* dW = nullptr;
+    const size_t w_bytes = sizeof(uint16_t) * static_cast<size_t>(N) * K;
+    if (cudaMalloc(&dW, w_bytes) != cudaSuccess) { cudaGetLastError(); return PRQ_ERR_OOM; }
+    if (cudaMemcpy(dW, W, w_bytes, cudaMemcpyHostToDevice) != cudaSuccess) { cudaFree(dW); return PRQ_ERR_CUDA; }
     for (int a = 0; a < n_alphas && st == PRQ_OK; ++a) {
         prq_weights* w = nullptr;
-        st = prq_prepare_weights(W, 1, N, K, amax.data(), alphas[a], k_tail, &w);
+        st = prq_prepare_weights_device(dW, 1, N, K, amax.data(), alphas[a], k_tail, nullptr, nullptr, &w);
         if (st != PRQ_OK) break;
         if (!dx) {
             ws_bytes = prq_linear_workspace_bytes(w, T);
@@ -526,7 +531,7 @@ prq_status prq_prepare_weights_search(const uint16_t* W, int N, int K, const uin
             prq_weights_free(w);
         }
     }
-    cudaFree(dx); cudaFree(dc); cudaFree(dsf); cudaFree(dy); cudaFree(dws);
+    cudaFree(dx); cudaFree(dc); cudaFree(dsf); cudaFree(dy); cudaFree(dws); cudaFree(dW);
     if (st != PRQ_OK) { prq_weights_free(best); return st; }
     *out = best;
     return PRQ_OK;
