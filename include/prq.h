@@ -152,6 +152,20 @@ void prq_weights_free(prq_weights *w);
  * Not part of the paper's method.  Free it with prq_weights_free. */
 prq_status prq_weights_clone(const prq_weights *w, prq_weights **out);
 
+/* The "offline copy" form of a prepared layer (Kernel design paragraph: the producer layers emit the k tail
+ * channels a second time, so that the activation already has K + k columns and nothing is re-read).
+ * Returns an independent handle (its own device copy, free it with prq_weights_free) that presents the same
+ * bytes [Q(W D P) | Q(R)] as a plain MXFP4 layer with K' = K + k input channels and no tail:
+ *   prq_quantize_act(view, PRQ_ACT_IDENTITY, x_wide, ...)   x_wide: M x (K + k), columns [K, K + k) a copy of
+ *                                                           columns [K - k, K) of the permuted, scaled activation
+ *   prq_linear / prq_linear_fused / prq_linear_grouped(view, ...)
+ * give bit for bit what the original handle gives on the first K columns (block alignment makes quantising
+ * the widened row equal to widening the quantised row).  Scaling and permutation are the producer's job in
+ * this form: the view's perm is the identity on K + k channels and its scales are 1.
+ * INVALID_ARG if k > 0 and K is not a multiple of 256 (the residual columns would not start on a stage of the
+ * scale-byte layout; all of the paper's shapes satisfy it). */
+prq_status prq_weights_offline_copy(const prq_weights *w, prq_weights **out);
+
 /* Shape of a handle.  Any output pointer may be NULL. */
 prq_status prq_weights_info(const prq_weights *w, int *n_experts, int *N, int *K, int *k_tail, float *alpha);
 

@@ -23,7 +23,7 @@ BUF_CODES, BUF_SCALES_ROW, BUF_SCALES_SF = range(3)
 
 EXPORTS = [
     "prq_prepare_weights", "prq_prepare_weights_opts", "prq_prepare_weights_device", "prq_prepare_weights_host", "prq_prepare_weights_host_opts", "prq_prepare_weights_search", "prq_weights_free",
-    "prq_weights_clone", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
+    "prq_weights_clone", "prq_weights_offline_copy", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
     "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_multi", "prq_quantize_act_multi",
     "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
@@ -55,6 +55,7 @@ def lib():
         L.prq_prepare_weights_search.argtypes = [vp, ci, ci, vp, ci, vp, ci, ci, ctypes.POINTER(vp),
                                                  ctypes.POINTER(cf), vp]
         L.prq_weights_clone.argtypes = [vp, ctypes.POINTER(vp)]
+        L.prq_weights_offline_copy.argtypes = [vp, ctypes.POINTER(vp)]
         L.prq_weights_free.argtypes = [vp]
         L.prq_weights_free.restype = None
         L.prq_weights_info.argtypes = [vp] + [ctypes.POINTER(ci)] * 4 + [ctypes.POINTER(cf)]
@@ -140,6 +141,13 @@ class Weights:
     def clone(self) -> "Weights":
         h = ctypes.c_void_p()
         _check(lib().prq_weights_clone(self._h, ctypes.byref(h)), "prq_weights_clone")
+        return Weights(h)
+
+    def offline_copy(self) -> "Weights":
+        """The same prepared bytes as a plain MXFP4 layer over K + k input channels (the producer emits the tail
+        channels twice; nothing is re-read)."""
+        h = ctypes.c_void_p()
+        _check(lib().prq_weights_offline_copy(self._h, ctypes.byref(h)), "prq_weights_offline_copy")
         return Weights(h)
 
     def free(self):

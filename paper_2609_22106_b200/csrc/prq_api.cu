@@ -608,6 +608,46 @@ prq_status prq_weights_clone(const prq_weights* w, prq_weights** out) {
     return PRQ_OK;
 }
 
+prq_status prq_weights_offline_copy(const prq_weights* w, prq_weights** out) {
+    if (!w || !out) return PRQ_ERR_INVALID_ARG;
+    // [Q(W D P) | Q(R)] read as a plain matrix of K + k reduction columns has the stage order of this layer's
+    // layout only if the residual stages start on a stage boundary
+    if (w->k_tail > 0 && w->K % kStageK != 0) return PRQ_ERR_INVALID_ARG;
+    prq_weights* c = nullptr;
+    prq_status st = prq_weights_clone(w, &c);
+    if (st != PRQ_OK) return st;
+    const int Kw = w->K + w->k_tail;
+    const size_t E = static_cast<size_t>(w->n_experts);
+    int cur = 0;
+    cudaGetDevice(&cur);
+    if (cur != c->device) cudaSetDevice(c->device);
+    try {
+        c->K = Kw; c->k_tail = 0; c->plan = StagePlan(Kw, 0);
+        // the activation arrives permuted, scaled and with its tail columns doubled: nothing is left to apply
+        c->h_perm.resize(E * Kw);
+        for (size_t e = 0; e < E; ++e)
+            for (int j = 0; j < Kw; ++j) c->h_perm[e * Kw + j] = j;
+        c->h_s.assign(E * Kw, 1.f);
+        c->h_inv_s.assign(E * Kw, 1.f);
+        c->h_col_err.assign(E * Kw, 0.0);
+        cudaFree(c->d_perm); c->d_perm = nullptr;
+        cudaFree(c->d_inv_s_perm); c->d_inv_s_perm = nullptr;
+        bool ok = cudaMalloc(&c->d_perm, sizeof(int32_t) * E * Kw) == cudaSuccess &&
+                  cudaMalloc(&c->d_inv_s_perm, sizeof(float) * E * Kw) == cudaSuccess;
+        if (!ok) { cudaGetLastError(); st = PRQ_ERR_OOM; }
+        ok = ok && cudaMemcpy(c->d_perm, c->h_perm.data(), sizeof(int32_t) * E * Kw, cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(c->d_inv_s_perm, c->h_inv_s.data(), sizeof(float) * E * Kw, cudaMemcpyHostToDevice) == cudaSuccess;
+        if (!ok && st == PRQ_OK) st = PRQ_ERR_CUDA;
+    } catch (const std::bad_alloc&) {
+        st = PRQ_ERR_OOM;
+    }
+    if (st == PRQ_OK) st = build_weight_maps(c);
+    if (cur != c->device) cudaSetDevice(cur);
+    if (st != PRQ_OK) { prq_weights_free(c); return st; }
+    *out = c;
+    return PRQ_OK;
+}
+
 prq_status prq_weights_info(const prq_weights* w, int* n_experts, int* N, int* K, int* k_tail, float* alpha) {
     if (!w) return PRQ_ERR_INVALID_ARG;
     if (n_experts) *n_experts = w->n_experts;

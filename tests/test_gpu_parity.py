@@ -536,3 +536,50 @@ def test_device_prep_experts_and_errors(prq, oracle):
     with pytest.raises(prq.PrqError) as ei:
         prq.prepare_weights_device(torch.from_numpy(bad.view(np.int16)).cuda(), amax[0], 0.5, k)
     assert ei.value.code == 7                        # PRQ_ERR_NONFINITE
+
+
+@pytest.mark.parametrize("N,K,k,M", [(256, 512, 64, 16), (512, 2560, 128, 300), (256, 768, 64, 1), (384, 1024, 256, 128)])
+def test_offline_copy_form_equals_the_revisit_form(prq, oracle, N, K, k, M):
+    """Kernel design paragraph, second implementation: the producer emits the k tail channels twice, the
+    activation has K + k columns, and the layer is a plain MXFP4 product over K + k.  Quantising the widened
+    row must equal widening the quantised row (block alignment), so codes, scale bytes and the product are
+    bit for bit those of the form that re-reads the tail -- and within tolerance of the oracle."""
+    L = synth.layer(4, N, K, M, T_cal=32, tag=K + k + M)
+    amax = oracle.channel_amax(L["zcal"])
+    w = prq.prepare_weights(L["W"], amax, 0.5, k)
+    o = oracle.prepare(L["W"], amax, float(np.float32(0.5)), k)
+    wide = w.offline_copy()
+    assert (wide.K, wide.k_tail, wide.N) == (K + k, 0, N)
+    assert np.array_equal(wide.get(prq.FIELD_CODES), o["wcodes"])
+    assert np.array_equal(wide.get(prq.FIELD_SCALES), o["wscales"])
+    x = L["x"]                                             # taken as already permuted and scaled (identity mode)
+    x_wide = np.concatenate([x, x[:, K - k:]], axis=1)
+    oc, osc = oracle.quantize_act(x)
+    ca, sa = oracle.augment_act(oc, osc, k)
+    codes_w, srow_w, sf_w = prq.quantize_act(wide, to_dev_bf16(x_wide), prq.ACT_IDENTITY, row_scales=True)
+    Ka = K + k
+    assert np.array_equal(codes_w.cpu().numpy()[: M * Ka // 2].reshape(M, Ka // 2), ca)
+    assert np.array_equal(srow_w.cpu().numpy()[: M * Ka // 32].reshape(M, Ka // 32), sa)
+    codes, _, sf = prq.quantize_act(w, to_dev_bf16(x), prq.ACT_IDENTITY)
+    y_revisit = prq.linear(w, codes, sf, M)
+    y_wide = prq.linear(wide, codes_w, sf_w, M)
+    assert torch.equal(y_revisit, y_wide)
+    y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+    assert np.abs(y_wide.cpu().numpy().astype(np.float64) - y_ref).max() <= prq_ref.tolerance(y_ref)
+    if M <= prq.FUSED_MAX_M:
+        assert torch.equal(prq.linear_fused(wide, to_dev_bf16(x_wide)), y_wide)
+    assert prq.last_device_status() == 0
+    wide.free()
+    w.free()
+
+
+def test_offline_copy_form_needs_stage_aligned_tail(prq, oracle):
+    W = synth.weights(8, 64, 160)
+    w = prq.prepare_weights(W, np.ones(160, np.float32), 0.0, 32)     # K = 160 is not a multiple of 256
+    with pytest.raises(prq.PrqError) as ei:
+        w.offline_copy()
+    assert ei.value.code == 1                                          # PRQ_ERR_INVALID_ARG
+    w0 = prq.prepare_weights(W, np.ones(160, np.float32), 0.0, 0)      # no tail: nothing to align
+    v = w0.offline_copy()
+    assert (v.K, v.k_tail) == (160, 0)
+    v.free(); w0.free(); w.free()
