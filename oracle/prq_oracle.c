@@ -389,6 +389,47 @@ int orc_matmul_bf16(const uint16_t *x_bf16, long M, const uint16_t *W_bf16, long
     return 0;
 }
 
+/* A finite double rounded once to bf16 (8 significant bits, fp32's exponent range, subnormals kept), ties to the
+ * even significand; returns the bf16 bit pattern. */
+static uint16_t orc_double_to_bf16(double v) {
+    double a = fabs(v), r;
+    float f;
+    uint32_t u;
+    if (a == 0.0) {
+        r = 0.0;
+    } else if (a < ldexp(1.0, -126)) {
+        r = ldexp(nearbyint(ldexp(a, 133)), -133);          /* subnormal range: fixed quantum 2^-133 */
+    } else {
+        int e;
+        double m = frexp(a, &e);                            /* a = m 2^e, m in [0.5, 1) */
+        r = ldexp(nearbyint(ldexp(m, 8)), e - 8);           /* 8 significant bits; nearbyint = ties to even */
+    }
+    f = (float)(v < 0.0 || (v == 0.0 && signbit(v)) ? -r : r);   /* exact, or +-infinity past the top of the range */
+    memcpy(&u, &f, 4);
+    return (uint16_t)(u >> 16);
+}
+
+/* Eq. (1), middle line, and the "offline copy" of the Activation tail construction paragraph: the producer
+ * weights that make the gated FFN emit Z D^-1 P directly.  Row j' of the folded up projection is row perm[j'] of
+ * W_up times inv_s[perm[j']] (the exact product rounded once to bf16), row j' of the folded gate projection is
+ * row perm[j'] of W_gate; with dup != 0 rows C .. C+k-1 of both repeat rows C-k .. C-1, so that the FFN emits
+ * [Z~, Z~_tail].  W_up, W_gate: C x H bf16 (C = input channels of the down projection); outputs (C or C+k) x H.
+ * W_gate / out_gate may be NULL. */
+int orc_fold_producer(const uint16_t *W_up, const uint16_t *W_gate, long C, long H, const int32_t *perm,
+                      const float *inv_s, long k, int dup, uint16_t *out_up, uint16_t *out_gate) {
+    long rows = C + (dup ? k : 0), jp, h;
+    if (k < 0 || k > C) return 1;
+    for (jp = 0; jp < rows; ++jp) {
+        long src_new = jp < C ? jp : C - k + (jp - C);      /* position in the permuted order */
+        long j = perm[src_new];                             /* original channel */
+        for (h = 0; h < H; ++h) {
+            out_up[jp * H + h] = orc_double_to_bf16((double)orc_bf16_to_f32(W_up[j * H + h]) * (double)inv_s[j]);
+            if (W_gate && out_gate) out_gate[jp * H + h] = W_gate[j * H + h];
+        }
+    }
+    return 0;
+}
+
 int orc_num_threads(void) {
 #ifdef _OPENMP
     return omp_get_max_threads();

@@ -204,6 +204,26 @@ def linear(x_bf16, prep: dict, identity: bool = False):
     return matmul(ca, sa, prep["wcodes"], prep["wscales"]), ac, asc
 
 
+def fold_producer(W_up, W_gate, perm, inv_s, k: int, dup: bool = False):
+    """Eq. (1), middle line: up- and gate-projection weights with the down projection's inverse scale and
+    permutation folded in (rows permuted, the up projection's rows scaled and rounded once to bf16); with dup the
+    last k rows are repeated (the 'offline copy' of the Activation tail construction paragraph).
+    W_up, W_gate: uint16 (C, H); returns (up, gate) of (C or C + k, H)."""
+    Wu = _c(W_up, np.uint16)
+    Wg = _c(W_gate, np.uint16)
+    pm = _c(perm, np.int32)
+    iv = _c(inv_s, np.float32)
+    C, H = Wu.shape
+    rows = C + (k if dup else 0)
+    ou = np.empty((rows, H), np.uint16)
+    og = np.empty((rows, H), np.uint16)
+    rc = _load().orc_fold_producer(_p(Wu), _p(Wg), ctypes.c_long(C), ctypes.c_long(H), _p(pm), _p(iv),
+                                   ctypes.c_long(k), ctypes.c_int(1 if dup else 0), _p(ou), _p(og))
+    if rc != 0:
+        raise ValueError("k must lie in [0, C]")
+    return ou, og
+
+
 def nrmse(y_hat, y):
     """Normalised reconstruction error ||Yhat - Y||_F / ||Y||_F (text after Eq. (3))."""
     return float(np.linalg.norm(y_hat - y) / np.linalg.norm(y))
