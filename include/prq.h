@@ -152,7 +152,7 @@ void prq_weights_free(prq_weights *w);
  * Not part of the paper's method.  Free it with prq_weights_free. */
 prq_status prq_weights_clone(const prq_weights *w, prq_weights **out);
 
-/* The "offline copy" form of a prepared layer (Kernel design paragraph: the producer layers emit the k tail
+/* The "offline copy" form of a prepared layer (Activation tail construction paragraph: the producer layers emit the k tail
  * channels a second time, so that the activation already has K + k columns and nothing is re-read).
  * Returns an independent handle (its own device copy, free it with prq_weights_free) that presents the same
  * bytes [Q(W D P) | Q(R)] as a plain MXFP4 layer with K' = K + k input channels and no tail:
@@ -165,6 +165,22 @@ prq_status prq_weights_clone(const prq_weights *w, prq_weights **out);
  * INVALID_ARG if k > 0 and K is not a multiple of 256 (the residual columns would not start on a stage of the
  * scale-byte layout; all of the paper's shapes satisfy it). */
 prq_status prq_weights_offline_copy(const prq_weights *w, prq_weights **out);
+
+/* Eq. (1), middle line: fold a down projection's inverse scaling and permutation into the layers that produce
+ * its input, so that the gated FFN emits Z D^-1 P directly and prq_quantize_act runs in PRQ_ACT_IDENTITY mode:
+ *   out_up  [j', :] = bf16( W_up[perm[j'], :] * inv_s[perm[j']] )     (exact product, rounded once, ties to even)
+ *   out_gate[j', :] =       W_gate[perm[j'], :]
+ * for j' in [0, C); with duplicate_tail != 0 rows C .. C + k_tail - 1 of both outputs repeat rows C - k_tail ..
+ * C - 1 (the "offline copy" of the Activation tail construction paragraph; pair it with
+ * prq_weights_offline_copy).  All pointers are HOST memory:
+ *   perm, inv_s   C entries each, as prq_weights_get returns them (PRQ_FIELD_PERM, PRQ_FIELD_INV_S)
+ *   W_up, W_gate  C x H bf16 row-major (C = input channels of the down projection = output features of the
+ *                 producers, H = their input features); W_gate and out_gate may both be NULL
+ *   out_up, out_gate   (C or C + k_tail) x H bf16, caller-owned
+ * INVALID_ARG for a perm entry outside [0, C), a non-finite inv_s, k_tail outside [0, C]. */
+prq_status prq_fold_producer(const int32_t *perm, const float *inv_s, int C, int k_tail, const uint16_t *W_up,
+                             const uint16_t *W_gate, int H, int duplicate_tail, uint16_t *out_up,
+                             uint16_t *out_gate);
 
 /* Shape of a handle.  Any output pointer may be NULL. */
 prq_status prq_weights_info(const prq_weights *w, int *n_experts, int *N, int *K, int *k_tail, float *alpha);

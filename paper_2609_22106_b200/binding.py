@@ -23,7 +23,7 @@ BUF_CODES, BUF_SCALES_ROW, BUF_SCALES_SF = range(3)
 
 EXPORTS = [
     "prq_prepare_weights", "prq_prepare_weights_opts", "prq_prepare_weights_device", "prq_prepare_weights_host", "prq_prepare_weights_host_opts", "prq_prepare_weights_search", "prq_weights_free",
-    "prq_weights_clone", "prq_weights_offline_copy", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
+    "prq_weights_clone", "prq_weights_offline_copy", "prq_fold_producer", "prq_weights_info", "prq_weights_get", "prq_act_bytes", "prq_quantize_act", "prq_linear_workspace_bytes",
     "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_multi", "prq_quantize_act_multi",
     "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
@@ -56,6 +56,7 @@ def lib():
                                                  ctypes.POINTER(cf), vp]
         L.prq_weights_clone.argtypes = [vp, ctypes.POINTER(vp)]
         L.prq_weights_offline_copy.argtypes = [vp, ctypes.POINTER(vp)]
+        L.prq_fold_producer.argtypes = [vp, vp, ci, ci, vp, vp, ci, ci, vp, vp]
         L.prq_weights_free.argtypes = [vp]
         L.prq_weights_free.restype = None
         L.prq_weights_info.argtypes = [vp] + [ctypes.POINTER(ci)] * 4 + [ctypes.POINTER(cf)]
@@ -224,6 +225,26 @@ def prepare_weights_host(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float,
                                                _np_ptr(out["inv_s"]), _np_ptr(out["col_err"])),
            "prq_prepare_weights_host_opts")
     return out
+
+
+def fold_producer(perm: np.ndarray, inv_s: np.ndarray, k_tail: int, W_up: np.ndarray, W_gate: np.ndarray = None,
+                  duplicate_tail: bool = False):
+    """Eq. (1): the up / gate projection weights with the down projection's 1 / s and permutation folded in.
+    W_up, W_gate: uint16 (C, H).  Returns (up, gate or None) of (C or C + k_tail, H)."""
+    pm = np.ascontiguousarray(perm, np.int32)
+    iv = np.ascontiguousarray(inv_s, np.float32)
+    Wu = np.ascontiguousarray(W_up, np.uint16)
+    C, H = Wu.shape
+    rows = C + (k_tail if duplicate_tail else 0)
+    ou = np.empty((rows, H), np.uint16)
+    Wg = og = None
+    if W_gate is not None:
+        Wg = np.ascontiguousarray(W_gate, np.uint16)
+        og = np.empty((rows, H), np.uint16)
+    _check(lib().prq_fold_producer(_np_ptr(pm), _np_ptr(iv), C, k_tail, _np_ptr(Wu), _np_ptr(Wg) if Wg is not None else None,
+                                   H, 1 if duplicate_tail else 0, _np_ptr(ou), _np_ptr(og) if og is not None else None),
+           "prq_fold_producer")
+    return ou, og
 
 
 def prepare_weights_search(W_bf16, zcal_bf16, alphas, k_tail: int):

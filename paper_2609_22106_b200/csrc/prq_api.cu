@@ -648,6 +648,13 @@ prq_status prq_weights_offline_copy(const prq_weights* w, prq_weights** out) {
     return PRQ_OK;
 }
 
+prq_status prq_fold_producer(const int32_t* perm, const float* inv_s, int C, int k_tail, const uint16_t* W_up,
+                             const uint16_t* W_gate, int H, int duplicate_tail, uint16_t* out_up, uint16_t* out_gate) {
+    if (!perm || !inv_s || !W_up || !out_up || C < 1 || H < 1 || k_tail < 0 || k_tail > C) return PRQ_ERR_INVALID_ARG;
+    if ((W_gate == nullptr) != (out_gate == nullptr)) return PRQ_ERR_INVALID_ARG;
+    return fold_producer(perm, inv_s, C, k_tail, W_up, W_gate, H, duplicate_tail != 0, out_up, out_gate);
+}
+
 prq_status prq_weights_info(const prq_weights* w, int* n_experts, int* N, int* K, int* k_tail, float* alpha) {
     if (!w) return PRQ_ERR_INVALID_ARG;
     if (n_experts) *n_experts = w->n_experts;

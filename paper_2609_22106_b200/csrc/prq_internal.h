@@ -64,6 +64,10 @@ prq_status channel_scales(const float* amax, int K, float alpha, std::vector<flo
 // ... and the error-ranked top-k with its permutation [unselected ascending | selected ascending]
 // (ties: the lower channel index ranks first).
 void rank_and_permute(const std::vector<double>& col_err, int K, int k_tail, std::vector<int32_t>& perm);
+// Eq. (1), middle line: rows of the producer weights permuted (and, for the up projection, scaled by 1 / s and
+// rounded once to bf16); with duplicate_tail the last k_tail rows are repeated.  Host buffers.
+prq_status fold_producer(const int32_t* perm, const float* inv_s, int C, int k_tail, const uint16_t* W_up,
+                         const uint16_t* W_gate, int H, bool duplicate_tail, uint16_t* out_up, uint16_t* out_gate);
 // The same result computed on the current device from a DEVICE copy of W (column errors, permuted
 // quantisation, residual and packing as kernels; scales and ranking on the host in between).  Allocates its
 // temporaries, runs on `stream` and synchronises it.

@@ -141,6 +141,40 @@ double scale_power(double a, float alpha) {
 
 }  // namespace
 
+// bf16 of the exact product of a bf16 weight and an fp32 scale, rounded once.  The product has up to 32
+// significant bits: it is first brought to fp32 with round-to-odd (truncate toward zero, then set the last bit if
+// anything was lost), after which the usual round-to-nearest-even to 8 bits cannot double-round.
+static uint16_t scaled_bf16(uint16_t w, float s) {
+    const double p = static_cast<double>(bf16_bits_to_float(w)) * static_cast<double>(s);   // exact
+    float f = static_cast<float>(p);
+    if (static_cast<double>(f) != p && std::isfinite(f)) {
+        if (std::fabs(static_cast<double>(f)) > std::fabs(p)) f = std::nextafterf(f, 0.f);   // now truncated
+        f = bits_float(float_bits(f) | 1u);                                                 // sticky bit
+    }
+    const uint32_t u = float_bits(f);
+    if ((u & 0x7f800000u) == 0x7f800000u) return static_cast<uint16_t>(u >> 16);            // infinity stays
+    return static_cast<uint16_t>((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
+}
+
+prq_status fold_producer(const int32_t* perm, const float* inv_s, int C, int k_tail, const uint16_t* W_up,
+                         const uint16_t* W_gate, int H, bool duplicate_tail, uint16_t* out_up, uint16_t* out_gate) {
+    const long rows = static_cast<long>(C) + (duplicate_tail ? k_tail : 0);
+    for (int j = 0; j < C; ++j)
+        if (perm[j] < 0 || perm[j] >= C || !std::isfinite(inv_s[j])) return PRQ_ERR_INVALID_ARG;
+    parallel_for(rows, [&](long lo, long hi) {
+        for (long jp = lo; jp < hi; ++jp) {
+            const long pos = jp < C ? jp : C - k_tail + (jp - C);   // position in the permuted order
+            const long j = perm[pos];
+            const float s = inv_s[j];
+            const uint16_t* src = W_up + j * H;
+            uint16_t* dst = out_up + jp * H;
+            for (int h = 0; h < H; ++h) dst[h] = scaled_bf16(src[h], s);
+            if (W_gate && out_gate) std::memcpy(out_gate + jp * H, W_gate + j * H, sizeof(uint16_t) * H);
+        }
+    });
+    return PRQ_OK;
+}
+
 prq_status channel_scales(const float* amax, int K, float alpha, std::vector<float>& s, std::vector<float>& inv_s) {
     s.resize(K);
     inv_s.resize(K);

@@ -540,7 +540,7 @@ def test_device_prep_experts_and_errors(prq, oracle):
 
 @pytest.mark.parametrize("N,K,k,M", [(256, 512, 64, 16), (512, 2560, 128, 300), (256, 768, 64, 1), (384, 1024, 256, 128)])
 def test_offline_copy_form_equals_the_revisit_form(prq, oracle, N, K, k, M):
-    """Kernel design paragraph, second implementation: the producer emits the k tail channels twice, the
+    """Activation tail construction paragraph, offline copy: the producer emits the k tail channels twice, the
     activation has K + k columns, and the layer is a plain MXFP4 product over K + k.  Quantising the widened
     row must equal widening the quantised row (block alignment), so codes, scale bytes and the product are
     bit for bit those of the form that re-reads the tail -- and within tolerance of the oracle."""
@@ -583,3 +583,70 @@ def test_offline_copy_form_needs_stage_aligned_tail(prq, oracle):
     v = w0.offline_copy()
     assert (v.K, v.k_tail) == (160, 0)
     v.free(); w0.free(); w.free()
+
+
+def test_folded_producers_feed_the_identity_path(prq, oracle):
+    """Eq. (1) end to end on a small gated FFN: with 1 / s and the permutation folded into the up / gate projections
+    (prq_fold_producer) the down projection runs in identity mode; with the tail rows duplicated as well it runs
+    as a plain product over C + k (prq_weights_offline_copy).  Each route is checked against the oracle on its
+    own activation (codes bit-exact, product within tolerance); across routes the outputs agree up to the bf16
+    roundings of the folded weights and of the activation."""
+    C, H, N, M, k = 512, 256, 256, 64, 64
+    rng = np.random.default_rng(77)
+    Wu, Wg, Wd = synth.weights(61, C, H), synth.weights(62, C, H), synth.weights(63, N, C)
+    X = torch.from_numpy(rng.standard_normal((M + 128, H)).astype(np.float32) * 8).cuda()
+
+    def ffn(up_bits, gate_bits, x):
+        up = torch.from_numpy(up_bits.view(np.int16)).cuda().view(torch.bfloat16).float()
+        gate = torch.from_numpy(gate_bits.view(np.int16)).cuda().view(torch.bfloat16).float()
+        return (torch.nn.functional.silu(x @ gate.T) * (x @ up.T)).to(torch.bfloat16)
+
+    def bits(t):
+        return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+    h_all = ffn(Wu, Wg, X)
+    amax = oracle.channel_amax(bits(h_all[M:]))            # calibration rows
+    w = prq.prepare_weights(Wd, amax, 0.5, k)
+    o = oracle.prepare(Wd, amax, float(np.float32(0.5)), k)
+    x = X[:M]
+
+    # route A: online scale + permute
+    h = h_all[:M].contiguous()
+    ca, _, sfa = prq.quantize_act(w, h, prq.ACT_SCALE_PERM)
+    y_a = prq.linear(w, ca, sfa, M).cpu().numpy().astype(np.float64)
+
+    # route B: folded producers, identity mode
+    up_f, gate_f = prq.fold_producer(w.get(prq.FIELD_PERM), w.get(prq.FIELD_INV_S), k, Wu, Wg)
+    ht = ffn(up_f, gate_f, x).contiguous()
+    cb, srow_b, sfb = prq.quantize_act(w, ht, prq.ACT_IDENTITY, row_scales=True)
+    y_b = prq.linear(w, cb, sfb, M).cpu().numpy().astype(np.float64)
+    oc, osc = oracle.quantize_act(bits(ht))
+    assert np.array_equal(cb.cpu().numpy()[: M * C // 2].reshape(M, C // 2), oc)
+    assert np.array_equal(srow_b.cpu().numpy()[: M * C // 32].reshape(M, C // 32), osc)
+    cao, sao = oracle.augment_act(oc, osc, k)
+    y_ref_b = oracle.matmul(cao, sao, o["wcodes"], o["wscales"])
+    assert np.abs(y_b - y_ref_b).max() <= prq_ref.tolerance(y_ref_b)
+
+    # route C: tail rows duplicated in the producers, plain product over C + k
+    up_w, gate_w = prq.fold_producer(w.get(prq.FIELD_PERM), w.get(prq.FIELD_INV_S), k, Wu, Wg, duplicate_tail=True)
+    hw = ffn(up_w, gate_w, x).contiguous()
+    wide = w.offline_copy()
+    cc, _, sfc = prq.quantize_act(wide, hw, prq.ACT_IDENTITY)
+    y_c = prq.linear(wide, cc, sfc, M).cpu().numpy().astype(np.float64)
+    ocw, oscw = oracle.quantize_act(bits(hw))
+    assert np.array_equal(cc.cpu().numpy()[: M * (C + k) // 2].reshape(M, (C + k) // 2), ocw)
+    y_ref_c = oracle.matmul(ocw, oscw, o["wcodes"], o["wscales"])
+    assert np.abs(y_c - y_ref_c).max() <= prq_ref.tolerance(y_ref_c)
+
+    # Across routes the activations differ in their last bf16 bit here and there, which flips some 4-bit codes: the
+    # outputs cannot agree closer than a fraction of the quantisation error itself.  All three must sit at the
+    # same distance from the unquantised product, and nearer to each other than to it.
+    y_exact = oracle.matmul_bf16(bits(h), Wd)
+    err = {n: np.linalg.norm(y - y_exact) / np.linalg.norm(y_exact) for n, y in (("a", y_a), ("b", y_b), ("c", y_c))}
+    assert abs(err["b"] - err["a"]) < 0.15 * err["a"] and abs(err["c"] - err["a"]) < 0.15 * err["a"], err
+    nrm = np.linalg.norm(y_exact)
+    assert np.linalg.norm(y_b - y_a) / nrm < 0.6 * err["a"], (np.linalg.norm(y_b - y_a) / nrm, err)
+    assert np.linalg.norm(y_c - y_b) / nrm < 0.6 * err["a"], (np.linalg.norm(y_c - y_b) / nrm, err)
+    assert prq.last_device_status() == 0
+    wide.free()
+    w.free()

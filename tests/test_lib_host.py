@@ -153,3 +153,37 @@ def test_host_prep_rejects_non_finite(prq):
     amax[0] = np.nan
     with pytest.raises(prq.PrqError):
         prq.prepare_weights_host(synth.f32_to_bf16(np.ones((2, 64), np.float32)), amax, 0.5, 0)
+
+
+def test_fold_producer_bit_exact(prq, oracle):
+    """prq_fold_producer (Eq. (1), host buffers) against the oracle: the hand-worked roundings (double-rounding
+    traps and subnormals included), a heavy-tailed random case with the duplicated tail, and without a gate."""
+    import os
+
+    golden = os.path.join(os.path.dirname(__file__), "golden", "bf16_fold_roundings.txt")
+    for line in open(golden):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        w, s, e, _ = [p.strip() for p in line.split(";")]
+        W = np.array([[int(w, 16)]], np.uint16)
+        inv_s = np.array([int(s, 16)], np.uint32).view(np.float32)
+        up, gate = prq.fold_producer(np.array([0], np.int32), inv_s, 0, W, W)
+        assert int(up[0, 0]) == int(e, 16), line
+        assert int(gate[0, 0]) == int(w, 16)
+    rng = np.random.default_rng(5)
+    C, H, k = 384, 200, 64
+    Wu, Wg = synth.weights(31, C, H), synth.weights(32, C, H)
+    Wu[0, :3] = [0x0001, 0x8003, 0x7F7F]
+    perm = rng.permutation(C).astype(np.int32)
+    inv_s = np.exp(rng.normal(0, 4, C)).astype(np.float32)
+    for dup in (False, True):
+        up, gate = prq.fold_producer(perm, inv_s, k, Wu, Wg, duplicate_tail=dup)
+        oup, ogate = oracle.fold_producer(Wu, Wg, perm, inv_s, k, dup=dup)
+        assert np.array_equal(up, oup) and np.array_equal(gate, ogate)
+    up, gate = prq.fold_producer(perm, inv_s, k, Wu)
+    assert gate is None and np.array_equal(up, oracle.fold_producer(Wu, Wg, perm, inv_s, k)[0])
+    bad = perm.copy()
+    bad[3] = C
+    with pytest.raises(prq.PrqError):
+        prq.fold_producer(bad, inv_s, k, Wu)
