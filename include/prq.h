@@ -195,7 +195,7 @@ prq_status prq_weights_get(const prq_weights *w, int expert, prq_field which, vo
  * dense calls pass n_groups = 1.  Returns 0 for invalid arguments. */
 size_t prq_act_bytes(int M, int K, int k_tail, int n_groups, prq_buf which);
 
-/* "The kernel quantizes the reordered activation to MXFP4 once" (Kernel design paragraph).
+/* The single MXFP4 quantisation of the reordered activation that the Kernel design paragraph calls for.
  * One launch: optional scale + permute (Eq. (1), activation side), per-32 amax, E8M0 scale,
  * E2M1 round-to-nearest-even codes.  The quantised tail is not copied: only its k_tail/32 scale
  * bytes per row are duplicated into the tile-ordered scale buffer, the GEMM re-reads the codes.

@@ -316,7 +316,7 @@ int orc_prepare(const uint16_t *W_bf16, long N, long K, const float *amax, doubl
 
 /* Eq. (1), activation side: Zt = Z D^-1 P, i.e. xt[t,j'] = fl32(x[t,perm[j']] * inv_s[perm[j']]);
  * identity when perm and inv_s are NULL (folded into the producer layers).  Then Q by rows
- * ("quantizes the reordered activation once", Kernel design paragraph). */
+ * (the one quantisation of the reordered activation of the Kernel design paragraph). */
 int orc_quantize_act(const uint16_t *x_bf16, long M, long K, const int32_t *perm, const float *inv_s,
                      uint8_t *codes, uint8_t *scales) {
     if (K % ORC_BLOCK) return 1;

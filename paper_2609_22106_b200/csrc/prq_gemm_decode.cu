@@ -24,7 +24,8 @@
 // their CTA -- one 32-element block per thread and stage, codes written straight into the 128-byte-
 // swizzled token tile of the pipeline slot, scale bytes into the slot's scale atom -- so that the
 // separate quantiser launch, its round trip through global memory and one kernel-to-kernel hand-over
-// leave the decode step ("the kernel quantizes the reordered activation once", Kernel design paragraph).
+// leave the decode step (the Kernel design paragraph asks for one quantisation of the reordered activation
+// per layer call; here it happens inside the product kernel).
 // Every cluster quantises the K-range it reduces over, i.e. the bf16 activation is read once per 128-row
 // weight tile; that extra L2 traffic grows with the token count and is why the variant stops at 16 tokens.
 #include <cuda.h>

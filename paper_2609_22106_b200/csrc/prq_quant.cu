@@ -1,5 +1,5 @@
-// Activation quantisation kernel ("the kernel quantizes the reordered activation to MXFP4 once",
-// Kernel design paragraph; Eq. (1) activation side when the scale and permutation are applied online).
+// Activation quantisation kernel: the one MXFP4 quantisation of the reordered activation per layer call
+// (Kernel design paragraph; Eq. (1) activation side when the scale and permutation are applied online).
 //
 // One CTA owns 128 rows x 128 columns: exactly one 512-byte scale atom of the GEMM's layout.  In
 // identity mode a lane takes one whole 32-element block (a row of the tile is 4 lanes, a warp covers
