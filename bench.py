@@ -180,8 +180,20 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
             sf = torch.empty(prq.act_bytes(M, K, k, 1, prq.BUF_SCALES_SF), dtype=torch.uint8, device=dev)
             y = torch.empty((M, N), dtype=torch.bfloat16, device=dev)
             lin[name] = dict(w=w, x=x, codes=codes, sf=sf, y=y, ws=prq.new_workspace(w, M, dev), N=N, K=K, k=k,
-                             mode=prq.ACT_IDENTITY if name == "down" else prq.ACT_SCALE_PERM,
+                             mode=prq.ACT_IDENTITY if name == "down" else prq.ACT_SCALE_PERM, amax=amax,
                              Wb=torch.from_numpy(L["W"].view(np.int16)).to(dev).view(torch.bfloat16))
+        # The layers that read the same activation, prepared as ONE layer each: q / k / v stacked to 6144 output
+        # features and gate / up to 19456, with one scaling, one permutation and one tail per group (the stacked
+        # matrix goes through Algorithm 1 like any other; its column errors are the sums over the group's rows).
+        # One quantisation then serves the whole group.
+        for gname, members in (("qkv", ("q", "k", "v")), ("gate_up", ("gate", "up"))):
+            first = lin[members[0]]
+            Wcat = torch.cat([lin[nm]["Wb"] for nm in members]).contiguous()
+            w = prq.prepare_weights_device(Wcat.view(torch.int16), first["amax"], 0.5, first["k"])
+            Ng = Wcat.shape[0]
+            lin[gname] = dict(w=w, x=first["x"], codes=first["codes"], sf=first["sf"], N=Ng, K=first["K"], k=first["k"],
+                              y=torch.empty((M, Ng), dtype=torch.bfloat16, device=dev), ws=prq.new_workspace(w, M, dev),
+                              mode=prq.ACT_SCALE_PERM, Wb=Wcat)
         layers.append(lin)
 
     def q(d):
@@ -206,6 +218,17 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
                           bound="tensor" if fl / fp4_peak / 1e6 > by / pk["hbm_gbs"] / 1e3 else "hbm")
     step_fns = [(lambda lin=lin: [f() for name in BLOCK_LINEARS for f in (q(lin[name]), g(lin[name]))]) for lin in layers]
     t_step = timer.run(step_fns, n, n_layers) / n
+    grouped = ("qkv", "o", "gate_up", "down")
+    step_grouped = [(lambda lin=lin: [f() for name in grouped for f in (q(lin[name]), g(lin[name]))]) for lin in layers]
+    t_step_grouped = timer.run(step_grouped, n, n_layers) / n
+    t_bf16_grouped = timer.run([(lambda lin=lin: [torch.matmul(lin[name]["x"], lin[name]["Wb"].t()) for name in grouped])
+                                for lin in layers], n, n_layers) / n
+    grouped_rows = {}
+    for name in ("qkv", "gate_up"):
+        ds = [lin[name] for lin in layers]
+        grouped_rows[name] = dict(N=ds[0]["N"], K=ds[0]["K"], k=ds[0]["k"],
+                                  quant_us=timer.run([q(d) for d in ds], n, n_layers) / n * 1e6,
+                                  gemm_us=timer.run([g(d) for d in ds], n, n_layers) / n * 1e6)
     # At decode batch sizes a launch costs as much as the work in it: the layers that read the same activation
     # (q / k / v and gate / up) also go through one quantiser launch and one GEMM launch per group.
     t_step_multi = None
@@ -241,6 +264,8 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
     extra = {}
     if t_step_multi is not None:
         extra = dict(step_multi_launch_us=t_step_multi * 1e6, bf16_fused_qkv_gateup_us=bf16_fused * 1e6)
+    extra.update(step_grouped_prep_us=t_step_grouped * 1e6, bf16_grouped_us=t_bf16_grouped * 1e6,
+                 grouped_linears=grouped_rows)
     return dict(workload=tag, M=M, layers=n_layers, step_us=t_step * 1e6, step_tflops=total_flops / t_step / 1e12, **extra,
                 gemm_us_sum=sum(r["gemm_us"] for r in rows.values()), quant_us_sum=sum(r["quant_us"] for r in rows.values()),
                 bf16_us_sum=sum(r["bf16_matmul_us"] for r in rows.values()), device_status=status, linears=rows)

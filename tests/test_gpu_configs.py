@@ -14,7 +14,10 @@ torch = pytest.importorskip("torch")
 
 # (name, N, K, k) of one Qwen3-4B-shaped decoder block; k and v share a shape, so do gate and up
 BLOCK = [("q", 4096, 2560, 128), ("kv", 1024, 2560, 128), ("o", 2560, 4096, 128),
-         ("gate_up", 9728, 2560, 128), ("down", 2560, 9728, 256)]
+         ("gate_up", 9728, 2560, 128), ("down", 2560, 9728, 256),
+         # q, k and v stacked into one layer (one scaling, permutation and tail for the group), as the
+         # benchmark's grouped-preparation step runs them
+         ("qkv_stacked", 6144, 2560, 128)]
 
 
 def to_dev_bf16(x_u16):
