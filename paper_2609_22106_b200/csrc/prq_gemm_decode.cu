@@ -49,13 +49,18 @@ constexpr uint32_t kHiPlain = (128u >> 4) | (1u << 14);
 __device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo) { return (static_cast<uint64_t>(hi) << 32) | lo; }
 constexpr int pow2_cols(int x) { int p = 32; while (p < x) p *= 2; return p; }
 
-template <int BN>
+// kDense: the variant for layers with more 128-row weight tiles than the GPU has SMs (from 64 tokens on one
+// CTA fills an SM, so tile 149 would wait for a second wave that leaves most SMs idle).  Such a layer is not
+// K-split, so its CTAs need no receive buffer; with a 3-slot ring two of them share an SM and all tiles are
+// resident at once (stacked gate / up projection, 152 tiles: 16.2 -> 12.1 us at 64 tokens, 20.0 -> 14.1 at 128).
+template <int BN, bool kDense = false>
 struct DCfg {
+    static_assert(!kDense || BN >= 64, "up to 32 tokens two CTAs share an SM anyway");
     static constexpr int kQTile = BN * 128;
     static constexpr int kStageBytes = kPTile + kQTile + 2 * kSf;
     // ring depth: 5 / 4 stages leave room for two CTAs per SM at 16 / 32 tokens
-    static constexpr int kStages = BN == 16 ? 5 : BN == 32 ? 4 : BN == 64 ? 6 : 4;
-    static constexpr int kCtasPerSm = BN <= 32 ? 2 : 1;
+    static constexpr int kStages = kDense ? 3 : BN == 16 ? 5 : BN == 32 ? 4 : BN == 64 ? 6 : 4;
+    static constexpr int kCtasPerSm = (kDense || BN <= 32) ? 2 : 1;
     // epilogue warps: four (one per tensor-memory lane quarter); eight from 64 tokens on, where moving the
     // partial sums is most of the kernel -- two warps per quarter then take alternate 16-token chunks
     static constexpr int kEpiWarps = BN >= 64 ? 8 : 4;
@@ -66,7 +71,7 @@ struct DCfg {
     static constexpr bool kAsyncExchange = BN <= 32;
     // receive buffer of the split-K exchange: [peer][token slot][128 rows] fp32, ceil(BN / splits) token
     // slots per peer, i.e. at most BN + 7 token rows of 512 bytes
-    static constexpr int kRecvBytes = (BN + 7) * 512;
+    static constexpr int kRecvBytes = kDense ? 0 : (BN + 7) * 512;
     static constexpr int kSmemBytes = kStages * kStageBytes + kRecvBytes + 1024;
     static constexpr int kAccCols = BN < 32 ? 32 : BN;
     static constexpr int kSfCol = kAccCols;          // 8 weight-scale + 8 token-scale columns behind the accumulator
@@ -110,10 +115,10 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
     tc_commit(empty_bar0 + slot * 8);
 }
 
-template <int BN, bool kFused, bool kBatch>
-__global__ void __launch_bounds__(DCfg<BN>::kThreads, DCfg<BN>::kCtasPerSm)
+template <int BN, bool kFused, bool kBatch, bool kDense = false>
+__global__ void __launch_bounds__(DCfg<BN, kDense>::kThreads, DCfg<BN, kDense>::kCtasPerSm)
 decode_kernel(const __grid_constant__ DecodeMaps maps, const DecodeBatch b) {
-    using C = DCfg<BN>;
+    using C = DCfg<BN, kDense>;
     // which of the batched layers this cluster works for (one launch may run several layers over the same
     // tokens, each with its own weights, activation codes and output)
     const int tile_all = static_cast<int>(blockIdx.x) / b.splits;
@@ -466,14 +471,15 @@ decode_kernel(const __grid_constant__ DecodeMaps maps, const DecodeBatch b) {
     if (threadIdx.x == 0 && abort_flag_s) atomicExch(p.status, static_cast<int>(PRQ_ERR_TIMEOUT));
 }
 
-template <int BN, bool kFused, bool kBatch>
+template <int BN, bool kFused, bool kBatch, bool kDense = false>
 cudaError_t launch_one(const DecodeMaps& maps, const DecodeBatch& b, cudaStream_t stream) {
     const DecodeBatch& p = b;
     const int n_tiles = b.lay[b.n_lin - 1].tile_end;
-    using C = DCfg<BN>;
+    using C = DCfg<BN, kDense>;
+    if (kDense && p.splits != 1) return cudaErrorInvalidValue;   // the dense variant has no receive buffer
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(decode_kernel<BN, kFused, kBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel<BN, kFused, kBatch, kDense>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -491,7 +497,20 @@ cudaError_t launch_one(const DecodeMaps& maps, const DecodeBatch& b, cudaStream_
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, decode_kernel<BN, kFused, kBatch>, maps, b);
+    return cudaLaunchKernelEx(&cfg, decode_kernel<BN, kFused, kBatch, kDense>, maps, b);
+}
+
+// more weight tiles than SMs, no K split, 64 tokens or more: the two-CTAs-per-SM variant
+bool wants_dense(int bn, const DecodeBatch& b) {
+    if (bn < 64 || b.splits != 1) return false;
+    static int sm_count[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (sm_count[dev] == 0 && cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return b.lay[b.n_lin - 1].tile_end > sm_count[dev];
 }
 
 template <int BN>
@@ -520,14 +539,17 @@ cudaError_t launch_decode_batch(int bn, const DecodeMaps& maps, const DecodeBatc
     if (b.n_lin < 1 || b.n_lin > kMaxBatch) return cudaErrorInvalidValue;
     if (b.x != nullptr)   // fused activation quantiser: one layer, the 16-token tile only
         return (bn == 16 && b.n_lin == 1) ? launch_one<16, true, false>(maps, b, stream) : cudaErrorInvalidValue;
+    const bool dense = wants_dense(bn, b);
     if (b.n_lin > 1) {
         switch (bn) {
             case 16: return launch_one<16, false, true>(maps, b, stream);
             case 32: return launch_one<32, false, true>(maps, b, stream);
-            case 64: return launch_one<64, false, true>(maps, b, stream);
-            default: return launch_one<128, false, true>(maps, b, stream);
+            case 64: return dense ? launch_one<64, false, true, true>(maps, b, stream) : launch_one<64, false, true>(maps, b, stream);
+            default: return dense ? launch_one<128, false, true, true>(maps, b, stream) : launch_one<128, false, true>(maps, b, stream);
         }
     }
+    if (dense)
+        return bn == 64 ? launch_one<64, false, false, true>(maps, b, stream) : launch_one<128, false, false, true>(maps, b, stream);
     switch (bn) {
         case 16: return launch_one<16, false, false>(maps, b, stream);
         case 32: return launch_one<32, false, false>(maps, b, stream);

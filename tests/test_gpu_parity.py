@@ -650,3 +650,37 @@ def test_folded_producers_feed_the_identity_path(prq, oracle):
     assert prq.last_device_status() == 0
     wide.free()
     w.free()
+
+
+@pytest.mark.parametrize("M", [64, 100, 128])
+def test_decode_more_weight_tiles_than_sms(prq, oracle, M):
+    """A layer with more 128-row weight tiles than the GPU has SMs (152 here, like a stacked gate / up
+    projection) at 64 to 128 tokens takes the decode kernel's two-CTAs-per-SM variant; so does a two-layer
+    launch whose layers have 76 tiles each.  Sampled rows against the oracle, and the two-layer launch against
+    single-layer calls."""
+    N, K, k = 19456, 512, 64
+    L = synth.layer(6, N, K, M, T_cal=32, tag=M)
+    amax = oracle.channel_amax(L["zcal"])
+    w = prq.prepare_weights(L["W"], amax, 0.5, k)
+    o = oracle.prepare(L["W"], amax, float(np.float32(0.5)), k)
+    assert np.array_equal(w.get(prq.FIELD_CODES), o["wcodes"])
+    x = to_dev_bf16(L["x"])
+    codes, _, sf = prq.quantize_act(w, x, prq.ACT_SCALE_PERM)
+    y = prq.linear(w, codes, sf, M)
+    assert prq.last_device_status() == 0
+    oc, osc = oracle.quantize_act(L["x"], o["perm"], o["inv_s"])
+    ca, sa = oracle.augment_act(oc, osc, k)
+    y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+    assert np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max() <= prq_ref.tolerance(y_ref)
+    yb = prq.linear(w, codes, sf, M, prq.BF16).float().cpu().numpy().astype(np.float64)
+    assert np.abs(yb - y_ref).max() <= prq_ref.tolerance(y_ref) + np.abs(y_ref).max() * 2.0 ** -7
+    w.free()
+    # two layers of 76 tiles in one launch
+    halves = [prq.prepare_weights(L["W"][i * 9728:(i + 1) * 9728], amax, 0.5, k) for i in range(2)]
+    acts = prq.quantize_act_multi(halves, x, prq.ACT_SCALE_PERM)
+    ys = prq.linear_multi(halves, acts, M)
+    for h, a, ym in zip(halves, acts, ys):
+        assert torch.equal(ym, prq.linear(h, a[0], a[1], M))
+    assert prq.last_device_status() == 0
+    for h in halves:
+        h.free()
