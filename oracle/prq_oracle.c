@@ -40,8 +40,9 @@
  * Pins (see tests/test_oracle_*.py): hand-worked encodings, a brute-force
  * nearest-value quantiser in exact rational arithmetic, the worked prep example,
  * k = 0 reducing to plain MXFP4, Eq. (1) invariance, exact residual identity,
- * brute-force top-k, Eq. (3) = main + correction.  The alpha selection is
- * "parity unpinned": the paper fixes only "argmin of the normalised error".
+ * brute-force top-k, Eq. (3) = main + correction.  The normalised error and the alpha
+ * selection of the Python front end (first minimum over the grid) are pinned by a hand-worked
+ * error norm and a hand-decided three-candidate search (tests/test_oracle_alpha.py).
  */
 #include <math.h>
 #include <stdint.h>
