@@ -19,10 +19,12 @@
  *   - bf16 values are raw 16-bit patterns.  MXFP4 storage: 32-element blocks along
  *     the reduction axis, one E8M0 scale byte per block (value 2^(byte-127)),
  *     E2M1 elements packed two per byte with the even column in the low nibble.
- *   - K % 32 == 0, k_tail % 32 == 0 and 0 <= k_tail <= K are required ("the tail and
- *     concatenation boundaries are aligned with the MXFP4 quantization blocks").
+ *   - K % 32 == 0, k_tail % 32 == 0 and 0 <= k_tail <= K are required: the tail starts and
+ *     ends on 32-element block boundaries, which is the condition of the Kernel design
+ *     paragraph under which copying the quantised tail equals quantising the widened row.
  *   - A prq_weights handle is immutable after creation and may be used from several
- *     streams at once.  It belongs to the device that was current when it was made.
+ *     streams at once.  It belongs to the device that was current when it was made, and
+ *     every online call must be made with that device current (else INVALID_ARG).
  *   - A kernel that gives up on a bounded wait records PRQ_ERR_TIMEOUT in a device
  *     status word that prq_last_device_status() reads; it never traps or spins forever.
  */
@@ -207,6 +209,11 @@ size_t prq_act_bytes(int M, int K, int k_tail, int n_groups, prq_buf which);
  *   codes           device out, PRQ_BUF_CODES bytes (16-byte aligned)
  *   scales_row      device out or NULL, PRQ_BUF_SCALES_ROW bytes
  *   scales_sf       device out, PRQ_BUF_SCALES_SF bytes (16-byte aligned)
+ * A single layer (n_experts == 1) may also be given a two-entry expert_offsets {0, M}: the buffers then have
+ * the grouped layout with one group, which prq_linear_grouped consumes.
+ * Precondition: x is finite.  The kernel does not look for NaN or infinities (a scan would cost a second pass
+ * over a memory-bound kernel); a block that holds one gets a meaningless scale byte and the product is
+ * undefined for that row.  The offline calls do check W and amax (NONFINITE).
  * M == 0 is a no-op. */
 prq_status prq_quantize_act(const prq_weights *w, prq_act_mode mode, const void *x, int M, int ldx,
                             const int32_t *expert_offsets, void *codes, void *scales_row, void *scales_sf,
@@ -225,7 +232,8 @@ size_t prq_linear_workspace_bytes(const prq_weights *w, int M);
  *                     (only columns [0, N) of a row are written: y may be a column slice of a wider matrix)
  *   workspace         device, at least prq_linear_workspace_bytes(w, M) bytes, 16-byte aligned (may be NULL
  *                     when that is 0); zero-filled by the caller before its first use, the kernel leaves
- *                     its flags zeroed again
+ *                     its flags zeroed again -- except after a wait inside the kernel ran out
+ *                     (prq_last_device_status returned PRQ_ERR_TIMEOUT): zero-fill it again then
  * M <= 128 takes the weight-streaming cluster split-K kernel, larger M the stream-K prefill kernel.
  * Errors: INVALID_ARG, ALIGNMENT (y, ldy, workspace), WORKSPACE (too small), CUDA (launch failed). */
 prq_status prq_linear(const prq_weights *w, const void *codes, const void *scales_sf, int M, void *y, int ldy,
@@ -238,7 +246,8 @@ prq_status prq_linear(const prq_weights *w, const void *codes, const void *scale
  * prq_linear's; the stream-K scratch (tile flags and fp32 partial tiles) lives in an array that is part
  * of the library image instead of in caller memory.
  *   - Arguments as for prq_linear, minus the workspace.  The handle's device must be the current device.
- *   - Limits: at most 8192 output half-tiles (2 * ceil(M/256) * ceil(N/224)) and at most 160 SMs; beyond
+ *   - Limits: at most 8192 output half-tiles, counted as 2 * ceil(M/256) * ceil(N/224) (an upper bound: the
+ *     kernel may pick 240-column tiles, of which there are no more), and at most 160 SMs; beyond
  *     that the call returns PRQ_ERR_STATIC_SCRATCH and launches nothing.  M <= 128 needs no scratch and is
  *     passed on.
  *   - Cost: the array is 42,008,576 bytes (64 KB of counters + 2 x 160 partial tiles of 128 KB) on every
@@ -305,8 +314,10 @@ prq_status prq_forward_host(const prq_weights *w, prq_act_mode mode, const uint1
 
 const char *prq_status_string(prq_status s);
 
-/* Synchronises `stream`, then reads and clears the device status word that a kernel sets when a
- * bounded wait expired (PRQ_ERR_TIMEOUT).  PRQ_OK when nothing went wrong. */
+/* Synchronises `stream`, then reads and clears the status word of the CURRENT device, which a kernel sets
+ * when a bounded wait expired (PRQ_ERR_TIMEOUT).  PRQ_OK when nothing went wrong.  After PRQ_ERR_TIMEOUT the
+ * outputs of the calls since the last check are undefined and a prq_linear workspace must be zero-filled
+ * again; the context stays usable. */
 prq_status prq_last_device_status(prq_stream_t stream);
 
 /* Number of kernels this library has launched in this process (for benchmark bookkeeping). */

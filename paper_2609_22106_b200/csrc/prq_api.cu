@@ -43,8 +43,14 @@ prq_status device_info(int dev, DeviceInfo** out) {
         if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return PRQ_ERR_CUDA;
         if (prop.major != 10) return PRQ_ERR_UNSUPPORTED_ARCH;
         d.num_sms = prop.multiProcessorCount;
+        // the address of a __device__ variable belongs to the device that is current during the look-up
+        int cur = -1;
+        if (cudaGetDevice(&cur) != cudaSuccess) return PRQ_ERR_CUDA;
+        if (cur != dev && cudaSetDevice(dev) != cudaSuccess) return PRQ_ERR_CUDA;
         void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return PRQ_ERR_CUDA;
+        const cudaError_t e = cudaGetSymbolAddress(&p, g_device_status);
+        if (cur != dev) cudaSetDevice(cur);
+        if (e != cudaSuccess) return PRQ_ERR_CUDA;
         d.status_ptr = static_cast<int*>(p);
         d.ok = true;
     }
@@ -121,11 +127,11 @@ prq_status build_weight_maps(prq_weights* w) {
     if (w->n_experts != 1) return PRQ_OK;
     const uint64_t Ka = static_cast<uint64_t>(w->K) + w->k_tail;
     prq_status st = make_code_map(&w->tm_w_decode, w->d_codes, Ka / 2, w->N, 128);
-    for (int v = 0; v < 2; ++v) {   // 224- and 240-row tilings: scale layouts 2 and 3
+    for (int v = 0; v < 2; ++v) {   // 224- and 240-row tilings
         if (st == PRQ_OK) st = make_code_map(&w->tm_w_pair[v], w->d_codes, Ka / 2, w->N, (v ? kPrefillTileWide : kPrefillTileN) / 2);
-        if (st == PRQ_OK && w->d_sf_alt[2 + v])
-            st = make_sf_map(&w->tm_sfw_pair[v], w->d_sf_alt[2 + v],
-                             static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[2 + v] * kSfGroupBytes, 8);
+        if (st == PRQ_OK && w->d_sf_alt[v])
+            st = make_sf_map(&w->tm_sfw_pair[v], w->d_sf_alt[v],
+                             static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[v] * kSfGroupBytes, 8);
     }
     if (st == PRQ_OK) w->maps_ready = true;
     return st;
@@ -147,8 +153,16 @@ long long* trace_ptr() {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// Online calls launch on the current device with pointers and tensor maps of the handle's device.
+bool handle_device_is_current(const prq_weights* w) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == w->device;
+}
+
 int dense_groups(int M) { return (M + kGroupRows - 1) / kGroupRows; }
-int grouped_groups(int M, int n_groups) { return (M + kGroupRows - 1) / kGroupRows + n_groups; }
+// Scale groups of a grouped buffer: every expert's rows are padded to whole 128-row groups, which costs at most
+// one group per expert; a single expert needs exactly the dense count, so that the two layouts coincide.
+int grouped_groups(int M, int n_groups) { return n_groups == 1 ? dense_groups(M) : (M + kGroupRows - 1) / kGroupRows + n_groups; }
 
 int decode_bn(int M) { return M <= 16 ? 16 : M <= 32 ? 32 : M <= 64 ? 64 : 128; }
 
@@ -190,24 +204,8 @@ int decode_splits(const prq_weights* w, int M, DeviceInfo* di) {
     return decode_splits_for((w->N + 127) / 128, w->plan.S, M, di);
 }
 
-int prefill_bn(const prq_weights* w, int M, int num_sms) {
-    int forced = env_int("PRQ_PREFILL_BN", 0);
-    if (forced) return forced;
-    const int cand[4] = {256, 192, 160, 128};
-    const long m_tiles = (M + 127) / 128;
-    long best_cost = -1;
-    int best = 256;
-    for (int bn : cand) {
-        const long units = m_tiles * ((w->N + bn - 1) / bn);
-        const long waves = (units + num_sms - 1) / num_sms;
-        const long cost = waves * bn;  // MMA time per tile is proportional to bn
-        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = bn; }
-    }
-    return best;
-}
-
-constexpr int kNumAlt = 4;
-constexpr int kAltTileRows[kNumAlt] = {160, 192, 224, 240};  // weight tile widths with their own scale layout
+constexpr int kNumAlt = 2;
+constexpr int kAltTileRows[kNumAlt] = {kPrefillTileN, kPrefillTileWide};  // weight tile widths of the prefill kernel, each with its own scale layout
 
 // How the pair kernel shares out the tiles of one call: every pair gets `whole` whole tiles; the `sk`
 // tiles left over are each cut into equal pieces for `base` (the first `extra` tiles: base + 1)
@@ -706,7 +704,10 @@ prq_status prq_quantize_act(const prq_weights* w, prq_act_mode mode, const void*
     if (mode != PRQ_ACT_IDENTITY && mode != PRQ_ACT_SCALE_PERM) return PRQ_ERR_INVALID_ARG;
     if (M == 0) return PRQ_OK;
     if (!x || !codes || !scales_sf || ldx < w->K) return PRQ_ERR_INVALID_ARG;
-    if ((w->n_experts > 1) != (expert_offsets != nullptr)) return PRQ_ERR_INVALID_ARG;
+    // stacked experts need their row boundaries; a single layer may be given a two-entry offsets array too
+    // (the grouped layout with one group), as prq_linear_grouped accepts it
+    if (w->n_experts > 1 && expert_offsets == nullptr) return PRQ_ERR_INVALID_ARG;
+    if (!handle_device_is_current(w)) return PRQ_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(codes) || !aligned16(scales_sf) || ldx % 8) return PRQ_ERR_ALIGNMENT;
     QuantParams p;
     p.x = static_cast<const uint16_t*>(x);
@@ -734,6 +735,7 @@ prq_status prq_quantize_act_multi(int n, const prq_weights* const* ws, prq_act_m
     }
     if (M == 0) return PRQ_OK;
     if (!x || ldx < ws[0]->K) return PRQ_ERR_INVALID_ARG;
+    if (!handle_device_is_current(ws[0])) return PRQ_ERR_INVALID_ARG;
     if (!aligned16(x) || ldx % 8) return PRQ_ERR_ALIGNMENT;
     for (int i = 0; i < n; ++i)
         if (!aligned16(codes[i]) || !aligned16(scales_sf[i])) return PRQ_ERR_ALIGNMENT;
@@ -779,10 +781,10 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
     prq_status st = check_linear_common(w, codes, scales_sf, y, ldy, y_dtype);
     if (st != PRQ_OK) return st;
     if (M < 0 || w->n_experts != 1 || !w->maps_ready) return PRQ_ERR_INVALID_ARG;
+    if (!handle_device_is_current(w)) return PRQ_ERR_INVALID_ARG;
     DeviceInfo* di;
     st = device_info(w->device, &di);
     if (st != PRQ_OK) return st;
-    const size_t Ka = static_cast<size_t>(w->K) + w->k_tail;
 
     GemmParams p;
     std::memset(&p, 0, sizeof(p));
@@ -797,9 +799,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
     p.trace = trace_ptr();
     p.dbg = env_int("PRQ_DBG", 0);
 
-    CUtensorMap tm_act, tm_w;
-    GemmKind kind;
-    int bn, grid;
+    CUtensorMap tm_act;
     if (M <= 128) {
         // weight-streaming kernel: weights on the MMA M axis, K split over a thread-block cluster
         DecodeParams q;
@@ -810,13 +810,13 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         q.y = y; q.ldy = ldy; q.y_bf16 = p.y_bf16;
         q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
         q.splits = decode_splits(w, M, di);
-        bn = decode_bn(M);
+        const int bn = decode_bn(M);
         st = make_code_map(&tm_act, codes, w->K / 2, M, bn);
         if (st != PRQ_OK) return st;
         cudaError_t e = launch_decode(bn, tm_act, w->tm_w_decode, q, (w->N + 127) / 128, static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
-    } else if (env_int("PRQ_PREFILL_BN", 0) == 0) {
+    } else {
         // stream-K kernel on CTA pairs with 256 x 224 or 256 x 240 tiles (scale bytes grouped per weight tile)
         PrefillParams q;
         std::memset(&q, 0, sizeof(q));
@@ -828,10 +828,13 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         if (pairs < 1) return PRQ_ERR_CUDA;
         q.M = M; q.N = w->N; q.K = w->K; q.k_tail = w->k_tail;
         q.m_tiles = (M + 255) / 256; q.n_tiles = (w->N + pair_bn - 1) / pair_bn;
-        q.act_groups = p.act_groups; q.w_groups = w->w_groups_alt[2 + variant];
-        q.act_sf = p.act_sf; q.w_sf = w->d_sf_alt[2 + variant];
+        q.act_groups = p.act_groups; q.w_groups = w->w_groups_alt[variant];
+        q.act_sf = p.act_sf; q.w_sf = w->d_sf_alt[variant];
         q.y = y; q.ldy = ldy;
         q.y_bf16 = p.y_bf16; q.status = p.status; q.trace = p.trace; q.dbg = p.dbg;
+        // developer switch: a short limit lets a test watch a wait run out (cycles; default about two seconds)
+        const int short_limit = env_int("PRQ_WAIT_LIMIT_CYCLES", 0);
+        q.wait_limit = short_limit > 0 ? short_limit : kDefaultWaitLimitCycles;
         const size_t flag_bytes = prefill_flag_bytes(w, M);
         const long long tiles = ps.tiles, whole = ps.whole, sk = ps.sk;
         if (sk > 0 && !env_int("PRQ_SK_RANGES", 0)) {
@@ -856,22 +859,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
                                             static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
-    } else {
-        kind = GemmKind::kPrefill;
-        bn = prefill_bn(w, M, di->num_sms);
-        const long units = static_cast<long>((M + 127) / 128) * ((w->N + bn - 1) / bn);
-        grid = static_cast<int>(std::min<long>(units, di->num_sms));
-        for (int a = 0; a < kNumAlt; ++a)
-            if (bn == kAltTileRows[a]) { p.w_sf = w->d_sf_alt[a]; p.w_groups = w->w_groups_alt[a]; }
-        st = make_code_map(&tm_act, codes, w->K / 2, M, 128);
-        if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, w->N, bn);
     }
-    if (st != PRQ_OK) return st;
-    bool unsupported = false;
-    cudaError_t e = launch_gemm(kind, bn, tm_act, tm_w, p, grid, static_cast<cudaStream_t>(stream), &unsupported);
-    if (unsupported) return PRQ_ERR_INVALID_ARG;
-    g_launches.fetch_add(1);
-    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
 }
 
 prq_status prq_linear_multi(int n, const prq_weights* const* ws, const void* const* codes, const void* const* scales_sf,
@@ -888,6 +876,7 @@ prq_status prq_linear_multi(int n, const prq_weights* const* ws, const void* con
         if (ws[i]->K != ws[0]->K || ws[i]->k_tail != ws[0]->k_tail || ws[i]->device != ws[0]->device) return PRQ_ERR_INVALID_ARG;
     }
     if (M == 0) return PRQ_OK;
+    if (!handle_device_is_current(ws[0])) return PRQ_ERR_INVALID_ARG;
     DeviceInfo* di;
     prq_status st = device_info(ws[0]->device, &di);
     if (st != PRQ_OK) return st;
@@ -922,6 +911,7 @@ prq_status prq_linear_fused(const prq_weights* w, prq_act_mode mode, const void*
     if (!x || !y || ldx < w->K || ldy < w->N) return PRQ_ERR_INVALID_ARG;
     if (y_dtype != PRQ_F32 && y_dtype != PRQ_BF16) return PRQ_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(y) || ldx % 8 || ldy % (y_dtype == PRQ_F32 ? 4 : 8)) return PRQ_ERR_ALIGNMENT;
+    if (!handle_device_is_current(w)) return PRQ_ERR_INVALID_ARG;
     DeviceInfo* di;
     prq_status st = device_info(w->device, &di);
     if (st != PRQ_OK) return st;
@@ -947,6 +937,7 @@ prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const voi
     prq_status st = check_linear_common(w, codes, scales_sf, y, ldy, y_dtype);
     if (st != PRQ_OK) return st;
     if (M_total < 0 || !expert_offsets) return PRQ_ERR_INVALID_ARG;
+    if (!handle_device_is_current(w)) return PRQ_ERR_INVALID_ARG;
     DeviceInfo* di;
     st = device_info(w->device, &di);
     if (st != PRQ_OK) return st;
@@ -964,20 +955,13 @@ prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const voi
     p.y = y; p.ldy = ldy; p.y_bf16 = y_dtype == PRQ_BF16;
     p.status = di->status_ptr;
     p.trace = trace_ptr();
-    // Default: output features on the MMA M axis, one 128-token group of an expert on the N axis (coalesced
-    // stores straight from the accumulator, cheap for experts with few tokens).  PRQ_GROUPED_BN selects the
-    // tokens-on-M variant with that weight-tile width instead.
-    int bn = env_int("PRQ_GROUPED_BN", 0);
-    const bool swap = bn == 0;
-    if (swap) bn = 128;
+    // output features on the MMA M axis, one 128-token group of an expert on the N axis (contiguous stores per
+    // token, cheap for experts with few tokens)
     CUtensorMap tm_act, tm_w;
     st = make_code_map(&tm_act, codes, w->K / 2, M_total, 128);
-    if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, static_cast<uint64_t>(w->n_experts) * w->N, bn);
+    if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, static_cast<uint64_t>(w->n_experts) * w->N, 128);
     if (st != PRQ_OK) return st;
-    bool unsupported = false;
-    cudaError_t e = launch_gemm(swap ? GemmKind::kGroupedSwap : GemmKind::kGrouped, bn, tm_act, tm_w, p, di->num_sms,
-                                static_cast<cudaStream_t>(stream), &unsupported);
-    if (unsupported) return PRQ_ERR_INVALID_ARG;
+    cudaError_t e = launch_gemm_grouped(tm_act, tm_w, p, di->num_sms, static_cast<cudaStream_t>(stream));
     g_launches.fetch_add(1);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
 }

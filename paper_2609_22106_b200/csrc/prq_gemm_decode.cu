@@ -456,6 +456,11 @@ decode_kernel(const __grid_constant__ DecodeMaps maps, const DecodeBatch b) {
             }
             if (trace && et == 0) trace[194] = clock64();
         }
+        // A CTA that gave up pushes nothing and sums nothing, but healthy peers still deliver their partial
+        // sums into its receive buffer and count them on its barrier: it stays until they have (bounded), so
+        // that no store of a peer reaches the shared memory of a CTA that has left.
+        if (C::kAsyncExchange && abort_flag_s && n_own > 0 && threadIdx.x == 64)
+            mbar_wait_after_abort(smem_u32(&bar_recv), 0);
     }
 
     // ------------------------------------------------------------ teardown (normal and aborted)

@@ -219,6 +219,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     __shared__ __align__(8) uint64_t bar_full[kStages], bar_empty[kStages], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag_s;
+    __shared__ int fixup_gave_up_s;   // an epilogue warp's wait for a stream-K tile's pieces ended without them
     volatile int* abort_flag = &abort_flag_s;
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -247,6 +248,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             mbar_init(smem_u32(&bar_acc_empty[i]), 8);   // four epilogue warps of each CTA
         }
         abort_flag_s = 0;
+        fixup_gave_up_s = 0;
         fence_mbar_init();
         tma_prefetch_desc(&tm_act);
         tma_prefetch_desc(&tm_w);
@@ -318,7 +320,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             const int sfa_row0 = (mi * 2 + static_cast<int>(rank)) * 4, sfa_stride = p.act_groups * 4;
             const int sfw_row0 = ni * 8, sfw_stride = p.w_groups * 4;
             for (int s = sg.s0; s < sg.s1; ++s, ++it) {
-                if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                 if (trace && lane == 0 && it < 64) trace[it] = clock64();
                 if (elect_one()) {
                     if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bar_full[st]), 2 * kStageBytes);
@@ -355,12 +357,12 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             bool ready = false;
             while (ok && r.next(sg)) {
                 const int buf = seg_it & 1;
-                if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), ((seg_it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), ((seg_it >> 1) & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 uint32_t accumulate = 0;
                 for (int s = sg.s0; s < sg.s1; ++s, ++it) {
-                    if (!ready && !mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
+                    if (!ready && !mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag, p.wait_limit)) { ok = false; break; }
                     if (trace && lane == 0 && it < 64) trace[64 + it] = clock64();
                     const int rem = s < S1 ? p.K - s * kStageK : p.k_tail - (s - S1) * kStageK;
                     const int nst = st + 1 == kStages ? 0 : st + 1;
@@ -500,12 +502,15 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                     volatile int* a = arrived;
                     const long long t0 = clock64();
                     while (*a < fx.P) {
-                        if (*abort_flag) break;
-                        if (clock64() - t0 > kWaitLimitCycles) { *abort_flag = 1; break; }
+                        if (*abort_flag) { fixup_gave_up_s = 1; break; }
+                        if (clock64() - t0 > p.wait_limit) { *abort_flag = 1; fixup_gave_up_s = 1; break; }
                     }
                 }
-                __syncwarp();
-                if (*abort_flag) { ok = false; break; }
+                // The four warps decide together, on a word that is written only before this barrier: a warp
+                // that saw the counter complete must not go on to the barrier at the end of the fix-up while
+                // another one gave up a moment earlier and will never arrive there.
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (*reinterpret_cast<volatile int*>(&fixup_gave_up_s)) { ok = false; break; }
                 __threadfence();
                 const int mi = fx.tile % p.m_tiles, ni = fx.tile / p.m_tiles;
                 const int y_row = mi * 256 + static_cast<int>(rank) * 128 + q4 * 32;
@@ -567,7 +572,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             // all of this pair's pieces are published: fix up now, overlapping the main loop of this whole tile
             if (!piece && n_fix > 0 && r.cur >= r.end) run_fixups();
             if (!ok) break;
-            if (!mbar_wait(smem_u32(&bar_acc_full[buf]), (seg_it >> 1) & 1, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(smem_u32(&bar_acc_full[buf]), (seg_it >> 1) & 1, abort_flag, p.wait_limit)) { ok = false; break; }
             if (trace && row_in_tile == 0 && seg_it < 8) trace[192 + 2 * seg_it] = clock64();
             tc_fence_after_sync();
             const uint32_t acc_t = tmem_base + buf * BN + (static_cast<uint32_t>(q4 * 32) << 16);

@@ -14,6 +14,10 @@ namespace prq {
 #endif
 constexpr bool kTraceBuild = PRQ_TRACE != 0;
 
+// Default limit of every wait inside a kernel, in SM clock cycles (about two seconds).  A wait that runs out
+// makes its CTA unwind and record PRQ_ERR_TIMEOUT; it never spins without bound.
+constexpr long long kDefaultWaitLimitCycles = 4000000000ll;
+
 struct QuantParams {
     const uint16_t* x;       // M x K bf16, row stride ldx
     int M, ldx, K, k_tail;
@@ -54,13 +58,6 @@ struct QuantBatch {
 };
 cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStream_t stream);
 
-// Which GEMM variant to run.
-enum class GemmKind {
-    kPrefill,  // tokens on the MMA M axis (128-row tiles), weights on the N axis, persistent CTAs
-    kGrouped,  // prefill layout with per-expert row ranges
-    kGroupedSwap  // per-expert row ranges with the weights on the MMA M axis and a 128-token group on N
-};
-
 struct GemmParams {
     int M;                   // activation rows (all experts)
     int N, K, k_tail;
@@ -78,11 +75,10 @@ struct GemmParams {
     int dbg;                 // developer switches for timing experiments (0 in normal use)
 };
 
-// Creates the tensor maps and launches.  `bn` is the N-axis tile (weights rows for prefill / grouped,
-// tokens for decode).  Returns cudaSuccess or the launch error; sets *unsupported when `bn` has no
-// compiled instance.
-cudaError_t launch_gemm(GemmKind kind, int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w,
-                        const GemmParams& p, int grid, cudaStream_t stream, bool* unsupported);
+// Grouped (MoE) kernel: 128 output features of one expert on the MMA M axis, one 128-token group of that expert
+// on the N axis; `grid` persistent CTAs.  `tm_act` / `tm_w` have 128-row boxes.
+cudaError_t launch_gemm_grouped(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
+                                cudaStream_t stream);
 
 
 // Decode kernel (M <= 128): cluster split-K with a distributed-shared-memory reduction.
@@ -153,6 +149,7 @@ struct PrefillParams {
     int* status;
     long long* trace;
     int dbg;
+    long long wait_limit;       // SM clock cycles after which a wait inside the kernel gives up (PRQ_ERR_TIMEOUT)
 };
 // `bn` = tile width (kPrefillTileN or kPrefillTileWide).  `tm_w` has boxes of bn / 2 rows; `tm_sfa` / `tm_sfw` view the scale bytes as rows of 256 bytes with boxes of
 // 4 / 8 rows (one / two 128-row groups); `tm_y` has 32 x 32 boxes.

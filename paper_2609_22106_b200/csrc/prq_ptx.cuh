@@ -77,7 +77,8 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 // then raises the flag itself.  The caller unwinds to the common teardown.
 constexpr long long kWaitLimitCycles = 4000000000ll;  // about two seconds
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit_cycles = kWaitLimitCycles) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
@@ -85,12 +86,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 0xff) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 *abort_flag = 1;
                 return false;
             }
         }
     }
+}
+// The same wait for a CTA that has already given up (its abort flag is set, so mbar_wait would return at
+// once) but must not leave while peers may still deliver into its shared memory: bounded by cycles only.
+__device__ __forceinline__ bool mbar_wait_after_abort(uint32_t bar, uint32_t parity, long long limit_cycles = kWaitLimitCycles) {
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0xff) == 0 && clock64() - t0 > limit_cycles) return false;
+    }
+    return true;
 }
 
 // ---------------------------------------------------------------- TMA

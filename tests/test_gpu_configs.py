@@ -79,6 +79,24 @@ def test_stack_layers_decode_64(prq, oracle, layer):
                    n_rows=4, bf16_too=False)
 
 
+@pytest.mark.parametrize("name,N,K", [(n, N, K) for n, N, K, _ in BLOCK])
+def test_stack_layer_prefill_4096(prq, oracle, name, N, K):
+    """The stack workload's prefill leg: block shapes with k = 256 on EVERY linear at 4096 tokens (K + k = 2816 is
+    eleven reduction stages on the q / k / v / gate / up shapes), online scale + permutation, one layer's weights."""
+    i = [b[0] for b in BLOCK].index(name)
+    dense_case(prq, oracle, config=4, tag=500 + i, N=N, K=K, k=256, M=4096, mode=prq.ACT_SCALE_PERM, n_rows=6,
+               bf16_too=(name in ("kv", "down")))
+
+
+def test_gate_up_stacked_prefill_and_decode(prq, oracle):
+    """gate and up stacked into one 19456-row layer (one scaling, permutation and tail for the pair), as the
+    benchmark's grouped-preparation step runs them: 4096 tokens and decode batch 64."""
+    dense_case(prq, oracle, config=2, tag=7, N=19456, K=2560, k=128, M=4096, mode=prq.ACT_SCALE_PERM, n_rows=4,
+               bf16_too=False)
+    dense_case(prq, oracle, config=4, tag=507, N=19456, K=2560, k=256, M=64, mode=prq.ACT_SCALE_PERM, n_rows=4,
+               bf16_too=False)
+
+
 @pytest.mark.parametrize("T", [64, 1024, 8192])
 def test_moe_grouped_zipf(prq, oracle, T):
     """128 experts 2048 x 768 with k = 64, T tokens routed top-8 with Zipf(1.1) popularity.  The library preps

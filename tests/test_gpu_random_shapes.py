@@ -72,7 +72,7 @@ def test_random_grouped_shapes_against_oracle(prq, oracle, seed):
     """Stacked experts with random row counts (empty experts included), strided activations and outputs."""
     rng = np.random.default_rng(seed)
     for case in range(8):
-        E = int(rng.choice([2, 3, 5, 8, 16]))
+        E = int(rng.choice([1, 2, 3, 5, 8, 16]))   # one expert: the grouped layout coincides with the dense one
         K = int(rng.integers(1, 16)) * 32
         k = int(rng.integers(0, min(K // 32, 4) + 1)) * 32
         N = int(rng.choice([16, 100, 128, 136, 256, 300]))
