@@ -403,7 +403,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         // (rows and columns outside M x N are clipped by the tensor map)
         // first column of a right edge narrower than 16 bytes, or -1 if N is a multiple of 16 bytes
         const int ragged_col = (p.N % (p.y_bf16 ? 8 : 4)) ? p.N - p.N % (p.y_bf16 ? 8 : 4) : -1;
-        auto store_chunk = [&](const uint32_t (&v)[32], int x, int y_row, int cols) {
+        // `own_buf`: shared address of a staging buffer that belongs to this chunk alone (the CTA's last tile, see
+        // below), or 0 for the warp's two alternating buffers
+        auto store_chunk = [&](const uint32_t (&v)[32], int x, int y_row, int cols, uint32_t own_buf = 0) {
             // A tiled store clips at the tensor's edge in units of 16 bytes: where N is not a multiple of that,
             // it would fill the last column group up with zeros, i.e. write into the caller's bytes between
             // column N and the row stride.  That one chunk goes out with plain stores instead.
@@ -448,10 +450,12 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 }
                 return;
             }
-            const uint32_t sbuf = stage_smem + (store_it & 1) * 4096;
-            // the store issued two chunks ago has finished reading this buffer
-            if (lane == 0) bulk_wait_read<1>();
-            __syncwarp();
+            const uint32_t sbuf = own_buf ? own_buf : stage_smem + (store_it & 1) * 4096;
+            if (!own_buf) {
+                // the store issued two chunks ago has finished reading this buffer
+                if (lane == 0) bulk_wait_read<1>();
+                __syncwarp();
+            }
             if (!p.y_bf16) {
                 // 128-byte staging rows, 16-byte unit index ^= row % 8
 #pragma unroll
@@ -601,6 +605,21 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                 int first, P;
                 plan_sk.participants(sg.tile, g, first, P);
                 fix[n_fix++] = Fixup{sg.tile, first, P};
+            } else if (r.cur >= r.end && r.whole_left == 0 && !(kTraceBuild && (p.dbg & 4))) {
+                // The CTA's last tile.  Nothing overlaps this epilogue, and with two staging buffers per warp it
+                // runs at the latency of the stores (a chunk waits for the store issued two chunks earlier).  The
+                // pipeline ring is idle by now -- the accumulator is complete, so every load has landed and every
+                // tensor-core read of both CTAs' shared memory is done -- and gives every chunk a staging buffer
+                // of its own: the warp reads the accumulator and issues its stores without ever waiting for one.
+                const int y_row = mi * 256 + static_cast<int>(rank) * 128 + q4 * 32;
+                const uint32_t own0 = smem_base + static_cast<uint32_t>((warp - 2) * kChunks) * 4096u;
+                static_assert(4 * kChunks * 4096 <= kStages * kStageBytes, "one staging buffer per warp and chunk fits the ring");
+#pragma unroll 1
+                for (int c = 0; c < kChunks; ++c) {
+                    uint32_t v[32];
+                    const int cols = load_chunk(acc_t, c, v);
+                    store_chunk(v, ni * BN + c * kChunkCols, y_row, cols, own0 + c * 4096u);
+                }
             } else {
                 const int y_row = mi * 256 + static_cast<int>(rank) * 128 + q4 * 32;
 #pragma unroll 1
