@@ -27,9 +27,12 @@ if ROOT not in sys.path:
 METRIC = "PRQuant W4A4 GEMM µs & TFLOP/s, Qwen3-4B down_proj; % of FP4/HBM roofline"
 N_OUT, K_IN, K_TAIL, M_TOK = 2560, 9728, 256, 2048
 FP4_OVER_BF16 = 4.0  # nominal dense tensor ratio (9 vs 2.25 PFLOP/s)
-# DRAM bytes of one prefill GEMM launch at this workload from the ncu capture summarised in
-# profiles/prefill_pair_M2048.txt (dram__bytes_read.sum + dram__bytes_write.sum; the outputs were still in L2).
+# DRAM bytes of one prefill GEMM launch at this workload: not a quantity of this run but the figure of the ncu
+# capture summarised in the file named here (dram__bytes_read.sum + dram__bytes_write.sum; the 21 MB of outputs
+# were still in L2 when the kernel ended, which is why it is below the algorithmic bytes).
 NCU_PREFILL_DRAM_BYTES = 24.34e6 + 2.18e6
+NCU_PREFILL_SOURCE = "profiles/prefill_pair_M2048.txt"
+LONG_RUN_LAUNCHES = 2000   # GEMM launches of the power-capped regime reported as roofline.frac_long_run
 
 
 def peaks():
@@ -600,6 +603,56 @@ def main():
     bf16_us = {M: time_bf16(M, side_steps) for M in (1, 16, 128, M_TOK)}
     k0 = detail[f"M{M_TOK}_k0"]
 
+    # ---- the headline GEMM over a fixed, long run: LONG_RUN_LAUNCHES launches back to back, whatever --steps was,
+    # so that the fraction cannot move with the step count (a short run stays ahead of the power cap) ----
+    with ClockSampler(physical_gpu_index(local_rank)) as long_clocks:
+        long_s = run_timed(main_graphs["gemm"], LONG_RUN_LAUNCHES, main_graphs["R"])
+    long_us = long_s / LONG_RUN_LAUNCHES * 1e6
+
+    # ---- the floor under the latency-bound decode calls: what one dependent launch costs with nothing in it
+    # (programmatic dependent launch, the decode GEMM's grid of 160 CTAs in clusters of 8) ----
+    def handover_us(grid, threads, cluster, n=200):
+        g = timer.capture([lambda: prq.handover_probe(n, grid, threads, cluster)])
+        g.replay()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(5):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) * 1e3 / (5 * n)
+    decode_floor = {"handover_us_160x192_cluster8": handover_us(160, 192, 8), "handover_us_148x192": handover_us(148, 192, 1),
+                    "hbm_floor_us": {f"M{M}": gemm_bytes(M, K_TAIL) / pk["hbm_gbs"] / 1e3 for M in (1, 16, 128)},
+                    "what": "time per launch of a chain of empty kernels that wait for one another, launched like the "
+                            "decode GEMM; a dependent decode call cannot take less than this plus its HBM time"}
+    for M in (1, 16, 128):
+        d = detail[f"M{M}_k{K_TAIL}"]
+        d["gemm_us_over_floor"] = d["gemm_us"] - (decode_floor["hbm_floor_us"][f"M{M}"] + decode_floor["handover_us_160x192_cluster8"])
+
+    # ---- the host link the end-to-end number rides on ----
+    def copy_gbs(dst, src, n=5):
+        dst.copy_(src, non_blocking=True)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            dst.copy_(src, non_blocking=True)
+        b.record()
+        torch.cuda.synchronize()
+        return src.numel() * src.element_size() * n / (a.elapsed_time(b) * 1e-3) / 1e9
+    xdev = torch.empty_like(xh0, device=dev)
+    link = {"h2d_gbs": copy_gbs(xdev, lanes[0]["x"]), "d2h_gbs": copy_gbs(lanes[0]["x"], xdev)}
+    try:
+        import pynvml
+
+        pynvml.nvmlInit()
+        h = pynvml.nvmlDeviceGetHandleByIndex(physical_gpu_index(local_rank))
+        link["pcie_gen"] = int(pynvml.nvmlDeviceGetCurrPcieLinkGeneration(h))
+        link["pcie_width"] = int(pynvml.nvmlDeviceGetCurrPcieLinkWidth(h))
+    except Exception:
+        pass
+
     # ---- CPU baseline: the oracle on a bounded sample of the same workload ----
     cpu = None
     if not args.no_cpu_baseline:
@@ -634,7 +687,7 @@ def main():
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "mxfp4 (e2m1 x e8m0), f32 accumulate", "data": "synthetic",
-        "config": {"workload": f"qwen3-4b down_proj N={N_OUT} K={K_IN} k_tail={K_TAIL} M={M_TOK} (BASELINE configs[1]); "
+        "config": {"workload": f"qwen3-4b down_proj N={N_OUT} K={K_IN} k_tail={K_TAIL} M={M_TOK}; "
                                "step = prq_quantize_act + prq_linear, fp32 output",
                    "l2": f"inputs larger than L2: steps rotate over {main_t['rotation_sets']} independent operand sets "
                          "(weights, activations, outputs), more than twice the 126 MB L2 per rotation; no flush",
@@ -645,14 +698,19 @@ def main():
                "bf16_matmul": bf16_us[M_TOK], "gemm_speedup_vs_bf16": bf16_us[M_TOK] / main_t["gemm_us"]},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": fp4_peak, "unit": "TFLOP/s",
                      "frac": achieved / fp4_peak, "frac_of_sustained": achieved / (pk["bf16_tflops_sustained"] * FP4_OVER_BF16),
-                     "traffic": NCU_PREFILL_DRAM_BYTES, "algorithmic_bytes": gemm_bytes(M_TOK, K_TAIL),
+                     "frac_long_run": flops(M_TOK, K_TAIL) / long_us / 1e6 / fp4_peak, "long_run_launch_us": long_us,
+                     "long_run_launches": LONG_RUN_LAUNCHES, "long_run_clocks": long_clocks.summary(),
+                     "traffic": NCU_PREFILL_DRAM_BYTES, "traffic_source": NCU_PREFILL_SOURCE + " (ncu capture, not this run)",
+                     "algorithmic_bytes": gemm_bytes(M_TOK, K_TAIL),
                      "kernel": "prefill_pair_kernel<240> (CTA pairs, 256x240 tiles, whole tiles + stream-K pieces)", "launch_us": gemm_us,
                      "peak_source": f"4 x bf16 burst, of {pk['source']}",
                      "frac_of_measured_mxf4_probe": achieved / mxf4_probe["burst_1.5ms"],
                      "frac_of_nominal_9pf": achieved / 9000.0},
         "mxf4_probe": mxf4_probe,
         "cpu_baseline": cpu,
-        "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": M_TOK * K_IN * 2, "d2h_bytes_per_step": M_TOK * N_OUT * 4},
+        "e2e": {"value": e2e_val, "unit": "TFLOP/s", "h2d_bytes_per_step": M_TOK * K_IN * 2, "d2h_bytes_per_step": M_TOK * N_OUT * 4,
+                "link": link},
+        "decode_floor": decode_floor,
         "gpu_launches": int(launches),
         "clocks": clocks.summary(),
         "device_status": status,

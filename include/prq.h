@@ -331,6 +331,13 @@ unsigned long long prq_kernel_launch_count(void);
  * the number of CTAs launched.  Errors: INVALID_ARG, CUDA. */
 prq_status prq_mxf4_peak_probe(int n_mma, int *n_ctas, prq_stream_t stream);
 
+/* Benchmark utility (the paper has no counterpart): enqueues, on `stream`, n empty kernels, each launched the way
+ * the decode GEMM is (programmatic dependent launch; `grid` CTAs of `threads` threads in clusters of `cluster`
+ * CTAs) and each waiting for the one before it.  The caller times the chain; time / n is what one dependent
+ * launch costs on this GPU before any work is done -- the floor under every latency-bound call of this library.
+ * n: 1 .. 4096; grid a multiple of cluster; cluster 1 .. 8.  Errors: INVALID_ARG, CUDA. */
+prq_status prq_handover_probe(int n, int grid, int threads, int cluster, prq_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

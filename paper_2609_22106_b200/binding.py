@@ -27,6 +27,7 @@ EXPORTS = [
     "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_multi", "prq_quantize_act_multi",
     "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
+    "prq_handover_probe",
 ]
 
 
@@ -80,6 +81,7 @@ def lib():
         L.prq_last_device_status.argtypes = [vp]
         L.prq_kernel_launch_count.restype = ctypes.c_ulonglong
         L.prq_mxf4_peak_probe.argtypes = [ci, ctypes.POINTER(ci), vp]
+        L.prq_handover_probe.argtypes = [ci, ci, ci, ci, vp]
         _lib = L
     return _lib
 
@@ -300,10 +302,11 @@ def linear(w: Weights, codes, scales_sf, M: int, y_dtype: int = F32, workspace=N
 
     if out is None:
         out = torch.empty((M, w.N), dtype=torch.float32 if y_dtype == F32 else torch.bfloat16, device=codes.device)
-    if workspace is None:
+    if workspace is None and M > 128:   # up to 128 tokens the kernel needs no scratch: nothing to allocate or clear
         workspace = new_workspace(w, M, codes.device)
     _check(lib().prq_linear(w.handle, _dptr(codes), _dptr(scales_sf), M, _dptr(out), out.stride(0) if M else w.N,
-                            y_dtype, _dptr(workspace), workspace.numel(), _stream_ptr(stream)), "prq_linear")
+                            y_dtype, _dptr(workspace), workspace.numel() if workspace is not None else 0,
+                            _stream_ptr(stream)), "prq_linear")
     return out
 
 
@@ -416,3 +419,9 @@ def mxf4_peak_probe(n_mma: int, stream=None) -> int:
     n = ctypes.c_int()
     _check(lib().prq_mxf4_peak_probe(int(n_mma), ctypes.byref(n), _stream_ptr(stream)), "prq_mxf4_peak_probe")
     return n.value
+
+
+def handover_probe(n: int, grid: int, threads: int = 192, cluster: int = 1, stream=None) -> None:
+    """Enqueues n empty, dependent launches shaped like the decode GEMM's (see include/prq.h); the caller times them."""
+    _check(lib().prq_handover_probe(int(n), int(grid), int(threads), int(cluster), _stream_ptr(stream)),
+           "prq_handover_probe")

@@ -20,6 +20,7 @@ namespace prq {
 namespace {
 
 __device__ int g_device_status = 0;
+__device__ int g_probe_sink = 0;   // the hand-over probe's kernels count themselves here; nothing reads it
 
 std::atomic<unsigned long long> g_launches{0};
 
@@ -299,6 +300,21 @@ prq_status prq_mxf4_peak_probe(int n_mma, int* n_ctas, prq_stream_t stream) {
     if (n_ctas) *n_ctas = di->num_sms;
     cudaError_t e = launch_mxf4_peak_probe(n_mma, di->num_sms, di->status_ptr, static_cast<cudaStream_t>(stream));
     g_launches.fetch_add(1);
+    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
+prq_status prq_handover_probe(int n, int grid, int threads, int cluster, prq_stream_t stream) {
+    if (n < 1 || n > 4096 || grid < 1 || threads < 32 || threads > 1024 || cluster < 1 || cluster > 8 || grid % cluster)
+        return PRQ_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return PRQ_ERR_CUDA;
+    DeviceInfo* di;
+    prq_status st = device_info(dev, &di);
+    if (st != PRQ_OK) return st;
+    void* sink = nullptr;
+    if (cudaGetSymbolAddress(&sink, g_probe_sink) != cudaSuccess) return PRQ_ERR_CUDA;
+    cudaError_t e = launch_handover_probe(n, grid, threads, cluster, static_cast<int*>(sink), static_cast<cudaStream_t>(stream));
+    g_launches.fetch_add(n);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
 }
 

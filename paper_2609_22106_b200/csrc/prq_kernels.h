@@ -162,4 +162,8 @@ int prefill_pair_max_clusters(int bn);
 // Benchmark utility: `grid` CTAs each issuing n_mma block-scaled FP4 MMAs (128 x 256 x 64) from shared memory.
 cudaError_t launch_mxf4_peak_probe(int n_mma, int grid, int* status, cudaStream_t stream);
 
+// Benchmark utility: `n` empty kernels in a row, each launched like the decode GEMM (programmatic dependent
+// launch, `grid` CTAs of `threads` threads in clusters of `cluster`) and each waiting for the one before it.
+cudaError_t launch_handover_probe(int n, int grid, int threads, int cluster, int* sink, cudaStream_t stream);
+
 }  // namespace prq

@@ -68,7 +68,37 @@ __global__ void __launch_bounds__(64, 1) mxf4_peak_kernel(int n_mma, int* status
     if (threadIdx.x == 0 && abort_s) atomicExch(status, static_cast<int>(PRQ_ERR_TIMEOUT));
 }
 
+// One link of a chain of dependent launches with nothing in it: every CTA lets the next kernel of the stream be
+// scheduled, waits for the previous one to finish, writes one word (so that the dependency is a real one) and
+// leaves.  `grid` CTAs of `threads` threads in clusters of `cluster` -- the launch shape of the decode GEMM.
+__global__ void handover_probe_kernel(int* sink) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    if (threadIdx.x == 0 && blockIdx.x == 0) atomicAdd(sink, 1);
+}
+
 }  // namespace
+
+cudaError_t launch_handover_probe(int n, int grid, int threads, int cluster, int* sink, cudaStream_t stream) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(threads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = cluster;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    for (int i = 0; i < n; ++i) {
+        cudaError_t e = cudaLaunchKernelEx(&cfg, handover_probe_kernel, sink);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
 
 cudaError_t launch_mxf4_peak_probe(int n_mma, int grid, int* status, cudaStream_t stream) {
     static bool configured = false;
