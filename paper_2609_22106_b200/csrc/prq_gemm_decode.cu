@@ -182,14 +182,12 @@ decode_kernel(const __grid_constant__ DecodeMaps maps, const DecodeBatch b) {
     tc_fence_after_sync();
     // Split-K exchange, receiving side: this CTA owns tokens split, split + splits, ...; every CTA of the
     // cluster (itself included) delivers 512 bytes per owned token, counted on bar_recv.  The cluster
-    // barrier only tells the peers that the barrier exists before they push.
+    // barrier only tells the peers that the barrier exists before they push: arrive here, wait just before
+    // the pushes, so that it costs nothing.
     const int n_own = split < p.M ? (p.M - split + splits - 1) / splits : 0;
     if (C::kAsyncExchange && splits > 1) {
         if (threadIdx.x == 0) mbar_arrive_expect_tx(smem_u32(&bar_recv), static_cast<uint32_t>(n_own) * splits * 512u);
-        // Both halves of the barrier here, in the set-up: under programmatic dependent launch this part of the
-        // kernel runs while the previous kernel is still busy, whereas a wait placed in front of the pushes sits
-        // in the dependent chain.
-        cluster_sync_all();
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     }
     // set-up done: let the next kernel of the stream be scheduled (its launch latency then overlaps this
     // kernel).  The roles that touch what earlier kernels wrote (activation codes and scales) or may
@@ -391,6 +389,8 @@ decode_kernel(const __grid_constant__ DecodeMaps maps, const DecodeBatch b) {
         const int slots = (p.M + splits - 1) / splits;        // token slots per peer in a receive buffer
         const int et = threadIdx.x - 64;                        // 0..127 for the epilogue warps
         const int j = et & 31, tq = et >> 5;
+        if constexpr (C::kAsyncExchange)
+            asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // every peer's bar_recv exists
         if (warp >= 2 && !abort_flag_s) {
             asm volatile("bar.sync 1, %0;" ::"n"(32 * C::kEpiWarps) : "memory");   // the parked tile is complete
             for (int tok = tq; tok < p.M; tok += C::kEpiWarps) {
