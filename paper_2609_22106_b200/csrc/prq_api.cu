@@ -122,18 +122,24 @@ prq_status make_out_map(CUtensorMap* map, void* y, int M, int N, int ldy, bool b
     return r == CUDA_SUCCESS ? PRQ_OK : PRQ_ERR_CUDA;
 }
 
+constexpr int kNumAlt = 3;
+constexpr int kAltTileRows[kNumAlt] = {kPrefillTileN, kPrefillTileWide, kPrefillTileOneWave};  // weight tile widths of the prefill kernel, each with its own scale layout
+
 // Weight-side tensor maps of a dense handle, encoded once at creation (cloning re-encodes: other addresses).
 prq_status build_weight_maps(prq_weights* w) {
     w->maps_ready = false;
     if (w->n_experts != 1) return PRQ_OK;
     const uint64_t Ka = static_cast<uint64_t>(w->K) + w->k_tail;
     prq_status st = make_code_map(&w->tm_w_decode, w->d_codes, Ka / 2, w->N, 128);
-    for (int v = 0; v < 2; ++v) {   // 224- and 240-row tilings
-        if (st == PRQ_OK) st = make_code_map(&w->tm_w_pair[v], w->d_codes, Ka / 2, w->N, (v ? kPrefillTileWide : kPrefillTileN) / 2);
+    for (int v = 0; v < kNumAlt; ++v) {   // 224-, 240- and 288-row tilings
+        const int rows = kAltTileRows[v], gpt = (rows + kGroupRows - 1) / kGroupRows;
+        // each CTA of a pair loads half a tile; the 288-row tile as 128 + 16 rows (second map)
+        if (st == PRQ_OK) st = make_code_map(&w->tm_w_pair[v], w->d_codes, Ka / 2, w->N, rows > 256 ? 128 : rows / 2);
         if (st == PRQ_OK && w->d_sf_alt[v])
             st = make_sf_map(&w->tm_sfw_pair[v], w->d_sf_alt[v],
-                             static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[v] * kSfGroupBytes, 8);
+                             static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[v] * kSfGroupBytes, 4 * gpt);
     }
+    if (st == PRQ_OK) st = make_code_map(&w->tm_w_tail, w->d_codes, Ka / 2, w->N, 16);
     if (st == PRQ_OK) w->maps_ready = true;
     return st;
 }
@@ -205,8 +211,6 @@ int decode_splits(const prq_weights* w, int M, DeviceInfo* di) {
     return decode_splits_for((w->N + 127) / 128, w->plan.S, M, di);
 }
 
-constexpr int kNumAlt = 2;
-constexpr int kAltTileRows[kNumAlt] = {kPrefillTileN, kPrefillTileWide};  // weight tile widths of the prefill kernel, each with its own scale layout
 
 // How the pair kernel shares out the tiles of one call: every pair gets `whole` whole tiles; the `sk`
 // tiles left over are each cut into equal pieces for `base` (the first `extra` tiles: base + 1)
@@ -247,13 +251,23 @@ PairSchedule pair_schedule(int bn, int M, int N, int S, int max_pairs) {
 // (33792 with 224-column tiles, 34816 with 240-column ones), so the width whose busiest pair takes in
 // fewer bytes wins; 224 on a tie.  With the paper's down projection that is 240 from 2048 tokens on
 // (11 instead of 12 column tiles) and 224 below (the tile counts do not fill the pairs either way).
+// Third width, 288 columns with a single accumulator: only where every tile of the call fits ONE wave of pairs at
+// that width while the narrower tilings would leave tiles over (so that they need a second wave or stream-K
+// pieces).  Every pair then runs one tile's reduction and one epilogue, nothing is published or fixed up.  The
+// paper's down projection at 2048 tokens is such a call: 8 x 9 = 72 tiles on 74 pairs instead of 88 tiles of which
+// 14 are cut into four pieces.
 PairSchedule choose_pair_schedule(int M, int N, int S, int max_pairs) {
     const PairSchedule narrow = pair_schedule(kPrefillTileN, M, N, S, max_pairs);
     const PairSchedule wide = pair_schedule(kPrefillTileWide, M, N, S, max_pairs);
+    const PairSchedule one = pair_schedule(kPrefillTileOneWave, M, N, S, max_pairs);
+    const bool one_ok = one.tiles <= max_pairs && one.whole == 0 && one.base == 1 && one.extra == 0;
     const int forced = env_int("PRQ_PAIR_BN", 0);
     if (forced == kPrefillTileN) return narrow;
     if (forced == kPrefillTileWide) return wide;
-    return wide.stages_per_pair * 34816 < narrow.stages_per_pair * 33792 ? wide : narrow;
+    if (forced == kPrefillTileOneWave && one_ok) return one;
+    const PairSchedule best = wide.stages_per_pair * 34816 < narrow.stages_per_pair * 33792 ? wide : narrow;
+    if (one_ok && forced == 0 && best.stages_per_pair > S) return one;
+    return best;
 }
 
 // Two counters ("arrived", "finished") per 128-row half of a 256 x 224 pair tile: first all the "arrived"
@@ -404,7 +418,7 @@ static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_
         std::vector<float> inv_s_perm(E * K);
         std::vector<uint8_t> sf_alt[kNumAlt];
         for (int a = 0; a < kNumAlt && E == 1; ++a) {
-            w->w_groups_alt[a] = ((N + kAltTileRows[a] - 1) / kAltTileRows[a]) * 2;
+            w->w_groups_alt[a] = ((N + kAltTileRows[a] - 1) / kAltTileRows[a]) * ((kAltTileRows[a] + kGroupRows - 1) / kGroupRows);
             sf_alt[a].assign((static_cast<size_t>(S) * w->w_groups_alt[a] + 4) * kSfGroupBytes, 0);
         }
         PrepResult r;
@@ -429,8 +443,8 @@ static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_
                     const int bis = b < nblk_main ? b % nb : (b - nblk_main) % nb;
                     sf[((e * S + stage) * w->w_groups + g) * kSfGroupBytes + sf_offset_in_group(rr, bis)] = srow[b];
                     for (int a = 0; a < kNumAlt && E == 1; ++a) {
-                        const int tile_rows = kAltTileRows[a];
-                        const int ga = (n / tile_rows) * 2 + (n % tile_rows) / kGroupRows;
+                        const int tile_rows = kAltTileRows[a], gpt = (tile_rows + kGroupRows - 1) / kGroupRows;
+                        const int ga = (n / tile_rows) * gpt + (n % tile_rows) / kGroupRows;
                         sf_alt[a][(static_cast<size_t>(stage) * w->w_groups_alt[a] + ga) * kSfGroupBytes +
                                   sf_offset_in_group((n % tile_rows) % kGroupRows, bis)] = srow[b];
                     }
@@ -837,10 +851,10 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         PrefillParams q;
         std::memset(&q, 0, sizeof(q));
         if (di->max_pairs == 0)
-            di->max_pairs = std::min(std::min(prefill_pair_max_clusters(kPrefillTileN), prefill_pair_max_clusters(kPrefillTileWide)),
-                                     di->num_sms / 2);
+            di->max_pairs = std::min(std::min(std::min(prefill_pair_max_clusters(kPrefillTileN), prefill_pair_max_clusters(kPrefillTileWide)),
+                                              prefill_pair_max_clusters(kPrefillTileOneWave)), di->num_sms / 2);
         const PairSchedule ps = choose_pair_schedule(M, w->N, w->plan.S, std::min(di->max_pairs, env_int("PRQ_GRID", 1 << 20)));
-        const int pair_bn = ps.bn, variant = pair_bn == kPrefillTileWide ? 1 : 0, pairs = ps.pairs;
+        const int pair_bn = ps.bn, variant = pair_bn == kPrefillTileOneWave ? 2 : pair_bn == kPrefillTileWide ? 1 : 0, pairs = ps.pairs;
         if (pairs < 1) return PRQ_ERR_CUDA;
         q.M = M; q.N = w->N; q.K = w->K; q.k_tail = w->k_tail;
         q.m_tiles = (M + 255) / 256; q.n_tiles = (w->N + pair_bn - 1) / pair_bn;
@@ -871,8 +885,8 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         if (st == PRQ_OK) st = make_sf_map(&tm_sfa, p.act_sf, Sg * p.act_groups * kSfGroupBytes, 4);
         if (st == PRQ_OK) st = make_out_map(&tm_y, y, M, w->N, ldy, y_dtype == PRQ_BF16);
         if (st != PRQ_OK) return st;
-        cudaError_t e = launch_prefill_pair(pair_bn, tm_act, w->tm_w_pair[variant], tm_sfa, w->tm_sfw_pair[variant], tm_y, q, pairs,
-                                            static_cast<cudaStream_t>(stream));
+        cudaError_t e = launch_prefill_pair(pair_bn, tm_act, w->tm_w_pair[variant], w->tm_w_tail, tm_sfa, w->tm_sfw_pair[variant], tm_y, q,
+                                            pairs, static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     }

@@ -49,32 +49,39 @@ namespace {
 constexpr int kThreads = 192;
 constexpr int kPTile = 128 * 128;                 // activation tile bytes (128 rows x 256 codes)
 constexpr int kSfp = kSfGroupBytes;               // 1 group of 128 activation rows
-constexpr int kSfq = 2 * kSfGroupBytes;           // 2 groups (128 + up to 128 weight rows)
 constexpr int kStages = 5;
 constexpr int kStagingPerWarp = 2 * 4096;         // two 32-row x 128-byte chunks per epilogue warp
 constexpr int kTmemCols = 512;
-constexpr int kSfSetCols = 24;                    // 8 activation + 16 weight scale columns
 constexpr int kChunkCols = 32;                    // accumulator columns per epilogue chunk
 
-// Everything that depends on the tile width BN (weight rows per tile): 224 or 240.  Two accumulators of
-// BN columns and the scale columns must fit the 512 columns of tensor memory, which 240 still does; the
-// wider tile needs fewer operand bytes per multiply-add, its main loop runs within a few percent of the tensor
-// time, and it pads N = 2560 less (11 x 240 against 12 x 224).
+// Everything that depends on the tile width BN (weight rows per tile): 224, 240 or 288.
+//   224 / 240: two accumulators of BN columns and the scale columns must fit the 512 columns of tensor memory,
+//   which 240 still does; the wider tile needs fewer operand bytes per multiply-add, its main loop runs within a
+//   few percent of the tensor time, and it pads N = 2560 less (11 x 240 against 12 x 224).
+//   288: ONE accumulator, for calls whose tiles all fit one wave of pairs at this width (the host decides): no
+//   pair takes a second tile, so nothing needs a second accumulator, and no tile is split along K.  An MMA takes at
+//   most 256 columns, so a reduction step is two instructions (256 + 32 columns); each CTA loads 128 + 16 weight
+//   rows so that the accumulator's columns are the tile's weight rows in order.
 template <int BN>
 struct PCfg {
+    static constexpr bool kWide = BN > 256;
     static constexpr int kHalfN = BN / 2;                    // weight rows each CTA of the pair loads
     static constexpr int kQTile = kHalfN * 128;              // half weight tile bytes
-    static constexpr int kStageBytes = kPTile + kQTile + kSfp + kSfq;  // 33792 / 34816
+    static constexpr int kSfqGroups = (BN + 127) / 128;      // 128-row scale groups of a weight tile
+    static constexpr int kSfq = kSfqGroups * kSfGroupBytes;
+    static constexpr int kStageBytes = kPTile + kQTile + kSfp + kSfq;  // 33792 / 34816 / 38912
     static constexpr int kSmemBytes = kStages * kStageBytes + 4 * kStagingPerWarp + 1024;
-    static constexpr int kSfCol = 2 * BN;                    // scale columns start behind the two accumulators
-    static constexpr int kChunks = (BN + kChunkCols - 1) / kChunkCols;   // 7, or 7 and a 16-column one
+    static constexpr int kAccBufs = kWide ? 1 : 2;
+    static constexpr int kSfCol = kAccBufs * BN;             // scale columns start behind the accumulator(s)
+    static constexpr int kSfSetCols = 8 + 8 * kSfqGroups;    // 8 activation + 8 per weight group
+    static constexpr int kChunks = (BN + kChunkCols - 1) / kChunkCols;   // 7, 7 and a 16-column one, or 9
     static constexpr int kLastCols = BN - (kChunks - 1) * kChunkCols;    // 32 or 16
     static constexpr int kSlotUnits = kChunks * 8 * 128;     // float4 per workspace slot (128 rows)
     static_assert(kQTile % 1024 == 0 && kStageBytes % 1024 == 0, "operand tiles must keep 1024-byte alignment");
     static_assert(kSmemBytes <= 232448 - 256, "shared memory budget");
     static_assert(kSfCol + kSfSetCols <= kTmemCols, "tensor memory budget");
     static_assert(kLastCols == 32 || kLastCols == 16, "epilogue chunks are 32 columns, the last one 32 or 16");
-    static_assert(static_cast<size_t>(kSlotUnits) * 16 <= kPrefillSlotBytes, "workspace slot");
+    static_assert(kWide || static_cast<size_t>(kSlotUnits) * 16 <= kPrefillSlotBytes, "workspace slot");
 };
 
 __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src_smem, int x, int y) {
@@ -177,39 +184,61 @@ __device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo) { return (s
 
 // One reduction stage of the issue loop with the ring slot Q known at compile time: every
 // shared-memory descriptor is `lo_base` plus a constant.  Scale atoms first -- activation group
-// (columns +0 / +4 for the two halves of the stage), weight groups 0 and 1 (columns +8, +12 / +16, +20)
-// -- then up to four K = 64 MMAs, then the commit that frees the slot in both CTAs.  The copies and
-// the MMAs are issued by one thread, so tensor memory sees them in order and one set of scale columns
-// is enough.  `rem` = reduction elements this stage still covers.
+// (columns +0 / +4 for the two halves of the stage), then the weight groups (G = 2 or 3 of them: columns
+// +8 + 4 g for the first half of the stage, +8 + 4 G + 4 g for the second) -- then up to four K = 64 steps,
+// then the commit that frees the slot in both CTAs.  A step is one MMA over all BN columns, or for the
+// 288-column tile two (256 columns, then the 32 columns of the third weight group into accumulator
+// columns 256 ..).  The copies and the MMAs are issued by one thread, so tensor memory sees them in order
+// and one set of scale columns is enough.  `rem` = reduction elements this stage still covers.
 template <int BN, int Q>
 __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, uint32_t sf_t, int rem,
                                             uint32_t accumulate, uint32_t empty_bar0) {
-    constexpr int kStageBytes = PCfg<BN>::kStageBytes, kQTile = PCfg<BN>::kQTile;
+    using C = PCfg<BN>;
+    constexpr int kStageBytes = C::kStageBytes, kQTile = C::kQTile, G = C::kSfqGroups;
     constexpr uint32_t so = (Q * kStageBytes) >> 4;  // stage offset in 16-byte units
     constexpr uint32_t sfo = so + ((kPTile + kQTile) >> 4);
-    // E2M1 x E2M1, E8M0 scales, both operands K-major, N = BN, M = 256 (two CTAs)
-    constexpr uint32_t idesc0 = (1u << 7) | (1u << 10) | ((BN >> 3) << 17) | (1u << 23) | ((256u >> 4) << 24);
+    // E2M1 x E2M1, E8M0 scales, both operands K-major, N = N1 (and N2), M = 256 (two CTAs)
+    constexpr int N1 = C::kWide ? 256 : BN, N2 = BN - N1;
+    constexpr uint32_t idesc0 = (1u << 7) | (1u << 10) | ((N1 >> 3) << 17) | (1u << 23) | ((256u >> 4) << 24);
     constexpr uint32_t idesc2 = idesc0 | (2u << 4) | (2u << 29);
+    constexpr uint32_t jdesc0 = (1u << 7) | (1u << 10) | (((N2 > 0 ? N2 : 16) >> 3) << 17) | (1u << 23) | ((256u >> 4) << 24);
+    constexpr uint32_t jdesc2 = jdesc0 | (2u << 4) | (2u << 29);
     const uint32_t plo = lo_base + so, qlo = lo_base + so + (kPTile >> 4), slo = lo_base + sfo;
     const uint32_t sfp_t = sf_t, sfq_t = sf_t + 8;
     tc_copy_sf_atom_pair(sf_t, desc64(kHiPlain, slo));
-    tc_copy_sf_atom_pair(sf_t + 8, desc64(kHiPlain, slo + (kSfp >> 4)));
-    tc_copy_sf_atom_pair(sf_t + 12, desc64(kHiPlain, slo + ((kSfp + kSfGroupBytes) >> 4)));
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+        tc_copy_sf_atom_pair(sfq_t + 4 * g, desc64(kHiPlain, slo + ((kSfp + g * kSfGroupBytes) >> 4)));
     if (rem > 128) {
         tc_copy_sf_atom_pair(sf_t + 4, desc64(kHiPlain, slo + (512 >> 4)));
-        tc_copy_sf_atom_pair(sf_t + 16, desc64(kHiPlain, slo + ((kSfp + 512) >> 4)));
-        tc_copy_sf_atom_pair(sf_t + 20, desc64(kHiPlain, slo + ((kSfp + kSfGroupBytes + 512) >> 4)));
+#pragma unroll
+        for (int g = 0; g < G; ++g)
+            tc_copy_sf_atom_pair(sfq_t + 4 * G + 4 * g, desc64(kHiPlain, slo + ((kSfp + g * kSfGroupBytes + 512) >> 4)));
     }
+    // the second instruction of a step reads the CTA's weight rows from row N1 / 2 on and the scale columns of
+    // the last group
+    constexpr uint32_t q2 = ((N1 / 2) * 128) >> 4, s2 = 4 * (G - 1);
     tc_mma_mxf4_pair(d_tmem, desc64(kHiSw128, plo), desc64(kHiSw128, qlo), idesc0, sfp_t, sfq_t, accumulate);
-    if (rem > 64) tc_mma_mxf4_pair(d_tmem, desc64(kHiSw128, plo + 2), desc64(kHiSw128, qlo + 2), idesc2, sfp_t, sfq_t, 1);
-    if (rem > 128) tc_mma_mxf4_pair(d_tmem, desc64(kHiSw128, plo + 4), desc64(kHiSw128, qlo + 4), idesc0, sfp_t + 4, sfq_t + 8, 1);
-    if (rem > 192) tc_mma_mxf4_pair(d_tmem, desc64(kHiSw128, plo + 6), desc64(kHiSw128, qlo + 6), idesc2, sfp_t + 4, sfq_t + 8, 1);
+    if (N2 > 0) tc_mma_mxf4_pair(d_tmem + N1, desc64(kHiSw128, plo), desc64(kHiSw128, qlo + q2), jdesc0, sfp_t, sfq_t + s2, accumulate);
+    if (rem > 64) {
+        tc_mma_mxf4_pair(d_tmem, desc64(kHiSw128, plo + 2), desc64(kHiSw128, qlo + 2), idesc2, sfp_t, sfq_t, 1);
+        if (N2 > 0) tc_mma_mxf4_pair(d_tmem + N1, desc64(kHiSw128, plo + 2), desc64(kHiSw128, qlo + q2 + 2), jdesc2, sfp_t, sfq_t + s2, 1);
+    }
+    if (rem > 128) {
+        tc_mma_mxf4_pair(d_tmem, desc64(kHiSw128, plo + 4), desc64(kHiSw128, qlo + 4), idesc0, sfp_t + 4, sfq_t + 4 * G, 1);
+        if (N2 > 0) tc_mma_mxf4_pair(d_tmem + N1, desc64(kHiSw128, plo + 4), desc64(kHiSw128, qlo + q2 + 4), jdesc0, sfp_t + 4, sfq_t + 4 * G + s2, 1);
+    }
+    if (rem > 192) {
+        tc_mma_mxf4_pair(d_tmem, desc64(kHiSw128, plo + 6), desc64(kHiSw128, qlo + 6), idesc2, sfp_t + 4, sfq_t + 4 * G, 1);
+        if (N2 > 0) tc_mma_mxf4_pair(d_tmem + N1, desc64(kHiSw128, plo + 6), desc64(kHiSw128, qlo + q2 + 6), jdesc2, sfp_t + 4, sfq_t + 4 * G + s2, 1);
+    }
     tc_commit_pair(empty_bar0 + Q * 8, 3);
 }
 
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
+                    const __grid_constant__ CUtensorMap tm_w_tail,
                     const __grid_constant__ CUtensorMap tm_sfa, const __grid_constant__ CUtensorMap tm_sfw,
                     const __grid_constant__ CUtensorMap tm_y, const PrefillParams p) {
     using C = PCfg<BN>;
@@ -252,6 +281,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         fence_mbar_init();
         tma_prefetch_desc(&tm_act);
         tma_prefetch_desc(&tm_w);
+        if (C::kWide) tma_prefetch_desc(&tm_w_tail);
         tma_prefetch_desc(&tm_sfa);
         tma_prefetch_desc(&tm_sfw);
         tma_prefetch_desc(&tm_y);
@@ -292,19 +322,27 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         // The weights do not depend on earlier kernels of the stream: the weight tiles and weight scales of
         // the first ring pass are requested before the dependency wait, so that their latency overlaps the
         // tail of the previous kernel.
+        // this CTA's half of the weight tile `ni` and the scale bytes of the whole tile, reduction stage s.
+        // 224 / 240 columns: rows [rank * BN / 2, + BN / 2) of the tile.  288 columns: rows [rank * 128, + 128) and
+        // [256 + rank * 16, + 16), so that the first instruction of a step covers the tile's first 256 rows in
+        // order and the second one the last 32.
+        auto load_weights = [&](uint32_t sb, int ni, int s, uint32_t full) {
+            const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
+            if (C::kWide) {
+                tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * 128, full);
+                tma_load_2d_pair(sb + kPTile + 128 * 128, &tm_w_tail, xw, ni * BN + 256 + static_cast<int>(rank) * 16, full);
+            } else {
+                tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * kHalfN, full);
+            }
+            tma_load_2d_pair(sb + kPTile + kQTile + kSfp, &tm_sfw, 0, ni * 4 * C::kSfqGroups + s * p.w_groups * 4, full);
+        };
         int pre = 0;
         {
             Range rr = r;
             while (pre < kStages && rr.next(sg)) {
                 const int ni = sg.tile / p.m_tiles;
                 for (int s = sg.s0; s < sg.s1 && pre < kStages; ++s, ++pre) {
-                    if (elect_one()) {
-                        const uint32_t full = leader_full0 + pre * 8;
-                        const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
-                        const uint32_t sb = smem_base + pre * kStageBytes;
-                        tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * kHalfN, full);
-                        tma_load_2d_pair(sb + kPTile + kQTile + kSfp, &tm_sfw, 0, ni * 8 + s * p.w_groups * 4, full);
-                    }
+                    if (elect_one()) load_weights(smem_base + pre * kStageBytes, ni, s, leader_full0 + pre * 8);
                 }
             }
         }
@@ -318,22 +356,17 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             const int mi = sg.tile % p.m_tiles, ni = sg.tile / p.m_tiles;
             // scale bytes: rows of 256 bytes, 4 per 128-row group
             const int sfa_row0 = (mi * 2 + static_cast<int>(rank)) * 4, sfa_stride = p.act_groups * 4;
-            const int sfw_row0 = ni * 8, sfw_stride = p.w_groups * 4;
             for (int s = sg.s0; s < sg.s1; ++s, ++it) {
                 if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                 if (trace && lane == 0 && it < 64) trace[it] = clock64();
                 if (elect_one()) {
                     if (rank == 0) mbar_arrive_expect_tx(smem_u32(&bar_full[st]), 2 * kStageBytes);
                     const uint32_t full = leader_full0 + st * 8;
-                    const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
                     const int xa = s < S1 ? s * 128 : (p.K - p.k_tail) / 2 + (s - S1) * 128;
                     const uint32_t sb = smem_base + st * kStageBytes;
                     tma_load_2d_pair(sb, &tm_act, xa, mi * 256 + static_cast<int>(rank) * 128, full);
                     tma_load_2d_pair(sb + kPTile + kQTile, &tm_sfa, 0, sfa_row0 + s * sfa_stride, full);
-                    if (it >= pre) {
-                        tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * kHalfN, full);
-                        tma_load_2d_pair(sb + kPTile + kQTile + kSfp, &tm_sfw, 0, sfw_row0 + s * sfw_stride, full);
-                    }
+                    if (it >= pre) load_weights(sb, ni, s, full);
                 }
                 if (++st == kStages) { st = 0; ph ^= 1; }
             }
@@ -356,7 +389,8 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             // earlier (before that stage's tcgen05 instructions, so that the probe's latency hides behind them)
             bool ready = false;
             while (ok && r.next(sg)) {
-                const int buf = seg_it & 1;
+                // (the 288-column tile has one accumulator: the host gives such a call one tile per pair at most)
+                const int buf = C::kAccBufs == 2 ? (seg_it & 1) : 0;
                 if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), ((seg_it >> 1) & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
@@ -571,7 +605,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
 
         while (ok && r.next(sg)) {
             const int mi = sg.tile % p.m_tiles, ni = sg.tile / p.m_tiles;
-            const int buf = seg_it & 1;
+            const int buf = C::kAccBufs == 2 ? (seg_it & 1) : 0;
             const bool piece = sg.s1 - sg.s0 < S;
             // all of this pair's pieces are published: fix up now, overlapping the main loop of this whole tile
             if (!piece && n_fix > 0 && r.cur >= r.end) run_fixups();
@@ -688,7 +722,7 @@ int max_clusters_bn() {
 }
 
 template <int BN>
-cudaError_t launch_bn(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
+cudaError_t launch_bn(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_w_tail, const CUtensorMap& tm_sfa,
                       const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
                       int pairs, cudaStream_t stream) {
     constexpr int kSmemBytes = PCfg<BN>::kSmemBytes;
@@ -712,20 +746,26 @@ cudaError_t launch_bn(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const 
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BN>, tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p);
+    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BN>, tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p);
 }
 
 }  // namespace
 
 int prefill_pair_max_clusters(int bn) {
-    return bn == kPrefillTileWide ? max_clusters_bn<kPrefillTileWide>() : max_clusters_bn<kPrefillTileN>();
+    return bn == kPrefillTileOneWave ? max_clusters_bn<kPrefillTileOneWave>()
+           : bn == kPrefillTileWide ? max_clusters_bn<kPrefillTileWide>() : max_clusters_bn<kPrefillTileN>();
 }
 
-cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
-                                const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
-                                int pairs, cudaStream_t stream) {
-    if (bn == kPrefillTileWide) return launch_bn<kPrefillTileWide>(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
-    if (bn == kPrefillTileN) return launch_bn<kPrefillTileN>(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_w_tail,
+                                const CUtensorMap& tm_sfa, const CUtensorMap& tm_sfw, const CUtensorMap& tm_y,
+                                const PrefillParams& p, int pairs, cudaStream_t stream) {
+    if (bn == kPrefillTileOneWave) {
+        // one accumulator: no pair may be given a second tile or a piece of one
+        if (p.whole_tiles + (p.sk_tiles > 0 ? 1 : 0) > 1 || (p.sk_tiles > 0 && p.sk_base != 1) || p.sk_extra != 0) return cudaErrorInvalidValue;
+        return launch_bn<kPrefillTileOneWave>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+    }
+    if (bn == kPrefillTileWide) return launch_bn<kPrefillTileWide>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+    if (bn == kPrefillTileN) return launch_bn<kPrefillTileN>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
     return cudaErrorInvalidValue;
 }
 

@@ -90,14 +90,14 @@ struct prq_weights {
     // device copies
     uint8_t* d_codes = nullptr;      // E x N x (K + k)/2
     uint8_t* d_sf = nullptr;         // E x S x w_groups x 1024 (+ padding)
-    // Dense layers also keep the scale bytes grouped per 224- and 240-row weight tile of the prefill kernel
-    // (two 128-row groups per tile, the second partly empty) so that those tile widths need no re-alignment.
-    uint8_t* d_sf_alt[2] = {nullptr, nullptr};
-    int w_groups_alt[2] = {0, 0};
+    // Dense layers also keep the scale bytes grouped per 224-, 240- and 288-row weight tile of the prefill kernel
+    // (two or three 128-row groups per tile, the last partly empty) so that those tile widths need no re-alignment.
+    uint8_t* d_sf_alt[3] = {nullptr, nullptr, nullptr};
+    int w_groups_alt[3] = {0, 0, 0};
     // tensor maps of the weight side, encoded once (dense layers; a handle is immutable afterwards):
     // codes with 128-row boxes (decode kernel), codes with half-tile boxes and the scale bytes of the
-    // 224-row [0] and 240-row [1] tilings (CTA-pair prefill kernel)
-    CUtensorMap tm_w_decode, tm_w_pair[2], tm_sfw_pair[2];
+    // 224-row [0], 240-row [1] and 288-row [2] tilings (CTA-pair prefill kernel)
+    CUtensorMap tm_w_decode, tm_w_pair[3], tm_sfw_pair[3], tm_w_tail;   // tm_w_tail: 16-row boxes (288-row tiling)
     bool maps_ready = false;
     int32_t* d_perm = nullptr;       // E x K
     float* d_inv_s_perm = nullptr;   // E x K : inv_s[perm[j]] in the new channel order

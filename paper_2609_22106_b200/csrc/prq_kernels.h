@@ -130,6 +130,7 @@ int decode_max_active_clusters(int bn, int splits);
 // Prefill kernel (M > 128): 256 x 224 or 256 x 240 output tiles, each computed by two CTAs of a cluster.
 constexpr int kPrefillTileN = 224;
 constexpr int kPrefillTileWide = 240;
+constexpr int kPrefillTileOneWave = 288;   // one accumulator: only for calls whose tiles fit one wave of pairs at this width
 constexpr size_t kPrefillSlotBytes = 128 * 256 * sizeof(float);   // workspace per partial tile of one CTA
 struct PrefillParams {
     int M, N, K, k_tail;
@@ -151,11 +152,12 @@ struct PrefillParams {
     int dbg;
     long long wait_limit;       // SM clock cycles after which a wait inside the kernel gives up (PRQ_ERR_TIMEOUT)
 };
-// `bn` = tile width (kPrefillTileN or kPrefillTileWide).  `tm_w` has boxes of bn / 2 rows; `tm_sfa` / `tm_sfw` view the scale bytes as rows of 256 bytes with boxes of
-// 4 / 8 rows (one / two 128-row groups); `tm_y` has 32 x 32 boxes.
-cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
-                                const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
-                                int pairs, cudaStream_t stream);
+// `bn` = tile width (kPrefillTileN, kPrefillTileWide or kPrefillTileOneWave).  `tm_w` has boxes of bn / 2 rows (288: 128 rows,
+// and `tm_w_tail` boxes of 16 rows; any valid map otherwise); `tm_sfa` / `tm_sfw` view the scale bytes as rows of 256 bytes
+// with boxes of 4 / 8 (288: 12) rows (one / two / three 128-row groups); `tm_y` has 32 x 32 boxes.
+cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_w_tail,
+                                const CUtensorMap& tm_sfa, const CUtensorMap& tm_sfw, const CUtensorMap& tm_y,
+                                const PrefillParams& p, int pairs, cudaStream_t stream);
 // How many pairs of the pair kernel can be resident at once on the current device.
 int prefill_pair_max_clusters(int bn);
 

@@ -173,11 +173,12 @@ def test_decode_split_counts(prq, oracle, splits, monkeypatch):
     layer_case(prq, oracle, N=300, K=2560, M=8, k=128, alpha=0.5, mode=prq.ACT_IDENTITY)
 
 
-@pytest.mark.parametrize("bn", [224, 240])
+@pytest.mark.parametrize("bn", [224, 240, 288])
 @pytest.mark.parametrize("shape", [(300, 608, 2336, 96), (1000, 2560, 1024, 0), (260, 328, 512, 512)])
 def test_prefill_tiles(prq, oracle, bn, shape, monkeypatch):
-    """M > 128: the stream-K prefill kernel with both tile widths; ragged M and N, a reduction that is not a
-    multiple of the stage, k = 0 and k = K."""
+    """M > 128: the prefill kernel with its three tile widths (288 columns: the one-wave variant with a single
+    accumulator, which all three shapes admit); ragged M and N, a reduction that is not a multiple of the stage,
+    k = 0 and k = K."""
     monkeypatch.setenv("PRQ_PAIR_BN", str(bn))
     M, N, K, k = shape
     layer_case(prq, oracle, N=N, K=K, M=M, k=k, alpha=0.5, mode=prq.ACT_SCALE_PERM, seed=bn)

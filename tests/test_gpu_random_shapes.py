@@ -119,10 +119,10 @@ def test_random_grouped_shapes_against_oracle(prq, oracle, seed):
         w.free()
 
 
-@pytest.mark.parametrize("bn", [224, 240])
+@pytest.mark.parametrize("bn", [224, 240, 288])
 @pytest.mark.parametrize("seed", [31, 32])
 def test_prefill_tile_widths_against_oracle(prq, oracle, monkeypatch, bn, seed):
-    """Both tile widths of the CTA-pair prefill kernel on shapes whose last column tile is ragged in every way
+    """All tile widths of the CTA-pair prefill kernel on shapes whose last column tile is ragged in every way
     (narrower than the closing 16-column chunk, inside it, an odd number of 16-byte groups, not a multiple of
     16 bytes), with fp32 and bf16 outputs in padded rows."""
     monkeypatch.setenv("PRQ_PAIR_BN", str(bn))
@@ -130,7 +130,7 @@ def test_prefill_tile_widths_against_oracle(prq, oracle, monkeypatch, bn, seed):
     for case in range(8):
         K = int(rng.integers(2, 24)) * 32
         k = int(rng.integers(0, min(K // 32, 4) + 1)) * 32
-        N = int(rng.choice([100, 224, 228, 232, 236, 240, 250, 256, 464, 472, 476, 480, 490, 500, 730]))
+        N = int(rng.choice([100, 224, 228, 232, 236, 240, 250, 256, 260, 288, 300, 464, 472, 476, 480, 490, 500, 570, 580, 730]))
         M = int(rng.choice([129, 256, 300, 520, 700, 1100]))
         dt = prq.F32 if rng.random() < 0.5 else prq.BF16
         if dt == prq.BF16 and N % 2:

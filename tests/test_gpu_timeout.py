@@ -20,8 +20,10 @@ torch = pytest.importorskip("torch")
 PRQ_ERR_TIMEOUT = 6
 
 
-def test_fixup_wait_runs_out_and_the_next_call_is_correct(prq, oracle):
-    # 88 or 96 output tiles on 74 CTA pairs: every pair takes a whole tile, the rest is cut into two pieces each
+def test_fixup_wait_runs_out_and_the_next_call_is_correct(prq, oracle, monkeypatch):
+    # 240-column tiles (forced: the library would give this shape one 288-column tile per pair, which exchanges
+    # nothing): 88 output tiles on 74 CTA pairs, every pair takes a whole tile, the rest is cut into two pieces each
+    monkeypatch.setenv("PRQ_PAIR_BN", "240")
     N, K, k, M = 2560, 4608, 256, 2048
     L = synth.layer(77, N, K, M, T_cal=64)
     amax = oracle.channel_amax(L["zcal"])
