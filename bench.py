@@ -702,7 +702,7 @@ def main():
                      "long_run_launches": LONG_RUN_LAUNCHES, "long_run_clocks": long_clocks.summary(),
                      "traffic": NCU_PREFILL_DRAM_BYTES, "traffic_source": NCU_PREFILL_SOURCE + " (ncu capture, not this run)",
                      "algorithmic_bytes": gemm_bytes(M_TOK, K_TAIL),
-                     "kernel": "prefill_pair_kernel<240> (CTA pairs, 256x240 tiles, whole tiles + stream-K pieces)", "launch_us": gemm_us,
+                     "kernel": "prefill_pair_kernel<288> (CTA pairs, one 256x288 tile per pair, one wave: 72 tiles on 74 pairs)", "launch_us": gemm_us,
                      "peak_source": f"4 x bf16 burst, of {pk['source']}",
                      "frac_of_measured_mxf4_probe": achieved / mxf4_probe["burst_1.5ms"],
                      "frac_of_nominal_9pf": achieved / 9000.0},
