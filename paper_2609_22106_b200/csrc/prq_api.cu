@@ -873,6 +873,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
             q.sk_extra = ps.extra;
         }
         q.sk_tiles = static_cast<int>(sk); q.whole_tiles = static_cast<int>(whole);
+        q.total_tiles = static_cast<int>(tiles);
         if (sk * w->plan.S * pairs >= (1ll << 32) || tiles >= (1ll << 30)) return PRQ_ERR_INVALID_ARG;  // 32-bit range arithmetic
         if (!workspace || workspace_bytes < flag_bytes + static_cast<size_t>(4 * pairs) * kPrefillSlotBytes) return PRQ_ERR_WORKSPACE;
         q.flag_stride = static_cast<int>(prefill_flag_count(w, M));

@@ -42,6 +42,7 @@
 
 #include "prq_kernels.h"
 #include "prq_ptx.cuh"
+#include "prq_quant_block.cuh"
 
 namespace prq {
 namespace {
@@ -112,7 +113,7 @@ struct Segment {
 struct Range {
     uint32_t cur, end;
     int S;
-    int next_whole, whole_left, G;
+    int next_whole, whole_left, G, total;
     __device__ __forceinline__ bool next(Segment& g) {
         if (cur < end) {
             g.tile = static_cast<int>(cur / static_cast<uint32_t>(S));
@@ -122,7 +123,7 @@ struct Range {
             cur += g.s1 - g.s0;
             return true;
         }
-        if (whole_left > 0) {
+        if (whole_left > 0 && next_whole < total) {
             g.tile = next_whole;
             g.s0 = 0;
             g.s1 = S;
@@ -235,7 +236,7 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
     tc_commit_pair(empty_bar0 + Q * 8, 3);
 }
 
-template <int BN>
+template <int BN, bool kGated = false>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
                     const __grid_constant__ CUtensorMap tm_w_tail,
@@ -313,7 +314,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer (both CTAs)
-        Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G};
+        Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G, p.total_tiles};
         Segment sg;
         int st = 0, it = 0;
         uint32_t ph = 0;
@@ -378,7 +379,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (rank == 0) {
-            Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G};
+            Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G, p.total_tiles};
             Segment sg;
             const bool leader = elect_one();
             int it = 0, st = 0, seg_it = 0;
@@ -428,7 +429,7 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         const int row_in_tile = q4 * 32 + lane;  // row of this CTA's 128-row half
         const uint32_t stage_smem = staging_base + (warp - 2) * kStagingPerWarp;
         const uint32_t leader_acc_empty0 = cluster_map(smem_u32(&bar_acc_empty[0]), 0);
-        Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G};
+        Range r{sk_b, sk_e, S, p.sk_tiles + g, p.whole_tiles, G, p.total_tiles};
         Segment sg;
         int seg_it = 0, store_it = 0;
         bool ok = true;
@@ -614,7 +615,62 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             if (trace && row_in_tile == 0 && seg_it < 8) trace[192 + 2 * seg_it] = clock64();
             tc_fence_after_sync();
             const uint32_t acc_t = tmem_base + buf * BN + (static_cast<uint32_t>(q4 * 32) << 16);
-            if (piece) {
+            if constexpr (kGated) {
+                // Gated-producer epilogue (Eq. (1), middle line, with the activation function inside the producer):
+                // the tile's columns are (gate, up) groups of 32 + 32 output features.  Per group a thread holds,
+                // for its token row, 32 gate and 32 up sums: h = bf16(silu(gate) * up) is one 32-element block of
+                // the down projection's input, quantised here exactly as the activation quantiser would (same
+                // function), and written as 16 bytes of codes and one scale byte.  The product never exists in
+                // global memory (unless the caller asks for it to check).
+                static_assert(!kGated || BN % 64 == 0, "whole (gate, up) groups per tile");
+                const int row = mi * 256 + static_cast<int>(rank) * 128 + row_in_tile;
+                const int grp = row >> 7, rg = row & 127;
+                const int C = p.out_C;
+                const int tail_blk0 = (C - p.out_k_tail) / kBlock, S1o = C / kStageK;
+#pragma unroll 1
+                for (int j = 0; j < BN / 64; ++j) {
+                    uint32_t vg[32], vu[32];
+                    tmem_ld_32x32(acc_t + j * 64, vg);
+                    tmem_ld_32x32(acc_t + j * 64 + 32, vu);
+                    tmem_ld_wait();
+                    if (j == BN / 64 - 1) {
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(leader_acc_empty0 + buf * 8);
+                    }
+                    const int fb = (ni * BN) / 64 + j;            // 32-channel block of the down projection's input
+                    if (fb * kBlock >= C || grp >= p.out_groups) continue;
+                    uint4 q[4];
+                    uint32_t* qw = reinterpret_cast<uint32_t*>(q);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float g0 = __uint_as_float(vg[2 * i]), g1 = __uint_as_float(vg[2 * i + 1]);
+                        const float h0 = __fdividef(g0, 1.f + __expf(-g0)) * __uint_as_float(vu[2 * i]);
+                        const float h1 = __fdividef(g1, 1.f + __expf(-g1)) * __uint_as_float(vu[2 * i + 1]);
+                        const __nv_bfloat162 hh = __floats2bfloat162_rn(h0, h1);
+                        qw[i] = *reinterpret_cast<const uint32_t*>(&hh);
+                    }
+                    const bool live = row < p.M;
+                    if (!live) { q[0] = q[1] = q[2] = q[3] = make_uint4(0, 0, 0, 0); }
+                    uint4 codes;
+                    const uint32_t byte = live ? quant_block32(q, codes) : 0u;   // rows past M: scale bytes stay 2^-127
+                    if (live) {
+                        *reinterpret_cast<uint4*>(p.out_codes + static_cast<size_t>(row) * (C / 2) + fb * 16) = codes;
+                        if (p.out_scales_row) p.out_scales_row[static_cast<size_t>(row) * (C / kBlock) + fb] = static_cast<uint8_t>(byte);
+                        if (p.out_h) {
+                            uint4* hp = reinterpret_cast<uint4*>(p.out_h + static_cast<size_t>(row) * C + fb * kBlock);
+                            hp[0] = q[0]; hp[1] = q[1]; hp[2] = q[2]; hp[3] = q[3];
+                        }
+                    }
+                    uint8_t* sfg = p.out_sf + static_cast<size_t>(grp) * kSfGroupBytes;
+                    const size_t stage_stride = static_cast<size_t>(p.out_groups) * kSfGroupBytes;
+                    sfg[(fb >> 3) * stage_stride + sf_offset_in_group(rg, fb & 7)] = static_cast<uint8_t>(byte);
+                    if (fb >= tail_blk0) {   // the tail's scale bytes a second time, in the residual stages
+                        const int t = fb - tail_blk0;
+                        sfg[(S1o + (t >> 3)) * stage_stride + sf_offset_in_group(rg, t & 7)] = static_cast<uint8_t>(byte);
+                    }
+                }
+            } else if (piece) {
                 // publish this piece: partial accumulator -> workspace slot (one 512-byte line per warp store)
                 const int k = plan_sk.slot_index(g, sg.tile);
                 float4* slot = reinterpret_cast<float4*>(p.partial) +
@@ -698,12 +754,12 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     if (threadIdx.x == 0 && abort_flag_s) atomicExch(p.status, static_cast<int>(PRQ_ERR_TIMEOUT));
 }
 
-template <int BN>
+template <int BN, bool kGated = false>
 int max_clusters_bn() {
     constexpr int kSmemBytes = PCfg<BN>::kSmemBytes;
     static int cached = -1;
     if (cached >= 0) return cached;
-    if (cudaFuncSetAttribute(prefill_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return 0;
+    if (cudaFuncSetAttribute(prefill_pair_kernel<BN, kGated>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) return 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2);
     cfg.blockDim = dim3(kThreads);
@@ -716,19 +772,19 @@ int max_clusters_bn() {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, prefill_pair_kernel<BN>, &cfg) != cudaSuccess) return 0;
+    if (cudaOccupancyMaxActiveClusters(&n, prefill_pair_kernel<BN, kGated>, &cfg) != cudaSuccess) return 0;
     cached = n;
     return n;
 }
 
-template <int BN>
+template <int BN, bool kGated = false>
 cudaError_t launch_bn(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_w_tail, const CUtensorMap& tm_sfa,
                       const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
                       int pairs, cudaStream_t stream) {
     constexpr int kSmemBytes = PCfg<BN>::kSmemBytes;
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_pair_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(prefill_pair_kernel<BN, kGated>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
@@ -746,12 +802,13 @@ cudaError_t launch_bn(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const 
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BN>, tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p);
+    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BN, kGated>, tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p);
 }
 
 }  // namespace
 
 int prefill_pair_max_clusters(int bn) {
+    if (bn == kPrefillTileGated) return max_clusters_bn<kPrefillTileGated, true>();
     return bn == kPrefillTileOneWave ? max_clusters_bn<kPrefillTileOneWave>()
            : bn == kPrefillTileWide ? max_clusters_bn<kPrefillTileWide>() : max_clusters_bn<kPrefillTileN>();
 }
@@ -763,6 +820,11 @@ cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtenso
         // one accumulator: no pair may be given a second tile or a piece of one
         if (p.whole_tiles + (p.sk_tiles > 0 ? 1 : 0) > 1 || (p.sk_tiles > 0 && p.sk_base != 1) || p.sk_extra != 0) return cudaErrorInvalidValue;
         return launch_bn<kPrefillTileOneWave>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+    }
+    if (bn == kPrefillTileGated) {
+        // whole tiles only: a piece of a tile has no (gate, up) sums to put through the activation function
+        if (p.sk_tiles != 0 || !p.out_codes || !p.out_sf) return cudaErrorInvalidValue;
+        return launch_bn<kPrefillTileGated, true>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
     }
     if (bn == kPrefillTileWide) return launch_bn<kPrefillTileWide>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
     if (bn == kPrefillTileN) return launch_bn<kPrefillTileN>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);

@@ -54,6 +54,8 @@ struct QuantBatch {
     int act_groups;
     int n_lin;                           // 1 .. kMaxBatch
     int groups_per_lin;                  // blockIdx.y = layer * groups_per_lin + group
+    int n_atoms, n_tail, tail_split;     // set by the launcher: 128-column atoms, how many of them are tail atoms
+                                         // (scale + permute mode), and into how many row shares each of those is cut
     QuantLayer lay[kMaxBatch];
 };
 cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStream_t stream);
@@ -131,6 +133,7 @@ int decode_max_active_clusters(int bn, int splits);
 constexpr int kPrefillTileN = 224;
 constexpr int kPrefillTileWide = 240;
 constexpr int kPrefillTileOneWave = 288;   // one accumulator: only for calls whose tiles fit one wave of pairs at this width
+constexpr int kPrefillTileGated = 192;     // gated-producer epilogue: three (gate, up) groups of 32 + 32 columns per tile
 constexpr size_t kPrefillSlotBytes = 128 * 256 * sizeof(float);   // workspace per partial tile of one CTA
 struct PrefillParams {
     int M, N, K, k_tail;
@@ -151,8 +154,17 @@ struct PrefillParams {
     long long* trace;
     int dbg;
     long long wait_limit;       // SM clock cycles after which a wait inside the kernel gives up (PRQ_ERR_TIMEOUT)
+    int total_tiles;            // m_tiles * n_tiles: whole-tile waves stop here (the last wave may be short)
+    // Gated-producer epilogue (kPrefillTileGated only): the layer is a gate and an up projection interleaved in
+    // groups of 32 output features; instead of y the kernel writes Q(silu(gate) * up), the MXFP4 activation of the
+    // down projection that follows (C input channels, tail k_tail), straight into that layer's buffers.
+    uint8_t* out_codes;         // M x C/2
+    uint8_t* out_sf;            // scale bytes in the GEMM's tile order, tail bytes duplicated
+    uint8_t* out_scales_row;    // M x C/32, or null
+    uint16_t* out_h;            // M x C bf16 (the product before quantisation), or null: for checks
+    int out_C, out_k_tail, out_groups;
 };
-// `bn` = tile width (kPrefillTileN, kPrefillTileWide or kPrefillTileOneWave).  `tm_w` has boxes of bn / 2 rows (288: 128 rows,
+// `bn` = tile width (kPrefillTileN, kPrefillTileWide, kPrefillTileOneWave, or kPrefillTileGated for the gated-producer epilogue).  `tm_w` has boxes of bn / 2 rows (288: 128 rows,
 // and `tm_w_tail` boxes of 16 rows; any valid map otherwise); `tm_sfa` / `tm_sfw` view the scale bytes as rows of 256 bytes
 // with boxes of 4 / 8 (288: 12) rows (one / two / three 128-row groups); `tm_y` has 32 x 32 boxes.
 cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_w_tail,

@@ -68,7 +68,28 @@ quant_act_kernel(const QuantBatch b) {
         p.k_tail = l.k_tail; p.perm = l.perm; p.inv_s_perm = l.inv_s_perm;
         p.codes = l.codes; p.scales_row = l.scales_row; p.scales_sf = l.scales_sf;
     }
-    const int atom = blockIdx.x;                  // 128-column slice of the reduction axis
+    // Which (128-column atom, 128-row group, share of the group's rows) this CTA takes.  In scale + permute mode the
+    // atoms of the tail are some twenty times slower than the others: their source columns are scattered over the
+    // whole row, every 2-byte read is a 32-byte sector of its own, and the CTA runs at the rate at which its SM's L1
+    // takes sectors (about 20 us for 128 rows against 1 us for a head atom, whose window is nearly contiguous).  A
+    // launch could not end before its slowest CTA, which the next kernel of the stream then waited for (8 - 11 us
+    // per call at 4096 tokens).  So the tail atoms are cut into `tail_split` shares of the rows each and come first
+    // in the grid, the head atoms after them.
+    // (counted over the whole layer: the tail units of ALL row groups precede every head atom.)
+    int group = static_cast<int>(blockIdx.y) - lin * b.groups_per_lin;
+    int atom = blockIdx.x, tail_share = 0, tail_split = 1;
+    if (kScalePerm && b.n_tail > 0) {
+        const int units = b.n_tail * b.tail_split, n_head = b.n_atoms - b.n_tail;
+        const int id = group * static_cast<int>(gridDim.x) + atom, first = units * b.groups_per_lin;
+        if (id < first) {
+            group = id / units;
+            const int u = id - group * units;
+            tail_split = b.tail_split; tail_share = u % tail_split; atom = n_head + u / tail_split;
+        } else {
+            const int r = id - first;
+            group = r / n_head; atom = r - group * n_head;
+        }
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int half = lane >> 4, hl = lane & 15;   // which of the warp's two rows, lane inside the row
     float inv_s[8];
@@ -93,7 +114,6 @@ quant_act_kernel(const QuantBatch b) {
     // Which rows does this CTA own?  Dense: group g covers rows [128 g, 128 g + 128).  Grouped: the
     // scale groups are padded per expert, so walk the expert offsets to find ours.
     int row0, row_end, expert = 0;
-    const int group = static_cast<int>(blockIdx.y) - lin * b.groups_per_lin;
     if (p.expert_offsets == nullptr) {
         row0 = group * kGroupRows;
         row_end = min(p.M, row0 + kGroupRows);
@@ -135,8 +155,8 @@ quant_act_kernel(const QuantBatch b) {
     const int n_rows = row_end - row0;            // 1..128
     // With few groups the rows of a group are split over gridDim.z CTAs (1, 2, 4 or 8 parts of whole
     // 16-row steps) so that a small batch still fills the GPU; only the scale + permute mode is split.
-    const int n_parts = kScalePerm ? static_cast<int>(gridDim.z) : 1;
-    const int part = kScalePerm ? static_cast<int>(blockIdx.z) : 0;
+    const int n_parts = kScalePerm ? static_cast<int>(gridDim.z) * tail_split : 1;
+    const int part = kScalePerm ? static_cast<int>(blockIdx.z) * tail_split + tail_share : 0;
     const int part_steps = kSteps / n_parts;
 
     if (kScalePerm && !dense) load_layer_constants(expert);   // grouped: the expert is known only now
@@ -271,7 +291,7 @@ quant_act_kernel(const QuantBatch b) {
             *reinterpret_cast<const uint32_t*>(sf_atom + off);
     }
     if (part != 0) return;
-    const int n_atoms = gridDim.x;
+    const int n_atoms = b.n_atoms;
     // An odd atom count leaves the second half of the last main stage without an owner: zero it.
     if (atom == n_atoms - 1 && (n_atoms & 1) && threadIdx.x >= 32 && threadIdx.x < 64)
         reinterpret_cast<uint4*>(sf_group + stage * sf_stage_stride + 512)[threadIdx.x - 32] = make_uint4(0, 0, 0, 0);
@@ -313,7 +333,17 @@ cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStr
         if (parts == 4 && tiles * parts < 4LL * sm_count[dev]) parts = 8;
         if (const char* ev = dev_knobs_enabled() ? getenv("PRQ_QUANT_PARTS") : nullptr) { const int v = atoi(ev); if (v == 1 || v == 2 || v == 4 || v == 8) parts = v; }
     }
-    cfg.gridDim = dim3(n_atoms, grid_groups, parts);
+    // the tail atoms of the scale + permute mode in shares of 16 rows (128 / 8), see the kernel
+    QuantBatch bb = b;
+    bb.n_atoms = n_atoms;
+    bb.n_tail = 0; bb.tail_split = 1;
+    if (scale_perm) {
+        int k_max = 0;
+        for (int i = 0; i < b.n_lin; ++i) k_max = b.lay[i].k_tail > k_max ? b.lay[i].k_tail : k_max;
+        bb.n_tail = (k_max + kAtomK - 1) / kAtomK < n_atoms ? (k_max + kAtomK - 1) / kAtomK : n_atoms;
+        bb.tail_split = 8 / parts;
+    }
+    cfg.gridDim = dim3(n_atoms - bb.n_tail + bb.n_tail * bb.tail_split, grid_groups, parts);
     cfg.blockDim = dim3(kQuantThreads);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -322,10 +352,10 @@ cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStr
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (b.n_lin > 1)
-        return scale_perm ? cudaLaunchKernelEx(&cfg, quant_act_kernel<true, true>, b)
-                          : cudaLaunchKernelEx(&cfg, quant_act_kernel<false, true>, b);
-    return scale_perm ? cudaLaunchKernelEx(&cfg, quant_act_kernel<true, false>, b)
-                      : cudaLaunchKernelEx(&cfg, quant_act_kernel<false, false>, b);
+        return scale_perm ? cudaLaunchKernelEx(&cfg, quant_act_kernel<true, true>, bb)
+                          : cudaLaunchKernelEx(&cfg, quant_act_kernel<false, true>, bb);
+    return scale_perm ? cudaLaunchKernelEx(&cfg, quant_act_kernel<true, false>, bb)
+                      : cudaLaunchKernelEx(&cfg, quant_act_kernel<false, false>, bb);
 }
 
 cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_groups, cudaStream_t stream) {
