@@ -100,10 +100,16 @@ prq_status prq_prepare_weights(const uint16_t *W, int n_experts, int N, int K, c
  *                           two neighbours, the one with the smallest squared quantisation error (a
  *                           neighbour only if strictly better).  Channel ranking, permutation and scales s
  *                           are not affected; R is the residual of the searched quantisation.  The GEMM is
- *                           untouched. */
+ *                           untouched.
+ *   gated_producer       0 (default): an ordinary layer.
+ *                        1: the layer is the stacked gate / up projection of a gated FFN in the row order of
+ *                           prq_stack_gate_up, to be run by prq_linear_gated.  The prepared weights are the same;
+ *                           the handle keeps the scale-byte tiling of that call's kernel instead of those of
+ *                           prq_linear, which therefore refuses it for more than 128 tokens. */
 typedef struct prq_prep_opts {
     size_t struct_size;
     int weight_scale_search;
+    int gated_producer;
 } prq_prep_opts;
 
 /* prq_prepare_weights with options (opts may be NULL).  Errors as prq_prepare_weights, plus INVALID_ARG for a
@@ -184,6 +190,14 @@ prq_status prq_fold_producer(const int32_t *perm, const float *inv_s, int C, int
                              const uint16_t *W_gate, int H, int duplicate_tail, uint16_t *out_up,
                              uint16_t *out_gate);
 
+/* Rows of a gate and an up projection interleaved in groups of 32, the row order prq_linear_gated expects:
+ *   out[64 b + i] = W_gate[32 b + i],  out[64 b + 32 + i] = W_up[32 b + i]     (b < C / 32, i < 32)
+ * so that 64 consecutive output features of the stacked layer are the gate and the up sums of ONE 32-channel block
+ * of the down projection's input.  All pointers are HOST memory: W_gate, W_up C x H bf16 row-major (normally the
+ * outputs of prq_fold_producer, so that the product arrives scaled and in the down projection's channel order),
+ * out 2 C x H.  INVALID_ARG unless C % 32 == 0. */
+prq_status prq_stack_gate_up(const uint16_t *W_gate, const uint16_t *W_up, int C, int H, uint16_t *out);
+
 /* Shape of a handle.  Any output pointer may be NULL. */
 prq_status prq_weights_info(const prq_weights *w, int *n_experts, int *N, int *K, int *k_tail, float *alpha);
 
@@ -261,6 +275,32 @@ prq_status prq_linear(const prq_weights *w, const void *codes, const void *scale
  *     overlapping callers prq_linear with workspaces of their own. */
 prq_status prq_linear_static_scratch(const prq_weights *w, const void *codes, const void *scales_sf, int M, void *y,
                                      int ldy, prq_dtype y_dtype, prq_stream_t stream);
+
+/* Eq. (1), middle line, with the producer's activation function inside the producer's GEMM: the gate and up
+ * projections of a gated FFN as one layer whose output never exists in bf16.  One launch computes
+ *   g, u = the two halves of prq_linear(w_gu, codes, scales_sf)      (fp32 sums, never stored)
+ *   h    = bf16( silu(g) * u ),  silu(g) = g / (1 + exp(-g)) in fp32
+ *   Q(h) = the MXFP4 quantisation prq_quantize_act(w_down, PRQ_ACT_IDENTITY, h) would give
+ * and writes Q(h) -- codes, tile-ordered scale bytes with the tail's bytes duplicated, optionally row-major scale
+ * bytes -- ready for prq_linear(w_down, ...).  With the down projection's 1 / s and permutation folded into the
+ * producers (prq_fold_producer, then prq_stack_gate_up) this is the whole activation side of Eq. (1): the separate
+ * quantiser launch and the bf16 round trip of h (2 x M x C bytes written, M x C read back) are gone.
+ *   w_gu              handle of the stacked layer (2 C output features), prepared with gated_producer = 1
+ *   codes, scales_sf  device, the quantised hidden state as prq_quantize_act wrote it for w_gu and M
+ *   w_down            handle of the down projection (gives C = its input channels and its tail k); needs
+ *                     C % 256 == 0 and k % 256 == 0 (whole reduction stages; the paper's shapes have both)
+ *   out_codes         device out, prq_act_bytes(M, C, k, 1, PRQ_BUF_CODES) bytes, 16-byte aligned
+ *   out_scales_row    device out or NULL, PRQ_BUF_SCALES_ROW bytes
+ *   out_scales_sf     device out, PRQ_BUF_SCALES_SF bytes, 16-byte aligned
+ *   h_check           device out or NULL: M x C bf16, the product before quantisation (for checks; costs the traffic
+ *                     the call exists to avoid)
+ * The exponential is the GPU's fast one: h is within one bf16 unit in the last place of the exactly evaluated
+ * product, and Q(h) is bit-for-bit the quantisation of the h this call forms.  Every token count takes the same
+ * kernel (256-token tiles); a decode-shaped instance is not built.  Needs no workspace.
+ * Errors: INVALID_ARG (shapes, a handle not prepared as gated producer, devices), ALIGNMENT, CUDA. */
+prq_status prq_linear_gated(const prq_weights *w_gu, const void *codes, const void *scales_sf, int M,
+                            const prq_weights *w_down, void *out_codes, void *out_scales_row, void *out_scales_sf,
+                            void *h_check, prq_stream_t stream);
 
 /* Decode step in one launch (Kernel design paragraph: the kernel quantises the reordered activation once
  * and multiplies): y = prq_linear(prq_quantize_act(x)) for up to PRQ_FUSED_MAX_M tokens, with the

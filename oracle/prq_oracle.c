@@ -42,7 +42,8 @@
  * k = 0 reducing to plain MXFP4, Eq. (1) invariance, exact residual identity,
  * brute-force top-k, Eq. (3) = main + correction.  The normalised error and the alpha
  * selection of the Python front end (first minimum over the grid) are pinned by a hand-worked
- * error norm and a hand-decided three-candidate search (tests/test_oracle_alpha.py).
+ * error norm and a hand-decided three-candidate search (tests/test_oracle_alpha.py).  The gated activation
+ * silu(g) * u of the producer is pinned by closed-form values and identities (tests/test_oracle_gated.py).
  */
 #include <math.h>
 #include <stdint.h>
@@ -429,6 +430,17 @@ int orc_fold_producer(const uint16_t *W_up, const uint16_t *W_gate, long C, long
         }
     }
     return 0;
+}
+
+/* Gated FFN activation of the producer (the function f of Eq. (1), middle line, for a SiLU-gated FFN):
+ * h[i] = bf16( silu(g[i]) * u[i] ) with silu(g) = g / (1 + exp(-g)), evaluated in FP64 and rounded once.
+ * g, u: n doubles (the gate and up projections' sums); h: n bf16 bit patterns. */
+void orc_silu_mul_bf16(const double *g, const double *u, long n, uint16_t *h) {
+    long i;
+    for (i = 0; i < n; ++i) {
+        double s = g[i] / (1.0 + exp(-g[i]));
+        h[i] = orc_double_to_bf16(s * u[i]);
+    }
 }
 
 int orc_num_threads(void) {

@@ -224,6 +224,29 @@ def fold_producer(W_up, W_gate, perm, inv_s, k: int, dup: bool = False):
     return ou, og
 
 
+def silu_mul_bf16(g, u):
+    """The producer's gated activation (f of Eq. (1), middle line, for a SiLU-gated FFN): bf16(silu(g) * u) from
+    FP64 gate / up sums, rounded once; returns uint16 bit patterns of the same shape."""
+    g = _c(g, np.float64)
+    u = _c(u, np.float64)
+    h = np.empty(g.shape, np.uint16)
+    _load().orc_silu_mul_bf16(_p(g), _p(u), ctypes.c_long(g.size), _p(h))
+    return h
+
+
+def stack_gate_up(W_gate, W_up):
+    """Rows of the gate and up projections interleaved in groups of 32 (gate rows 32 b .., then up rows 32 b ..): the
+    stacked producer layer whose 64-feature output groups are the two factors of one 32-channel block."""
+    Wg = _c(W_gate, np.uint16)
+    Wu = _c(W_up, np.uint16)
+    C, H = Wg.shape
+    out = np.empty((2 * C, H), np.uint16)
+    o4 = out.reshape(C // BLOCK, 2, BLOCK, H)
+    o4[:, 0] = Wg.reshape(C // BLOCK, BLOCK, H)
+    o4[:, 1] = Wu.reshape(C // BLOCK, BLOCK, H)
+    return out
+
+
 def nrmse(y_hat, y):
     """Normalised reconstruction error ||Yhat - Y||_F / ||Y||_F (text after Eq. (3))."""
     return float(np.linalg.norm(y_hat - y) / np.linalg.norm(y))

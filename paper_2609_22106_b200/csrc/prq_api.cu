@@ -30,6 +30,7 @@ struct DeviceInfo {
     int* status_ptr = nullptr;
     int max_clusters[4][9] = {};  // decode kernel: [token-tile index][cluster size], 0 = not queried yet
     int max_pairs = 0;            // prefill pair kernel: co-resident CTA pairs, 0 = not queried yet
+    int max_pairs_gated = 0;      // the same for its gated-producer instance
 };
 std::mutex g_dev_mutex;
 DeviceInfo g_dev[64];
@@ -122,8 +123,12 @@ prq_status make_out_map(CUtensorMap* map, void* y, int M, int N, int ldy, bool b
     return r == CUDA_SUCCESS ? PRQ_OK : PRQ_ERR_CUDA;
 }
 
-constexpr int kNumAlt = 3;
-constexpr int kAltTileRows[kNumAlt] = {kPrefillTileN, kPrefillTileWide, kPrefillTileOneWave};  // weight tile widths of the prefill kernel, each with its own scale layout
+constexpr int kNumAlt = 4;
+// weight tile widths of the prefill kernel, each with its own scale layout; the last one only in gated-producer handles,
+// which in turn have none of the others
+constexpr int kAltTileRows[kNumAlt] = {kPrefillTileN, kPrefillTileWide, kPrefillTileOneWave, kPrefillTileGated};
+constexpr int kAltGated = 3;
+bool alt_wanted(bool gated, int a) { return gated ? a == kAltGated : a != kAltGated; }
 
 // Weight-side tensor maps of a dense handle, encoded once at creation (cloning re-encodes: other addresses).
 prq_status build_weight_maps(prq_weights* w) {
@@ -131,7 +136,8 @@ prq_status build_weight_maps(prq_weights* w) {
     if (w->n_experts != 1) return PRQ_OK;
     const uint64_t Ka = static_cast<uint64_t>(w->K) + w->k_tail;
     prq_status st = make_code_map(&w->tm_w_decode, w->d_codes, Ka / 2, w->N, 128);
-    for (int v = 0; v < kNumAlt; ++v) {   // 224-, 240- and 288-row tilings
+    for (int v = 0; v < kNumAlt; ++v) {   // 224-, 240- and 288-row tilings, or the 192-row one
+        if (!alt_wanted(w->gated, v)) continue;
         const int rows = kAltTileRows[v], gpt = (rows + kGroupRows - 1) / kGroupRows;
         // each CTA of a pair loads half a tile; the 288-row tile as 128 + 16 rows (second map)
         if (st == PRQ_OK) st = make_code_map(&w->tm_w_pair[v], w->d_codes, Ka / 2, w->N, rows > 256 ? 128 : rows / 2);
@@ -385,8 +391,10 @@ static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_
                                 const float* act_amax, float alpha, int k_tail, const prq_prep_opts* opts, prq_weights** out) {
     if (opts && opts->struct_size < sizeof(prq_prep_opts)) return PRQ_ERR_INVALID_ARG;
     const bool scale_search = opts && opts->weight_scale_search != 0;
+    const bool gated = opts && opts->gated_producer != 0;
     if (!W || !act_amax || !out) return PRQ_ERR_INVALID_ARG;
     if (n_experts < 1 || n_experts > kMaxExperts || N < 1 || K < kBlock) return PRQ_ERR_INVALID_ARG;
+    if (gated && (n_experts != 1 || N % 64)) return PRQ_ERR_INVALID_ARG;   // whole (gate, up) groups of 32 + 32 rows
     if (K % kBlock || k_tail % kBlock || k_tail < 0 || k_tail > K) return PRQ_ERR_INVALID_ARG;
     if (!std::isfinite(alpha)) return PRQ_ERR_INVALID_ARG;
     if (static_cast<long long>(n_experts) * N > 0x7fffffffll) return PRQ_ERR_INVALID_ARG;
@@ -402,6 +410,7 @@ static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_
     w->plan = StagePlan(K, k_tail);
     w->w_groups = (N + kGroupRows - 1) / kGroupRows;
     w->device = dev;
+    w->gated = gated;
     const size_t Ka = static_cast<size_t>(K) + k_tail;
     const size_t E = n_experts;
     try {
@@ -418,6 +427,7 @@ static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_
         std::vector<float> inv_s_perm(E * K);
         std::vector<uint8_t> sf_alt[kNumAlt];
         for (int a = 0; a < kNumAlt && E == 1; ++a) {
+            if (!alt_wanted(gated, a)) continue;
             w->w_groups_alt[a] = ((N + kAltTileRows[a] - 1) / kAltTileRows[a]) * ((kAltTileRows[a] + kGroupRows - 1) / kGroupRows);
             sf_alt[a].assign((static_cast<size_t>(S) * w->w_groups_alt[a] + 4) * kSfGroupBytes, 0);
         }
@@ -443,6 +453,7 @@ static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_
                     const int bis = b < nblk_main ? b % nb : (b - nblk_main) % nb;
                     sf[((e * S + stage) * w->w_groups + g) * kSfGroupBytes + sf_offset_in_group(rr, bis)] = srow[b];
                     for (int a = 0; a < kNumAlt && E == 1; ++a) {
+                        if (!alt_wanted(gated, a)) continue;
                         const int tile_rows = kAltTileRows[a], gpt = (tile_rows + kGroupRows - 1) / kGroupRows;
                         const int ga = (n / tile_rows) * gpt + (n % tile_rows) / kGroupRows;
                         sf_alt[a][(static_cast<size_t>(stage) * w->w_groups_alt[a] + ga) * kSfGroupBytes +
@@ -464,6 +475,7 @@ static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_
         ok = ok && cudaMemcpy(w->d_perm, w->h_perm.data(), sizeof(int32_t) * E * K, cudaMemcpyHostToDevice) == cudaSuccess;
         ok = ok && cudaMemcpy(w->d_inv_s_perm, inv_s_perm.data(), sizeof(float) * E * K, cudaMemcpyHostToDevice) == cudaSuccess;
         for (int a = 0; a < kNumAlt && E == 1 && ok; ++a) {
+            if (!alt_wanted(gated, a)) continue;
             if (cudaMalloc(&w->d_sf_alt[a], sf_alt[a].size()) != cudaSuccess) {
                 cudaGetLastError();
                 prq_weights_free(w);
@@ -606,7 +618,7 @@ prq_status prq_weights_clone(const prq_weights* w, prq_weights** out) {
     prq_status st = PRQ_OK;
     try {
         c->n_experts = w->n_experts; c->N = w->N; c->K = w->K; c->k_tail = w->k_tail; c->alpha = w->alpha;
-        c->plan = w->plan; c->w_groups = w->w_groups; c->device = w->device;
+        c->plan = w->plan; c->w_groups = w->w_groups; c->device = w->device; c->gated = w->gated;
         c->h_codes = w->h_codes; c->h_scales = w->h_scales; c->h_perm = w->h_perm;
         c->h_s = w->h_s; c->h_inv_s = w->h_inv_s; c->h_col_err = w->h_col_err;
         c->d_codes_bytes = w->d_codes_bytes; c->d_sf_bytes = w->d_sf_bytes;
@@ -848,6 +860,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
     } else {
         // stream-K kernel on CTA pairs with 256 x 224 or 256 x 240 tiles (scale bytes grouped per weight tile)
+        if (w->gated) return PRQ_ERR_INVALID_ARG;   // a gated-producer handle has the tiling of prq_linear_gated only
         PrefillParams q;
         std::memset(&q, 0, sizeof(q));
         if (di->max_pairs == 0)
@@ -930,6 +943,58 @@ prq_status prq_linear_multi(int n, const prq_weights* const* ws, const void* con
     }
     b.splits = decode_splits_for(tiles, ws[0]->plan.S, M, di);
     cudaError_t e = launch_decode_batch(bn, maps, b, static_cast<cudaStream_t>(stream));
+    g_launches.fetch_add(1);
+    return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+}
+
+prq_status prq_stack_gate_up(const uint16_t* W_gate, const uint16_t* W_up, int C, int H, uint16_t* out) {
+    if (!W_gate || !W_up || !out || C < kBlock || C % kBlock || H < 1) return PRQ_ERR_INVALID_ARG;
+    stack_gate_up(W_gate, W_up, C, H, out);
+    return PRQ_OK;
+}
+
+prq_status prq_linear_gated(const prq_weights* w, const void* codes, const void* scales_sf, int M, const prq_weights* wd,
+                            void* out_codes, void* out_scales_row, void* out_scales_sf, void* h_check, prq_stream_t stream) {
+    if (!w || !wd || M < 0) return PRQ_ERR_INVALID_ARG;
+    if (!w->gated || !w->maps_ready || w->n_experts != 1 || wd->n_experts != 1 || w->device != wd->device) return PRQ_ERR_INVALID_ARG;
+    const int C = wd->K, kd = wd->k_tail;
+    if (w->N != 2 * C || C % kStageK || kd % kStageK) return PRQ_ERR_INVALID_ARG;
+    if (M == 0) return PRQ_OK;
+    if (!codes || !scales_sf || !out_codes || !out_scales_sf) return PRQ_ERR_INVALID_ARG;
+    if (!aligned16(codes) || !aligned16(scales_sf) || !aligned16(out_codes) || !aligned16(out_scales_sf) || !aligned16(h_check))
+        return PRQ_ERR_ALIGNMENT;
+    if (!handle_device_is_current(w)) return PRQ_ERR_INVALID_ARG;
+    DeviceInfo* di;
+    prq_status st = device_info(w->device, &di);
+    if (st != PRQ_OK) return st;
+    if (di->max_pairs_gated == 0)
+        di->max_pairs_gated = std::max(1, std::min(prefill_pair_max_clusters(kPrefillTileGated), di->num_sms / 2));
+
+    PrefillParams q;
+    std::memset(&q, 0, sizeof(q));
+    q.M = M; q.N = w->N; q.K = w->K; q.k_tail = w->k_tail;
+    q.m_tiles = (M + 255) / 256; q.n_tiles = (w->N + kPrefillTileGated - 1) / kPrefillTileGated;
+    const long long tiles = static_cast<long long>(q.m_tiles) * q.n_tiles;
+    if (tiles >= (1ll << 30)) return PRQ_ERR_INVALID_ARG;
+    // whole tiles only, wave after wave (a piece of a tile has no gate and up sums to put through the activation)
+    const int pairs = static_cast<int>(std::min<long long>(tiles, di->max_pairs_gated));
+    q.sk_tiles = 0; q.whole_tiles = static_cast<int>((tiles + pairs - 1) / pairs); q.total_tiles = static_cast<int>(tiles);
+    q.act_groups = dense_groups(M); q.w_groups = w->w_groups_alt[kAltGated];
+    q.act_sf = static_cast<const uint8_t*>(scales_sf); q.w_sf = w->d_sf_alt[kAltGated];
+    q.status = di->status_ptr; q.trace = trace_ptr(); q.dbg = env_int("PRQ_DBG", 0);
+    q.wait_limit = kDefaultWaitLimitCycles;
+    q.out_codes = static_cast<uint8_t*>(out_codes);
+    q.out_sf = static_cast<uint8_t*>(out_scales_sf);
+    q.out_scales_row = static_cast<uint8_t*>(out_scales_row);
+    q.out_h = static_cast<uint16_t*>(h_check);
+    q.out_C = C; q.out_k_tail = kd; q.out_groups = dense_groups(M);
+    CUtensorMap tm_act, tm_sfa;
+    st = make_code_map(&tm_act, codes, w->K / 2, M, 128);
+    if (st == PRQ_OK) st = make_sf_map(&tm_sfa, q.act_sf, static_cast<uint64_t>(w->plan.S) * q.act_groups * kSfGroupBytes, 4);
+    if (st != PRQ_OK) return st;
+    // (the kernel stores nothing through an output map in this mode: the activation map fills the parameter)
+    cudaError_t e = launch_prefill_pair(kPrefillTileGated, tm_act, w->tm_w_pair[kAltGated], w->tm_w_tail, tm_sfa, w->tm_sfw_pair[kAltGated],
+                                        tm_act, q, pairs, static_cast<cudaStream_t>(stream));
     g_launches.fetch_add(1);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
 }

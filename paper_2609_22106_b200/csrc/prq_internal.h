@@ -68,6 +68,9 @@ void rank_and_permute(const std::vector<double>& col_err, int K, int k_tail, std
 // rounded once to bf16); with duplicate_tail the last k_tail rows are repeated.  Host buffers.
 prq_status fold_producer(const int32_t* perm, const float* inv_s, int C, int k_tail, const uint16_t* W_up,
                          const uint16_t* W_gate, int H, bool duplicate_tail, uint16_t* out_up, uint16_t* out_gate);
+// Gate and up projection rows interleaved in groups of 32 (rows 64 b .. 64 b + 31 = gate rows 32 b .., rows 64 b + 32 ..
+// 64 b + 63 = up rows 32 b ..): the layout prq_linear_gated expects.  Host buffers, C % 32 == 0.
+void stack_gate_up(const uint16_t* W_gate, const uint16_t* W_up, int C, int H, uint16_t* out);
 // The same result computed on the current device from a DEVICE copy of W (column errors, permuted
 // quantisation, residual and packing as kernels; scales and ranking on the host in between).  Allocates its
 // temporaries, runs on `stream` and synchronises it.
@@ -92,12 +95,15 @@ struct prq_weights {
     uint8_t* d_sf = nullptr;         // E x S x w_groups x 1024 (+ padding)
     // Dense layers also keep the scale bytes grouped per 224-, 240- and 288-row weight tile of the prefill kernel
     // (two or three 128-row groups per tile, the last partly empty) so that those tile widths need no re-alignment.
-    uint8_t* d_sf_alt[3] = {nullptr, nullptr, nullptr};
-    int w_groups_alt[3] = {0, 0, 0};
+    // A handle prepared as a gated producer (prq_prep_opts::gated_producer) keeps the 192-row tiling instead, the
+    // one prq_linear_gated runs.
+    uint8_t* d_sf_alt[4] = {nullptr, nullptr, nullptr, nullptr};
+    int w_groups_alt[4] = {0, 0, 0, 0};
+    bool gated = false;
     // tensor maps of the weight side, encoded once (dense layers; a handle is immutable afterwards):
     // codes with 128-row boxes (decode kernel), codes with half-tile boxes and the scale bytes of the
-    // 224-row [0], 240-row [1] and 288-row [2] tilings (CTA-pair prefill kernel)
-    CUtensorMap tm_w_decode, tm_w_pair[3], tm_sfw_pair[3], tm_w_tail;   // tm_w_tail: 16-row boxes (288-row tiling)
+    // 224-row [0], 240-row [1], 288-row [2] and 192-row [3] tilings (CTA-pair prefill kernel)
+    CUtensorMap tm_w_decode, tm_w_pair[4], tm_sfw_pair[4], tm_w_tail;   // tm_w_tail: 16-row boxes (288-row tiling)
     bool maps_ready = false;
     int32_t* d_perm = nullptr;       // E x K
     float* d_inv_s_perm = nullptr;   // E x K : inv_s[perm[j]] in the new channel order

@@ -271,4 +271,12 @@ prq_status prepare_layer(const uint16_t* W, int N, int K, const float* amax, flo
     return PRQ_OK;
 }
 
+void stack_gate_up(const uint16_t* W_gate, const uint16_t* W_up, int C, int H, uint16_t* out) {
+    const size_t row = static_cast<size_t>(H) * sizeof(uint16_t);
+    for (int b = 0; b < C / kBlock; ++b) {
+        std::memcpy(out + static_cast<size_t>(2 * b) * kBlock * H, W_gate + static_cast<size_t>(b) * kBlock * H, row * kBlock);
+        std::memcpy(out + static_cast<size_t>(2 * b + 1) * kBlock * H, W_up + static_cast<size_t>(b) * kBlock * H, row * kBlock);
+    }
+}
+
 }  // namespace prq
