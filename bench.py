@@ -197,7 +197,18 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
             lin[gname] = dict(w=w, x=first["x"], codes=first["codes"], sf=first["sf"], N=Ng, K=first["K"], k=first["k"],
                               y=torch.empty((M, Ng), dtype=torch.bfloat16, device=dev), ws=prq.new_workspace(w, M, dev),
                               mode=prq.ACT_SCALE_PERM, Wb=Wcat)
+        # gate / up once more as a gated producer: rows interleaved in (gate, up) groups of 32, the product
+        # silu(gate) * up quantised inside the GEMM's epilogue straight into the down projection's buffers
+        # (timing only: the producers' fold of the down projection's 1 / s and permutation does not change the work)
+        C, Hd = lin["gate"]["N"], lin["gate"]["K"]
+        Wst = torch.stack([lin["gate"]["Wb"].view(C // 32, 32, Hd), lin["up"]["Wb"].view(C // 32, 32, Hd)], dim=1).reshape(2 * C, Hd).contiguous()
+        lin["gate_up_gated"] = dict(w=prq.prepare_weights_device(Wst.view(torch.int16), lin["gate"]["amax"], 0.5, lin["gate"]["k"], gated_producer=True),
+                                    x=lin["gate"]["x"], codes=lin["gate"]["codes"], sf=lin["gate"]["sf"], mode=prq.ACT_SCALE_PERM)
         layers.append(lin)
+
+    def gg(lin):
+        d, dn = lin["gate_up_gated"], lin["down"]
+        return lambda: prq.linear_gated(d["w"], d["codes"], d["sf"], M, dn["w"], out=(dn["codes"], None, dn["sf"]))
 
     def q(d):
         return lambda: prq.quantize_act(d["w"], d["x"], d["mode"], out=(d["codes"], None, d["sf"]))
@@ -226,6 +237,11 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
     t_step_grouped = timer.run(step_grouped, n, n_layers) / n
     t_bf16_grouped = timer.run([(lambda lin=lin: [torch.matmul(lin[name]["x"], lin[name]["Wb"].t()) for name in grouped])
                                 for lin in layers], n, n_layers) / n
+    # the same block with the gated producer: no quantiser launch for the down projection, no bf16 gate / up output
+    step_gated = [(lambda lin=lin: [f() for f in (q(lin["qkv"]), g(lin["qkv"]), q(lin["o"]), g(lin["o"]),
+                                                   q(lin["gate_up_gated"]), gg(lin), g(lin["down"]))]) for lin in layers]
+    t_step_gated = timer.run(step_gated, n, n_layers) / n
+    t_gated = timer.run([gg(lin) for lin in layers], n, n_layers) / n
     grouped_rows = {}
     for name in ("qkv", "gate_up"):
         ds = [lin[name] for lin in layers]
@@ -268,7 +284,7 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
     if t_step_multi is not None:
         extra = dict(step_multi_launch_us=t_step_multi * 1e6, bf16_fused_qkv_gateup_us=bf16_fused * 1e6)
     extra.update(step_grouped_prep_us=t_step_grouped * 1e6, bf16_grouped_us=t_bf16_grouped * 1e6,
-                 grouped_linears=grouped_rows)
+                 grouped_linears=grouped_rows, step_gated_producer_us=t_step_gated * 1e6, gated_producer_gemm_us=t_gated * 1e6)
     return dict(workload=tag, M=M, layers=n_layers, step_us=t_step * 1e6, step_tflops=total_flops / t_step / 1e12, **extra,
                 gemm_us_sum=sum(r["gemm_us"] for r in rows.values()), quant_us_sum=sum(r["quant_us"] for r in rows.values()),
                 bf16_us_sum=sum(r["bf16_matmul_us"] for r in rows.values()), device_status=status, linears=rows)

@@ -27,7 +27,7 @@ EXPORTS = [
     "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_multi", "prq_quantize_act_multi",
     "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
-    "prq_handover_probe",
+    "prq_handover_probe", "prq_stack_gate_up", "prq_linear_gated",
 ]
 
 
@@ -82,6 +82,8 @@ def lib():
         L.prq_kernel_launch_count.restype = ctypes.c_ulonglong
         L.prq_mxf4_peak_probe.argtypes = [ci, ctypes.POINTER(ci), vp]
         L.prq_handover_probe.argtypes = [ci, ci, ci, ci, vp]
+        L.prq_stack_gate_up.argtypes = [vp, vp, ci, ci, vp]
+        L.prq_linear_gated.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -166,17 +168,18 @@ class Weights:
 
 
 class PrepOpts(ctypes.Structure):
-    _fields_ = [("struct_size", ctypes.c_size_t), ("weight_scale_search", ctypes.c_int)]
+    _fields_ = [("struct_size", ctypes.c_size_t), ("weight_scale_search", ctypes.c_int), ("gated_producer", ctypes.c_int)]
 
 
-def _opts(scale_search: bool):
-    return PrepOpts(ctypes.sizeof(PrepOpts), 1 if scale_search else 0)
+def _opts(scale_search: bool, gated_producer: bool = False):
+    return PrepOpts(ctypes.sizeof(PrepOpts), 1 if scale_search else 0, 1 if gated_producer else 0)
 
 
 def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_tail: int,
-                    scale_search: bool = False) -> Weights:
+                    scale_search: bool = False, gated_producer: bool = False) -> Weights:
     """W_bf16: uint16 (N, K) or (E, N, K); act_amax: float32 (K,) or (E, K).  scale_search: the E8M0-W
-    variant (weight-side block-scale search)."""
+    variant (weight-side block-scale search).  gated_producer: W is a stacked gate / up projection in the row order
+    of stack_gate_up, to be run by linear_gated."""
     W = np.ascontiguousarray(W_bf16, np.uint16)
     amax = np.ascontiguousarray(act_amax, np.float32)
     if W.ndim == 2:
@@ -184,7 +187,7 @@ def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_ta
         amax = amax[None]
     E, N, K = W.shape
     h = ctypes.c_void_p()
-    o = _opts(scale_search)
+    o = _opts(scale_search, gated_producer)
     _check(lib().prq_prepare_weights_opts(_np_ptr(W), E, N, K, _np_ptr(amax), alpha, k_tail,
                                           ctypes.cast(ctypes.pointer(o), ctypes.c_void_p), ctypes.byref(h)),
            "prq_prepare_weights_opts")
@@ -192,7 +195,7 @@ def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_ta
 
 
 def prepare_weights_device(W, act_amax: np.ndarray, alpha: float, k_tail: int, scale_search: bool = False,
-                           stream=None) -> Weights:
+                           stream=None, gated_producer: bool = False) -> Weights:
     """W: torch CUDA tensor, bf16 (or its uint16 / int16 bit pattern), (N, K) or (E, N, K), contiguous.  The prep
     runs on the GPU; the handle equals the one prepare_weights builds from a host copy."""
     assert W.is_cuda and W.is_contiguous() and W.element_size() == 2
@@ -203,7 +206,7 @@ def prepare_weights_device(W, act_amax: np.ndarray, alpha: float, k_tail: int, s
         amax = amax[None]
     E, N, K = shape
     h = ctypes.c_void_p()
-    o = _opts(scale_search)
+    o = _opts(scale_search, gated_producer)
     _check(lib().prq_prepare_weights_device(W.data_ptr(), E, N, K, _np_ptr(amax), alpha, k_tail,
                                             ctypes.cast(ctypes.pointer(o), ctypes.c_void_p), _stream_ptr(stream),
                                             ctypes.byref(h)),
@@ -425,3 +428,33 @@ def handover_probe(n: int, grid: int, threads: int = 192, cluster: int = 1, stre
     """Enqueues n empty, dependent launches shaped like the decode GEMM's (see include/prq.h); the caller times them."""
     _check(lib().prq_handover_probe(int(n), int(grid), int(threads), int(cluster), _stream_ptr(stream)),
            "prq_handover_probe")
+
+
+def stack_gate_up(W_gate: np.ndarray, W_up: np.ndarray) -> np.ndarray:
+    """Gate and up projection rows (C, H) uint16 interleaved in groups of 32: the stacked layer linear_gated runs."""
+    Wg = np.ascontiguousarray(W_gate, np.uint16)
+    Wu = np.ascontiguousarray(W_up, np.uint16)
+    C, H = Wg.shape
+    out = np.empty((2 * C, H), np.uint16)
+    _check(lib().prq_stack_gate_up(_np_ptr(Wg), _np_ptr(Wu), C, H, _np_ptr(out)), "prq_stack_gate_up")
+    return out
+
+
+def linear_gated(w_gu: Weights, codes, scales_sf, M: int, w_down: Weights, row_scales: bool = False, h_check: bool = False,
+                 out=None, stream=None):
+    """Q(silu(gate) * up) of the stacked producer layer, written as the down projection's quantised activation.
+    Returns (codes, scales_row or None, scales_sf, h or None) -- h only on request, for checks."""
+    import torch
+
+    C, k = w_down.K, w_down.k_tail
+    dev = codes.device
+    if out is None:
+        oc = torch.empty(max(act_bytes(M, C, k, 1, BUF_CODES), 16), dtype=torch.uint8, device=dev)
+        osf = torch.empty(max(act_bytes(M, C, k, 1, BUF_SCALES_SF), 16), dtype=torch.uint8, device=dev)
+        orow = torch.empty(max(act_bytes(M, C, k, 1, BUF_SCALES_ROW), 16), dtype=torch.uint8, device=dev) if row_scales else None
+    else:
+        oc, orow, osf = out
+    h = torch.empty((M, C), dtype=torch.bfloat16, device=dev) if h_check else None
+    _check(lib().prq_linear_gated(w_gu.handle, _dptr(codes), _dptr(scales_sf), M, w_down.handle, _dptr(oc), _dptr(orow),
+                                  _dptr(osf), _dptr(h), _stream_ptr(stream)), "prq_linear_gated")
+    return oc, orow, osf, h
