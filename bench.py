@@ -30,7 +30,7 @@ FP4_OVER_BF16 = 4.0  # nominal dense tensor ratio (9 vs 2.25 PFLOP/s)
 # DRAM bytes of one prefill GEMM launch at this workload: not a quantity of this run but the figure of the ncu
 # capture summarised in the file named here (dram__bytes_read.sum + dram__bytes_write.sum; the 21 MB of outputs
 # were still in L2 when the kernel ended, which is why it is below the algorithmic bytes).
-NCU_PREFILL_DRAM_BYTES = 24.34e6 + 2.18e6
+NCU_PREFILL_DRAM_BYTES = 24.53e6 + 0.006e6
 NCU_PREFILL_SOURCE = "profiles/prefill_pair_M2048.txt"
 LONG_RUN_LAUNCHES = 2000   # GEMM launches of the power-capped regime reported as roofline.frac_long_run
 
