@@ -337,7 +337,10 @@ cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStr
     QuantBatch bb = b;
     bb.n_atoms = n_atoms;
     bb.n_tail = 0; bb.tail_split = 1;
-    if (scale_perm) {
+    // (dense launches only: a grouped launch has a CTA per expert group and column atom already, each with the fixed
+    // cost of finding its expert -- eight times as many tail CTAs made the 128-expert quantiser 35-50 % slower, and its
+    // launches are long enough for a 20 us CTA not to be their end)
+    if (scale_perm && b.expert_offsets == nullptr) {
         int k_max = 0;
         for (int i = 0; i < b.n_lin; ++i) k_max = b.lay[i].k_tail > k_max ? b.lay[i].k_tail : k_max;
         bb.n_tail = (k_max + kAtomK - 1) / kAtomK < n_atoms ? (k_max + kAtomK - 1) / kAtomK : n_atoms;
