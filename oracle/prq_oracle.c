@@ -43,7 +43,9 @@
  * brute-force top-k, Eq. (3) = main + correction.  The normalised error and the alpha
  * selection of the Python front end (first minimum over the grid) are pinned by a hand-worked
  * error norm and a hand-decided three-candidate search (tests/test_oracle_alpha.py).  The gated activation
- * silu(g) * u of the producer is pinned by closed-form values and identities (tests/test_oracle_gated.py).
+ * silu(g) * u of the producer is pinned by closed-form values and identities (tests/test_oracle_gated.py); the
+ * second format (MXFP8) by hand-worked encodings and a brute-force nearest-value search over the whole code
+ * table (tests/test_oracle_mxfp8.py).
  */
 #include <math.h>
 #include <stdint.h>
@@ -429,6 +431,127 @@ int orc_fold_producer(const uint16_t *W_up, const uint16_t *W_gate, long C, long
             if (W_gate && out_gate) out_gate[jp * H + h] = W_gate[j * H + h];
         }
     }
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------------------------------------
+ * Second format: MXFP8 (OCP MX, E4M3 elements), the format the paper's end-to-end setting runs the attention
+ * linears in (Experimental setup); plain W8A8 -- Eq. (2)'s compensation is defined for MXFP4 and is not applied.
+ * The paper gives only the format's name; the reading mirrors the MXFP4 one:
+ *   - blocks of 32 along the reduction axis, E8M0 scale 2^e with e = clamp(floor(log2 amax) - 8, -127, 127)
+ *     (8 = exponent of the largest E4M3 magnitude 448 = 1.75 * 2^8), byte e + 127; all-zero block: byte 0;
+ *   - elements: E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; subnormals below 2^-6 in steps of
+ *     2^-9; no infinities; the all-ones pattern is NaN and never produced), round to nearest, ties to the even
+ *     mantissa, magnitudes above 448 saturate to 448 (so amax / 2^e in (448, 512) saturates, as (6, 8) does in
+ *     MXFP4); the sign of values that round to zero is kept. */
+static double orc_e4m3_value(uint8_t code) {
+    int ex = (code >> 3) & 15, man = code & 7;
+    double mag = ex == 0 ? ldexp((double)man, -9) : ldexp(1.0 + man / 8.0, ex - 7);
+    return (code & 0x80) ? -mag : mag;
+}
+
+static uint8_t orc_fp8_block_scale_byte(const float *v) {
+    double amax = 0.0;
+    for (int i = 0; i < ORC_BLOCK; ++i) {
+        double a = fabs((double)v[i]);
+        if (a > amax) amax = a;
+    }
+    if (amax == 0.0) return 0;
+    int ex;
+    (void)frexp(amax, &ex);
+    int e = (ex - 1) - 8;
+    if (e < -127) e = -127;
+    if (e > 127) e = 127;
+    return (uint8_t)(e + 127);
+}
+
+static uint8_t orc_e4m3_code(float v, int e) {
+    double a = ldexp(fabs((double)v), -e);   /* exact */
+    uint8_t sign = (uint8_t)(orc_signbit_f32(v) << 7);
+    if (a >= 464.0) return (uint8_t)(sign | 0x7E);          /* past the midpoint to the next step: saturate at 448 */
+    if (a < ldexp(1.0, -6)) {                                /* subnormal range: multiples of 2^-9 */
+        int q = (int)nearbyint(ldexp(a, 9));                 /* ties to even */
+        return (uint8_t)(sign | (q == 8 ? 0x08 : q));
+    }
+    int ex;
+    double m = frexp(a, &ex);                                /* a = m 2^ex, m in [0.5, 1) */
+    int q = (int)nearbyint(ldexp(m, 4));                     /* 4 significant bits: 8 .. 16 */
+    int eu = ex - 1;
+    if (q == 16) { q = 8; eu += 1; }
+    if (eu > 8 || (eu == 8 && q > 14)) return (uint8_t)(sign | 0x7E);
+    return (uint8_t)(sign | ((eu + 7) << 3) | (q - 8));
+}
+
+/* Q of the second format, storage half: rows x cols fp32 -> codes (rows x cols bytes), scale bytes (rows x cols/32). */
+int orc_fp8_quantize_rows(const float *v, long rows, long cols, uint8_t *codes, uint8_t *scales) {
+    if (cols % ORC_BLOCK) return 1;
+    for (long r = 0; r < rows; ++r)
+        for (long b = 0; b < cols / ORC_BLOCK; ++b) {
+            const float *blk = v + r * cols + b * ORC_BLOCK;
+            uint8_t byte = orc_fp8_block_scale_byte(blk);
+            scales[r * (cols / ORC_BLOCK) + b] = byte;
+            for (int i = 0; i < ORC_BLOCK; ++i) codes[r * cols + b * ORC_BLOCK + i] = orc_e4m3_code(blk[i], (int)byte - 127);
+        }
+    return 0;
+}
+
+int orc_fp8_dequantize_rows(const uint8_t *codes, const uint8_t *scales, long rows, long cols, double *out) {
+    if (cols % ORC_BLOCK) return 1;
+    for (long r = 0; r < rows; ++r)
+        for (long j = 0; j < cols; ++j)
+            out[r * cols + j] = ldexp(orc_e4m3_value(codes[r * cols + j]), (int)scales[r * (cols / ORC_BLOCK) + j / ORC_BLOCK] - 127);
+    return 0;
+}
+
+/* Offline half for one alpha: s as in the MXFP4 path, W0 = fl32(W * s), Q by rows.  No permutation, no tail. */
+int orc_fp8_prepare(const uint16_t *W_bf16, long N, long K, const float *amax, double alpha, float *s, float *inv_s,
+                    uint8_t *wcodes, uint8_t *wscales) {
+    if (K % ORC_BLOCK) return 1;
+    orc_scales_from_amax(amax, K, alpha, s, inv_s);
+    float *W0 = (float *)malloc(sizeof(float) * N * K);
+    for (long n = 0; n < N; ++n)
+        for (long j = 0; j < K; ++j)
+            W0[n * K + j] = (float)((double)orc_bf16_to_f32(W_bf16[n * K + j]) * (double)s[j]);
+    orc_fp8_quantize_rows(W0, N, K, wcodes, wscales);
+    free(W0);
+    return 0;
+}
+
+/* Online half, activation side: xt[t,j] = fl32(x[t,j] * inv_s[j]) (inv_s may be NULL: identity), then Q by rows. */
+int orc_fp8_quantize_act(const uint16_t *x_bf16, long M, long K, const float *inv_s, uint8_t *codes, uint8_t *scales) {
+    if (K % ORC_BLOCK) return 1;
+    float *row = (float *)malloc(sizeof(float) * K);
+    for (long t = 0; t < M; ++t) {
+        for (long j = 0; j < K; ++j) {
+            double v = (double)orc_bf16_to_f32(x_bf16[t * K + j]);
+            if (inv_s) v = v * (double)inv_s[j];
+            row[j] = (float)v;
+        }
+        orc_fp8_quantize_rows(row, 1, K, codes + t * K, scales + t * (K / ORC_BLOCK));
+    }
+    free(row);
+    return 0;
+}
+
+/* y[t,n] = sum_j deq(A)[t,j] deq(W)[n,j] in FP64, ascending j. */
+int orc_fp8_matmul(const uint8_t *acodes, const uint8_t *ascales, const uint8_t *wcodes, const uint8_t *wscales,
+                   long M, long N, long K, double *y) {
+    if (K % ORC_BLOCK) return 1;
+    double *a = (double *)malloc(sizeof(double) * M * K);
+    double *w = (double *)malloc(sizeof(double) * N * K);
+    orc_fp8_dequantize_rows(acodes, ascales, M, K, a);
+    orc_fp8_dequantize_rows(wcodes, wscales, N, K, w);
+    long t;
+#ifdef _OPENMP
+#pragma omp parallel for schedule(static)
+#endif
+    for (t = 0; t < M; ++t)
+        for (long n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (long j = 0; j < K; ++j) acc += a[t * K + j] * w[n * K + j];
+            y[t * N + n] = acc;
+        }
+    free(a); free(w);
     return 0;
 }
 

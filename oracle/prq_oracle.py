@@ -247,6 +247,69 @@ def stack_gate_up(W_gate, W_up):
     return out
 
 
+# ---- second format: MXFP8 (E4M3 elements, E8M0 block scales), plain W8A8 ----
+
+def fp8_quantize_rows(v):
+    """fp32 (rows, cols) -> (E4M3 codes (rows, cols), scale bytes (rows, cols/32))."""
+    v = _c(v, np.float32)
+    rows, cols = v.shape
+    codes = np.empty((rows, cols), np.uint8)
+    scales = np.empty((rows, cols // BLOCK), np.uint8)
+    if _load().orc_fp8_quantize_rows(_p(v), ctypes.c_long(rows), ctypes.c_long(cols), _p(codes), _p(scales)):
+        raise ValueError("cols must be a multiple of 32")
+    return codes, scales
+
+
+def fp8_dequantize_rows(codes, scales):
+    codes = _c(codes, np.uint8)
+    scales = _c(scales, np.uint8)
+    rows, cols = codes.shape
+    out = np.empty((rows, cols), np.float64)
+    if _load().orc_fp8_dequantize_rows(_p(codes), _p(scales), ctypes.c_long(rows), ctypes.c_long(cols), _p(out)):
+        raise ValueError("cols must be a multiple of 32")
+    return out
+
+
+def fp8_prepare(W_bf16, amax, alpha: float):
+    """Offline half of the MXFP8 layer for one alpha: scale by s = amax^alpha, quantise by rows."""
+    W = _c(W_bf16, np.uint16)
+    am = _c(amax, np.float32)
+    N, K = W.shape
+    s = np.empty(K, np.float32)
+    inv_s = np.empty(K, np.float32)
+    wc = np.empty((N, K), np.uint8)
+    wsc = np.empty((N, K // BLOCK), np.uint8)
+    if _load().orc_fp8_prepare(_p(W), ctypes.c_long(N), ctypes.c_long(K), _p(am), ctypes.c_double(alpha), _p(s), _p(inv_s),
+                               _p(wc), _p(wsc)):
+        raise ValueError("K must be a multiple of 32")
+    return dict(alpha=alpha, s=s, inv_s=inv_s, wcodes=wc, wscales=wsc)
+
+
+def fp8_quantize_act(x_bf16, inv_s=None):
+    x = _c(x_bf16, np.uint16)
+    M, K = x.shape
+    iv = _c(inv_s, np.float32) if inv_s is not None else None
+    codes = np.empty((M, K), np.uint8)
+    scales = np.empty((M, K // BLOCK), np.uint8)
+    if _load().orc_fp8_quantize_act(_p(x), ctypes.c_long(M), ctypes.c_long(K), _p(iv) if iv is not None else None,
+                                    _p(codes), _p(scales)):
+        raise ValueError("K must be a multiple of 32")
+    return codes, scales
+
+
+def fp8_matmul(acodes, ascales, wcodes, wscales):
+    a = _c(acodes, np.uint8)
+    asc = _c(ascales, np.uint8)
+    w = _c(wcodes, np.uint8)
+    wsc = _c(wscales, np.uint8)
+    M, K = a.shape
+    N = w.shape[0]
+    y = np.empty((M, N), np.float64)
+    if _load().orc_fp8_matmul(_p(a), _p(asc), _p(w), _p(wsc), ctypes.c_long(M), ctypes.c_long(N), ctypes.c_long(K), _p(y)):
+        raise ValueError("K must be a multiple of 32")
+    return y
+
+
 def nrmse(y_hat, y):
     """Normalised reconstruction error ||Yhat - Y||_F / ||Y||_F (text after Eq. (3))."""
     return float(np.linalg.norm(y_hat - y) / np.linalg.norm(y))
