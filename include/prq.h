@@ -105,15 +105,24 @@ prq_status prq_prepare_weights(const uint16_t *W, int n_experts, int N, int K, c
  *                        1: the layer is the stacked gate / up projection of a gated FFN in the row order of
  *                           prq_stack_gate_up, to be run by prq_linear_gated.  The prepared weights are the same;
  *                           the handle keeps the scale-byte tiling of that call's kernel instead of those of
- *                           prq_linear, which therefore refuses it for more than 128 tokens. */
+ *                           prq_linear, which therefore refuses it for more than 128 tokens.
+ *   format               PRQ_FMT_MXFP4 (default): the paper's format for the FFN / expert layers.
+ *                        PRQ_FMT_MXFP8: E4M3 elements with the same 32-element E8M0 block scales, the format the
+ *                           paper's end-to-end setting runs the attention linears in (Experimental setup), as plain
+ *                           W8A8: k_tail must be 0 (Eq. (2)'s compensation is defined for MXFP4), alpha still scales.
+ *                           Served by prq_quantize_act and prq_linear (dense layers, any M); buffer sizes come from
+ *                           prq_act_bytes_for.  The other online calls return INVALID_ARG for such a handle.
+ * A caller compiled against an earlier header may pass its smaller struct: fields beyond struct_size read as 0. */
+typedef enum { PRQ_FMT_MXFP4 = 0, PRQ_FMT_MXFP8 = 1 } prq_format;
 typedef struct prq_prep_opts {
     size_t struct_size;
     int weight_scale_search;
     int gated_producer;
+    int format;
 } prq_prep_opts;
 
 /* prq_prepare_weights with options (opts may be NULL).  Errors as prq_prepare_weights, plus INVALID_ARG for a
- * struct_size smaller than this header's. */
+ * struct_size smaller than the first version of the struct (16 bytes). */
 prq_status prq_prepare_weights_opts(const uint16_t *W, int n_experts, int N, int K, const float *act_amax,
                                     float alpha, int k_tail, const prq_prep_opts *opts, prq_weights **out);
 
@@ -138,7 +147,8 @@ prq_status prq_prepare_weights_host(const uint16_t *W, int N, int K, const float
                                     int k_tail, uint8_t *codes, uint8_t *scales, int32_t *perm, float *s,
                                     float *inv_s, double *col_err);
 
-/* prq_prepare_weights_host with options (opts may be NULL). */
+/* prq_prepare_weights_host with options (opts may be NULL).  With format = PRQ_FMT_MXFP8: k_tail must be 0, codes is
+ * N x K bytes, perm comes back as the identity and col_err as zeros. */
 prq_status prq_prepare_weights_host_opts(const uint16_t *W, int N, int K, const float *act_amax, float alpha,
                                          int k_tail, const prq_prep_opts *opts, uint8_t *codes, uint8_t *scales,
                                          int32_t *perm, float *s, float *inv_s, double *col_err);
@@ -201,7 +211,11 @@ prq_status prq_stack_gate_up(const uint16_t *W_gate, const uint16_t *W_up, int C
 /* Shape of a handle.  Any output pointer may be NULL. */
 prq_status prq_weights_info(const prq_weights *w, int *n_experts, int *N, int *K, int *k_tail, float *alpha);
 
-/* Copy one canonical host-side view of expert `expert` into dst (host, dst_bytes must match). */
+/* Format of a handle (a prq_format).  INVALID_ARG for NULL. */
+prq_status prq_weights_format(const prq_weights *w, int *format);
+
+/* Copy one canonical host-side view of expert `expert` into dst (host, dst_bytes must match).  For an MXFP8 handle
+ * PRQ_FIELD_CODES is N x K bytes of E4M3 codes. */
 prq_status prq_weights_get(const prq_weights *w, int expert, prq_field which, void *dst, size_t dst_bytes);
 
 /* ---- online ------------------------------------------------------------------------------ */
@@ -210,6 +224,10 @@ prq_status prq_weights_get(const prq_weights *w, int expert, prq_field which, vo
  * count and n_groups = number of experts (each group's scale tiles are padded to 128 rows);
  * dense calls pass n_groups = 1.  Returns 0 for invalid arguments. */
 size_t prq_act_bytes(int M, int K, int k_tail, int n_groups, prq_buf which);
+
+/* The same sizes for the layer behind a handle, whatever its format (MXFP8: one byte per code, scale bytes in
+ * 512-byte groups per 128-element stage).  Dense layers; returns 0 for invalid arguments. */
+size_t prq_act_bytes_for(const prq_weights *w, int M, prq_buf which);
 
 /* The single MXFP4 quantisation of the reordered activation that the Kernel design paragraph calls for.
  * One launch: optional scale + permute (Eq. (1), activation side), per-32 amax, E8M0 scale,

@@ -27,7 +27,7 @@ EXPORTS = [
     "prq_linear", "prq_linear_static_scratch", "prq_linear_fused", "prq_linear_multi", "prq_quantize_act_multi",
     "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
-    "prq_handover_probe", "prq_stack_gate_up", "prq_linear_gated",
+    "prq_handover_probe", "prq_stack_gate_up", "prq_linear_gated", "prq_weights_format", "prq_act_bytes_for",
 ]
 
 
@@ -82,6 +82,9 @@ def lib():
         L.prq_kernel_launch_count.restype = ctypes.c_ulonglong
         L.prq_mxf4_peak_probe.argtypes = [ci, ctypes.POINTER(ci), vp]
         L.prq_handover_probe.argtypes = [ci, ci, ci, ci, vp]
+        L.prq_weights_format.argtypes = [vp, ctypes.POINTER(ci)]
+        L.prq_act_bytes_for.argtypes = [vp, ci, ci]
+        L.prq_act_bytes_for.restype = cs
         L.prq_stack_gate_up.argtypes = [vp, vp, ci, ci, vp]
         L.prq_linear_gated.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, vp, vp]
         _lib = L
@@ -123,6 +126,9 @@ class Weights:
         a = ctypes.c_float()
         _check(lib().prq_weights_info(handle, ne, N, K, k, a), "prq_weights_info")
         self.n_experts, self.N, self.K, self.k_tail, self.alpha = ne.value, N.value, K.value, k.value, a.value
+        f = ctypes.c_int()
+        _check(lib().prq_weights_format(handle, ctypes.byref(f)), "prq_weights_format")
+        self.format = f.value
 
     @property
     def handle(self):
@@ -131,7 +137,7 @@ class Weights:
     def get(self, field: int, expert: int = 0) -> np.ndarray:
         Ka = self.K + self.k_tail
         shape, dt = {
-            FIELD_CODES: ((self.N, Ka // 2), np.uint8),
+            FIELD_CODES: ((self.N, Ka // 2 if self.format == FMT_MXFP4 else self.K), np.uint8),
             FIELD_SCALES: ((self.N, Ka // 32), np.uint8),
             FIELD_PERM: ((self.K,), np.int32),
             FIELD_TOPK: ((self.k_tail,), np.int32),
@@ -167,16 +173,20 @@ class Weights:
             pass
 
 
+FMT_MXFP4, FMT_MXFP8 = 0, 1
+
+
 class PrepOpts(ctypes.Structure):
-    _fields_ = [("struct_size", ctypes.c_size_t), ("weight_scale_search", ctypes.c_int), ("gated_producer", ctypes.c_int)]
+    _fields_ = [("struct_size", ctypes.c_size_t), ("weight_scale_search", ctypes.c_int), ("gated_producer", ctypes.c_int),
+                ("format", ctypes.c_int)]
 
 
-def _opts(scale_search: bool, gated_producer: bool = False):
-    return PrepOpts(ctypes.sizeof(PrepOpts), 1 if scale_search else 0, 1 if gated_producer else 0)
+def _opts(scale_search: bool, gated_producer: bool = False, fmt: int = FMT_MXFP4):
+    return PrepOpts(ctypes.sizeof(PrepOpts), 1 if scale_search else 0, 1 if gated_producer else 0, fmt)
 
 
 def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_tail: int,
-                    scale_search: bool = False, gated_producer: bool = False) -> Weights:
+                    scale_search: bool = False, gated_producer: bool = False, fmt: int = FMT_MXFP4) -> Weights:
     """W_bf16: uint16 (N, K) or (E, N, K); act_amax: float32 (K,) or (E, K).  scale_search: the E8M0-W
     variant (weight-side block-scale search).  gated_producer: W is a stacked gate / up projection in the row order
     of stack_gate_up, to be run by linear_gated."""
@@ -187,7 +197,7 @@ def prepare_weights(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_ta
         amax = amax[None]
     E, N, K = W.shape
     h = ctypes.c_void_p()
-    o = _opts(scale_search, gated_producer)
+    o = _opts(scale_search, gated_producer, fmt)
     _check(lib().prq_prepare_weights_opts(_np_ptr(W), E, N, K, _np_ptr(amax), alpha, k_tail,
                                           ctypes.cast(ctypes.pointer(o), ctypes.c_void_p), ctypes.byref(h)),
            "prq_prepare_weights_opts")
@@ -215,15 +225,15 @@ def prepare_weights_device(W, act_amax: np.ndarray, alpha: float, k_tail: int, s
 
 
 def prepare_weights_host(W_bf16: np.ndarray, act_amax: np.ndarray, alpha: float, k_tail: int,
-                         scale_search: bool = False) -> dict:
+                         scale_search: bool = False, fmt: int = FMT_MXFP4) -> dict:
     W = np.ascontiguousarray(W_bf16, np.uint16)
     amax = np.ascontiguousarray(act_amax, np.float32)
     N, K = W.shape
     Ka = K + k_tail
-    out = dict(codes=np.empty((N, Ka // 2), np.uint8), scales=np.empty((N, Ka // 32), np.uint8),
+    out = dict(codes=np.empty((N, Ka // 2 if fmt == FMT_MXFP4 else K), np.uint8), scales=np.empty((N, Ka // 32), np.uint8),
                perm=np.empty(K, np.int32), s=np.empty(K, np.float32), inv_s=np.empty(K, np.float32),
                col_err=np.empty(K, np.float64))
-    o = _opts(scale_search)
+    o = _opts(scale_search, False, fmt)
     _check(lib().prq_prepare_weights_host_opts(_np_ptr(W), N, K, _np_ptr(amax), alpha, k_tail,
                                                ctypes.cast(ctypes.pointer(o), ctypes.c_void_p), _np_ptr(out["codes"]),
                                                _np_ptr(out["scales"]), _np_ptr(out["perm"]), _np_ptr(out["s"]),
@@ -279,10 +289,11 @@ def quantize_act(w: Weights, x, mode: int = ACT_IDENTITY, expert_offsets=None, r
     M = x.shape[0]
     ng = w.n_experts
     if out is None:
-        codes = torch.empty(max(act_bytes(M, w.K, w.k_tail, ng, BUF_CODES), 16), dtype=torch.uint8, device=x.device)
-        sf = torch.empty(max(act_bytes(M, w.K, w.k_tail, ng, BUF_SCALES_SF), 16), dtype=torch.uint8, device=x.device)
-        srow = torch.empty(max(act_bytes(M, w.K, w.k_tail, ng, BUF_SCALES_ROW), 16), dtype=torch.uint8,
-                           device=x.device) if row_scales else None
+        size = (lambda which: act_bytes(M, w.K, w.k_tail, ng, which)) if w.format == FMT_MXFP4 else \
+               (lambda which: int(lib().prq_act_bytes_for(w.handle, M, which)))
+        codes = torch.empty(max(size(BUF_CODES), 16), dtype=torch.uint8, device=x.device)
+        sf = torch.empty(max(size(BUF_SCALES_SF), 16), dtype=torch.uint8, device=x.device)
+        srow = torch.empty(max(size(BUF_SCALES_ROW), 16), dtype=torch.uint8, device=x.device) if row_scales else None
     else:
         codes, srow, sf = out
     _check(lib().prq_quantize_act(w.handle, mode, _dptr(x), M, x.stride(0) if M else w.K, _dptr(expert_offsets),

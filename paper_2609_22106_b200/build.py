@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 TRACE = os.environ.get("PRQ_TRACE") == "1"   # developer build: clock-stamp tracing compiled into the kernels
 LIB = os.path.join(HERE, "libprq_trace.so" if TRACE else "libprq.so")
-SOURCES = ["prq_api.cu", "prq_prep.cu", "prq_prep_device.cu", "prq_quant.cu", "prq_gemm.cu", "prq_gemm_prefill_pair.cu", "prq_gemm_decode.cu", "prq_peak_probe.cu"]
+SOURCES = ["prq_api.cu", "prq_prep.cu", "prq_prep_device.cu", "prq_quant.cu", "prq_gemm.cu", "prq_gemm_prefill_pair.cu", "prq_gemm_decode.cu", "prq_peak_probe.cu", "prq_fp8.cu"]
 
 
 def _newest_source_mtime() -> float:

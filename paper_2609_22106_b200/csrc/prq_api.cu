@@ -363,6 +363,7 @@ void prq_weights_free(prq_weights* w) {
     cudaFree(w->d_sf);
     cudaFree(w->d_perm);
     cudaFree(w->d_inv_s_perm);
+    cudaFree(w->d_inv_s);
     for (uint8_t* p : w->d_sf_alt) cudaFree(p);
     if (w->device >= 0 && w->device != cur) cudaSetDevice(cur);
     delete w;
@@ -387,11 +388,39 @@ prq_status prq_prepare_weights_device(const uint16_t* W_device, int n_experts, i
     return create_handle(W_device, true, stream, n_experts, N, K, act_amax, alpha, k_tail, opts, out);
 }
 
+// Options as this version of the library understands them; a caller built against an earlier header passes a shorter
+// struct, whose missing fields read as zero.
+struct PrepOptions { bool scale_search = false, gated = false; int format = PRQ_FMT_MXFP4; bool valid = true; };
+static PrepOptions read_opts(const prq_prep_opts* opts) {
+    PrepOptions o;
+    if (!opts) return o;
+    if (opts->struct_size < 16) { o.valid = false; return o; }
+    o.scale_search = opts->weight_scale_search != 0;
+    if (opts->struct_size >= offsetof(prq_prep_opts, gated_producer) + sizeof(int)) o.gated = opts->gated_producer != 0;
+    if (opts->struct_size >= offsetof(prq_prep_opts, format) + sizeof(int)) o.format = opts->format;
+    if (o.format != PRQ_FMT_MXFP4 && o.format != PRQ_FMT_MXFP8) o.valid = false;
+    return o;
+}
+
+static prq_status create_handle_fp8(const uint16_t* W, int N, int K, const float* act_amax, float alpha, int dev, prq_weights** out);
+
 static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_t stream, int n_experts, int N, int K,
                                 const float* act_amax, float alpha, int k_tail, const prq_prep_opts* opts, prq_weights** out) {
-    if (opts && opts->struct_size < sizeof(prq_prep_opts)) return PRQ_ERR_INVALID_ARG;
-    const bool scale_search = opts && opts->weight_scale_search != 0;
-    const bool gated = opts && opts->gated_producer != 0;
+    const PrepOptions po = read_opts(opts);
+    if (!po.valid) return PRQ_ERR_INVALID_ARG;
+    const bool scale_search = po.scale_search;
+    const bool gated = po.gated;
+    if (po.format == PRQ_FMT_MXFP8) {
+        // plain W8A8: no tail, no expert stack, no search; the preparation runs on the host
+        if (k_tail != 0 || n_experts != 1 || scale_search || gated || w_on_device) return PRQ_ERR_INVALID_ARG;
+        if (!W || !act_amax || !out || N < 1 || K < kBlock || K % kBlock || !std::isfinite(alpha)) return PRQ_ERR_INVALID_ARG;
+        int dev8 = 0;
+        if (cudaGetDevice(&dev8) != cudaSuccess) return PRQ_ERR_CUDA;
+        DeviceInfo* di8;
+        prq_status st8 = device_info(dev8, &di8);
+        if (st8 != PRQ_OK) return st8;
+        return create_handle_fp8(W, N, K, act_amax, alpha, dev8, out);
+    }
     if (!W || !act_amax || !out) return PRQ_ERR_INVALID_ARG;
     if (n_experts < 1 || n_experts > kMaxExperts || N < 1 || K < kBlock) return PRQ_ERR_INVALID_ARG;
     if (gated && (n_experts != 1 || N % 64)) return PRQ_ERR_INVALID_ARG;   // whole (gate, up) groups of 32 + 32 rows
@@ -493,6 +522,68 @@ static prq_status create_handle(const uint16_t* W, bool w_on_device, prq_stream_
     return PRQ_OK;
 }
 
+// Second format: host preparation, scale bytes in [128-element stage][128-row group][512], one upload.
+static prq_status create_handle_fp8(const uint16_t* W, int N, int K, const float* act_amax, float alpha, int dev, prq_weights** out) {
+    prq_weights* w = new (std::nothrow) prq_weights;
+    if (!w) return PRQ_ERR_OOM;
+    w->n_experts = 1; w->N = N; w->K = K; w->k_tail = 0; w->alpha = alpha;
+    w->plan = StagePlan(K, 0);
+    w->w_groups = (N + kGroupRows - 1) / kGroupRows;
+    w->device = dev;
+    w->format = PRQ_FMT_MXFP8;
+    try {
+        prq_status st = prepare_layer_fp8(W, N, K, act_amax, alpha, w->h_s, w->h_inv_s, w->h_codes, w->h_scales);
+        if (st != PRQ_OK) { delete w; return st; }
+        w->h_perm.resize(K);
+        for (int j = 0; j < K; ++j) w->h_perm[j] = j;
+        w->h_col_err.assign(K, 0.0);
+        const int S8 = (K + 127) / 128, nblk = K / kBlock;
+        w->d_sf_bytes = (static_cast<size_t>(S8) * w->w_groups + 4) * 512;
+        std::vector<uint8_t> sf(w->d_sf_bytes, 0);
+        for (int n = 0; n < N; ++n)
+            for (int b = 0; b < nblk; ++b)
+                sf[(static_cast<size_t>(b / 4) * w->w_groups + n / kGroupRows) * 512 + sf_offset_in_group(n % kGroupRows, b % 4)] =
+                    w->h_scales[static_cast<size_t>(n) * nblk + b];
+        w->d_codes_bytes = w->h_codes.size() + 256;
+        if (cudaMalloc(&w->d_codes, w->d_codes_bytes) != cudaSuccess || cudaMalloc(&w->d_sf, w->d_sf_bytes) != cudaSuccess ||
+            cudaMalloc(&w->d_inv_s, sizeof(float) * K) != cudaSuccess) {
+            cudaGetLastError();
+            prq_weights_free(w);
+            return PRQ_ERR_OOM;
+        }
+        bool ok = cudaMemcpy(w->d_codes, w->h_codes.data(), w->h_codes.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(w->d_sf, sf.data(), sf.size(), cudaMemcpyHostToDevice) == cudaSuccess;
+        ok = ok && cudaMemcpy(w->d_inv_s, w->h_inv_s.data(), sizeof(float) * K, cudaMemcpyHostToDevice) == cudaSuccess;
+        if (!ok || make_code_map(&w->tm_w_fp8, w->d_codes, static_cast<uint64_t>(K), N, 128) != PRQ_OK) {
+            prq_weights_free(w);
+            return PRQ_ERR_CUDA;
+        }
+        w->maps_ready = true;
+    } catch (const std::bad_alloc&) {
+        prq_weights_free(w);
+        return PRQ_ERR_OOM;
+    }
+    *out = w;
+    return PRQ_OK;
+}
+
+prq_status prq_weights_format(const prq_weights* w, int* format) {
+    if (!w || !format) return PRQ_ERR_INVALID_ARG;
+    *format = w->format;
+    return PRQ_OK;
+}
+
+size_t prq_act_bytes_for(const prq_weights* w, int M, prq_buf which) {
+    if (!w || M < 0 || w->n_experts != 1) return 0;
+    if (w->format == PRQ_FMT_MXFP4) return prq_act_bytes(M, w->K, w->k_tail, 1, which);
+    switch (which) {
+        case PRQ_BUF_CODES: return static_cast<size_t>(M) * w->K;
+        case PRQ_BUF_SCALES_ROW: return static_cast<size_t>(M) * w->K / kBlock;
+        case PRQ_BUF_SCALES_SF: return static_cast<size_t>((w->K + 127) / 128) * std::max(dense_groups(M), 1) * 512;
+    }
+    return 0;
+}
+
 prq_status prq_prepare_weights_search(const uint16_t* W, int N, int K, const uint16_t* Zcal, int T, const float* alphas,
                                       int n_alphas, int k_tail, prq_weights** out, float* alpha_star, double* nrmse) {
     if (!W || !Zcal || !alphas || !out || !alpha_star || T < 1 || n_alphas < 1) return PRQ_ERR_INVALID_ARG;
@@ -587,9 +678,29 @@ prq_status prq_prepare_weights_host(const uint16_t* W, int N, int K, const float
 prq_status prq_prepare_weights_host_opts(const uint16_t* W, int N, int K, const float* act_amax, float alpha,
                                          int k_tail, const prq_prep_opts* opts, uint8_t* codes, uint8_t* scales,
                                          int32_t* perm, float* s_out, float* inv_s_out, double* col_err) {
-    if (opts && opts->struct_size < sizeof(prq_prep_opts)) return PRQ_ERR_INVALID_ARG;
-    const bool scale_search = opts && opts->weight_scale_search != 0;
+    const PrepOptions po = read_opts(opts);
+    if (!po.valid) return PRQ_ERR_INVALID_ARG;
+    const bool scale_search = po.scale_search;
     if (!W || !act_amax || !codes || !scales || !perm) return PRQ_ERR_INVALID_ARG;
+    if (po.format == PRQ_FMT_MXFP8) {
+        // second format: codes N x K bytes, scales N x K/32, identity permutation, no ranking
+        if (N < 1 || K < kBlock || K % kBlock || k_tail != 0 || scale_search || !std::isfinite(alpha)) return PRQ_ERR_INVALID_ARG;
+        try {
+            std::vector<float> s8, inv8;
+            std::vector<uint8_t> c8, sc8;
+            prq_status st8 = prepare_layer_fp8(W, N, K, act_amax, alpha, s8, inv8, c8, sc8);
+            if (st8 != PRQ_OK) return st8;
+            std::memcpy(codes, c8.data(), c8.size());
+            std::memcpy(scales, sc8.data(), sc8.size());
+            for (int j = 0; j < K; ++j) perm[j] = j;
+            if (s_out) std::memcpy(s_out, s8.data(), sizeof(float) * K);
+            if (inv_s_out) std::memcpy(inv_s_out, inv8.data(), sizeof(float) * K);
+            if (col_err) std::fill(col_err, col_err + K, 0.0);
+        } catch (const std::bad_alloc&) {
+            return PRQ_ERR_OOM;
+        }
+        return PRQ_OK;
+    }
     if (N < 1 || K < kBlock || K % kBlock || k_tail % kBlock || k_tail < 0 || k_tail > K) return PRQ_ERR_INVALID_ARG;
     if (!std::isfinite(alpha)) return PRQ_ERR_INVALID_ARG;
     PrepResult r;
@@ -609,7 +720,7 @@ prq_status prq_prepare_weights_host_opts(const uint16_t* W, int N, int K, const 
 }
 
 prq_status prq_weights_clone(const prq_weights* w, prq_weights** out) {
-    if (!w || !out) return PRQ_ERR_INVALID_ARG;
+    if (!w || !out || w->format != PRQ_FMT_MXFP4) return PRQ_ERR_INVALID_ARG;
     prq_weights* c = new (std::nothrow) prq_weights;
     if (!c) return PRQ_ERR_OOM;
     int cur = 0;
@@ -711,7 +822,7 @@ prq_status prq_weights_get(const prq_weights* w, int expert, prq_field which, vo
     const void* src = nullptr;
     size_t bytes = 0;
     switch (which) {
-        case PRQ_FIELD_CODES: bytes = N * Ka / 2; src = &w->h_codes[e * bytes]; break;
+        case PRQ_FIELD_CODES: bytes = w->format == PRQ_FMT_MXFP8 ? N * K : N * Ka / 2; src = &w->h_codes[e * bytes]; break;
         case PRQ_FIELD_SCALES: bytes = N * Ka / kBlock; src = &w->h_scales[e * bytes]; break;
         case PRQ_FIELD_PERM: bytes = K * sizeof(int32_t); src = &w->h_perm[e * K]; break;
         case PRQ_FIELD_TOPK: bytes = w->k_tail * sizeof(int32_t); src = w->h_perm.data() + e * K + (K - w->k_tail); break;
@@ -746,6 +857,16 @@ prq_status prq_quantize_act(const prq_weights* w, prq_act_mode mode, const void*
     if (mode != PRQ_ACT_IDENTITY && mode != PRQ_ACT_SCALE_PERM) return PRQ_ERR_INVALID_ARG;
     if (M == 0) return PRQ_OK;
     if (!x || !codes || !scales_sf || ldx < w->K) return PRQ_ERR_INVALID_ARG;
+    if (w->format == PRQ_FMT_MXFP8) {
+        if (expert_offsets) return PRQ_ERR_INVALID_ARG;
+        if (!aligned16(x) || !aligned16(codes) || !aligned16(scales_sf) || ldx % 8) return PRQ_ERR_ALIGNMENT;
+        if (!handle_device_is_current(w)) return PRQ_ERR_INVALID_ARG;
+        cudaError_t e8 = launch_quant_act_fp8(static_cast<const uint16_t*>(x), M, ldx, w->K, mode == PRQ_ACT_SCALE_PERM ? w->d_inv_s : nullptr,
+                                              static_cast<uint8_t*>(codes), static_cast<uint8_t*>(scales_row),
+                                              static_cast<uint8_t*>(scales_sf), static_cast<cudaStream_t>(stream));
+        g_launches.fetch_add(1);
+        return e8 == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+    }
     // stacked experts need their row boundaries; a single layer may be given a two-entry offsets array too
     // (the grouped layout with one group), as prq_linear_grouped accepts it
     if (w->n_experts > 1 && expert_offsets == nullptr) return PRQ_ERR_INVALID_ARG;
@@ -773,6 +894,7 @@ prq_status prq_quantize_act_multi(int n, const prq_weights* const* ws, prq_act_m
     if (mode != PRQ_ACT_IDENTITY && mode != PRQ_ACT_SCALE_PERM) return PRQ_ERR_INVALID_ARG;
     for (int i = 0; i < n; ++i) {
         if (!ws[i] || ws[i]->n_experts != 1 || ws[i]->K != ws[0]->K || ws[i]->device != ws[0]->device) return PRQ_ERR_INVALID_ARG;
+        if (ws[i]->format != PRQ_FMT_MXFP4) return PRQ_ERR_INVALID_ARG;
         if (M > 0 && (!codes[i] || !scales_sf[i])) return PRQ_ERR_INVALID_ARG;
     }
     if (M == 0) return PRQ_OK;
@@ -798,7 +920,7 @@ prq_status prq_quantize_act_multi(int n, const prq_weights* const* ws, prq_act_m
 
 size_t prq_linear_workspace_bytes(const prq_weights* w, int M) {
     if (!w || M < 0) return 0;
-    if (M > 128) {
+    if (M > 128 && w->format == PRQ_FMT_MXFP4) {
         // stream-K prefill: one flag per 128 x 256 tile, one fp32 partial tile per CTA (at most one CTA per SM)
         DeviceInfo* di;
         if (device_info(w->device, &di) != PRQ_OK) return 0;
@@ -833,6 +955,20 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
     p.M = M; p.N = w->N; p.K = w->K; p.k_tail = w->k_tail;
     p.n_experts = 1;
     p.act_groups = dense_groups(M);
+    if (w->format == PRQ_FMT_MXFP8) {
+        // second format: the tile-per-CTA kernel (128 output features x 128 tokens) over the layer as one expert
+        p.w_groups = w->w_groups;
+        p.act_sf = static_cast<const uint8_t*>(scales_sf);
+        p.w_sf = w->d_sf;
+        p.y = y; p.ldy = ldy; p.y_bf16 = y_dtype == PRQ_BF16;
+        p.status = di->status_ptr;
+        CUtensorMap tm_act8;
+        st = make_code_map(&tm_act8, codes, static_cast<uint64_t>(w->K), M, 128);
+        if (st != PRQ_OK) return st;
+        cudaError_t e8 = launch_gemm_fp8(tm_act8, w->tm_w_fp8, p, di->num_sms, static_cast<cudaStream_t>(stream));
+        g_launches.fetch_add(1);
+        return e8 == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
+    }
     p.w_groups = w->w_groups;
     p.act_sf = static_cast<const uint8_t*>(scales_sf);
     p.w_sf = w->d_sf;
@@ -915,7 +1051,7 @@ prq_status prq_linear_multi(int n, const prq_weights* const* ws, const void* con
         if (M == 0) continue;
         prq_status st = check_linear_common(ws[i], codes[i], scales_sf[i], y[i], ldy[i], y_dtype);
         if (st != PRQ_OK) return st;
-        if (ws[i]->n_experts != 1 || !ws[i]->maps_ready) return PRQ_ERR_INVALID_ARG;
+        if (ws[i]->n_experts != 1 || !ws[i]->maps_ready || ws[i]->format != PRQ_FMT_MXFP4) return PRQ_ERR_INVALID_ARG;
         // one stage plan and one cluster size for the whole launch
         if (ws[i]->K != ws[0]->K || ws[i]->k_tail != ws[0]->k_tail || ws[i]->device != ws[0]->device) return PRQ_ERR_INVALID_ARG;
     }
@@ -957,6 +1093,7 @@ prq_status prq_linear_gated(const prq_weights* w, const void* codes, const void*
                             void* out_codes, void* out_scales_row, void* out_scales_sf, void* h_check, prq_stream_t stream) {
     if (!w || !wd || M < 0) return PRQ_ERR_INVALID_ARG;
     if (!w->gated || !w->maps_ready || w->n_experts != 1 || wd->n_experts != 1 || w->device != wd->device) return PRQ_ERR_INVALID_ARG;
+    if (w->format != PRQ_FMT_MXFP4 || wd->format != PRQ_FMT_MXFP4) return PRQ_ERR_INVALID_ARG;
     const int C = wd->K, kd = wd->k_tail;
     if (w->N != 2 * C || C % kStageK || kd % kStageK) return PRQ_ERR_INVALID_ARG;
     if (M == 0) return PRQ_OK;
@@ -1001,7 +1138,8 @@ prq_status prq_linear_gated(const prq_weights* w, const void* codes, const void*
 
 prq_status prq_linear_fused(const prq_weights* w, prq_act_mode mode, const void* x, int M, int ldx, void* y, int ldy,
                             prq_dtype y_dtype, prq_stream_t stream) {
-    if (!w || M < 0 || M > PRQ_FUSED_MAX_M || mode != PRQ_ACT_IDENTITY || w->n_experts != 1 || !w->maps_ready)
+    if (!w || M < 0 || M > PRQ_FUSED_MAX_M || mode != PRQ_ACT_IDENTITY || w->n_experts != 1 || !w->maps_ready ||
+        w->format != PRQ_FMT_MXFP4)
         return PRQ_ERR_INVALID_ARG;
     if (M == 0) return PRQ_OK;
     if (!x || !y || ldx < w->K || ldy < w->N) return PRQ_ERR_INVALID_ARG;
@@ -1032,7 +1170,7 @@ prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const voi
     if (w && M_total == 0) return PRQ_OK;
     prq_status st = check_linear_common(w, codes, scales_sf, y, ldy, y_dtype);
     if (st != PRQ_OK) return st;
-    if (M_total < 0 || !expert_offsets) return PRQ_ERR_INVALID_ARG;
+    if (M_total < 0 || !expert_offsets || w->format != PRQ_FMT_MXFP4) return PRQ_ERR_INVALID_ARG;
     if (!handle_device_is_current(w)) return PRQ_ERR_INVALID_ARG;
     DeviceInfo* di;
     st = device_info(w->device, &di);
@@ -1081,13 +1219,13 @@ HostFwdLayout host_fwd_layout(const prq_weights* w, int M) {
 }  // namespace
 
 size_t prq_forward_host_scratch_bytes(const prq_weights* w, int M) {
-    if (!w || M < 0 || w->n_experts != 1) return 0;
+    if (!w || M < 0 || w->n_experts != 1 || w->format != PRQ_FMT_MXFP4) return 0;
     return host_fwd_layout(w, M).total;
 }
 
 prq_status prq_forward_host(const prq_weights* w, prq_act_mode mode, const uint16_t* x_host, int M, void* y_host,
                             prq_dtype y_dtype, void* dev_scratch, size_t scratch_bytes, prq_stream_t stream) {
-    if (!w || w->n_experts != 1 || M < 0) return PRQ_ERR_INVALID_ARG;
+    if (!w || w->n_experts != 1 || M < 0 || w->format != PRQ_FMT_MXFP4) return PRQ_ERR_INVALID_ARG;
     if (M == 0) return PRQ_OK;
     if (!x_host || !y_host || !dev_scratch) return PRQ_ERR_INVALID_ARG;
     if (y_dtype != PRQ_F32 && y_dtype != PRQ_BF16) return PRQ_ERR_INVALID_ARG;

@@ -47,14 +47,20 @@ constexpr uint32_t kHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 constexpr uint32_t kHiPlain = (128u >> 4) | (1u << 14);
 __device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo) { return (static_cast<uint64_t>(hi) << 32) | lo; }
 
+// kFp8: the second format (MXFP8: one byte per element, E4M3).  A stage is still one 128-byte swizzled row per operand
+// row, which then holds 128 elements = 4 blocks = ONE scale atom per 128-row group instead of two, and a K = 32 step
+// per MMA (kind::mxf8f6f4) that takes one scale byte per row: the scale-id fields walk the four bytes of the word.
+template <bool kFp8>
 struct Cfg {
+    static constexpr int kStageElems = kFp8 ? 128 : kStageK;
+    static constexpr int kSfBytes = kFp8 ? 512 : kSfGroupBytes;    // scale bytes per (stage, 128-row group)
     // eight epilogue warps, two per tensor-memory lane quarter taking alternate 16-token chunks: with
     // K + k = 832 a tile is only 3.25 stages, and the epilogue is what the main loop waits for
     static constexpr int kEpiWarps = 8;
     static constexpr int kThreads = 32 * (kMainWarps + kEpiWarps);
     static constexpr int kQTileBytes = BN * 128;
-    static constexpr int kSfpBytes = kSfGroupBytes;
-    static constexpr int kSfqBytes = kSfGroupBytes;
+    static constexpr int kSfpBytes = kSfBytes;
+    static constexpr int kSfqBytes = kSfBytes;
     static constexpr int kStageBytes = kPTileBytes + kQTileBytes + kSfpBytes + kSfqBytes;
     static constexpr int kStages = cmin(8, (232448 - 1024 - 16384 - 2048) / kStageBytes);
     // tensor memory columns: two accumulators, then scale words (2 atoms x 4 columns per operand)
@@ -82,15 +88,15 @@ struct Unit {
 struct GroupPos { int e, mt, ni; };
 
 __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_start, const int* row_start, int S,
-                                           const GroupPos& g) {
+                                           const GroupPos& g, int sf_bytes) {
     Unit t;
     const int e = g.e, mt = g.mt, ni = g.ni;
     t.p_row = e * p.N + ni * 128;
     t.q_row = row_start[e] + (mt - tile_start[e]) * 128;
-    t.sfp = p.w_sf + (static_cast<size_t>(e) * S * p.w_groups + ni) * kSfGroupBytes;
-    t.sfp_stride = static_cast<size_t>(p.w_groups) * kSfGroupBytes;
-    t.sfq = p.act_sf + static_cast<size_t>(mt) * kSfGroupBytes;
-    t.sfq_stride = static_cast<size_t>(p.act_groups) * kSfGroupBytes;
+    t.sfp = p.w_sf + (static_cast<size_t>(e) * S * p.w_groups + ni) * sf_bytes;
+    t.sfp_stride = static_cast<size_t>(p.w_groups) * sf_bytes;
+    t.sfq = p.act_sf + static_cast<size_t>(mt) * sf_bytes;
+    t.sfq_stride = static_cast<size_t>(p.act_groups) * sf_bytes;
     t.row0 = t.q_row; t.row_end = min(row_start[e + 1], t.q_row + 128);
     t.n0 = ni * 128;
     return t;
@@ -104,10 +110,10 @@ struct UnitIter {
     const GemmParams& p;
     const int* tile_start;
     const int* row_start;
-    int S, u, u_end;
+    int S, u, u_end, sf_bytes;
     GroupPos g;
-    __device__ __forceinline__ UnitIter(const GemmParams& p_, const int* ts, const int* rs, int S_, int n_units)
-        : p(p_), tile_start(ts), row_start(rs), S(S_), g{0, 0, 0} {
+    __device__ __forceinline__ UnitIter(const GemmParams& p_, const int* ts, const int* rs, int S_, int n_units, int sf_bytes_)
+        : p(p_), tile_start(ts), row_start(rs), S(S_), sf_bytes(sf_bytes_), g{0, 0, 0} {
         const int per = (n_units + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
         u = min(n_units, static_cast<int>(blockIdx.x) * per);
         u_end = min(n_units, u + per);
@@ -123,7 +129,7 @@ struct UnitIter {
         }
     }
     __device__ __forceinline__ bool valid() const { return u < u_end; }
-    __device__ __forceinline__ Unit get() const { return make_unit(p, tile_start, row_start, S, g); }
+    __device__ __forceinline__ Unit get() const { return make_unit(p, tile_start, row_start, S, g, sf_bytes); }
     __device__ __forceinline__ void next() {
         if (++u < u_end) {
             if (++g.mt == tile_start[p.n_experts]) { g.mt = 0; g.e = 0; ++g.ni; }
@@ -132,10 +138,11 @@ struct UnitIter {
     }
 };
 
-__global__ void __launch_bounds__(Cfg::kThreads, 1)
+template <bool kFp8>
+__global__ void __launch_bounds__(Cfg<kFp8>::kThreads, 1)
 gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
                     const GemmParams p) {
-    using C = Cfg;
+    using C = Cfg<kFp8>;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[C::kStages], bar_empty[C::kStages], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_slot;
@@ -148,8 +155,9 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const StagePlan plan(p.K, p.k_tail);
-    const int S = plan.S, S1 = plan.S1;
+    // reduction stages: the K main columns, then the k tail columns (MXFP4 only; the second format has no tail)
+    const int S1 = (p.K + C::kStageElems - 1) / C::kStageElems;
+    const int S = S1 + (kFp8 ? 0 : (p.k_tail + C::kStageElems - 1) / C::kStageElems);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < C::kStages; ++i) { mbar_init(smem_u32(&bar_full[i]), 1); mbar_init(smem_u32(&bar_empty[i]), 1); }
@@ -161,8 +169,10 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     }
     // the expert row ranges are kept in shared memory (up to kRowCache experts): every role looks
     // them up once per tile, and a dependent global load there sits on the producer's critical path
+    // (no offsets array: a dense layer, i.e. one expert that owns all M rows)
     if (p.n_experts <= kRowCache)
-        for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x) row_cache[e] = p.expert_offsets[e];
+        for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x)
+            row_cache[e] = p.expert_offsets ? p.expert_offsets[e] : (e == 0 ? 0 : p.M);
     __syncthreads();
     if (threadIdx.x == 64) {
         int acc = 0;
@@ -193,7 +203,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         int it = 0, st = 0;
         uint32_t ph = 0;
         bool ok = true;
-        for (UnitIter ui(p, tile_start, row_start, S, n_units); ui.valid() && ok; ui.next()) {
+        for (UnitIter ui(p, tile_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next()) {
             const Unit t = ui.get();
             for (int s = 0; s < S; ++s, ++it) {
                 if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
@@ -202,6 +212,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                     const uint32_t full = smem_u32(&bar_full[st]);
                     mbar_arrive_expect_tx(full, C::kTxBytes);
                     // byte column of each operand in this stage
+                    // (a stage is 128 bytes of either format's row; residual stages exist for MXFP4 only)
                     const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
                     const int xa = s < S1 ? s * 128 : (p.K - p.k_tail) / 2 + (s - S1) * 128;
                     const uint32_t sb = smem_base + st * C::kStageBytes;
@@ -234,7 +245,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         const uint32_t sfp_t = tmem_base + C::kSfpCol;
         const uint32_t sfq_t = tmem_base + C::kSfqCol;
         const uint32_t lo_base = ((smem_base & 0x3FFFF) >> 4) | (1u << 16);
-        for (UnitIter ui(p, tile_start, row_start, S, n_units); ui.valid() && ok; ui.next(), ++acc_it) {
+        for (UnitIter ui(p, tile_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next(), ++acc_it) {
             const int buf = acc_it % C::kAcc;
             const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
             if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1, abort_flag)) { ok = false; break; }
@@ -244,8 +255,8 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             for (int s = 0; s < S; ++s, ++it) {
                 if (!ready && !mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
                 if (trace && lane == 0 && it < 64) trace[64 + it] = clock64();
-                const int rem = s < S1 ? p.K - s * kStageK : p.k_tail - (s - S1) * kStageK;
-                const int ksteps = min(4, (rem + 63) / 64);
+                const int rem = s < S1 ? p.K - s * C::kStageElems : p.k_tail - (s - S1) * C::kStageElems;
+                const int ksteps = min(4, (rem + C::kStageElems / 4 - 1) / (C::kStageElems / 4));
                 // probe the next slot now: the probe's latency hides behind this stage's tcgen05 instructions
                 const int nst = st + 1 == C::kStages ? 0 : st + 1;
                 const uint32_t nph = nst == 0 ? ph ^ 1 : ph;
@@ -257,21 +268,37 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                     const uint32_t plo = lo_base + st * (C::kStageBytes >> 4);
                     const uint32_t qlo = plo + (kPTileBytes >> 4);
                     const uint32_t sfp_lo = qlo + (C::kQTileBytes >> 4), sfq_lo = sfp_lo + (C::kSfpBytes >> 4);
+                    if constexpr (kFp8) {
+                        // one atom per operand covers the stage's four blocks; step j takes byte j of the scale word
+                        tc_copy_sf_atom(sfp_t, desc64(kHiPlain, sfp_lo));
+                        tc_copy_sf_atom(sfq_t, desc64(kHiPlain, sfq_lo));
+                        // E4M3 x E4M3 (format 0), E8M0 scales, both operands K-major, N = BN, M = 128
+                        constexpr uint32_t idesc = ((BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
 #pragma unroll
-                    for (int ka = 0; ka < 2; ++ka) {
-                        if (ka * 2 < ksteps) {
-                            tc_copy_sf_atom(sfp_t + ka * 4, desc64(kHiPlain, sfp_lo + ka * (512 >> 4)));
-                            tc_copy_sf_atom(sfq_t + ka * 4, desc64(kHiPlain, sfq_lo + ka * (512 >> 4)));
+                        for (int j = 0; j < 4; ++j) {
+                            if (j < ksteps) {
+                                tc_mma_mxf8(d_tmem, desc64(kHiSw128, plo + 2 * j), desc64(kHiSw128, qlo + 2 * j),
+                                            idesc | (static_cast<uint32_t>(j) << 4) | (static_cast<uint32_t>(j) << 29), sfp_t, sfq_t, accumulate);
+                                accumulate = 1;
+                            }
                         }
-                    }
-                    constexpr uint32_t idesc0 = (1u << 7) | (1u << 10) | ((BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
-                    constexpr uint32_t idesc2 = idesc0 | (2u << 4) | (2u << 29);
+                    } else {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        if (j < ksteps) {
-                            tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 2 * j), desc64(kHiSw128, qlo + 2 * j),
-                                        (j & 1) ? idesc2 : idesc0, sfp_t + (j >> 1) * 4, sfq_t + (j >> 1) * 4, accumulate);
-                            accumulate = 1;
+                        for (int ka = 0; ka < 2; ++ka) {
+                            if (ka * 2 < ksteps) {
+                                tc_copy_sf_atom(sfp_t + ka * 4, desc64(kHiPlain, sfp_lo + ka * (512 >> 4)));
+                                tc_copy_sf_atom(sfq_t + ka * 4, desc64(kHiPlain, sfq_lo + ka * (512 >> 4)));
+                            }
+                        }
+                        constexpr uint32_t idesc0 = (1u << 7) | (1u << 10) | ((BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+                        constexpr uint32_t idesc2 = idesc0 | (2u << 4) | (2u << 29);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            if (j < ksteps) {
+                                tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 2 * j), desc64(kHiSw128, qlo + 2 * j),
+                                            (j & 1) ? idesc2 : idesc0, sfp_t + (j >> 1) * 4, sfq_t + (j >> 1) * 4, accumulate);
+                                accumulate = 1;
+                            }
                         }
                     }
                     tc_commit(smem_u32(&bar_empty[st]));
@@ -290,7 +317,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         const int et = q * 32 + lane;           // 0..127: accumulator row
         int acc_it = 0;
         bool ok = true;
-        for (UnitIter ui(p, tile_start, row_start, S, n_units); ui.valid() && ok; ui.next(), ++acc_it) {
+        for (UnitIter ui(p, tile_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next(), ++acc_it) {
             const Unit t = ui.get();
             const int buf = acc_it % C::kAcc;
             const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
@@ -374,20 +401,32 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     if (threadIdx.x == 0 && abort_flag_s) atomicExch(p.status, static_cast<int>(PRQ_ERR_TIMEOUT));
 }
 
+
+template <bool kFp8>
+cudaError_t launch_grouped_impl(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
+                                cudaStream_t stream) {
+    using C = Cfg<kFp8>;
+    constexpr int smem = C::kStages * C::kStageBytes + 1024 + C::kEpiWarps * 2048;  // + store staging
+    static bool configured = false;  // the attribute is per function, setting it twice is harmless
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_grouped_kernel<kFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    gemm_grouped_kernel<kFp8><<<grid, C::kThreads, smem, stream>>>(tm_act, tm_w, p);
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 cudaError_t launch_gemm_grouped(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
                                 cudaStream_t stream) {
-    using C = Cfg;
-    constexpr int smem = C::kStages * C::kStageBytes + 1024 + C::kEpiWarps * 2048;  // + store staging
-    static bool configured = false;  // the attribute is per function, setting it twice is harmless
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_grouped_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
-    gemm_grouped_kernel<<<grid, C::kThreads, smem, stream>>>(tm_act, tm_w, p);
-    return cudaGetLastError();
+    return launch_grouped_impl<false>(tm_act, tm_w, p, grid, stream);
+}
+
+cudaError_t launch_gemm_fp8(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
+                            cudaStream_t stream) {
+    return launch_grouped_impl<true>(tm_act, tm_w, p, grid, stream);
 }
 
 }  // namespace prq

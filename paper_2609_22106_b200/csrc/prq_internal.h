@@ -68,6 +68,10 @@ void rank_and_permute(const std::vector<double>& col_err, int K, int k_tail, std
 // rounded once to bf16); with duplicate_tail the last k_tail rows are repeated.  Host buffers.
 prq_status fold_producer(const int32_t* perm, const float* inv_s, int C, int k_tail, const uint16_t* W_up,
                          const uint16_t* W_gate, int H, bool duplicate_tail, uint16_t* out_up, uint16_t* out_gate);
+// Offline half of a layer in the second format (MXFP8) for one alpha, on the host: scales as above, W0 = fl32(W * s),
+// E4M3 codes (N x K bytes) and E8M0 scale bytes (N x K/32) by rows.  No permutation, no tail.
+prq_status prepare_layer_fp8(const uint16_t* W, int N, int K, const float* amax, float alpha, std::vector<float>& s,
+                             std::vector<float>& inv_s, std::vector<uint8_t>& codes, std::vector<uint8_t>& scales);
 // Gate and up projection rows interleaved in groups of 32 (rows 64 b .. 64 b + 31 = gate rows 32 b .., rows 64 b + 32 ..
 // 64 b + 63 = up rows 32 b ..): the layout prq_linear_gated expects.  Host buffers, C % 32 == 0.
 void stack_gate_up(const uint16_t* W_gate, const uint16_t* W_up, int C, int H, uint16_t* out);
@@ -100,6 +104,11 @@ struct prq_weights {
     uint8_t* d_sf_alt[4] = {nullptr, nullptr, nullptr, nullptr};
     int w_groups_alt[4] = {0, 0, 0, 0};
     bool gated = false;
+    // Second format (prq_prep_opts::format = PRQ_FMT_MXFP8): d_codes holds N x K bytes of E4M3 codes, d_sf the scale
+    // bytes as [128-element stage][128-row group][512]; k_tail is 0, perm the identity; none of the MXFP4 tilings exist.
+    int format = 0;
+    CUtensorMap tm_w_fp8;
+    float* d_inv_s = nullptr;        // K: the activation side's factors (original = permuted order)
     // tensor maps of the weight side, encoded once (dense layers; a handle is immutable afterwards):
     // codes with 128-row boxes (decode kernel), codes with half-tile boxes and the scale bytes of the
     // 224-row [0], 240-row [1], 288-row [2] and 192-row [3] tilings (CTA-pair prefill kernel)

@@ -83,6 +83,17 @@ cudaError_t launch_gemm_grouped(const CUtensorMap& tm_act, const CUtensorMap& tm
                                 cudaStream_t stream);
 
 
+// The same kernel for the second format (MXFP8), dense layers of any M: `p.expert_offsets` null, `p.n_experts` 1;
+// scale bytes in 512-byte groups per (128-element stage, 128-row group); code maps over K-byte rows.
+cudaError_t launch_gemm_fp8(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
+                            cudaStream_t stream);
+
+// Activation quantiser of the second format: x (M x K bf16, row stride ldx), optionally times inv_s[j] (null: identity),
+// to E4M3 codes (M x K bytes), row-major scale bytes (or null) and tile-ordered scale bytes
+// [stage = 128 columns][128-row group][512].
+cudaError_t launch_quant_act_fp8(const uint16_t* x, int M, int ldx, int K, const float* inv_s, uint8_t* codes,
+                                 uint8_t* scales_row, uint8_t* scales_sf, cudaStream_t stream);
+
 // Decode kernel (M <= 128): cluster split-K with a distributed-shared-memory reduction.
 struct DecodeParams {
     int M, N, K, k_tail;

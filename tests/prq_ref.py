@@ -48,3 +48,16 @@ def unpack(codes):
 def tolerance(y_ref):
     """Acceptance bound of the GEMM: max |y - y_ref| <= 2e-3 (||y_ref||_inf + 1)."""
     return 2e-3 * (float(np.abs(y_ref).max()) + 1.0)
+
+
+def expected_sf_fp8(scales, K, groups=None):
+    """Tile-ordered scale buffer of the second format (MXFP8): [128-element stage][128-row group][512 bytes], the byte of
+    (row r of a group, block b of a stage) at (r % 32) * 16 + (r // 32) * 4 + b."""
+    M = scales.shape[0]
+    S = (K + 127) // 128
+    groups = (M + GROUP - 1) // GROUP if groups is None else groups
+    out = np.zeros((S, groups, 512), np.uint8)
+    r = np.arange(M)
+    for b in range(scales.shape[1]):
+        out[b // 4, r // GROUP, ((r % GROUP) % 32) * 16 + ((r % GROUP) // 32) * 4 + b % 4] = scales[:, b]
+    return out.reshape(-1)

@@ -187,3 +187,30 @@ def test_fold_producer_bit_exact(prq, oracle):
     bad[3] = C
     with pytest.raises(prq.PrqError):
         prq.fold_producer(bad, inv_s, k, Wu)
+
+
+def test_mxfp8_host_prep_is_bit_exact(prq, oracle):
+    """Second format: the library's host preparation (no device involved) against the oracle, code for code."""
+    for seed, (N, K), alpha in ((1, (40, 96), 0.5), (2, (17, 256), 0.0), (3, (64, 64), 0.75), (4, (8, 32), 0.3)):
+        L = synth.layer(60 + seed, N, K, 4, T_cal=32)
+        amax = oracle.channel_amax(L["zcal"])
+        amax[0] = 0.0                                         # a dead channel takes the floor
+        got = prq.prepare_weights_host(L["W"], amax, alpha, 0, fmt=prq.FMT_MXFP8)
+        o = oracle.fp8_prepare(L["W"], amax, float(np.float32(alpha)))
+        assert np.array_equal(got["s"], o["s"]) and np.array_equal(got["inv_s"], o["inv_s"])
+        assert np.array_equal(got["scales"], o["wscales"])
+        assert np.array_equal(got["codes"], o["wcodes"])
+        assert np.array_equal(got["perm"], np.arange(K))
+    # blocks on the format's decision boundaries (ties, saturation band, subnormal steps), unit scales
+    rows = []
+    for vals in ([448, 1, .5, -3, 2 ** -9, 296], [256, 17, 19, 272, 304], [500, 464, 462, -510], [512, 3, 1],
+                 [256, 7 * 2 ** -9, 7.5 * 2 ** -9, -0.5 * 2 ** -9], [2.0 ** -20, 2.0 ** -30, -2.0 ** -29]):
+        b = np.zeros(32, np.float32); b[: len(vals)] = vals; rows.append(b)
+    Wb = synth.f32_to_bf16(np.stack(rows))
+    assert np.array_equal(synth.bf16_to_f32(Wb), np.stack(rows))
+    got = prq.prepare_weights_host(Wb, np.ones(32, np.float32), 0.0, 0, fmt=prq.FMT_MXFP8)
+    o = oracle.fp8_prepare(Wb, np.ones(32, np.float32), 0.0)
+    assert np.array_equal(got["codes"], o["wcodes"]) and np.array_equal(got["scales"], o["wscales"])
+    # the format carries no tail
+    with pytest.raises(prq.PrqError):
+        prq.prepare_weights_host(Wb, np.ones(32, np.float32), 0.0, 32, fmt=prq.FMT_MXFP8)
