@@ -275,6 +275,24 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
                 torch.matmul(lin["gate"]["x"], fw["gu"].t()); torch.matmul(lin["down"]["x"], lin["down"]["Wb"].t())
             return run
         bf16_fused = timer.run([bf16_step(lin, fw) for lin, fw in zip(layers, fused_w)], n, n_layers) / n
+    # the attention linears in the second format (MXFP8, plain W8A8), as the paper's end-to-end setting runs them
+    fp8_rows = {}
+    if M > 128:
+        for name in ("q", "k", "o"):
+            ds = []
+            for lin in layers:
+                d = lin[name]
+                w8 = prq.prepare_weights(d["Wb"].view(torch.int16).cpu().numpy().view(np.uint16), d["amax"], 0.5, 0, fmt=prq.FMT_MXFP8)
+                c8, _, s8 = prq.quantize_act(w8, d["x"], prq.ACT_SCALE_PERM)
+                ds.append(dict(w=w8, x=d["x"], codes=c8, sf=s8, y=d["y"]))
+            tq8 = timer.run([(lambda e=e: prq.quantize_act(e["w"], e["x"], prq.ACT_SCALE_PERM, out=(e["codes"], None, e["sf"]))) for e in ds], n, n_layers) / n * 1e6
+            tg8 = timer.run([(lambda e=e: prq.linear(e["w"], e["codes"], e["sf"], M, prq.BF16, out=e["y"])) for e in ds], n, n_layers) / n * 1e6
+            N8, K8 = lin[name]["N"], lin[name]["K"]
+            fl8 = 2.0 * M * N8 * K8
+            fp8_rows[name] = dict(N=N8, K=K8, quant_us=tq8, gemm_us=tg8, gemm_tflops=fl8 / tg8 / 1e6,
+                                  gemm_roofline_frac=fl8 / (pk["bf16_tflops"] * 2.0) / 1e6 / tg8)
+            for e in ds:
+                e["w"].free()
     total_flops = sum(2.0 * M * N * (K + (k if k_override is None else k_override)) for N, K, k in BLOCK_LINEARS.values())
     status = prq.last_device_status()
     for lin in layers:
@@ -284,7 +302,8 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
     if t_step_multi is not None:
         extra = dict(step_multi_launch_us=t_step_multi * 1e6, bf16_fused_qkv_gateup_us=bf16_fused * 1e6)
     extra.update(step_grouped_prep_us=t_step_grouped * 1e6, bf16_grouped_us=t_bf16_grouped * 1e6,
-                 grouped_linears=grouped_rows, step_gated_producer_us=t_step_gated * 1e6, gated_producer_gemm_us=t_gated * 1e6)
+                 grouped_linears=grouped_rows, step_gated_producer_us=t_step_gated * 1e6, gated_producer_gemm_us=t_gated * 1e6,
+                 mxfp8_attention_linears=fp8_rows)
     return dict(workload=tag, M=M, layers=n_layers, step_us=t_step * 1e6, step_tflops=total_flops / t_step / 1e12, **extra,
                 gemm_us_sum=sum(r["gemm_us"] for r in rows.values()), quant_us_sum=sum(r["quant_us"] for r in rows.values()),
                 bf16_us_sum=sum(r["bf16_matmul_us"] for r in rows.values()), device_status=status, linears=rows)
