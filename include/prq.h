@@ -126,6 +126,18 @@ typedef struct prq_prep_opts {
 prq_status prq_prepare_weights_opts(const uint16_t *W, int n_experts, int N, int K, const float *act_amax,
                                     float alpha, int k_tail, const prq_prep_opts *opts, prq_weights **out);
 
+/* Several layers that read the SAME activation (q / k / v, gate / up), prepared as ONE PRQuant layer: their weights are
+ * stacked along the output axis and go through Algorithm 1 together -- the scale s depends on the shared input only,
+ * and one permutation and one tail are chosen from the stacked matrix's column errors -- so that one activation
+ * quantisation and one product serve the whole group.  (The paper applies the method per linear; this is the same method
+ * applied to the fused projection.)  The handle is an ordinary one with N = sum of N_i: layer i's outputs are columns
+ * [sum_{j<i} N_j, + N_i) of prq_linear's y.
+ *   Ws        host array of n host pointers, layer i: N_i x K bf16 row-major
+ *   Ns        host array of n row counts        act_amax  host, K floats        opts  may be NULL
+ * Errors as prq_prepare_weights_opts; INVALID_ARG for n < 1 or a NULL entry. */
+prq_status prq_prepare_weights_stacked(const uint16_t *const *Ws, const int *Ns, int n, int K, const float *act_amax,
+                                       float alpha, int k_tail, const prq_prep_opts *opts, prq_weights **out);
+
 /* prq_prepare_weights_opts for weights that already sit in DEVICE memory (Algorithm 1 steps 3-7 and 11 with
  * the heavy steps as kernels on the current device; the K channel scales and the ranking of the K column
  * errors stay on the host).  The handle is bit-for-bit the one prq_prepare_weights_opts builds from a host

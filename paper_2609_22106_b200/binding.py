@@ -28,6 +28,7 @@ EXPORTS = [
     "prq_linear_grouped", "prq_forward_host_scratch_bytes", "prq_forward_host",
     "prq_status_string", "prq_last_device_status", "prq_kernel_launch_count", "prq_mxf4_peak_probe",
     "prq_handover_probe", "prq_stack_gate_up", "prq_linear_gated", "prq_weights_format", "prq_act_bytes_for",
+    "prq_prepare_weights_stacked",
 ]
 
 
@@ -82,6 +83,7 @@ def lib():
         L.prq_kernel_launch_count.restype = ctypes.c_ulonglong
         L.prq_mxf4_peak_probe.argtypes = [ci, ctypes.POINTER(ci), vp]
         L.prq_handover_probe.argtypes = [ci, ci, ci, ci, vp]
+        L.prq_prepare_weights_stacked.argtypes = [vp, vp, ci, ci, vp, cf, ci, vp, ctypes.POINTER(vp)]
         L.prq_weights_format.argtypes = [vp, ctypes.POINTER(ci)]
         L.prq_act_bytes_for.argtypes = [vp, ci, ci]
         L.prq_act_bytes_for.restype = cs
@@ -469,3 +471,19 @@ def linear_gated(w_gu: Weights, codes, scales_sf, M: int, w_down: Weights, row_s
     _check(lib().prq_linear_gated(w_gu.handle, _dptr(codes), _dptr(scales_sf), M, w_down.handle, _dptr(oc), _dptr(orow),
                                   _dptr(osf), _dptr(h), _stream_ptr(stream)), "prq_linear_gated")
     return oc, orow, osf, h
+
+
+def prepare_weights_stacked(Ws, act_amax: np.ndarray, alpha: float, k_tail: int, scale_search: bool = False) -> Weights:
+    """Several layers over the same activation (list of uint16 (N_i, K) arrays) prepared as one layer; layer i's outputs
+    are columns [sum N_j for j < i, + N_i) of linear()'s result."""
+    mats = [np.ascontiguousarray(W, np.uint16) for W in Ws]
+    K = mats[0].shape[1]
+    ptrs = (ctypes.c_void_p * len(mats))(*[m.ctypes.data for m in mats])
+    ns = (ctypes.c_int * len(mats))(*[m.shape[0] for m in mats])
+    amax = np.ascontiguousarray(act_amax, np.float32)
+    h = ctypes.c_void_p()
+    o = _opts(scale_search)
+    _check(lib().prq_prepare_weights_stacked(ctypes.cast(ptrs, ctypes.c_void_p), ctypes.cast(ns, ctypes.c_void_p), len(mats), K,
+                                             _np_ptr(amax), alpha, k_tail, ctypes.cast(ctypes.pointer(o), ctypes.c_void_p),
+                                             ctypes.byref(h)), "prq_prepare_weights_stacked")
+    return Weights(h)

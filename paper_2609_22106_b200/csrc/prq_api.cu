@@ -382,6 +382,28 @@ prq_status prq_prepare_weights_opts(const uint16_t* W, int n_experts, int N, int
     return create_handle(W, false, nullptr, n_experts, N, K, act_amax, alpha, k_tail, opts, out);
 }
 
+prq_status prq_prepare_weights_stacked(const uint16_t* const* Ws, const int* Ns, int n, int K, const float* act_amax, float alpha,
+                                       int k_tail, const prq_prep_opts* opts, prq_weights** out) {
+    if (!Ws || !Ns || n < 1 || K < kBlock) return PRQ_ERR_INVALID_ARG;
+    long long N = 0;
+    for (int i = 0; i < n; ++i) {
+        if (!Ws[i] || Ns[i] < 1) return PRQ_ERR_INVALID_ARG;
+        N += Ns[i];
+    }
+    if (N > 0x7fffffffll) return PRQ_ERR_INVALID_ARG;
+    try {
+        std::vector<uint16_t> W(static_cast<size_t>(N) * K);
+        size_t row = 0;
+        for (int i = 0; i < n; ++i) {
+            std::memcpy(&W[row * K], Ws[i], sizeof(uint16_t) * static_cast<size_t>(Ns[i]) * K);
+            row += Ns[i];
+        }
+        return create_handle(W.data(), false, nullptr, 1, static_cast<int>(N), K, act_amax, alpha, k_tail, opts, out);
+    } catch (const std::bad_alloc&) {
+        return PRQ_ERR_OOM;
+    }
+}
+
 prq_status prq_prepare_weights_device(const uint16_t* W_device, int n_experts, int N, int K, const float* act_amax,
                                       float alpha, int k_tail, const prq_prep_opts* opts, prq_stream_t stream,
                                       prq_weights** out) {

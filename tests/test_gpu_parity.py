@@ -692,3 +692,27 @@ def test_production_switch_state_in_a_fresh_process():
     r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
     assert "smoke ok" in r.stdout
+
+
+def test_stacked_preparation_is_the_method_on_the_concatenated_matrix(prq, oracle):
+    """prq_prepare_weights_stacked: q / k / v-like layers over one activation as one layer -- equal, field by field, to
+    the oracle's preparation of the row-concatenated weight, and its product carries every layer's outputs in its
+    column slice."""
+    K, k, M = 512, 64, 200
+    Ns = (384, 96, 160)
+    Ws = [synth.weights(80 + i, n, K) for i, n in enumerate(Ns)]
+    ch = synth.HeavyTailChannels(83, K)
+    x, xcal = ch.rows(84, M), ch.rows(85, 64)
+    amax = oracle.channel_amax(xcal)
+    w = prq.prepare_weights_stacked(Ws, amax, 0.5, k)
+    Wcat = np.concatenate(Ws)
+    assert w.N == sum(Ns)
+    o = check_prep(prq, oracle, w, Wcat, amax, 0.5, k)
+    codes, sf, oc, osc = run_quant(prq, oracle, w, o, x, prq.ACT_SCALE_PERM)
+    y, y_ref = run_linear(prq, oracle, w, o, codes, sf, oc, osc, M)
+    # a layer's slice is the product with that layer's rows of the prepared weights
+    r0 = Ns[0]
+    ca, sa = oracle.augment_act(oc, osc, k)
+    y_k = oracle.matmul(ca, sa, o["wcodes"][r0: r0 + Ns[1]], o["wscales"][r0: r0 + Ns[1]])
+    assert np.abs(y[:, r0: r0 + Ns[1]] - y_k).max() <= prq_ref.tolerance(y_k)
+    w.free()
