@@ -126,7 +126,8 @@ prq_status make_out_map(CUtensorMap* map, void* y, int M, int N, int ldy, bool b
 constexpr int kNumAlt = 4;
 // weight tile widths of the prefill kernel, each with its own scale layout; the last one only in gated-producer handles,
 // which in turn have none of the others
-constexpr int kAltTileRows[kNumAlt] = {kPrefillTileN, kPrefillTileWide, kPrefillTileOneWave, kPrefillTileGated};
+// (the one-wave tile is tiled per 144-row half: its two MMAs per step take 144 columns each)
+constexpr int kAltTileRows[kNumAlt] = {kPrefillTileN, kPrefillTileWide, kPrefillTileOneWave / 2, kPrefillTileGated};
 constexpr int kAltGated = 3;
 bool alt_wanted(bool gated, int a) { return gated ? a == kAltGated : a != kAltGated; }
 
@@ -139,11 +140,12 @@ prq_status build_weight_maps(prq_weights* w) {
     for (int v = 0; v < kNumAlt; ++v) {   // 224-, 240- and 288-row tilings, or the 192-row one
         if (!alt_wanted(w->gated, v)) continue;
         const int rows = kAltTileRows[v], gpt = (rows + kGroupRows - 1) / kGroupRows;
-        // each CTA of a pair loads half a tile; the 288-row tile as 128 + 16 rows (second map)
-        if (st == PRQ_OK) st = make_code_map(&w->tm_w_pair[v], w->d_codes, Ka / 2, w->N, rows > 256 ? 128 : rows / 2);
+        const bool one_wave = v == 2;   // a 288-row tile = two 144-row halves: boxes of 72 weight rows, four scale groups
+        // each CTA of a pair loads half a tile (the 288-row tile: a quarter, twice)
+        if (st == PRQ_OK) st = make_code_map(&w->tm_w_pair[v], w->d_codes, Ka / 2, w->N, rows / 2);
         if (st == PRQ_OK && w->d_sf_alt[v])
             st = make_sf_map(&w->tm_sfw_pair[v], w->d_sf_alt[v],
-                             static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[v] * kSfGroupBytes, 4 * gpt);
+                             static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[v] * kSfGroupBytes, 4 * gpt * (one_wave ? 2 : 1));
     }
     if (st == PRQ_OK) st = make_code_map(&w->tm_w_tail, w->d_codes, Ka / 2, w->N, 16);
     if (st == PRQ_OK) w->maps_ready = true;

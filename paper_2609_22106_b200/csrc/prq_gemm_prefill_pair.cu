@@ -61,17 +61,23 @@ constexpr int kChunkCols = 32;                    // accumulator columns per epi
 //   few percent of the tensor time, and it pads N = 2560 less (11 x 240 against 12 x 224).
 //   288: ONE accumulator, for calls whose tiles all fit one wave of pairs at this width (the host decides): no
 //   pair takes a second tile, so nothing needs a second accumulator, and no tile is split along K.  An MMA takes at
-//   most 256 columns, so a reduction step is two instructions (256 + 32 columns); each CTA loads 128 + 16 weight
-//   rows so that the accumulator's columns are the tile's weight rows in order.
+//   most 256 columns, so a reduction step is two instructions of 144 columns each (an MMA of 32 columns costs about as
+//   much as one of 64: 256 + 32 measured 9 % slower than 144 + 144 predicts); each CTA loads 72 + 72 weight rows -- rows
+//   [72 r, +72) and [144 + 72 r, +72) of the tile -- so that the accumulator's columns are the tile's weight rows in
+//   order, and the scale bytes are tiled per 144-row half (two groups each).
 template <int BN>
 struct PCfg {
     static constexpr bool kWide = BN > 256;
     static constexpr int kHalfN = BN / 2;                    // weight rows each CTA of the pair loads
     static constexpr int kQTile = kHalfN * 128;              // half weight tile bytes
-    static constexpr int kSfqGroups = (BN + 127) / 128;      // 128-row scale groups of a weight tile
+    static constexpr int kHalfGroups = kWide ? (BN / 2 + 127) / 128 : 0;                    // scale groups per 144-row half
+    static constexpr int kSfqGroups = kWide ? 2 * kHalfGroups : (BN + 127) / 128;           // 128-row scale groups of a weight tile
     static constexpr int kSfq = kSfqGroups * kSfGroupBytes;
-    static constexpr int kStageBytes = kPTile + kQTile + kSfp + kSfq;  // 33792 / 34816 / 38912
-    static constexpr int kSmemBytes = kStages * kStageBytes + 4 * kStagingPerWarp + 1024;
+    static constexpr int kStageBytes = kPTile + kQTile + kSfp + kSfq;  // 33792 / 34816 / 39936
+    // the alternating staging buffers serve epilogues that run under a main loop; the one-wave tile has only a last
+    // epilogue, which stages in the idle ring
+    static constexpr int kStagingBytes = kWide ? 0 : 4 * kStagingPerWarp;
+    static constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + 1024;
     static constexpr int kAccBufs = kWide ? 1 : 2;
     static constexpr int kSfCol = kAccBufs * BN;             // scale columns start behind the accumulator(s)
     static constexpr int kSfSetCols = 8 + 8 * kSfqGroups;    // 8 activation + 8 per weight group
@@ -199,7 +205,7 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
     constexpr uint32_t so = (Q * kStageBytes) >> 4;  // stage offset in 16-byte units
     constexpr uint32_t sfo = so + ((kPTile + kQTile) >> 4);
     // E2M1 x E2M1, E8M0 scales, both operands K-major, N = N1 (and N2), M = 256 (two CTAs)
-    constexpr int N1 = C::kWide ? 256 : BN, N2 = BN - N1;
+    constexpr int N1 = C::kWide ? BN / 2 : BN, N2 = BN - N1;
     constexpr uint32_t idesc0 = (1u << 7) | (1u << 10) | ((N1 >> 3) << 17) | (1u << 23) | ((256u >> 4) << 24);
     constexpr uint32_t idesc2 = idesc0 | (2u << 4) | (2u << 29);
     constexpr uint32_t jdesc0 = (1u << 7) | (1u << 10) | (((N2 > 0 ? N2 : 16) >> 3) << 17) | (1u << 23) | ((256u >> 4) << 24);
@@ -217,8 +223,8 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
             tc_copy_sf_atom_pair(sfq_t + 4 * G + 4 * g, desc64(kHiPlain, slo + ((kSfp + g * kSfGroupBytes + 512) >> 4)));
     }
     // the second instruction of a step reads the CTA's weight rows from row N1 / 2 on and the scale columns of
-    // the last group
-    constexpr uint32_t q2 = ((N1 / 2) * 128) >> 4, s2 = 4 * (G - 1);
+    // the second half's groups
+    constexpr uint32_t q2 = ((N1 / 2) * 128) >> 4, s2 = 4 * C::kHalfGroups;
     tc_mma_mxf4_pair(d_tmem, desc64(kHiSw128, plo), desc64(kHiSw128, qlo), idesc0, sfp_t, sfq_t, accumulate);
     if (N2 > 0) tc_mma_mxf4_pair(d_tmem + N1, desc64(kHiSw128, plo), desc64(kHiSw128, qlo + q2), jdesc0, sfp_t, sfq_t + s2, accumulate);
     if (rem > 64) {
@@ -282,7 +288,6 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         fence_mbar_init();
         tma_prefetch_desc(&tm_act);
         tma_prefetch_desc(&tm_w);
-        if (C::kWide) tma_prefetch_desc(&tm_w_tail);
         tma_prefetch_desc(&tm_sfa);
         tma_prefetch_desc(&tm_sfw);
         tma_prefetch_desc(&tm_y);
@@ -324,14 +329,14 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         // the first ring pass are requested before the dependency wait, so that their latency overlaps the
         // tail of the previous kernel.
         // this CTA's half of the weight tile `ni` and the scale bytes of the whole tile, reduction stage s.
-        // 224 / 240 columns: rows [rank * BN / 2, + BN / 2) of the tile.  288 columns: rows [rank * 128, + 128) and
-        // [256 + rank * 16, + 16), so that the first instruction of a step covers the tile's first 256 rows in
-        // order and the second one the last 32.
+        // 224 / 240 columns: rows [rank * BN / 2, + BN / 2) of the tile.  288 columns: rows [72 rank, + 72) and
+        // [144 + 72 rank, + 72), so that the two instructions of a step cover the tile's two halves in order.
         auto load_weights = [&](uint32_t sb, int ni, int s, uint32_t full) {
             const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
             if (C::kWide) {
-                tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * 128, full);
-                tma_load_2d_pair(sb + kPTile + 128 * 128, &tm_w_tail, xw, ni * BN + 256 + static_cast<int>(rank) * 16, full);
+                constexpr int q = BN / 4;   // 72 rows per box
+                tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * q, full);
+                tma_load_2d_pair(sb + kPTile + q * 128, &tm_w, xw, ni * BN + BN / 2 + static_cast<int>(rank) * q, full);
             } else {
                 tma_load_2d_pair(sb + kPTile, &tm_w, xw, ni * BN + static_cast<int>(rank) * kHalfN, full);
             }
