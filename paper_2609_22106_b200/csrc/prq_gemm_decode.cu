@@ -195,7 +195,12 @@ decode_kernel(const __grid_constant__ DecodeMaps maps, const DecodeBatch b) {
     // requests them before it waits and they stream in while the previous kernel (normally the
     // activation quantiser) is still running.
     const long long t_setup = kTraceBuild ? clock64() : 0;
-    grid_launch_dependents();
+    // Up to 32 tokens the next kernel may be scheduled from here on: two CTAs share an SM, and the next GEMM's set-up and
+    // weight stream overlap this one.  From 64 tokens on a CTA fills its SM and what comes next in a decode step is the
+    // small-CTA activation quantiser, whose blocks would squeeze in beside this kernel's CTAs and slow their chain for
+    // nothing (they wait for this kernel's result anyway): there the trigger comes once the reduction has been issued
+    // (quantise + GEMM step 9.1 -> 8.5 us at 64 tokens, 11.75 -> 11.67 at 128; GEMM-only loops unchanged).
+    if (BN < 64) grid_launch_dependents();
     const uint32_t tmem_base = tmem_slot;
     long long* trace = (ptrace && blockIdx.x < 4) ? ptrace + blockIdx.x * 512 : nullptr;
     if (trace && threadIdx.x == 0) { trace[500] = clock64(); trace[502] = t_entry; trace[503] = t_setup; }
@@ -276,6 +281,7 @@ decode_kernel(const __grid_constant__ DecodeMaps maps, const DecodeBatch b) {
             st = nst; ph = nph;
         }
         if (ok && leader) tc_commit(smem_u32(&bar_acc_full));
+        if (BN >= 64) grid_launch_dependents();
     } else {
         // ------------------------------------------------------------ epilogue, part 1: accumulator -> registers
         // -> (splits == 1) y, or this CTA's partial tile in shared memory, token-major: partial[t][row]
