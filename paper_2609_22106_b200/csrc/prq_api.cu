@@ -147,7 +147,6 @@ prq_status build_weight_maps(prq_weights* w) {
             st = make_sf_map(&w->tm_sfw_pair[v], w->d_sf_alt[v],
                              static_cast<uint64_t>(w->plan.S) * w->w_groups_alt[v] * kSfGroupBytes, 4 * gpt * (one_wave ? 2 : 1));
     }
-    if (st == PRQ_OK) st = make_code_map(&w->tm_w_tail, w->d_codes, Ka / 2, w->N, 16);
     if (st == PRQ_OK) w->maps_ready = true;
     return st;
 }
@@ -1059,7 +1058,7 @@ prq_status prq_linear(const prq_weights* w, const void* codes, const void* scale
         if (st == PRQ_OK) st = make_sf_map(&tm_sfa, p.act_sf, Sg * p.act_groups * kSfGroupBytes, 4);
         if (st == PRQ_OK) st = make_out_map(&tm_y, y, M, w->N, ldy, y_dtype == PRQ_BF16);
         if (st != PRQ_OK) return st;
-        cudaError_t e = launch_prefill_pair(pair_bn, tm_act, w->tm_w_pair[variant], w->tm_w_tail, tm_sfa, w->tm_sfw_pair[variant], tm_y, q,
+        cudaError_t e = launch_prefill_pair(pair_bn, tm_act, w->tm_w_pair[variant], tm_sfa, w->tm_sfw_pair[variant], tm_y, q,
                                             pairs, static_cast<cudaStream_t>(stream));
         g_launches.fetch_add(1);
         return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
@@ -1154,7 +1153,7 @@ prq_status prq_linear_gated(const prq_weights* w, const void* codes, const void*
     if (st == PRQ_OK) st = make_sf_map(&tm_sfa, q.act_sf, static_cast<uint64_t>(w->plan.S) * q.act_groups * kSfGroupBytes, 4);
     if (st != PRQ_OK) return st;
     // (the kernel stores nothing through an output map in this mode: the activation map fills the parameter)
-    cudaError_t e = launch_prefill_pair(kPrefillTileGated, tm_act, w->tm_w_pair[kAltGated], w->tm_w_tail, tm_sfa, w->tm_sfw_pair[kAltGated],
+    cudaError_t e = launch_prefill_pair(kPrefillTileGated, tm_act, w->tm_w_pair[kAltGated], tm_sfa, w->tm_sfw_pair[kAltGated],
                                         tm_act, q, pairs, static_cast<cudaStream_t>(stream));
     g_launches.fetch_add(1);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;

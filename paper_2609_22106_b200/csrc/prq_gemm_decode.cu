@@ -17,7 +17,11 @@
 // epilogue and reduction.  The activation tail is re-read: stages past the K main columns load the
 // token tile from column K - k and the weight tile from column K onwards (Kernel design paragraph).
 // Every wait is bounded; the cluster barriers sit on the common path so that a CTA that gave up still
-// arrives and its peers are released.
+// arrives and its peers are released, and a CTA that gave up under the asynchronous exchange stays until its
+// peers' deliveries into its receive buffer have landed.
+// The kernel is latency-bound, not bandwidth-bound (with the weights resident in L2 it is only 0.5-1 us faster): what a
+// launch costs is the chain token copies -> five stages of tcgen05 issue -> accumulator read -> exchange -> store behind
+// its dependency, plus the hand-over to the next kernel.
 //
 // Fused variant (up to 16 tokens, activation already scaled and reordered by its producer): the kernel
 // takes the bf16 activation itself.  The four epilogue warps first act as the activation quantiser of

@@ -1,7 +1,9 @@
-// Prefill GEMM (M > 128) on CTA pairs: the block-scaled FP4 product of Eq. (3) with 256 x 224 (or
-// 256 x 240) output tiles computed by two CTAs of a cluster as one tcgen05 cta_group::2 unit, under a
-// stream-K schedule.  The text below speaks of the 224-column tile; the 240-column variant differs in the
-// constants only (120 weight rows per CTA, a 16-column chunk closing the epilogue).
+// Prefill GEMM (M > 128) on CTA pairs: the block-scaled FP4 product of Eq. (3) with output tiles of 256 rows computed
+// by two CTAs of a cluster as one tcgen05 cta_group::2 unit.  Three tile widths (template instances): 224 and 240
+// columns under a stream-K schedule, and 288 columns for calls whose tiles all fit ONE wave of pairs at that width (see
+// PCfg).  A fourth instance, 192 columns with a gated epilogue, serves prq_linear_gated.  The text below speaks of the
+// 224-column tile; the 240-column one differs in the constants only (120 weight rows per CTA, a 16-column chunk closing
+// the epilogue).
 //
 // Why pairs.  With one CTA per 128 x 224 tile every SM pulls (128 + 224) operand rows per reduction
 // stage from L2, and at the paper's down-projection shape the 148 SMs together ask for more than the
@@ -9,33 +11,34 @@
 // each CTA loads its own 128 activation rows and only 112 of the 224 weight rows, the tensor cores read
 // the other half from the peer's shared memory, and the bytes per SM and stage drop by 30 %.
 //
-// Schedule.  2048 tokens x 2560 features are 8 x 12 = 96 pair tiles on 74 pairs; tile-per-pair
-// scheduling would leave a third of the machine idle in its second wave.  So every pair gets the same
-// number of whole tiles (one here), and the tiles left over (22) are processed stream-K: their (tile,
-// reduction-stage) space is cut into equal contiguous ranges, one per pair, which the pairs work off
-// FIRST.  A range is a piece of one tile or the tail of one and the head of the next.  The pair that
-// holds a tile's first stage owns it; the others write their fp32 partial accumulators to workspace
-// slots (one per CTA) and raise the flags of the tile's two halves; the owner adds them in a fixed
-// order.  All of this fix-up traffic and waiting happens while the pairs' main loops are busy with
-// their whole tiles; what is exposed at the end of every pair is one plain tile epilogue, the same
-// for all of them.
+// Schedule (224 / 240 columns).  Every pair gets the same number of whole tiles, and the tiles left over are each cut
+// along K into equal pieces for consecutive pairs, which the pairs work off FIRST.  A pair that computed a piece
+// publishes its fp32 partial tile to a workspace slot and counts itself on the tile's "arrived" counters; once all
+// pieces are there, every participant sums (in piece order: deterministic) a share of the tile's column chunks and
+// stores them.  All of this fix-up traffic and waiting happens while the pairs' main loops are busy with their whole
+// tiles; what is exposed at the end of every pair is one plain tile epilogue, whose chunks are each staged in a buffer
+// of their own taken from the idle pipeline ring.  Stream-K is at its worst where the tiles exceed the pairs by little
+// (the paper's down projection at 2048 tokens: 88 tiles on 74 pairs); such a call takes the 288-column instance instead:
+// 72 tiles, one per pair, nothing published or fixed up.
 //
 // Roles (6 warps per CTA):
 //   warp 0    TMA producer (both CTAs): per 256-element reduction stage its own activation tile, its
-//             half of the weight tile, the scale bytes of its activation rows and of all 224 weight rows;
-//             all four copies of both CTAs are counted on the LEADER's "full" mbarrier;
-//   warp 1    leader CTA: tcgen05 issuer -- six scale-atom copies shared -> tensor memory (each CTA
-//             copies from its own shared memory), up to four K = 64 MMAs, one commit that arrives on
-//             the "empty" barrier of both CTAs.  In the other CTA this warp only allocates and frees
-//             tensor memory;
+//             half of the weight tile, the scale bytes of its activation rows and of all weight rows of the tile;
+//             all copies of both CTAs are counted on the LEADER's "full" mbarrier;
+//   warp 1    leader CTA: tcgen05 issuer -- the stage's scale-atom copies shared -> tensor memory (each CTA
+//             copies from its own shared memory), up to four K = 64 steps (one MMA each; two of 144 columns in the
+//             288-column instance), one commit that arrives on the "empty" barrier of both CTAs.  In the other CTA
+//             this warp only allocates and frees tensor memory;
 //   warps 2-5 epilogue (both CTAs): tcgen05.ld of their 32-lane quarter of the CTA's 128 accumulator
 //             rows, 32 columns at a time, into swizzled shared staging, then one TMA store per warp and
-//             chunk (rows and columns outside M x N are clipped by the tensor map).
+//             chunk (rows and columns outside M x N are clipped by the tensor map).  Gated instance: instead of
+//             storing y, form silu(gate) * up per (gate, up) group of 32 + 32 columns, quantise it to MXFP4 and write
+//             codes and scale bytes of the down projection's input (Eq. (1), middle line).
 //
 // The activation tail is re-read, not copied: stages past the K main columns load the activation tile
 // from column K - k and the weight tile from column K onwards (Kernel design paragraph).
-// Every wait is bounded; on expiry the CTA raises its abort flag and the peer's, all roles unwind, both
-// CTAs meet at the closing cluster barrier, tensor memory is freed and PRQ_ERR_TIMEOUT is recorded.
+// Every wait is bounded (the limit is a launch parameter); on expiry the CTA raises its abort flag and the peer's, all
+// roles unwind, both CTAs meet at the closing cluster barrier, tensor memory is freed and PRQ_ERR_TIMEOUT is recorded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -245,7 +248,6 @@ __device__ __forceinline__ void issue_stage(uint32_t lo_base, uint32_t d_tmem, u
 template <int BN, bool kGated = false>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
-                    const __grid_constant__ CUtensorMap tm_w_tail,
                     const __grid_constant__ CUtensorMap tm_sfa, const __grid_constant__ CUtensorMap tm_sfw,
                     const __grid_constant__ CUtensorMap tm_y, const PrefillParams p) {
     using C = PCfg<BN>;
@@ -783,7 +785,7 @@ int max_clusters_bn() {
 }
 
 template <int BN, bool kGated = false>
-cudaError_t launch_bn(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_w_tail, const CUtensorMap& tm_sfa,
+cudaError_t launch_bn(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_sfa,
                       const CUtensorMap& tm_sfw, const CUtensorMap& tm_y, const PrefillParams& p,
                       int pairs, cudaStream_t stream) {
     constexpr int kSmemBytes = PCfg<BN>::kSmemBytes;
@@ -807,7 +809,7 @@ cudaError_t launch_bn(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const 
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BN, kGated>, tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p);
+    return cudaLaunchKernelEx(&cfg, prefill_pair_kernel<BN, kGated>, tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p);
 }
 
 }  // namespace
@@ -818,21 +820,21 @@ int prefill_pair_max_clusters(int bn) {
            : bn == kPrefillTileWide ? max_clusters_bn<kPrefillTileWide>() : max_clusters_bn<kPrefillTileN>();
 }
 
-cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_w_tail,
+cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w,
                                 const CUtensorMap& tm_sfa, const CUtensorMap& tm_sfw, const CUtensorMap& tm_y,
                                 const PrefillParams& p, int pairs, cudaStream_t stream) {
     if (bn == kPrefillTileOneWave) {
         // one accumulator: no pair may be given a second tile or a piece of one
         if (p.whole_tiles + (p.sk_tiles > 0 ? 1 : 0) > 1 || (p.sk_tiles > 0 && p.sk_base != 1) || p.sk_extra != 0) return cudaErrorInvalidValue;
-        return launch_bn<kPrefillTileOneWave>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+        return launch_bn<kPrefillTileOneWave>(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
     }
     if (bn == kPrefillTileGated) {
         // whole tiles only: a piece of a tile has no (gate, up) sums to put through the activation function
         if (p.sk_tiles != 0 || !p.out_codes || !p.out_sf) return cudaErrorInvalidValue;
-        return launch_bn<kPrefillTileGated, true>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+        return launch_bn<kPrefillTileGated, true>(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
     }
-    if (bn == kPrefillTileWide) return launch_bn<kPrefillTileWide>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
-    if (bn == kPrefillTileN) return launch_bn<kPrefillTileN>(tm_act, tm_w, tm_w_tail, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+    if (bn == kPrefillTileWide) return launch_bn<kPrefillTileWide>(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
+    if (bn == kPrefillTileN) return launch_bn<kPrefillTileN>(tm_act, tm_w, tm_sfa, tm_sfw, tm_y, p, pairs, stream);
     return cudaErrorInvalidValue;
 }
 

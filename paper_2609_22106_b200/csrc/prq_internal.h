@@ -112,7 +112,7 @@ struct prq_weights {
     // tensor maps of the weight side, encoded once (dense layers; a handle is immutable afterwards):
     // codes with 128-row boxes (decode kernel), codes with half-tile boxes and the scale bytes of the
     // 224-row [0], 240-row [1], 288-row [2] and 192-row [3] tilings (CTA-pair prefill kernel)
-    CUtensorMap tm_w_decode, tm_w_pair[4], tm_sfw_pair[4], tm_w_tail;   // tm_w_tail: 16-row boxes (288-row tiling)
+    CUtensorMap tm_w_decode, tm_w_pair[4], tm_sfw_pair[4];
     bool maps_ready = false;
     int32_t* d_perm = nullptr;       // E x K
     float* d_inv_s_perm = nullptr;   // E x K : inv_s[perm[j]] in the new channel order

@@ -175,10 +175,11 @@ struct PrefillParams {
     uint16_t* out_h;            // M x C bf16 (the product before quantisation), or null: for checks
     int out_C, out_k_tail, out_groups;
 };
-// `bn` = tile width (kPrefillTileN, kPrefillTileWide, kPrefillTileOneWave, or kPrefillTileGated for the gated-producer epilogue).  `tm_w` has boxes of bn / 2 rows (288: 128 rows,
-// and `tm_w_tail` boxes of 16 rows; any valid map otherwise); `tm_sfa` / `tm_sfw` view the scale bytes as rows of 256 bytes
-// with boxes of 4 / 8 (288: 12) rows (one / two / three 128-row groups); `tm_y` has 32 x 32 boxes.
-cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const CUtensorMap& tm_w_tail,
+// `bn` = tile width (kPrefillTileN, kPrefillTileWide, kPrefillTileOneWave, or kPrefillTileGated for the gated-producer
+// epilogue).  `tm_w` has boxes of bn / 2 rows (288: bn / 4 = 72 rows, loaded twice per CTA and stage); `tm_sfa` / `tm_sfw`
+// view the scale bytes as rows of 256 bytes with boxes of 4 / 8 (288: 16) rows (one / two / four 128-row groups);
+// `tm_y` has 32 x 32 boxes (any valid map for the gated instance, which stores nothing through it).
+cudaError_t launch_prefill_pair(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w,
                                 const CUtensorMap& tm_sfa, const CUtensorMap& tm_sfw, const CUtensorMap& tm_y,
                                 const PrefillParams& p, int pairs, cudaStream_t stream);
 // How many pairs of the pair kernel can be resident at once on the current device.
