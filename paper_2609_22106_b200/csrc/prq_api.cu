@@ -1214,11 +1214,16 @@ prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const voi
     p.trace = trace_ptr();
     // output features on the MMA M axis, one 128-token group of an expert on the N axis (contiguous stores per
     // token, cheap for experts with few tokens)
+    // token tile: 64 rows when the experts hold a handful of tokens each (the smaller tile leaves room for a deeper
+    // ring of weight tiles in flight), 128 otherwise (every extra token tile of an expert re-reads its weight tiles)
+    int bn = static_cast<long long>(M_total) <= 8LL * w->n_experts ? 64 : 128;
+    bn = env_int("PRQ_GROUPED_BN", bn);   // developer switch
+    if (bn != 64 && bn != 128) return PRQ_ERR_INVALID_ARG;
     CUtensorMap tm_act, tm_w;
-    st = make_code_map(&tm_act, codes, w->K / 2, M_total, 128);
+    st = make_code_map(&tm_act, codes, w->K / 2, M_total, bn);
     if (st == PRQ_OK) st = make_code_map(&tm_w, w->d_codes, Ka / 2, static_cast<uint64_t>(w->n_experts) * w->N, 128);
     if (st != PRQ_OK) return st;
-    cudaError_t e = launch_gemm_grouped(tm_act, tm_w, p, di->num_sms, static_cast<cudaStream_t>(stream));
+    cudaError_t e = launch_gemm_grouped(bn, tm_act, tm_w, p, di->num_sms, static_cast<cudaStream_t>(stream));
     g_launches.fetch_add(1);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
 }

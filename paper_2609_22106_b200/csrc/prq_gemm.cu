@@ -36,7 +36,6 @@ namespace {
 constexpr int kMainWarps = 2;   // producer + issuer; the epilogue warps follow
 constexpr int kPTileBytes = 128 * 128;
 constexpr int kRowCache = 256;   // experts whose row ranges are cached in shared memory
-constexpr int BN = 128;          // tokens per tile (MMA N)
 
 constexpr int cmin(int a, int b) { return a < b ? a : b; }
 constexpr int pow2_at_least(int x) { int p = 32; while (p < x) p *= 2; return p; }
@@ -50,19 +49,30 @@ __device__ __forceinline__ uint64_t desc64(uint32_t hi, uint32_t lo) { return (s
 // kFp8: the second format (MXFP8: one byte per element, E4M3).  A stage is still one 128-byte swizzled row per operand
 // row, which then holds 128 elements = 4 blocks = ONE scale atom per 128-row group instead of two, and a K = 32 step
 // per MMA (kind::mxf8f6f4) that takes one scale byte per row: the scale-id fields walk the four bytes of the word.
-template <bool kFp8>
+// BN: tokens per tile (MMA N), 128 or 64.  The 64-token instance is for launches whose experts hold a handful of
+// tokens each (MoE decode): there the kernel is a stream of weight tiles, a CTA's throughput is the bytes its ring
+// keeps in flight over the memory latency, and an 8 KB token tile instead of a 16 KB one buys two more ring slots.
+// (The scale columns of a tile then start two tensor-memory columns into the group's atom.  A 32-token tile would
+// start at odd columns, which the block-scaled MMA does not take: such an instance raised a misaligned-address
+// error and was not pursued.)
+template <bool kFp8, int BN>
 struct Cfg {
+    static_assert(BN == 128 || BN == 64, "token tile");
     static constexpr int kStageElems = kFp8 ? 128 : kStageK;
     static constexpr int kSfBytes = kFp8 ? 512 : kSfGroupBytes;    // scale bytes per (stage, 128-row group)
     // eight epilogue warps, two per tensor-memory lane quarter taking alternate 16-token chunks: with
     // K + k = 832 a tile is only 3.25 stages, and the epilogue is what the main loop waits for
-    static constexpr int kEpiWarps = 8;
+    // (four with the 64-token tile, whose epilogues are short: their staging would cost the eighth ring slot)
+    static constexpr int kEpiWarps = BN == 128 ? 8 : 4;
     static constexpr int kThreads = 32 * (kMainWarps + kEpiWarps);
     static constexpr int kQTileBytes = BN * 128;
     static constexpr int kSfpBytes = kSfBytes;
     static constexpr int kSfqBytes = kSfBytes;
     static constexpr int kStageBytes = kPTileBytes + kQTileBytes + kSfpBytes + kSfqBytes;
-    static constexpr int kStages = cmin(8, (232448 - 1024 - 16384 - 2048) / kStageBytes);
+    // shared memory per CTA: 227 KB less the kernel's static arrays (barriers, per-expert tile and row tables), the
+    // alignment slack and the epilogue's staging tiles
+    static constexpr int kStaticBytes = 5632 + (BN == 128 ? 0 : 4 * (kMaxExperts + 1));
+    static constexpr int kStages = cmin(8, (232448 - kStaticBytes - 1024 - kEpiWarps * 2048) / kStageBytes);
     // tensor memory columns: two accumulators, then scale words (2 atoms x 4 columns per operand)
     static constexpr int kAccStride = BN;
     static constexpr int kSfpCols = 8, kSfqCols = 8;
@@ -84,20 +94,23 @@ struct Unit {
     int n0;                      // first output feature
 };
 
-// Where a unit sits: expert, 128-row token tile (counted over all experts), feature tile.
+// Where a unit sits: expert, BN-row token tile (counted over all experts), feature tile.
 struct GroupPos { int e, mt, ni; };
 
-__device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_start, const int* row_start, int S,
-                                           const GroupPos& g, int sf_bytes) {
+// The scale bytes of the activation come in 128-row groups, every expert's rows padded to whole groups
+// (group_start[e] = groups before expert e); a BN-row tile is rows [lt * BN, lt * BN + BN) of its expert.
+template <int BN>
+__device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_start, const int* group_start,
+                                           const int* row_start, int S, const GroupPos& g, int sf_bytes) {
     Unit t;
-    const int e = g.e, mt = g.mt, ni = g.ni;
+    const int e = g.e, lt = g.mt - tile_start[e], ni = g.ni;
     t.p_row = e * p.N + ni * 128;
-    t.q_row = row_start[e] + (mt - tile_start[e]) * 128;
+    t.q_row = row_start[e] + lt * BN;
     t.sfp = p.w_sf + (static_cast<size_t>(e) * S * p.w_groups + ni) * sf_bytes;
     t.sfp_stride = static_cast<size_t>(p.w_groups) * sf_bytes;
-    t.sfq = p.act_sf + static_cast<size_t>(mt) * sf_bytes;
+    t.sfq = p.act_sf + static_cast<size_t>(group_start[e] + lt * BN / 128) * sf_bytes;
     t.sfq_stride = static_cast<size_t>(p.act_groups) * sf_bytes;
-    t.row0 = t.q_row; t.row_end = min(row_start[e + 1], t.q_row + 128);
+    t.row0 = t.q_row; t.row_end = min(row_start[e + 1], t.q_row + BN);
     t.n0 = ni * 128;
     return t;
 }
@@ -106,14 +119,17 @@ __device__ __forceinline__ Unit make_unit(const GemmParams& p, const int* tile_s
 // the next one is a couple of shared-memory reads (the next token tile, usually of the same expert) instead
 // of a division and a search over the experts in every role's critical path; consecutive units of an expert
 // also reuse its weight tile from L2.
+template <int BN>
 struct UnitIter {
     const GemmParams& p;
     const int* tile_start;
+    const int* group_start;
     const int* row_start;
     int S, u, u_end, sf_bytes;
     GroupPos g;
-    __device__ __forceinline__ UnitIter(const GemmParams& p_, const int* ts, const int* rs, int S_, int n_units, int sf_bytes_)
-        : p(p_), tile_start(ts), row_start(rs), S(S_), sf_bytes(sf_bytes_), g{0, 0, 0} {
+    __device__ __forceinline__ UnitIter(const GemmParams& p_, const int* ts, const int* gs, const int* rs, int S_, int n_units,
+                                        int sf_bytes_)
+        : p(p_), tile_start(ts), group_start(gs), row_start(rs), S(S_), sf_bytes(sf_bytes_), g{0, 0, 0} {
         const int per = (n_units + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
         u = min(n_units, static_cast<int>(blockIdx.x) * per);
         u_end = min(n_units, u + per);
@@ -129,7 +145,9 @@ struct UnitIter {
         }
     }
     __device__ __forceinline__ bool valid() const { return u < u_end; }
-    __device__ __forceinline__ Unit get() const { return make_unit(p, tile_start, row_start, S, g, sf_bytes); }
+    __device__ __forceinline__ Unit get() const { return make_unit<BN>(p, tile_start, group_start, row_start, S, g, sf_bytes); }
+    // which BN-row part of its 128-row scale group the current tile is
+    __device__ __forceinline__ int sub() const { return (g.mt - tile_start[g.e]) % (128 / BN); }
     __device__ __forceinline__ void next() {
         if (++u < u_end) {
             if (++g.mt == tile_start[p.n_experts]) { g.mt = 0; g.e = 0; ++g.ni; }
@@ -138,19 +156,26 @@ struct UnitIter {
     }
 };
 
-template <bool kFp8>
-__global__ void __launch_bounds__(Cfg<kFp8>::kThreads, 1)
+template <bool kFp8, int BN>
+__global__ void __launch_bounds__(Cfg<kFp8, BN>::kThreads, 1)
 gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_constant__ CUtensorMap tm_w,
                     const GemmParams p) {
-    using C = Cfg<kFp8>;
+    using C = Cfg<kFp8, BN>;
+    using Iter = UnitIter<BN>;
     extern __shared__ uint8_t smem_raw[];
+    if (kTraceBuild && p.trace && threadIdx.x == 0 && blockIdx.x < 160) {
+        unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g));
+        p.trace[2048 + blockIdx.x * 4] = static_cast<long long>(g);
+    }
     __shared__ __align__(8) uint64_t bar_full[C::kStages], bar_empty[C::kStages], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag_s;
     __shared__ int tile_start[kMaxExperts + 1];
+    __shared__ int group_start_s[BN == 128 ? 1 : kMaxExperts + 1];
     __shared__ int row_cache[kRowCache + 1];
     volatile int* abort_flag = &abort_flag_s;
     const int* row_start = p.n_experts <= kRowCache ? row_cache : p.expert_offsets;
+    const int* group_start = BN == 128 ? tile_start : group_start_s;   // with 128-row tiles the two coincide
 
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t smem_base = smem_u32(smem);
@@ -174,14 +199,8 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         for (int e = threadIdx.x; e <= p.n_experts; e += blockDim.x)
             row_cache[e] = p.expert_offsets ? p.expert_offsets[e] : (e == 0 ? 0 : p.M);
     __syncthreads();
-    if (threadIdx.x == 64) {
-        int acc = 0;
-        for (int e = 0; e < p.n_experts; ++e) {
-            tile_start[e] = acc;
-            acc += (row_start[e + 1] - row_start[e] + 127) / 128;
-        }
-        tile_start[p.n_experts] = acc;
-    }
+    // first tile (and first 128-row scale group) of every expert
+    if (warp == 2) warp_expert_starts(row_start, p.n_experts, BN, tile_start, BN == 128 ? nullptr : group_start_s);
     if (warp == 1) {
         tmem_alloc(smem_u32(&tmem_slot), C::kTmemCols);
         tmem_relinquish();
@@ -194,6 +213,14 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     long long* const ptrace = kTraceBuild ? p.trace : nullptr;
     long long* trace = (ptrace && blockIdx.x < 4) ? ptrace + blockIdx.x * 512 : nullptr;
     if (trace && threadIdx.x == 0) trace[500] = clock64();
+    // ... and every CTA's entry, start of work and end on the global timer (ns)
+    auto gstamp = [&](int which) {
+        if (ptrace && threadIdx.x == 0 && blockIdx.x < 160) {
+            unsigned long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g));
+            ptrace[2048 + blockIdx.x * 4 + which] = static_cast<long long>(g);
+        }
+    };
+    gstamp(1);
     const int n_units = tile_start[p.n_experts] * ((p.N + 127) / 128);
 
     if (warp == 0) {
@@ -203,7 +230,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         int it = 0, st = 0;
         uint32_t ph = 0;
         bool ok = true;
-        for (UnitIter ui(p, tile_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next()) {
+        for (Iter ui(p, tile_start, group_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next()) {
             const Unit t = ui.get();
             for (int s = 0; s < S; ++s, ++it) {
                 if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
@@ -245,12 +272,15 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         const uint32_t sfp_t = tmem_base + C::kSfpCol;
         const uint32_t sfq_t = tmem_base + C::kSfqCol;
         const uint32_t lo_base = ((smem_base & 0x3FFFF) >> 4) | (1u << 16);
-        for (UnitIter ui(p, tile_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next(), ++acc_it) {
+        for (Iter ui(p, tile_start, group_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next(), ++acc_it) {
             const int buf = acc_it % C::kAcc;
             const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
             if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + buf * C::kAccStride;
+            // a scale atom holds the bytes of all 128 rows of the group: row r in lane r % 32 of column r / 32, so
+            // a BN-row tile's scales start BN / 32 columns further per tile
+            const uint32_t sfq_u = sfq_t + ui.sub() * (BN / 32);
             uint32_t accumulate = 0;
             for (int s = 0; s < S; ++s, ++it) {
                 if (!ready && !mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
@@ -278,7 +308,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                         for (int j = 0; j < 4; ++j) {
                             if (j < ksteps) {
                                 tc_mma_mxf8(d_tmem, desc64(kHiSw128, plo + 2 * j), desc64(kHiSw128, qlo + 2 * j),
-                                            idesc | (static_cast<uint32_t>(j) << 4) | (static_cast<uint32_t>(j) << 29), sfp_t, sfq_t, accumulate);
+                                            idesc | (static_cast<uint32_t>(j) << 4) | (static_cast<uint32_t>(j) << 29), sfp_t, sfq_u, accumulate);
                                 accumulate = 1;
                             }
                         }
@@ -296,7 +326,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                         for (int j = 0; j < 4; ++j) {
                             if (j < ksteps) {
                                 tc_mma_mxf4(d_tmem, desc64(kHiSw128, plo + 2 * j), desc64(kHiSw128, qlo + 2 * j),
-                                            (j & 1) ? idesc2 : idesc0, sfp_t + (j >> 1) * 4, sfq_t + (j >> 1) * 4, accumulate);
+                                            (j & 1) ? idesc2 : idesc0, sfp_t + (j >> 1) * 4, sfq_u + (j >> 1) * 4, accumulate);
                                 accumulate = 1;
                             }
                         }
@@ -317,7 +347,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
         const int et = q * 32 + lane;           // 0..127: accumulator row
         int acc_it = 0;
         bool ok = true;
-        for (UnitIter ui(p, tile_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next(), ++acc_it) {
+        for (Iter ui(p, tile_start, group_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next(), ++acc_it) {
             const Unit t = ui.get();
             const int buf = acc_it % C::kAcc;
             const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
@@ -393,6 +423,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     tc_fence_before_sync();
     __syncthreads();
     if (trace && threadIdx.x == 0) trace[501] = clock64();
+    gstamp(2);
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();
@@ -402,31 +433,33 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
 }
 
 
-template <bool kFp8>
+template <bool kFp8, int BN>
 cudaError_t launch_grouped_impl(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
                                 cudaStream_t stream) {
-    using C = Cfg<kFp8>;
+    using C = Cfg<kFp8, BN>;
     constexpr int smem = C::kStages * C::kStageBytes + 1024 + C::kEpiWarps * 2048;  // + store staging
     static bool configured = false;  // the attribute is per function, setting it twice is harmless
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_grouped_kernel<kFp8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        cudaError_t e = cudaFuncSetAttribute(gemm_grouped_kernel<kFp8, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    gemm_grouped_kernel<kFp8><<<grid, C::kThreads, smem, stream>>>(tm_act, tm_w, p);
+    gemm_grouped_kernel<kFp8, BN><<<grid, C::kThreads, smem, stream>>>(tm_act, tm_w, p);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t launch_gemm_grouped(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
+cudaError_t launch_gemm_grouped(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
                                 cudaStream_t stream) {
-    return launch_grouped_impl<false>(tm_act, tm_w, p, grid, stream);
+    if (bn == 64) return launch_grouped_impl<false, 64>(tm_act, tm_w, p, grid, stream);
+    if (bn != 128) return cudaErrorInvalidValue;
+    return launch_grouped_impl<false, 128>(tm_act, tm_w, p, grid, stream);
 }
 
 cudaError_t launch_gemm_fp8(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
                             cudaStream_t stream) {
-    return launch_grouped_impl<true>(tm_act, tm_w, p, grid, stream);
+    return launch_grouped_impl<true, 128>(tm_act, tm_w, p, grid, stream);
 }
 
 }  // namespace prq

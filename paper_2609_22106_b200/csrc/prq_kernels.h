@@ -77,9 +77,9 @@ struct GemmParams {
     int dbg;                 // developer switches for timing experiments (0 in normal use)
 };
 
-// Grouped (MoE) kernel: 128 output features of one expert on the MMA M axis, one 128-token group of that expert
-// on the N axis; `grid` persistent CTAs.  `tm_act` / `tm_w` have 128-row boxes.
-cudaError_t launch_gemm_grouped(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
+// Grouped (MoE) kernel: 128 output features of one expert on the MMA M axis, `bn` (128 or 64) tokens of that expert
+// on the N axis; `grid` persistent CTAs.  `tm_w` has 128-row boxes, `tm_act` bn-row boxes.
+cudaError_t launch_gemm_grouped(int bn, const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
                                 cudaStream_t stream);
 
 

@@ -273,4 +273,38 @@ __host__ __device__ __forceinline__ uint32_t make_idesc_mxf4(uint32_t n, uint32_
            (a_sf_id << 29);
 }
 
+// ---------------------------------------------------------------- expert tables
+// Grouped layers: rows are sorted by expert, row_start[e] .. row_start[e + 1], and every expert's rows are cut into
+// tiles of `tile_rows`.  One warp fills tile_start[0 .. n_experts] with the tiles before each expert (and, if asked,
+// group_start[0 .. n_experts) with the 128-row groups before it): each lane sums a contiguous share of the experts
+// and a warp scan turns the sums into starts.  (A single thread walking all experts costs several microseconds in
+// front of every CTA's work.)  Call with all 32 lanes; the caller synchronises before reading the tables.
+__device__ __forceinline__ void warp_expert_starts(const int* row_start, int n_experts, int tile_rows, int* tile_start,
+                                                   int* group_start) {
+    const int lane = threadIdx.x & 31;
+    const int per = (n_experts + 31) / 32;
+    const int e0 = min(n_experts, lane * per), e1 = min(n_experts, e0 + per);
+    int sum = 0, sum_g = 0;
+    for (int e = e0; e < e1; ++e) {
+        const int rows = row_start[e + 1] - row_start[e];
+        sum += (rows + tile_rows - 1) / tile_rows;
+        sum_g += (rows + 127) / 128;
+    }
+    int inc = sum, inc_g = sum_g;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const int a = __shfl_up_sync(0xffffffffu, inc, d), b = __shfl_up_sync(0xffffffffu, inc_g, d);
+        if (lane >= d) { inc += a; inc_g += b; }
+    }
+    int acc = inc - sum, acc_g = inc_g - sum_g;
+    for (int e = e0; e < e1; ++e) {
+        const int rows = row_start[e + 1] - row_start[e];
+        tile_start[e] = acc;
+        if (group_start) group_start[e] = acc_g;
+        acc += (rows + tile_rows - 1) / tile_rows;
+        acc_g += (rows + 127) / 128;
+    }
+    if (lane == 31) tile_start[n_experts] = inc;
+}
+
 }  // namespace prq

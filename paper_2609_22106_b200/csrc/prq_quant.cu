@@ -118,14 +118,7 @@ quant_act_kernel(const QuantBatch b) {
         row0 = group * kGroupRows;
         row_end = min(p.M, row0 + kGroupRows);
     } else {
-        if (threadIdx.x == 0) {
-            int acc = 0;
-            for (int e = 0; e < p.n_experts; ++e) {
-                s_tile_start[e] = acc;
-                acc += (p.expert_offsets[e + 1] - p.expert_offsets[e] + kGroupRows - 1) / kGroupRows;
-            }
-            s_tile_start[p.n_experts] = acc;
-        }
+        if (threadIdx.x < 32) warp_expert_starts(p.expert_offsets, p.n_experts, kGroupRows, s_tile_start, nullptr);
         __syncthreads();
         if (group >= s_tile_start[p.n_experts]) return;  // padding CTA of the launch grid
         int lo = 0, hi = p.n_experts - 1;

@@ -67,9 +67,13 @@ def test_random_shapes_against_oracle(prq, oracle, seed):
         w.free()
 
 
+@pytest.mark.parametrize("gbn", [0, 64, 128])
 @pytest.mark.parametrize("seed", [21, 22])
-def test_random_grouped_shapes_against_oracle(prq, oracle, seed):
-    """Stacked experts with random row counts (empty experts included), strided activations and outputs."""
+def test_random_grouped_shapes_against_oracle(prq, oracle, monkeypatch, seed, gbn):
+    """Stacked experts with random row counts (empty experts included), strided activations and outputs, with the
+    library's own choice of token tile (gbn 0) and with both tiles forced."""
+    if gbn:
+        monkeypatch.setenv("PRQ_GROUPED_BN", str(gbn))
     rng = np.random.default_rng(seed)
     for case in range(8):
         E = int(rng.choice([1, 2, 3, 5, 8, 16]))   # one expert: the grouped layout coincides with the dense one
@@ -83,7 +87,7 @@ def test_random_grouped_shapes_against_oracle(prq, oracle, seed):
         M = int(offsets[-1])
         mode = int(rng.integers(0, 2))
         dt = prq.F32 if rng.random() < 0.5 else prq.BF16
-        what = f"seed {seed} case {case}: E={E} N={N} K={K} k={k} counts={counts.tolist()} mode={mode} dt={dt}"
+        what = f"seed {seed} tile {gbn} case {case}: E={E} N={N} K={K} k={k} counts={counts.tolist()} mode={mode} dt={dt}"
         ch = synth.HeavyTailChannels(int(rng.integers(0, 10000)), K)
         Ws = np.stack([synth.weights(int(rng.integers(0, 10000)), N, K) for _ in range(E)])
         amax = np.stack([oracle.channel_amax(ch.rows(int(rng.integers(0, 10000)), 32)) for _ in range(E)])
