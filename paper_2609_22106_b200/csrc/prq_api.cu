@@ -1216,8 +1216,9 @@ prq_status prq_linear_grouped(const prq_weights* w, const void* codes, const voi
     // token, cheap for experts with few tokens)
     // token tile: 64 rows when the experts hold a handful of tokens each (the smaller tile leaves room for a deeper
     // ring of weight tiles in flight), 128 otherwise (every extra token tile of an expert re-reads its weight tiles)
-    int bn = static_cast<long long>(M_total) <= 8LL * w->n_experts ? 64 : 128;
+    int bn = static_cast<long long>(M_total) <= 64LL * w->n_experts ? 64 : 128;
     bn = env_int("PRQ_GROUPED_BN", bn);   // developer switch
+    if (bn == 0) bn = 128;
     if (bn != 64 && bn != 128) return PRQ_ERR_INVALID_ARG;
     CUtensorMap tm_act, tm_w;
     st = make_code_map(&tm_act, codes, w->K / 2, M_total, bn);

@@ -33,7 +33,8 @@
 namespace prq {
 namespace {
 
-constexpr int kMainWarps = 2;   // producer + issuer; the epilogue warps follow
+constexpr int kRings = 2;       // independent (producer, issuer) warp pairs, taking alternate units
+constexpr int kMainWarps = 2 * kRings;   // the epilogue warps follow
 constexpr int kPTileBytes = 128 * 128;
 constexpr int kRowCache = 256;   // experts whose row ranges are cached in shared memory
 
@@ -72,16 +73,18 @@ struct Cfg {
     // shared memory per CTA: 227 KB less the kernel's static arrays (barriers, per-expert tile and row tables), the
     // alignment slack and the epilogue's staging tiles
     static constexpr int kStaticBytes = 5632 + (BN == 128 ? 0 : 4 * (kMaxExperts + 1));
-    static constexpr int kStages = cmin(8, (232448 - kStaticBytes - 1024 - kEpiWarps * 2048) / kStageBytes);
+    static constexpr int kStages = cmin(8, (232448 - kStaticBytes - 1024 - kEpiWarps * 2048) / kStageBytes) & ~1;
+    static constexpr int kRing = kStages / kRings;   // slots of each pair's ring
     // tensor memory columns: two accumulators, then scale words (2 atoms x 4 columns per operand)
     static constexpr int kAccStride = BN;
-    static constexpr int kSfpCols = 8, kSfqCols = 8;
-    static constexpr int kAcc = 2;
-    static constexpr int kTmemCols = pow2_at_least(kAcc * kAccStride + kSfpCols + kSfqCols);
-    static constexpr int kSfpCol = kAcc * kAccStride;
+    static constexpr int kSfpCols = 8, kSfqCols = 8;   // per ring
+    static constexpr int kAcc = 2;                     // one accumulator per ring
+    static constexpr int kTmemCols = pow2_at_least(kAcc * kAccStride + kRings * (kSfpCols + kSfqCols));
+    static constexpr int kSfpCol = kAcc * kAccStride;  // + ring * (kSfpCols + kSfqCols)
     static constexpr int kSfqCol = kSfpCol + kSfpCols;
+    static_assert(kAcc == kRings, "every ring accumulates into its own buffer");
     static constexpr uint32_t kTxBytes = kStageBytes;
-    static_assert(kStages >= 2, "tile too large for shared memory");
+    static_assert(kRing >= 2, "tile too large for shared memory");
     static_assert(kTmemCols <= 512, "tile too large for tensor memory");
 };
 
@@ -223,58 +226,71 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
     gstamp(1);
     const int n_units = tile_start[p.n_experts] * ((p.N + 127) / 128);
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ producer
+    // Warps 0..3 are two (producer, issuer) pairs.  Pair r takes the CTA's units r, r + 2, ... through its own ring
+    // of kRing stage slots, its own scale columns and accumulator r: what a role spends per stage is mostly the
+    // issue cost of its own asynchronous instructions (four copies, or nine tcgen05 instructions), and with few
+    // tokens per expert that cost, not the memory system, paced a single pair.
+    const int ring = warp >> 1;
+    if (warp < kMainWarps && (warp & 1) == 0) {
+        // ------------------------------------------------------------ producers
         // The whole warp walks the loop (a lone diverged lane runs this code several times slower);
         // one elected lane arms the barrier and issues the copies.
         int it = 0, st = 0;
         uint32_t ph = 0;
         bool ok = true;
-        for (Iter ui(p, tile_start, group_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next()) {
+        uint64_t* const full_bars = bar_full + ring * C::kRing;
+        uint64_t* const empty_bars = bar_empty + ring * C::kRing;
+        Iter ui(p, tile_start, group_start, row_start, S, n_units, C::kSfBytes);
+        if (ring == 1) ui.next();
+        for (; ui.valid() && ok; ui.next(), ui.next()) {
             const Unit t = ui.get();
             for (int s = 0; s < S; ++s, ++it) {
-                if (!mbar_wait(smem_u32(&bar_empty[st]), ph ^ 1, abort_flag)) { ok = false; break; }
-                if (trace && lane == 0 && it < 64) trace[it] = clock64();
+                if (!mbar_wait(smem_u32(&empty_bars[st]), ph ^ 1, abort_flag)) { ok = false; break; }
+                if (trace && ring == 0 && lane == 0 && it < 64) trace[it] = clock64();
                 if (elect_one()) {
-                    const uint32_t full = smem_u32(&bar_full[st]);
+                    const uint32_t full = smem_u32(&full_bars[st]);
                     mbar_arrive_expect_tx(full, C::kTxBytes);
                     // byte column of each operand in this stage
                     // (a stage is 128 bytes of either format's row; residual stages exist for MXFP4 only)
                     const int xw = s < S1 ? s * 128 : p.K / 2 + (s - S1) * 128;
                     const int xa = s < S1 ? s * 128 : (p.K - p.k_tail) / 2 + (s - S1) * 128;
-                    const uint32_t sb = smem_base + st * C::kStageBytes;
+                    const uint32_t sb = smem_base + (ring * C::kRing + st) * C::kStageBytes;
                     tma_load_2d(sb, &tm_w, xw, t.p_row, full);
                     tma_load_2d(sb + kPTileBytes, &tm_act, xa, t.q_row, full);
                     bulk_load(sb + kPTileBytes + C::kQTileBytes, t.sfp + s * t.sfp_stride, C::kSfpBytes, full);
                     bulk_load(sb + kPTileBytes + C::kQTileBytes + C::kSfpBytes, t.sfq + s * t.sfq_stride,
                               C::kSfqBytes, full);
                 }
-                if (++st == C::kStages) { st = 0; ph ^= 1; }
+                if (++st == C::kRing) { st = 0; ph ^= 1; }
             }
         }
         if (!ok && lane == 0) {
-            // let this CTA's copies in flight land before shared memory is given up (bounded)
-            for (int j = max(0, it - C::kStages); j < it; ++j) {
-                const uint32_t bar = smem_u32(&bar_full[j % C::kStages]);
-                const uint32_t ph = (j / C::kStages) & 1;
+            // let this ring's copies in flight land before shared memory is given up (bounded)
+            for (int j = max(0, it - C::kRing); j < it; ++j) {
+                const uint32_t bar = smem_u32(&full_bars[j % C::kRing]);
+                const uint32_t ph = (j / C::kRing) & 1;
                 for (int tries = 0; tries < (1 << 16) && !mbar_try_wait(bar, ph); ++tries) {}
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
+    } else if (warp < kMainWarps) {
+        // ------------------------------------------------------------ MMA issuers
         // The whole warp walks the loop and waits on the barriers; one elected lane issues the
         // tensor-core instructions (and therefore also the commits that track them).
-        int it = 0, acc_it = 0, st = 0;
+        int it = 0, acc_it = 0, st = 0;   // acc_it counts this ring's units
         uint32_t ph = 0;
         bool ok = true;
         bool ready = false;   // the next slot was already seen full by the probe issued one stage earlier
         const bool leader = elect_one();
-        const uint32_t sfp_t = tmem_base + C::kSfpCol;
-        const uint32_t sfq_t = tmem_base + C::kSfqCol;
-        const uint32_t lo_base = ((smem_base & 0x3FFFF) >> 4) | (1u << 16);
-        for (Iter ui(p, tile_start, group_start, row_start, S, n_units, C::kSfBytes); ui.valid() && ok; ui.next(), ++acc_it) {
-            const int buf = acc_it % C::kAcc;
-            const uint32_t acc_ph = (acc_it / C::kAcc) & 1;
+        uint64_t* const full_bars = bar_full + ring * C::kRing;
+        uint64_t* const empty_bars = bar_empty + ring * C::kRing;
+        const uint32_t sfp_t = tmem_base + C::kSfpCol + ring * (C::kSfpCols + C::kSfqCols);
+        const uint32_t sfq_t = tmem_base + C::kSfqCol + ring * (C::kSfpCols + C::kSfqCols);
+        const uint32_t lo_base = (((smem_base + ring * C::kRing * C::kStageBytes) & 0x3FFFF) >> 4) | (1u << 16);
+        const int buf = ring;
+        Iter ui(p, tile_start, group_start, row_start, S, n_units, C::kSfBytes);
+        if (ring == 1) ui.next();
+        for (; ui.valid() && ok; ui.next(), ui.next(), ++acc_it) {
+            const uint32_t acc_ph = acc_it & 1;
             if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), acc_ph ^ 1, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + buf * C::kAccStride;
@@ -283,14 +299,14 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             const uint32_t sfq_u = sfq_t + ui.sub() * (BN / 32);
             uint32_t accumulate = 0;
             for (int s = 0; s < S; ++s, ++it) {
-                if (!ready && !mbar_wait(smem_u32(&bar_full[st]), ph, abort_flag)) { ok = false; break; }
-                if (trace && lane == 0 && it < 64) trace[64 + it] = clock64();
+                if (!ready && !mbar_wait(smem_u32(&full_bars[st]), ph, abort_flag)) { ok = false; break; }
+                if (trace && ring == 0 && lane == 0 && it < 64) trace[64 + it] = clock64();
                 const int rem = s < S1 ? p.K - s * C::kStageElems : p.k_tail - (s - S1) * C::kStageElems;
                 const int ksteps = min(4, (rem + C::kStageElems / 4 - 1) / (C::kStageElems / 4));
                 // probe the next slot now: the probe's latency hides behind this stage's tcgen05 instructions
-                const int nst = st + 1 == C::kStages ? 0 : st + 1;
+                const int nst = st + 1 == C::kRing ? 0 : st + 1;
                 const uint32_t nph = nst == 0 ? ph ^ 1 : ph;
-                ready = mbar_test_wait(smem_u32(&bar_full[nst]), nph);
+                ready = mbar_test_wait(smem_u32(&full_bars[nst]), nph);
                 if (leader) {
                     // Descriptors as (constant high word, 32-bit low word): the low word is the shared
                     // address in 16-byte units plus the leading-dimension field, so a stage's descriptors
@@ -331,10 +347,10 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                             }
                         }
                     }
-                    tc_commit(smem_u32(&bar_empty[st]));
+                    tc_commit(smem_u32(&empty_bars[st]));
                 }
                 accumulate = 1;
-                if (trace && lane == 0 && it < 64) trace[128 + it] = clock64();
+                if (trace && ring == 0 && lane == 0 && it < 64) trace[128 + it] = clock64();
                 st = nst; ph = nph;
             }
             if (!ok) break;
@@ -342,7 +358,7 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             __syncwarp();
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..9)
+        // ------------------------------------------------------------ epilogue (the warps after the two pairs)
         const int q = warp & 3;                 // tensor-memory lane quarter this warp may read
         const int et = q * 32 + lane;           // 0..127: accumulator row
         int acc_it = 0;
