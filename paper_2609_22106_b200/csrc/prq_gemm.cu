@@ -61,10 +61,11 @@ struct Cfg {
     static_assert(BN == 128 || BN == 64, "token tile");
     static constexpr int kStageElems = kFp8 ? 128 : kStageK;
     static constexpr int kSfBytes = kFp8 ? 512 : kSfGroupBytes;    // scale bytes per (stage, 128-row group)
-    // eight epilogue warps, two per tensor-memory lane quarter taking alternate 16-token chunks: with
+    // eight epilogue warps, two per tensor-memory lane quarter taking half of the tile's tokens each: with
     // K + k = 832 a tile is only 3.25 stages, and the epilogue is what the main loop waits for
-    // (four with the 64-token tile, whose epilogues are short: their staging would cost the eighth ring slot)
-    static constexpr int kEpiWarps = BN == 128 ? 8 : 4;
+    static constexpr int kEpiWarps = 8;
+    static constexpr int kWarpTokens = BN / (kEpiWarps / 4);
+    static constexpr int kStagingBytes = 1024;   // per epilogue warp
     static constexpr int kThreads = 32 * (kMainWarps + kEpiWarps);
     static constexpr int kQTileBytes = BN * 128;
     static constexpr int kSfpBytes = kSfBytes;
@@ -73,7 +74,7 @@ struct Cfg {
     // shared memory per CTA: 227 KB less the kernel's static arrays (barriers, per-expert tile and row tables), the
     // alignment slack and the epilogue's staging tiles
     static constexpr int kStaticBytes = 5632 + (BN == 128 ? 0 : 4 * (kMaxExperts + 1));
-    static constexpr int kStages = cmin(8, (232448 - kStaticBytes - 1024 - kEpiWarps * 2048) / kStageBytes) & ~1;
+    static constexpr int kStages = cmin(8, (232448 - kStaticBytes - 1024 - kEpiWarps * kStagingBytes) / kStageBytes) & ~1;
     static constexpr int kRing = kStages / kRings;   // slots of each pair's ring
     // tensor memory columns: two accumulators, then scale words (2 atoms x 4 columns per operand)
     static constexpr int kAccStride = BN;
@@ -371,29 +372,41 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             if (trace && et == 0 && acc_it < 8) trace[192 + 2 * acc_it] = clock64();
             tc_fence_after_sync();
             const uint32_t acc_t = tmem_base + buf * C::kAccStride + (static_cast<uint32_t>(q * 32) << 16);
-            // accumulator row = output feature n, column = token of this expert's 128-row group.  Sixteen
-            // tokens at a time, every warp parks its 32 features per token in a small shared tile (one
-            // contiguous row per token) and writes the rows out in 16-byte pieces: 64 (bf16) or 128 (fp32)
-            // contiguous bytes per token and warp.  A group with few tokens costs few stores.
+            // accumulator row = output feature n, column = token of this tile.  A warp takes 64 tokens of its
+            // lane quarter (the two warps of a quarter take one half of a 128-token tile each): it reads all of
+            // them into registers and hands the accumulator back to the issuer at once, so that the next tile
+            // of this ring accumulates while the stores below run.  Sixteen tokens at a time, the warp then
+            // parks its 32 features per token in a small shared tile (one contiguous row per token) and writes
+            // the rows out in 16-byte pieces: 64 (bf16) or 128 (fp32) contiguous bytes per token and warp.  A
+            // tile with few tokens costs few reads and few stores.
             const int n_tok = t.row_end - t.row0;
             const int nw = t.n0 + q * 32;                   // first feature of this warp
-            const uint32_t stg = smem_base + C::kStages * C::kStageBytes + (warp - kMainWarps) * 2048;
-            constexpr int kPerQuarter = C::kEpiWarps / 4;   // warps sharing a lane quarter take alternate chunks
-#pragma unroll 1
-            for (int c = (warp - kMainWarps) >> 2; c * 16 < n_tok; c += kPerQuarter) {
-                uint32_t r[16];
-                tmem_ld_32x16(acc_t + c * 16, r);
-                tmem_ld_wait();
-                if (p.y_bf16) {
+            const uint32_t stg = smem_base + C::kStages * C::kStageBytes + (warp - kMainWarps) * C::kStagingBytes;
+            constexpr int kTW = C::kWarpTokens;
+            const int tok0 = ((warp - kMainWarps) >> 2) * kTW;   // first token of this warp
+            uint32_t r[kTW];
+#pragma unroll
+            for (int l = 0; l < kTW / 32; ++l)
+                if (tok0 + l * 32 < n_tok) tmem_ld_32x32(acc_t + tok0 + l * 32, *reinterpret_cast<uint32_t (*)[32]>(&r[l * 32]));
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
+            if (p.y_bf16) {
+                // 16 tokens x 32 features x 2 bytes fill the warp's 1 KB staging tile
+#pragma unroll
+                for (int cc = 0; cc < kTW / 16; ++cc) {
+                    const int c0 = tok0 + cc * 16;              // first token of the chunk
+                    if (c0 >= n_tok) break;
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const __nv_bfloat16 h = __float2bfloat16_rn(__uint_as_float(r[i]));
+                        const __nv_bfloat16 h = __float2bfloat16_rn(__uint_as_float(r[cc * 16 + i]));
                         asm volatile("st.shared.u16 [%0], %1;" ::"r"(stg + i * 64 + lane * 2), "h"(*reinterpret_cast<const uint16_t*>(&h)) : "memory");
                     }
                     __syncwarp();
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
-                        const int tok = c * 16 + j * 8 + (lane >> 2), col = nw + (lane & 3) * 8;
+                        const int tok = c0 + j * 8 + (lane >> 2), col = nw + (lane & 3) * 8;
                         uint4 v;
                         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg + j * 512 + lane * 16));
                         if (tok < n_tok && col < p.N) {
@@ -405,14 +418,21 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                             }
                         }
                     }
-                } else {
+                    __syncwarp();   // the tile is read before the next chunk overwrites it
+                }
+            } else {
+                // 8 tokens x 32 features x 4 bytes
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + i * 128 + lane * 4), "r"(r[i]) : "memory");
+                for (int cc = 0; cc < kTW / 8; ++cc) {
+                    const int c0 = tok0 + cc * 8;
+                    if (c0 >= n_tok) break;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(stg + i * 128 + lane * 4), "r"(r[cc * 8 + i]) : "memory");
                     __syncwarp();
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int tok = c * 16 + j * 4 + (lane >> 3), col = nw + (lane & 7) * 4;
+                    for (int j = 0; j < 2; ++j) {
+                        const int tok = c0 + j * 4 + (lane >> 3), col = nw + (lane & 7) * 4;
                         uint4 v;
                         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(stg + j * 512 + lane * 16));
                         if (tok < n_tok && col < p.N) {
@@ -424,13 +444,9 @@ gemm_grouped_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
                             }
                         }
                     }
+                    __syncwarp();
                 }
-                __syncwarp();   // the tile is read before the next chunk overwrites it
             }
-            // hand the accumulator back to the MMA issuer
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
             if (trace && et == 0 && acc_it < 8) trace[193 + 2 * acc_it] = clock64();
         }
     }
@@ -453,7 +469,7 @@ template <bool kFp8, int BN>
 cudaError_t launch_grouped_impl(const CUtensorMap& tm_act, const CUtensorMap& tm_w, const GemmParams& p, int grid,
                                 cudaStream_t stream) {
     using C = Cfg<kFp8, BN>;
-    constexpr int smem = C::kStages * C::kStageBytes + 1024 + C::kEpiWarps * 2048;  // + store staging
+    constexpr int smem = C::kStages * C::kStageBytes + 1024 + C::kEpiWarps * C::kStagingBytes;  // + store staging
     static bool configured = false;  // the attribute is per function, setting it twice is harmless
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemm_grouped_kernel<kFp8, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
