@@ -906,6 +906,10 @@ prq_status prq_quantize_act(const prq_weights* w, prq_act_mode mode, const void*
     p.codes = static_cast<uint8_t*>(codes);
     p.scales_row = static_cast<uint8_t*>(scales_row);
     p.scales_sf = static_cast<uint8_t*>(scales_sf);
+    DeviceInfo* di;
+    prq_status st = device_info(w->device, &di);
+    if (st != PRQ_OK) return st;
+    p.status = di->status_ptr;
     cudaError_t e = launch_quant_act(p, mode == PRQ_ACT_SCALE_PERM, p.act_groups, static_cast<cudaStream_t>(stream));
     g_launches.fetch_add(1);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;
@@ -936,6 +940,10 @@ prq_status prq_quantize_act_multi(int n, const prq_weights* const* ws, prq_act_m
     for (int i = 0; i < n; ++i)
         b.lay[i] = QuantLayer{ws[i]->d_perm, ws[i]->d_inv_s_perm, static_cast<uint8_t*>(codes[i]), nullptr,
                               static_cast<uint8_t*>(scales_sf[i]), ws[i]->k_tail};
+    DeviceInfo* di;
+    prq_status st = device_info(ws[0]->device, &di);
+    if (st != PRQ_OK) return st;
+    b.status = di->status_ptr;
     cudaError_t e = launch_quant_act_batch(b, mode == PRQ_ACT_SCALE_PERM, static_cast<cudaStream_t>(stream));
     g_launches.fetch_add(1);
     return e == cudaSuccess ? PRQ_OK : PRQ_ERR_CUDA;

@@ -29,6 +29,7 @@ struct QuantParams {
     uint8_t* codes;          // M x K/2
     uint8_t* scales_row;     // M x K/32 or nullptr
     uint8_t* scales_sf;      // S x act_groups x 1024
+    int* status;             // device status word (a bounded wait that ran out is recorded there)
 };
 
 cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_groups, cudaStream_t stream);
@@ -57,6 +58,7 @@ struct QuantBatch {
     int n_atoms, n_tail, tail_split;     // set by the launcher: 128-column atoms, how many of them are tail atoms
                                          // (scale + permute mode), and into how many row shares each of those is cut
     QuantLayer lay[kMaxBatch];
+    int* status;                         // device status word
 };
 cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStream_t stream);
 

@@ -12,6 +12,11 @@
 // permute mode keeps 8 elements per lane and 4 lanes per block.)  The atom's scale bytes are collected in shared memory and
 // written out as one coalesced 512-byte piece; the bytes of tail blocks are also duplicated into the
 // residual stages, which is all the "tail copy" this design needs (the GEMM re-reads the tail codes).
+//
+// The scale + permute mode has two structures.  From 512 rows on (and while two slices of rows fit shared memory)
+// quant_act_rows_kernel runs: persistent CTAs that bring whole rows into shared memory by bulk copies and gather
+// from there (see that kernel).  Smaller batches keep the column-atom CTAs of quant_act_kernel, whose rows can be
+// cut into parts so that a few rows still fill the GPU.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -206,9 +211,7 @@ quant_act_kernel(const QuantBatch b) {
     } else {
         // ---- scale + permute: gathered 2-byte loads (the head of the permutation is nearly the identity,
         // so they coalesce), multiply by the stored reciprocal scale in fp32.  The loads of four steps
-        // (32 per lane) are issued before any arithmetic.  (Fetching each row's source window with
-        // 16-byte loads and gathering from shared memory was no faster: this mode is bound by its fp32
-        // arithmetic, not by the gathers.) ----
+        // (32 per lane) are issued before any arithmetic. ----
         // Everything that does not depend on the row is computed once: per-lane pointers that advance by
         // a fixed stride per 16-row step, the lane's slot in the residual stages, and -- for lanes past K --
         // zero sources and factors so that the arithmetic below needs no per-element select.
@@ -302,6 +305,260 @@ quant_act_kernel(const QuantBatch b) {
     }
 }
 
+
+// ---------------------------------------------------------------------------------------------------------
+// Scale + permute mode, second structure: whole rows through shared memory.  A persistent CTA takes slices of
+// kRowsR rows; the rows of the next slice arrive by bulk copies (one per row, no instruction per element) while
+// the current slice is quantised, and every gather of the permutation is a shared-memory read.  The lanes of a
+// warp are 8 different rows reading the SAME source column (for 4 blocks side by side): the rows are 16 bytes
+// further apart than a multiple of 128 bytes, so the 8 rows fall into different banks and a gather costs about
+// one pass however scattered the permutation is -- against one 32-byte sector per 2-byte read when the tail of
+// the permutation is gathered from global memory -- and the column's index and reciprocal scale are the same for
+// all rows, so they come as 16-byte broadcast loads, four columns at a time, instead of living in registers per
+// lane.  A lane takes one row of one block: 32 values held in registers (no shuffle), 16 bytes of codes and one
+// scale byte.  The scale bytes of the slice are collected in shared memory and then written out in every place
+// the GEMM reads them (main stages, duplicated tail bytes in the residual stages, zeros for rows and blocks that
+// do not exist) and, if asked for, row-major.  Several layers that read the same activation are quantised from
+// the one copy of the rows.
+constexpr int kRowsThreads = 256;
+constexpr int kRowsR = 8;                        // rows per slice
+static_assert(32 / kRowsR == 4, "a warp is 8 rows x the 4 blocks of an atom");
+constexpr int kRowsSlices = kGroupRows / kRowsR; // slices per 128-row group
+
+__global__ void __launch_bounds__(kRowsThreads, 2)
+quant_act_rows_kernel(const QuantBatch b, int n_slices) {
+    extern __shared__ __align__(16) uint8_t rows_smem_raw[];
+    // 256-byte aligned in the shared address space (the records are addressed with XORs)
+    uint8_t* const rows_smem = rows_smem_raw + ((256u - (smem_u32(rows_smem_raw) & 255u)) & 255u);
+    __shared__ int s_tile_start[kMaxExperts + 1];
+    __shared__ __align__(8) uint64_t bar_rows[2];
+    __shared__ int abort_flag_s;
+    volatile int* abort_flag = &abort_flag_s;
+    grid_launch_dependents();
+    const int K = b.K, nblk = K / kBlock;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t row_bytes = K * 2 + 16;       // staged row: 16 bytes past a multiple of 128
+    const uint32_t buf_bytes = kRowsR * row_bytes;
+    // per pair of destination columns: {byte offsets of the two source columns in a staged row, their two
+    // reciprocal scales}; the records come first so that a block's sixteen are 256 aligned bytes
+    uint4* rec = reinterpret_cast<uint4*>(rows_smem);
+    const uint32_t rec_base = smem_u32(rows_smem);
+    uint8_t* const rows_buf = rows_smem + (K / 2) * 16;
+    uint8_t* sfb = rows_buf + 2 * buf_bytes;     // 2 x [kRowsR][K / 32]: the tail blocks' scale bytes, per slice parity
+    int rec_lin = -1, rec_expert = -1;           // which layer's constants the records hold
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar_rows[0]), 1);
+        mbar_init(smem_u32(&bar_rows[1]), 1);
+        abort_flag_s = 0;
+        fence_mbar_init();
+    }
+
+    // The layer's (expert's) permutation and reciprocal scales as one 16-byte record per column pair, so that a
+    // lane fetches them with one shared-memory read (the same for all rows of a warp).  The loads of four records
+    // are in flight together: the build is in front of the first slice.
+    auto build_records = [&](int lin, int expert) {
+        const int2* perm2 = reinterpret_cast<const int2*>(b.lay[lin].perm + static_cast<size_t>(expert) * K);
+        const float2* inv2 = reinterpret_cast<const float2*>(b.lay[lin].inv_s_perm + static_cast<size_t>(expert) * K);
+#pragma unroll 1
+        for (int c0 = threadIdx.x; c0 < K / 2; c0 += 4 * kRowsThreads) {
+            int2 p2[4];
+            float2 s2[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int c2 = c0 + i * kRowsThreads;
+                if (c2 < K / 2) { p2[i] = __ldg(perm2 + c2); s2[i] = __ldg(inv2 + c2); }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int c2 = c0 + i * kRowsThreads;
+                if (c2 < K / 2)
+                    rec[c2] = make_uint4(static_cast<uint32_t>(p2[i].x) * 2, static_cast<uint32_t>(p2[i].y) * 2,
+                                         __float_as_uint(s2[i].x), __float_as_uint(s2[i].y));
+            }
+        }
+        rec_lin = lin; rec_expert = expert;
+    };
+    const bool dense = b.expert_offsets == nullptr;
+    // a dense layer's constants belong to the prepared weights, not to an earlier kernel of the stream: fetch them
+    // while that kernel may still be running
+    if (dense) build_records(0, 0);
+    grid_dependency_wait();
+    if (!dense && threadIdx.x < 32) warp_expert_starts(b.expert_offsets, b.n_experts, kGroupRows, s_tile_start, nullptr);
+    __syncthreads();
+    const int n_groups = dense ? b.groups_per_lin : s_tile_start[b.n_experts];
+
+    // where a slice sits: its group, its first row (in x) and how many of its rows exist
+    struct Slice { int group, expert, r_first, row0, n_rows; };
+    auto slice_at = [&](int sl) {
+        Slice t;
+        t.group = sl / kRowsSlices; t.r_first = (sl % kRowsSlices) * kRowsR; t.expert = 0;
+        int g_row0, g_end;
+        if (dense) {
+            g_row0 = t.group * kGroupRows; g_end = min(b.M, g_row0 + kGroupRows);
+        } else if (t.group >= n_groups) {   // padding of the launch grid
+            g_row0 = 0; g_end = 0;
+        } else {
+            int lo = 0, hi = b.n_experts - 1;
+            while (lo < hi) {  // last expert whose first group is <= group
+                const int mid = (lo + hi + 1) >> 1;
+                if (s_tile_start[mid] <= t.group) lo = mid; else hi = mid - 1;
+            }
+            t.expert = lo;
+            g_row0 = b.expert_offsets[lo] + (t.group - s_tile_start[lo]) * kGroupRows;
+            g_end = min(b.expert_offsets[lo + 1], g_row0 + kGroupRows);
+        }
+        t.row0 = g_row0 + t.r_first;
+        t.n_rows = max(0, min(kRowsR, g_end - t.row0));
+        return t;
+    };
+    auto request = [&](const Slice& t, int buf) {   // one thread
+        if (t.n_rows == 0) return;
+        const uint32_t bar = smem_u32(&bar_rows[buf]);
+        mbar_arrive_expect_tx(bar, t.n_rows * K * 2);
+        for (int r = 0; r < t.n_rows; ++r)
+            bulk_load(smem_u32(rows_buf + buf * buf_bytes + r * row_bytes), b.x + static_cast<size_t>(t.row0 + r) * b.ldx, K * 2, bar);
+    };
+
+    const int rl = lane % kRowsR, side = lane / kRowsR;
+    const uint32_t byte_sel = side == 0 ? 0x3210u : side == 1 ? 0x2301u : side == 2 ? 0x1032u : 0x0123u;
+    const size_t sf_stage_stride = static_cast<size_t>(b.act_groups) * kSfGroupBytes;
+    uint32_t phase[2] = {0, 0};
+    int sl = blockIdx.x;
+    Slice cur = slice_at(sl < n_slices ? sl : 0);
+    if (sl < n_slices && threadIdx.x == 0) request(cur, 0);
+    for (int it = 0; sl < n_slices; ++it, sl += gridDim.x) {
+        const int buf = it & 1;
+        const int sl_next = sl + gridDim.x;
+        Slice nxt = cur;
+        if (sl_next < n_slices) {
+            nxt = slice_at(sl_next);
+            if (threadIdx.x == 0) request(nxt, buf ^ 1);   // that buffer's readers passed the barrier of their slice
+        }
+        if (!dense && cur.group >= n_groups) { cur = nxt; continue; }
+        if (cur.n_rows > 0) {
+            if (!mbar_wait(smem_u32(&bar_rows[buf]), phase[buf], abort_flag)) break;
+            phase[buf] ^= 1;
+        }
+        const bool row_ok = rl < cur.n_rows;
+        const uint32_t xrow_a = smem_u32(rows_buf + buf * buf_bytes + rl * row_bytes);
+        const size_t row = static_cast<size_t>(cur.row0 + rl);
+        const int g = cur.r_first + rl;                        // row inside its 128-row group
+        const int sf_row_off = (g & 31) * 16 + (g >> 5) * 4;
+        uint8_t* tailb = sfb + (it & 1) * (kRowsR * nblk);     // [kRowsR][tail blocks] of this slice
+        for (int lin = 0; lin < b.n_lin; ++lin) {
+            const QuantLayer& l = b.lay[lin];
+            if (rec_lin != lin || rec_expert != cur.expert) {
+                if (rec_lin >= 0) __syncthreads();             // the old records are still being read
+                build_records(lin, cur.expert);
+                __syncthreads();
+            }
+            const StagePlan plan(K, l.k_tail);
+            const int tail_blk0 = (K - l.k_tail) / kBlock, n_tail_blk = l.k_tail / kBlock;
+            uint8_t* sf_group = l.scales_sf + static_cast<size_t>(cur.group) * kSfGroupBytes;
+            uint8_t* crow = l.codes + row * (K / 2);
+            // A warp takes whole 128-column atoms, its four sides one block each: the four scale bytes of
+            // (row, atom) meet by two shuffles and go out as the one word the GEMM's layout has for them.  Rows
+            // and blocks that do not exist contribute zero bytes (an odd atom count leaves half a stage of them).
+#pragma unroll 1
+            for (int a = warp; a < 2 * plan.S1; a += kRowsThreads / 32) {
+                const int blk = a * 4 + side;
+                const int j0 = blk * kBlock;
+                uint32_t byte = 0;
+                if (row_ok && blk < nblk) {
+                    // At step t a lane visits the block's column pair t ^ side: where the permutation is (nearly)
+                    // the identity, the four blocks side by side would otherwise read the same banks.  (A block's
+                    // records are 256 aligned bytes, so the exchange is one XOR on the address.)
+                    const uint32_t rec_blk = rec_base + (blk * 256 ^ (side << 4));
+                    float v[32];
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) {
+                        uint4 rc;
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(rc.x), "=r"(rc.y), "=r"(rc.z), "=r"(rc.w) : "r"(rec_blk ^ (t << 4)));
+                        uint16_t x0, x1;
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(x0) : "r"(xrow_a + rc.x));
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=h"(x1) : "r"(xrow_a + rc.y));
+                        v[2 * t] = __uint_as_float(static_cast<uint32_t>(x0) << 16) * __uint_as_float(rc.z);
+                        v[2 * t + 1] = __uint_as_float(static_cast<uint32_t>(x1) << 16) * __uint_as_float(rc.w);
+                    }
+                    float am;
+                    {
+                        float m[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            m[i] = fmaxf(fmaxf(fabsf(v[4 * i]), fabsf(v[4 * i + 1])), fmaxf(fabsf(v[4 * i + 2]), fabsf(v[4 * i + 3])));
+                        am = fmaxf(fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3])), fmaxf(fmaxf(m[4], m[5]), fmaxf(m[6], m[7])));
+                    }
+                    byte = scale_byte(__float_as_uint(am));
+                    const float inv = __uint_as_float((254u - byte) << 23);  // 2^(127 - byte), exact multiply
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int h = 0; h < 4; ++h)
+                        pk[h] = cvt_e2m1x8(v[8 * h] * inv, v[8 * h + 1] * inv, v[8 * h + 2] * inv, v[8 * h + 3] * inv,
+                                           v[8 * h + 4] * inv, v[8 * h + 5] * inv, v[8 * h + 6] * inv, v[8 * h + 7] * inv);
+                    // byte t of pk holds pair t ^ side: exchange the bytes inside every word accordingly
+                    *reinterpret_cast<uint4*>(crow + j0 / 2) =
+                        make_uint4(__byte_perm(pk[0], 0, byte_sel), __byte_perm(pk[1], 0, byte_sel),
+                                   __byte_perm(pk[2], 0, byte_sel), __byte_perm(pk[3], 0, byte_sel));
+                    if (l.scales_row) l.scales_row[row * nblk + blk] = static_cast<uint8_t>(byte);
+                    if (blk >= tail_blk0) tailb[rl * nblk + blk - tail_blk0] = static_cast<uint8_t>(byte);
+                }
+                uint32_t w = byte << (8 * side);
+                w |= __shfl_xor_sync(0xffffffffu, w, 8);
+                w |= __shfl_xor_sync(0xffffffffu, w, 16);
+                if (side == 0)
+                    *reinterpret_cast<uint32_t*>(sf_group + (a >> 1) * sf_stage_stride + (a & 1) * 512 + sf_row_off) = w;
+            }
+            // every warp is through with this slice's rows (their buffer may be refilled from now on) and the tail's
+            // bytes are in shared memory
+            __syncthreads();
+            if (n_tail_blk > 0) {
+                // the tail's bytes once more, where the residual stages read them (zeros past the tail and the rows)
+                for (int idx = threadIdx.x; idx < kRowsR * (plan.S - plan.S1) * 2; idx += kRowsThreads) {
+                    const int r = idx % kRowsR, sa = idx / kRowsR, ts = sa >> 1, ah = sa & 1;
+                    const int t0 = ts * 8 + ah * 4;
+                    uint32_t w = 0;
+                    if (r < cur.n_rows) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            if (t0 + i < n_tail_blk) w |= static_cast<uint32_t>(tailb[r * nblk + t0 + i]) << (8 * i);
+                    }
+                    const int gr = cur.r_first + r;
+                    *reinterpret_cast<uint32_t*>(sf_group + (plan.S1 + ts) * sf_stage_stride + ah * 512 + (gr & 31) * 16 + (gr >> 5) * 4) = w;
+                }
+            }
+        }
+        cur = nxt;
+    }
+    if (abort_flag_s) {
+        // copies may still be on their way into this CTA's shared memory: give them one more bounded wait
+        mbar_wait_after_abort(smem_u32(&bar_rows[0]), phase[0]);
+        mbar_wait_after_abort(smem_u32(&bar_rows[1]), phase[1]);
+        if (threadIdx.x == 0 && b.status) atomicExch(b.status, static_cast<int>(PRQ_ERR_TIMEOUT));
+    }
+}
+
+cudaError_t launch_rows_impl(const QuantBatch& b, size_t smem, int sm_count, cudaStream_t stream) {
+    static size_t configured = 0;   // the attribute is per function; raise it when a larger K comes
+    if (smem > configured) {
+        cudaError_t e = cudaFuncSetAttribute(quant_act_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
+        configured = smem;
+    }
+    const int n_slices = b.groups_per_lin * kRowsSlices;
+    const int per_sm = smem + 8192 <= 113 * 1024 ? 2 : 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_slices < per_sm * sm_count ? n_slices : per_sm * sm_count);
+    cfg.blockDim = dim3(kRowsThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, quant_act_rows_kernel, b, n_slices);
+}
+
 }  // namespace
 
 cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStream_t stream) {
@@ -325,6 +582,17 @@ cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStr
         while (parts < 4 && tiles * parts < 8LL * sm_count[dev]) parts *= 2;   // 3 CTAs per SM: keep the last wave short
         if (parts == 4 && tiles * parts < 4LL * sm_count[dev]) parts = 8;
         if (const char* ev = dev_knobs_enabled() ? getenv("PRQ_QUANT_PARTS") : nullptr) { const int v = atoi(ev); if (v == 1 || v == 2 || v == 4 || v == 8) parts = v; }
+        // Whole rows through shared memory when there are rows enough to fill the GPU that way, a slice's rows fit
+        // twice, and the rows can be fetched by bulk copies (16-byte aligned).
+        int rows = b.M >= 512 ? 1 : 0;
+        if (const char* ev = dev_knobs_enabled() ? getenv("PRQ_QUANT_ROWS") : nullptr) rows = atoi(ev);
+        const size_t smem = 2 * static_cast<size_t>(kRowsR) * (p.K * 2 + 16) + static_cast<size_t>(p.K) * 8 +
+                            2 * static_cast<size_t>(kRowsR) * (p.K / 32) + 256;   // + alignment slack
+        if (rows && smem <= 200 * 1024 && (reinterpret_cast<uintptr_t>(b.x) & 15) == 0 && b.ldx % 8 == 0) {
+            QuantBatch br = b;
+            br.n_atoms = n_atoms; br.n_tail = 0; br.tail_split = 1;
+            return launch_rows_impl(br, smem, sm_count[dev], stream);
+        }
     }
     // the tail atoms of the scale + permute mode in shares of 16 rows (128 / 8), see the kernel
     QuantBatch bb = b;
@@ -361,6 +629,7 @@ cudaError_t launch_quant_act(const QuantParams& p, bool scale_perm, int grid_gro
     b.n_lin = 1;
     b.groups_per_lin = grid_groups;
     b.lay[0] = QuantLayer{p.perm, p.inv_s_perm, p.codes, p.scales_row, p.scales_sf, p.k_tail};
+    b.status = p.status;
     return launch_quant_act_batch(b, scale_perm, stream);
 }
 

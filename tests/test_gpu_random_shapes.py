@@ -157,3 +157,84 @@ def test_prefill_tile_widths_against_oracle(prq, oracle, monkeypatch, bn, seed):
         slack = np.abs(y_ref).max() * 2.0 ** -7 if dt == prq.BF16 else 0.0
         assert np.abs(got - y_ref).max() <= prq_ref.tolerance(y_ref) + slack, what
         w.free()
+
+
+@pytest.mark.parametrize("rows", [0, 1])
+def test_permuting_quantiser_structures_against_oracle(prq, oracle, monkeypatch, rows):
+    """The two structures of the scale + permute quantiser (column atoms per CTA; whole rows through shared memory),
+    each forced on the same shapes: row counts that leave a ragged last slice and a ragged last group, K with a
+    partial last atom and an odd block count, tails that straddle atoms, strided x, several layers from one
+    activation, and stacked experts with empty ones."""
+    monkeypatch.setenv("PRQ_QUANT_ROWS", str(rows))
+    rng = np.random.default_rng(77)
+    for case, (M, K, k) in enumerate([(513, 96, 32), (700, 736, 160), (1029, 2560, 256), (130, 160, 0), (5, 2560, 128),
+                                      (640, 4096, 96), (1100, 32, 32)]):
+        what = f"structure {rows} case {case}: M={M} K={K} k={k}"
+        ch = synth.HeavyTailChannels(500 + case, K)
+        amax = oracle.channel_amax(ch.rows(600 + case, 32))
+        ws, os_ = [], []
+        for j in range(3):
+            W = synth.weights(700 + 10 * case + j, 64, K)
+            kj = max(0, k - 32 * j)
+            am = (amax * (1.0 + 0.25 * j)).astype(np.float32)
+            ws.append(prq.prepare_weights(W, am, 0.5, kj))
+            os_.append(oracle.prepare(W, am, 0.5, kj))
+        x = ch.rows(800 + case, M)
+        ldx = K + 8 * int(rng.integers(0, 3))
+        xs = torch.zeros((M, ldx), dtype=torch.bfloat16, device="cuda")
+        xs[:, :K] = dev_bf16(x)
+        # one layer, with row-major scales
+        codes, srow, sf = prq.quantize_act(ws[0], xs[:, :K], prq.ACT_SCALE_PERM, row_scales=True)
+        assert prq.last_device_status() == 0, what
+        oc, osc = oracle.quantize_act(x, os_[0]["perm"], os_[0]["inv_s"])
+        assert np.array_equal(codes.cpu().numpy()[: M * K // 2].reshape(M, K // 2), oc), what
+        assert np.array_equal(srow.cpu().numpy()[: M * K // 32].reshape(M, K // 32), osc), what
+        _, sa = oracle.augment_act(oc, osc, ws[0].k_tail)
+        want = prq_ref.expected_sf(sa, K, ws[0].k_tail)
+        assert np.array_equal(sf.cpu().numpy()[: want.size], want), what
+        # three layers from the one activation
+        acts = prq.quantize_act_multi(ws, xs[:, :K], prq.ACT_SCALE_PERM)
+        assert prq.last_device_status() == 0, what
+        for j in range(3):
+            oc, osc = oracle.quantize_act(x, os_[j]["perm"], os_[j]["inv_s"])
+            assert np.array_equal(acts[j][0].cpu().numpy()[: M * K // 2].reshape(M, K // 2), oc), (what, j)
+            _, sa = oracle.augment_act(oc, osc, ws[j].k_tail)
+            want = prq_ref.expected_sf(sa, K, ws[j].k_tail)
+            assert np.array_equal(acts[j][1].cpu().numpy()[: want.size], want), (what, j)
+        for w in ws:
+            w.free()
+    # stacked experts
+    for case, (E, K, k, counts) in enumerate([(5, 768, 64, [300, 0, 7, 129, 128]), (3, 160, 32, [0, 600, 1]),
+                                              (16, 96, 0, [40] * 16)]):
+        what = f"structure {rows} grouped case {case}"
+        offsets = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+        M = int(offsets[-1])
+        ch = synth.HeavyTailChannels(900 + case, K)
+        Ws = np.stack([synth.weights(910 + 20 * case + e, 32, K) for e in range(E)])
+        amax = np.stack([oracle.channel_amax(ch.rows(950 + 20 * case + e, 32)) for e in range(E)])
+        w = prq.prepare_weights(Ws, amax, 0.5, k)
+        x = ch.rows(990 + case, M)
+        d_off = torch.from_numpy(offsets).cuda()
+        codes, srow, sf = prq.quantize_act(w, dev_bf16(x), prq.ACT_SCALE_PERM, expert_offsets=d_off, row_scales=True)
+        assert prq.last_device_status() == 0, what
+        got_c = codes.cpu().numpy()[: M * K // 2].reshape(M, K // 2)
+        got_s = srow.cpu().numpy()[: M * K // 32].reshape(M, K // 32)
+        sa_all = np.zeros((M, (K + k) // 32), np.uint8)
+        row_group = np.zeros(M, np.int64)
+        row_in_group = np.zeros(M, np.int64)
+        g0 = 0
+        for e in range(E):
+            r0, r1 = int(offsets[e]), int(offsets[e + 1])
+            if r1 > r0:
+                o = oracle.prepare(Ws[e], amax[e], float(np.float32(0.5)), k)
+                oc, osc = oracle.quantize_act(x[r0:r1], o["perm"], o["inv_s"])
+                assert np.array_equal(got_c[r0:r1], oc) and np.array_equal(got_s[r0:r1], osc), (what, e)
+                _, sa_all[r0:r1] = oracle.augment_act(oc, osc, k)
+                row_group[r0:r1] = g0 + np.arange(r1 - r0) // 128
+                row_in_group[r0:r1] = np.arange(r1 - r0) % 128
+            g0 += (r1 - r0 + 127) // 128
+        groups = int(prq.act_bytes(M, K, k, E, prq.BUF_SCALES_SF)) // (1024 * prq_ref.stages(K, k)[1])
+        want = prq_ref.expected_sf(sa_all, K, k, groups=groups, row_group=row_group, row_in_group=row_in_group)
+        got = sf.cpu().numpy()[: want.size].reshape(-1, groups, 1024)[:, :g0]
+        assert np.array_equal(got, want.reshape(-1, groups, 1024)[:, :g0]), what
+        w.free()
