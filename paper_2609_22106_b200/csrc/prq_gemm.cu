@@ -3,20 +3,24 @@
 // with a = E2M1 codes of [Q(x) | Q(x)_tail] and w = E2M1 codes of [Q(W D P) | Q(R)] of the expert that
 // owns token row t (rows sorted by expert, boundaries in expert_offsets).
 //
-// sm_100a design.  One persistent CTA per SM, 10 warps:
-//   warp 0  producer: per 256-element reduction stage, one TMA tile load per operand (128-byte rows,
+// sm_100a design.  One persistent CTA per SM, 12 warps:
+//   warps 0, 2  producers: per 256-element reduction stage, one TMA tile load per operand (128-byte rows,
 //           128B swizzle) and one flat bulk copy per operand for the stage's scale bytes, all landing
 //           on the stage's "full" mbarrier;
-//   warp 1  MMA issuer: copies the stage's scale atoms shared -> tensor memory (tcgen05.cp), then issues
+//   warps 1, 3  MMA issuers: copy the stage's scale atoms shared -> tensor memory (tcgen05.cp), then issue
 //           up to four K = 64 tcgen05.mma.kind::mxf4.block_scale steps into a tensor-memory accumulator
-//           and commits to the stage's "empty" mbarrier; after the last stage commits "accumulator full";
-//   warps 2-9 epilogue: tcgen05.ld of their 32-lane quarter, store to y, release the accumulator.
+//           and commit to the stage's "empty" mbarrier; after the last stage commit "accumulator full";
+//           (warps 0 + 1 and 2 + 3 are two pairs, each with its own ring of stage slots, scale columns and
+//           accumulator, taking alternate units of the CTA)
+//   warps 4-11 epilogue: tcgen05.ld of their 32-lane quarter, store to y, release the accumulator.
+// A unit is 128 output features x one token tile of an expert: 128 tokens, or 64 when the experts hold few
+// tokens each (the smaller tile buys a deeper ring).
 // The augmented activation is never materialised: in the residual stages the activation tile is loaded
 // again from column K - k while the weight tile continues at column K (the Kernel design paragraph's point
 // that the tail is quantised once and used twice); only the tail's scale bytes were duplicated.
 //
 // Operand roles.  "P" is the operand on the MMA M axis: 128 output features of one expert.  "Q" is the
-// operand on the MMA N axis: one 128-token group of that expert.  With the features on M, the lanes of a
+// operand on the MMA N axis: one token tile of that expert.  With the features on M, the lanes of a
 // warp hold consecutive features of one token, stores are contiguous per token, and an expert with few
 // tokens costs few stores.  (Dense layers have kernels of their own: prq_gemm_decode.cu for M <= 128,
 // prq_gemm_prefill_pair.cu above.)
