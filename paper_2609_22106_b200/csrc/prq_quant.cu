@@ -320,12 +320,13 @@ quant_act_kernel(const QuantBatch b) {
 // the GEMM reads them (main stages, duplicated tail bytes in the residual stages, zeros for rows and blocks that
 // do not exist) and, if asked for, row-major.  Several layers that read the same activation are quantised from
 // the one copy of the rows.
-constexpr int kRowsThreads = 256;
+// threads per CTA: 256 where two CTAs share an SM, 512 where the rows of a wide layer leave room for one only
 constexpr int kRowsR = 8;                        // rows per slice
 static_assert(32 / kRowsR == 4, "a warp is 8 rows x the 4 blocks of an atom");
 constexpr int kRowsSlices = kGroupRows / kRowsR; // slices per 128-row group
 
-__global__ void __launch_bounds__(kRowsThreads, 2)
+template <int kRowsThreads>
+__global__ void __launch_bounds__(kRowsThreads, 512 / kRowsThreads)
 quant_act_rows_kernel(const QuantBatch b, int n_slices) {
     extern __shared__ __align__(16) uint8_t rows_smem_raw[];
     // 256-byte aligned in the shared address space (the records are addressed with XORs)
@@ -540,15 +541,17 @@ quant_act_rows_kernel(const QuantBatch b, int n_slices) {
     }
 }
 
+template <int kRowsThreads>
 cudaError_t launch_rows_impl(const QuantBatch& b, size_t smem, int sm_count, cudaStream_t stream) {
     static size_t configured = 0;   // the attribute is per function; raise it when a larger K comes
     if (smem > configured) {
-        cudaError_t e = cudaFuncSetAttribute(quant_act_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        cudaError_t e = cudaFuncSetAttribute(quant_act_rows_kernel<kRowsThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
         if (e != cudaSuccess) return e;
         configured = smem;
     }
     const int n_slices = b.groups_per_lin * kRowsSlices;
-    const int per_sm = smem + 8192 <= 113 * 1024 ? 2 : 1;
+    const int per_sm = 512 / kRowsThreads;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(n_slices < per_sm * sm_count ? n_slices : per_sm * sm_count);
     cfg.blockDim = dim3(kRowsThreads);
@@ -559,7 +562,7 @@ cudaError_t launch_rows_impl(const QuantBatch& b, size_t smem, int sm_count, cud
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, quant_act_rows_kernel, b, n_slices);
+    return cudaLaunchKernelEx(&cfg, quant_act_rows_kernel<kRowsThreads>, b, n_slices);
 }
 
 }  // namespace
@@ -596,7 +599,9 @@ cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStr
         if (rows && smem <= 200 * 1024 && (reinterpret_cast<uintptr_t>(b.x) & 15) == 0 && b.ldx % 8 == 0) {
             QuantBatch br = b;
             br.n_atoms = n_atoms; br.n_tail = 0; br.tail_split = 1;
-            return launch_rows_impl(br, smem, sm_count[dev], stream);
+            // (4.6 KB of static shared memory and 1 KB reserved per CTA beside the dynamic part)
+            return 2 * (smem + 6 * 1024) <= 227 * 1024 ? launch_rows_impl<256>(br, smem, sm_count[dev], stream)
+                                                       : launch_rows_impl<512>(br, smem, sm_count[dev], stream);
         }
     }
     // the tail atoms of the scale + permute mode in shares of 16 rows (128 / 8), see the kernel
