@@ -322,17 +322,19 @@ quant_act_kernel(const QuantBatch b) {
 // the one copy of the rows.
 // threads per CTA: 256 where two CTAs share an SM, 512 where the rows of a wide layer leave room for one only
 constexpr int kRowsR = 8;                        // rows per slice
+constexpr int kRowsMaxBufs = 8;                  // slices of rows in shared memory at most (at least 2)
 static_assert(32 / kRowsR == 4, "a warp is 8 rows x the 4 blocks of an atom");
 constexpr int kRowsSlices = kGroupRows / kRowsR; // slices per 128-row group
 
 template <int kRowsThreads>
 __global__ void __launch_bounds__(kRowsThreads, 512 / kRowsThreads)
-quant_act_rows_kernel(const QuantBatch b, int n_slices) {
+quant_act_rows_kernel(const QuantBatch b, int n_slices, int n_buf) {
     extern __shared__ __align__(16) uint8_t rows_smem_raw[];
     // 256-byte aligned in the shared address space (the records are addressed with XORs)
     uint8_t* const rows_smem = rows_smem_raw + ((256u - (smem_u32(rows_smem_raw) & 255u)) & 255u);
     __shared__ int s_tile_start[kMaxExperts + 1];
-    __shared__ __align__(8) uint64_t bar_rows[2];
+    __shared__ int s_row_start[kMaxExperts + 1];
+    __shared__ __align__(8) uint64_t bar_rows[kRowsMaxBufs];
     __shared__ int abort_flag_s;
     volatile int* abort_flag = &abort_flag_s;
     grid_launch_dependents();
@@ -345,11 +347,10 @@ quant_act_rows_kernel(const QuantBatch b, int n_slices) {
     uint4* rec = reinterpret_cast<uint4*>(rows_smem);
     const uint32_t rec_base = smem_u32(rows_smem);
     uint8_t* const rows_buf = rows_smem + (K / 2) * 16;
-    uint8_t* sfb = rows_buf + 2 * buf_bytes;     // 2 x [kRowsR][K / 32]: the tail blocks' scale bytes, per slice parity
+    uint8_t* sfb = rows_buf + n_buf * buf_bytes;     // 2 x [kRowsR][K / 32]: the tail blocks' scale bytes, per slice parity
     int rec_lin = -1, rec_expert = -1;           // which layer's constants the records hold
     if (threadIdx.x == 0) {
-        mbar_init(smem_u32(&bar_rows[0]), 1);
-        mbar_init(smem_u32(&bar_rows[1]), 1);
+        for (int i = 0; i < kRowsMaxBufs; ++i) mbar_init(smem_u32(&bar_rows[i]), 1);
         abort_flag_s = 0;
         fence_mbar_init();
     }
@@ -384,7 +385,13 @@ quant_act_rows_kernel(const QuantBatch b, int n_slices) {
     // while that kernel may still be running
     if (dense) build_records(0, 0);
     grid_dependency_wait();
-    if (!dense && threadIdx.x < 32) warp_expert_starts(b.expert_offsets, b.n_experts, kGroupRows, s_tile_start, nullptr);
+    if (!dense) {
+        // the experts' row ranges, once per CTA: every slice looks its expert up, and a dependent global load
+        // there would sit in front of each of them
+        for (int e = threadIdx.x; e <= b.n_experts; e += kRowsThreads) s_row_start[e] = b.expert_offsets[e];
+        __syncthreads();
+        if (threadIdx.x < 32) warp_expert_starts(s_row_start, b.n_experts, kGroupRows, s_tile_start, nullptr);
+    }
     __syncthreads();
     const int n_groups = dense ? b.groups_per_lin : s_tile_start[b.n_experts];
 
@@ -405,8 +412,8 @@ quant_act_rows_kernel(const QuantBatch b, int n_slices) {
                 if (s_tile_start[mid] <= t.group) lo = mid; else hi = mid - 1;
             }
             t.expert = lo;
-            g_row0 = b.expert_offsets[lo] + (t.group - s_tile_start[lo]) * kGroupRows;
-            g_end = min(b.expert_offsets[lo + 1], g_row0 + kGroupRows);
+            g_row0 = s_row_start[lo] + (t.group - s_tile_start[lo]) * kGroupRows;
+            g_end = min(s_row_start[lo + 1], g_row0 + kGroupRows);
         }
         t.row0 = g_row0 + t.r_first;
         t.n_rows = max(0, min(kRowsR, g_end - t.row0));
@@ -423,25 +430,24 @@ quant_act_rows_kernel(const QuantBatch b, int n_slices) {
     const int rl = lane % kRowsR, side = lane / kRowsR;
     const uint32_t byte_sel = side == 0 ? 0x3210u : side == 1 ? 0x2301u : side == 2 ? 0x1032u : 0x0123u;
     const size_t sf_stage_stride = static_cast<size_t>(b.act_groups) * kSfGroupBytes;
-    uint32_t phase[2] = {0, 0};
-    // a CTA's slices are consecutive: with stacked experts its records then change a few times, not per slice
+    uint32_t phases = 0;                         // bit i: parity of buffer i's next completion
+    // a CTA's slices are consecutive: with stacked experts its records then change a few times, not per slice.  The
+    // rows of the next n_buf - 1 slices are on their way while a slice is quantised: a narrow layer's slice is
+    // quantised in a fraction of the time its rows take to arrive.
     const int per_cta = (n_slices + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
     int sl = min(n_slices, static_cast<int>(blockIdx.x) * per_cta);
     const int sl_end = min(n_slices, sl + per_cta);
-    Slice cur = slice_at(sl < sl_end ? sl : 0);
-    if (sl < sl_end && threadIdx.x == 0) request(cur, 0);
+    if (threadIdx.x == 0)
+        for (int d = 0; d < n_buf - 1 && sl + d < sl_end; ++d) request(slice_at(sl + d), d);
     for (int it = 0; sl < sl_end; ++it, ++sl) {
-        const int buf = it & 1;
-        const int sl_next = sl + 1;
-        Slice nxt = cur;
-        if (sl_next < sl_end) {
-            nxt = slice_at(sl_next);
-            if (threadIdx.x == 0) request(nxt, buf ^ 1);   // that buffer's readers passed the barrier of their slice
-        }
-        if (!dense && cur.group >= n_groups) { cur = nxt; continue; }
+        const int buf = it % n_buf;
+        // the buffer of the slice before this one: its readers passed the barrier of their slice
+        if (threadIdx.x == 0 && sl + n_buf - 1 < sl_end) request(slice_at(sl + n_buf - 1), (it + n_buf - 1) % n_buf);
+        const Slice cur = slice_at(sl);
+        if (!dense && cur.group >= n_groups) continue;
         if (cur.n_rows > 0) {
-            if (!mbar_wait(smem_u32(&bar_rows[buf]), phase[buf], abort_flag)) break;
-            phase[buf] ^= 1;
+            if (!mbar_wait(smem_u32(&bar_rows[buf]), (phases >> buf) & 1u, abort_flag)) break;
+            phases ^= 1u << buf;
         }
         const bool row_ok = rl < cur.n_rows;
         const uint32_t xrow_a = smem_u32(rows_buf + buf * buf_bytes + rl * row_bytes);
@@ -531,18 +537,16 @@ quant_act_rows_kernel(const QuantBatch b, int n_slices) {
                 }
             }
         }
-        cur = nxt;
     }
     if (abort_flag_s) {
         // copies may still be on their way into this CTA's shared memory: give them one more bounded wait
-        mbar_wait_after_abort(smem_u32(&bar_rows[0]), phase[0]);
-        mbar_wait_after_abort(smem_u32(&bar_rows[1]), phase[1]);
+        for (int i = 0; i < n_buf; ++i) mbar_wait_after_abort(smem_u32(&bar_rows[i]), (phases >> i) & 1u);
         if (threadIdx.x == 0 && b.status) atomicExch(b.status, static_cast<int>(PRQ_ERR_TIMEOUT));
     }
 }
 
 template <int kRowsThreads>
-cudaError_t launch_rows_impl(const QuantBatch& b, size_t smem, int sm_count, cudaStream_t stream) {
+cudaError_t launch_rows_impl(const QuantBatch& b, size_t smem, int n_buf, int sm_count, cudaStream_t stream) {
     static size_t configured = 0;   // the attribute is per function; raise it when a larger K comes
     if (smem > configured) {
         cudaError_t e = cudaFuncSetAttribute(quant_act_rows_kernel<kRowsThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -562,7 +566,7 @@ cudaError_t launch_rows_impl(const QuantBatch& b, size_t smem, int sm_count, cud
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, quant_act_rows_kernel<kRowsThreads>, b, n_slices);
+    return cudaLaunchKernelEx(&cfg, quant_act_rows_kernel<kRowsThreads>, b, n_slices, n_buf);
 }
 
 }  // namespace
@@ -590,18 +594,27 @@ cudaError_t launch_quant_act_batch(const QuantBatch& b, bool scale_perm, cudaStr
         if (const char* ev = dev_knobs_enabled() ? getenv("PRQ_QUANT_PARTS") : nullptr) { const int v = atoi(ev); if (v == 1 || v == 2 || v == 4 || v == 8) parts = v; }
         // Whole rows through shared memory when there are rows enough to fill the GPU that way, a slice's rows fit
         // twice, and the rows can be fetched by bulk copies (16-byte aligned).
-        // (dense layers: with stacked experts every slice first has to find its expert and, where that changed,
-        // rebuild the records, and measured 25-40 % slower than the column atoms at 128 experts)
+        // (dense layers: with stacked experts of K = 768 the row structure measured 25-40 % slower than the column atoms
+        // at 128 experts -- 26.7 against 19.0 us at 1024 tokens, 78.7 against 63.5 at 8192 -- also with the experts' row
+        // ranges cached in shared memory and seven slices in flight: narrow rows leave two of the eight warps without
+        // an atom, and a slice of 8 rows is little work per barrier)
         int rows = b.M >= 512 && b.expert_offsets == nullptr ? 1 : 0;
         if (const char* ev = dev_knobs_enabled() ? getenv("PRQ_QUANT_ROWS") : nullptr) rows = atoi(ev);
-        const size_t smem = 2 * static_cast<size_t>(kRowsR) * (p.K * 2 + 16) + static_cast<size_t>(p.K) * 8 +
-                            2 * static_cast<size_t>(kRowsR) * (p.K / 32) + 256;   // + alignment slack
-        if (rows && smem <= 200 * 1024 && (reinterpret_cast<uintptr_t>(b.x) & 15) == 0 && b.ldx % 8 == 0) {
+        const size_t buf_bytes = static_cast<size_t>(kRowsR) * (p.K * 2 + 16);
+        const size_t fixed = static_cast<size_t>(p.K) * 8 + 2 * static_cast<size_t>(kRowsR) * (p.K / 32) + 256;   // + alignment slack
+        if (rows && 2 * buf_bytes + fixed <= 200 * 1024 && (reinterpret_cast<uintptr_t>(b.x) & 15) == 0 && b.ldx % 8 == 0) {
             QuantBatch br = b;
             br.n_atoms = n_atoms; br.n_tail = 0; br.tail_split = 1;
-            // (4.6 KB of static shared memory and 1 KB reserved per CTA beside the dynamic part)
-            return 2 * (smem + 6 * 1024) <= 227 * 1024 ? launch_rows_impl<256>(br, smem, sm_count[dev], stream)
-                                                       : launch_rows_impl<512>(br, smem, sm_count[dev], stream);
+            // Two CTAs per SM where two slices of rows fit twice (8.7 KB of static shared memory and 1 KB reserved per
+            // CTA beside the dynamic part); then as many slices in flight as the CTA's share of the SM holds.
+            const size_t half_sm = 227 * 1024 / 2 - 10 * 1024;
+            const bool two = 2 * buf_bytes + fixed <= half_sm;
+            const size_t budget = two ? half_sm : 200 * 1024;
+            int n_buf = static_cast<int>((budget - fixed) / buf_bytes);
+            n_buf = n_buf > kRowsMaxBufs ? kRowsMaxBufs : n_buf;
+            const size_t smem = n_buf * buf_bytes + fixed;
+            return two ? launch_rows_impl<256>(br, smem, n_buf, sm_count[dev], stream)
+                       : launch_rows_impl<512>(br, smem, n_buf, sm_count[dev], stream);
         }
     }
     // the tail atoms of the scale + permute mode in shares of 16 rows (128 / 8), see the kernel
