@@ -329,6 +329,11 @@ def run_moe_workload(args, torch, prq, synth, dev, pk, T):
     g = lambda: prq.linear_grouped(w, codes, sf, d_off, M, prq.BF16, out=y)
     n = 20
     tq = timer.run([q], n, 3) / n * 1e6
+    # the same rows in identity mode: what the quantiser costs once every expert's scale and permutation are folded
+    # into its producers (Eq. (1)); the codes it leaves behind are not the layer's, so it runs before the last q()
+    qi = lambda: prq.quantize_act(w, x, prq.ACT_IDENTITY, expert_offsets=d_off, out=(codes, None, sf))
+    tqi = timer.run([qi], n, 3) / n * 1e6
+    q()
     tg = timer.run([g], n, 3) / n * 1e6
     active = int((np.diff(offsets) > 0).sum())
     fl = 2.0 * M * N * (K + k)
@@ -336,7 +341,10 @@ def run_moe_workload(args, torch, prq, synth, dev, pk, T):
     t_roof = max(fl / (pk["bf16_tflops"] * FP4_OVER_BF16) / 1e6, by / pk["hbm_gbs"] / 1e3)
     status = prq.last_device_status()
     w.free()
-    return dict(workload="moe", T=T, rows=M, active_experts=active, quant_us=tq, gemm_us=tg, gemm_tflops=fl / tg / 1e6,
+    qby = 2.53125 * M * K
+    return dict(workload="moe", T=T, rows=M, active_experts=active, quant_us=tq, quant_identity_us=tqi,
+                quant_roofline_frac=qby / pk["hbm_gbs"] / 1e3 / tq, quant_identity_roofline_frac=qby / pk["hbm_gbs"] / 1e3 / tqi,
+                gemm_us=tg, gemm_tflops=fl / tg / 1e6,
                 gemm_gbs=by / tg / 1e3, gemm_roofline_frac=t_roof / tg, device_status=status,
                 note="weights (116 MB for 128 experts) are re-read every launch; they nearly fit the 126 MB L2")
 
