@@ -293,6 +293,22 @@ def run_block_workload(args, torch, prq, synth, dev, pk, M, k_override=None, n_l
                                   gemm_roofline_frac=fl8 / (pk["bf16_tflops"] * 2.0) / 1e6 / tg8)
             for e in ds:
                 e["w"].free()
+        # q / k / v of the second format prepared as one layer (one quantiser launch, one GEMM over 6144 output features)
+        ds = []
+        for lin in layers:
+            Ws8 = [lin[nm]["Wb"].view(torch.int16).cpu().numpy().view(np.uint16) for nm in ("q", "k", "v")]
+            w8 = prq.prepare_weights_stacked(Ws8, lin["q"]["amax"], 0.5, 0, fmt=prq.FMT_MXFP8)
+            c8, _, s8 = prq.quantize_act(w8, lin["q"]["x"], prq.ACT_SCALE_PERM)
+            ds.append(dict(w=w8, x=lin["q"]["x"], codes=c8, sf=s8,
+                           y=torch.empty((M, w8.N), dtype=torch.bfloat16, device=dev)))
+        tq8 = timer.run([(lambda e=e: prq.quantize_act(e["w"], e["x"], prq.ACT_SCALE_PERM, out=(e["codes"], None, e["sf"]))) for e in ds], n, n_layers) / n * 1e6
+        tg8 = timer.run([(lambda e=e: prq.linear(e["w"], e["codes"], e["sf"], M, prq.BF16, out=e["y"])) for e in ds], n, n_layers) / n * 1e6
+        N8, K8 = ds[0]["w"].N, ds[0]["w"].K
+        fl8 = 2.0 * M * N8 * K8
+        fp8_rows["qkv_stacked"] = dict(N=N8, K=K8, quant_us=tq8, gemm_us=tg8, gemm_tflops=fl8 / tg8 / 1e6,
+                                       gemm_roofline_frac=fl8 / (pk["bf16_tflops"] * 2.0) / 1e6 / tg8)
+        for e in ds:
+            e["w"].free()
     total_flops = sum(2.0 * M * N * (K + (k if k_override is None else k_override)) for N, K, k in BLOCK_LINEARS.values())
     status = prq.last_device_status()
     for lin in layers:

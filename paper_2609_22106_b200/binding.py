@@ -473,16 +473,17 @@ def linear_gated(w_gu: Weights, codes, scales_sf, M: int, w_down: Weights, row_s
     return oc, orow, osf, h
 
 
-def prepare_weights_stacked(Ws, act_amax: np.ndarray, alpha: float, k_tail: int, scale_search: bool = False) -> Weights:
+def prepare_weights_stacked(Ws, act_amax: np.ndarray, alpha: float, k_tail: int, scale_search: bool = False,
+                            fmt: int = FMT_MXFP4) -> Weights:
     """Several layers over the same activation (list of uint16 (N_i, K) arrays) prepared as one layer; layer i's outputs
-    are columns [sum N_j for j < i, + N_i) of linear()'s result."""
+    are columns [sum N_j for j < i, + N_i) of linear()'s result.  fmt as in prepare_weights (MXFP8: k_tail 0)."""
     mats = [np.ascontiguousarray(W, np.uint16) for W in Ws]
     K = mats[0].shape[1]
     ptrs = (ctypes.c_void_p * len(mats))(*[m.ctypes.data for m in mats])
     ns = (ctypes.c_int * len(mats))(*[m.shape[0] for m in mats])
     amax = np.ascontiguousarray(act_amax, np.float32)
     h = ctypes.c_void_p()
-    o = _opts(scale_search)
+    o = _opts(scale_search, False, fmt)
     _check(lib().prq_prepare_weights_stacked(ctypes.cast(ptrs, ctypes.c_void_p), ctypes.cast(ns, ctypes.c_void_p), len(mats), K,
                                              _np_ptr(amax), alpha, k_tail, ctypes.cast(ctypes.pointer(o), ctypes.c_void_p),
                                              ctypes.byref(h)), "prq_prepare_weights_stacked")

@@ -89,3 +89,34 @@ def test_mxfp8_refusals(prq, oracle):
     with pytest.raises(prq.PrqError):
         w.clone()
     w.free()
+
+
+def test_mxfp8_stacked_preparation(prq, oracle):
+    """q / k / v-like layers over one activation prepared as one MXFP8 layer: its fields are the oracle's for the
+    concatenated matrix, and its output columns are the separate layers' outputs, bit for bit."""
+    K, M = 320, 200
+    Ns = [96, 32, 40]
+    L = synth.layer(83, sum(Ns), K, M, T_cal=32)
+    amax = oracle.channel_amax(L["zcal"])
+    Ws, r = [], 0
+    for n in Ns:
+        Ws.append(L["W"][r: r + n]); r += n
+    w = prq.prepare_weights_stacked(Ws, amax, 0.5, 0, fmt=prq.FMT_MXFP8)
+    o = oracle.fp8_prepare(L["W"], amax, float(np.float32(0.5)))
+    assert w.format == prq.FMT_MXFP8 and w.N == sum(Ns)
+    assert np.array_equal(w.get(prq.FIELD_CODES), o["wcodes"]) and np.array_equal(w.get(prq.FIELD_SCALES), o["wscales"])
+    x = dev_bf16(L["x"])
+    codes, _, sf = prq.quantize_act(w, x, prq.ACT_SCALE_PERM)
+    y = prq.linear(w, codes, sf, M, prq.F32)
+    oc, osc = oracle.fp8_quantize_act(L["x"], o["inv_s"])
+    y_ref = oracle.fp8_matmul(oc, osc, o["wcodes"], o["wscales"])
+    assert np.abs(y.cpu().numpy().astype(np.float64) - y_ref).max() <= prq_ref.tolerance(y_ref)
+    r = 0
+    for n, Wi in zip(Ns, Ws):
+        wi = prq.prepare_weights(Wi, amax, 0.5, 0, fmt=prq.FMT_MXFP8)
+        ci, _, si = prq.quantize_act(wi, x, prq.ACT_SCALE_PERM)
+        assert torch.equal(ci, codes)
+        yi = prq.linear(wi, ci, si, M, prq.F32)
+        assert torch.equal(yi, y[:, r: r + n])
+        wi.free(); r += n
+    w.free()
