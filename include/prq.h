@@ -258,6 +258,10 @@ size_t prq_act_bytes_for(const prq_weights *w, int M, prq_buf which);
  * Precondition: x is finite.  The kernel does not look for NaN or infinities (a scan would cost a second pass
  * over a memory-bound kernel); a block that holds one gets a meaningless scale byte and the product is
  * undefined for that row.  The offline calls do check W and amax (NONFINITE).
+ * Errors: INVALID_ARG / ALIGNMENT before anything is enqueued.  In scale + permute mode a dense layer of 512 rows or
+ * more is fetched by bulk copies whose waits are bounded like every device wait of this library: if one ran out the
+ * kernel returns early and PRQ_ERR_TIMEOUT is recorded in the device status word (prq_last_device_status); the output
+ * buffers are then incomplete.
  * M == 0 is a no-op. */
 prq_status prq_quantize_act(const prq_weights *w, prq_act_mode mode, const void *x, int M, int ldx,
                             const int32_t *expert_offsets, void *codes, void *scales_row, void *scales_sf,
