@@ -307,20 +307,21 @@ quant_act_kernel(const QuantBatch b) {
 
 
 // ---------------------------------------------------------------------------------------------------------
-// Scale + permute mode, second structure: whole rows through shared memory.  A persistent CTA takes slices of
-// kRowsR rows; the rows of the next slice arrive by bulk copies (one per row, no instruction per element) while
-// the current slice is quantised, and every gather of the permutation is a shared-memory read.  The lanes of a
-// warp are 8 different rows reading the SAME source column (for 4 blocks side by side): the rows are 16 bytes
-// further apart than a multiple of 128 bytes, so the 8 rows fall into different banks and a gather costs about
-// one pass however scattered the permutation is -- against one 32-byte sector per 2-byte read when the tail of
-// the permutation is gathered from global memory -- and the column's index and reciprocal scale are the same for
-// all rows, so they come as 16-byte broadcast loads, four columns at a time, instead of living in registers per
-// lane.  A lane takes one row of one block: 32 values held in registers (no shuffle), 16 bytes of codes and one
-// scale byte.  The scale bytes of the slice are collected in shared memory and then written out in every place
-// the GEMM reads them (main stages, duplicated tail bytes in the residual stages, zeros for rows and blocks that
-// do not exist) and, if asked for, row-major.  Several layers that read the same activation are quantised from
-// the one copy of the rows.
-// threads per CTA: 256 where two CTAs share an SM, 512 where the rows of a wide layer leave room for one only
+// Scale + permute mode, second structure: whole rows through shared memory.  A persistent CTA takes consecutive
+// slices of kRowsR rows; the rows of the next slices arrive by bulk copies (one per row, no instruction per element)
+// while the current slice is quantised, and every gather of the permutation is a shared-memory read.  The lanes of
+// a warp are 8 different rows reading the SAME source column, for the 4 blocks of one 128-column atom side by side:
+// the staged rows are 16 bytes further apart than a multiple of 128 bytes, so the 8 rows fall into 8 different
+// groups of four banks and a gather costs about one pass however scattered the permutation is -- against one
+// 32-byte sector per 2-byte read when the tail of the permutation is gathered from global memory.  The column's
+// source offset and reciprocal scale are the same for all rows of a warp: they are kept as one 16-byte record per
+// column pair in shared memory (built once per layer and expert) instead of living in registers per lane.  A lane
+// takes one row of one block: 32 values held in registers (no shuffle for the amax), 16 bytes of codes, one scale
+// byte; the four bytes of (row, atom) meet by two shuffles and leave as the one word the GEMM's layout has for them.
+// The tail's bytes are also collected in shared memory and written once more where the residual stages read them;
+// rows and blocks that do not exist get zero bytes; row-major scales are written if asked for.  Several layers that
+// read the same activation are quantised from the one copy of the rows.
+// Threads per CTA: 256 where two CTAs share an SM, 512 where the rows of a wide layer leave room for one only.
 constexpr int kRowsR = 8;                        // rows per slice
 constexpr int kRowsMaxBufs = 8;                  // slices of rows in shared memory at most (at least 2)
 static_assert(32 / kRowsR == 4, "a warp is 8 rows x the 4 blocks of an atom");
