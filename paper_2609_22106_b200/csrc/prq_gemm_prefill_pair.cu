@@ -399,7 +399,9 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tm_act, const __grid_con
             while (ok && r.next(sg)) {
                 // (the 288-column tile has one accumulator: the host gives such a call one tile per pair at most)
                 const int buf = C::kAccBufs == 2 ? (seg_it & 1) : 0;
+                if (trace && lane == 0 && seg_it < 8) trace[216 + 2 * seg_it] = clock64();
                 if (!mbar_wait(smem_u32(&bar_acc_empty[buf]), ((seg_it >> 1) & 1) ^ 1, abort_flag, p.wait_limit)) { ok = false; break; }
+                if (trace && lane == 0 && seg_it < 8) trace[217 + 2 * seg_it] = clock64();
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + buf * BN;
                 uint32_t accumulate = 0;
