@@ -238,3 +238,41 @@ def test_permuting_quantiser_structures_against_oracle(prq, oracle, monkeypatch,
         got = sf.cpu().numpy()[: want.size].reshape(-1, groups, 1024)[:, :g0]
         assert np.array_equal(got, want.reshape(-1, groups, 1024)[:, :g0]), what
         w.free()
+
+
+@pytest.mark.parametrize("gbn", [0, 64, 128])
+def test_many_experts_beyond_the_row_cache(prq, oracle, monkeypatch, gbn):
+    """300 stacked experts (more than the kernels cache row ranges for), most with a handful of rows and many with
+    none: the per-expert tile tables are built by a warp scan over ten experts per lane."""
+    if gbn:
+        monkeypatch.setenv("PRQ_GROUPED_BN", str(gbn))
+    E, N, K, k = 300, 136, 96, 32
+    rng = np.random.default_rng(4242)
+    counts = rng.choice([0, 0, 0, 1, 2, 5, 9, 130], size=E, p=[.3, .1, .1, .2, .1, .1, .05, .05])
+    offsets = np.concatenate([[0], np.cumsum(counts)]).astype(np.int32)
+    M = int(offsets[-1])
+    ch = synth.HeavyTailChannels(77, K)
+    Ws = np.stack([synth.weights(5000 + e, N, K) for e in range(E)])
+    amax = np.stack([oracle.channel_amax(ch.rows(6000 + e, 16)) for e in range(E)])
+    w = prq.prepare_weights(Ws, amax, 0.5, k)
+    x = ch.rows(7000, M)
+    d_off = torch.from_numpy(offsets).cuda()
+    codes, srow, sf = prq.quantize_act(w, dev_bf16(x), prq.ACT_SCALE_PERM, expert_offsets=d_off, row_scales=True)
+    full = torch.full((M, N + 8), 7.0, dtype=torch.float32, device="cuda")
+    y = prq.linear_grouped(w, codes, sf, d_off, M, prq.F32, out=full[:, :N])
+    assert prq.last_device_status() == 0
+    assert bool((full[:, N:] == 7.0).all())
+    got_c = codes.cpu().numpy()[: M * K // 2].reshape(M, K // 2)
+    got_s = srow.cpu().numpy()[: M * K // 32].reshape(M, K // 32)
+    nonempty = np.flatnonzero(counts)
+    picks = set(int(e) for e in rng.choice(nonempty, size=12, replace=False)) | {int(nonempty[0]), int(nonempty[-1]), int(np.argmax(counts))}
+    for e in sorted(picks):
+        r0, r1 = int(offsets[e]), int(offsets[e + 1])
+        o = oracle.prepare(Ws[e], amax[e], float(np.float32(0.5)), k)
+        oc, osc = oracle.quantize_act(x[r0:r1], o["perm"], o["inv_s"])
+        assert np.array_equal(got_c[r0:r1], oc) and np.array_equal(got_s[r0:r1], osc), e
+        ca, sa = oracle.augment_act(oc, osc, k)
+        y_ref = oracle.matmul(ca, sa, o["wcodes"], o["wscales"])
+        got = y[r0:r1].cpu().numpy().astype(np.float64)
+        assert np.abs(got - y_ref).max() <= prq_ref.tolerance(y_ref), e
+    w.free()
